@@ -1,0 +1,205 @@
+/*
+ * plora.h — C ABI of the B200 (sm_100a) batched heterogeneous-adapter LoRA delta.
+ *
+ * For a batch of tokens, each tagged with an adapter id a_t, the library computes
+ *
+ *        y_t  +=  s_a * ( (x_t * A_a) * B_a ),        a = a_t
+ *
+ * over a pool of adapters held in this GPU's HBM.  A_a is [d_in, r_a], B_a is
+ * [r_a, d_out] (paper Section II-A: y = x (W + A B); Section III-A: Y = X A B).
+ * This is the paper's placement P1 / strategy E1 (Section V-A): both matrices are
+ * resident in GPU memory and the GPU computes the delta without touching any
+ * other device.  The shrink m = x A and expand y = m B halves (Section V-A,
+ * strategy E4) are also exported on their own.
+ *
+ * General conventions
+ *   - "dev" pointers are CUDA device pointers on the context's device; "host"
+ *     pointers are ordinary host memory.  The library never takes ownership of a
+ *     caller's buffer.
+ *   - bf16 tensors are raw 16-bit patterns; x is [n_tok, d_in] row-major
+ *     contiguous, y is fp32 [n_tok, d_out] row-major contiguous.  d_in and d_out
+ *     must be multiples of 8.
+ *   - adapter ids are int32 in [-1, n_adapters); -1 means "no adapter": the
+ *     token's row of y is left as it is.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Unless stated otherwise a call only enqueues work on `stream` and returns
+ *     without synchronising.
+ *   - Every function returns a plora_status (0 = ok, negative = error) and never
+ *     throws or aborts.  Errors that the host can see are returned before
+ *     anything is launched.  Conditions only the device can see (an id outside
+ *     [-1, n_adapters), a bounded wait that ran out) set a sticky device status
+ *     word, read with plora_device_status; the kernels stay inside their buffers
+ *     in that case (an out-of-range id is treated as -1).
+ *   - One context serves one stream at a time; calls on one context are not
+ *     thread-safe.
+ */
+#ifndef PLORA_H_
+#define PLORA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define PLORA_API __attribute__((visibility("default")))
+#else
+#define PLORA_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct plora_ctx plora_ctx; /* opaque, owned by the library */
+typedef int32_t plora_status;
+
+enum {
+    PLORA_OK = 0,
+    PLORA_ERR_INVALID_ARG = -1,    /* null pointer, negative size, size above the context's limits */
+    PLORA_ERR_NOT_REGISTERED = -2, /* no pool registered for (layer, proj) */
+    PLORA_ERR_BAD_ADAPTER_ID = -3, /* device status: an id outside [-1, n_adapters) was seen */
+    PLORA_ERR_WORKSPACE = -4,      /* slab or workspace too small */
+    PLORA_ERR_CUDA = -5,           /* a CUDA runtime call failed */
+    PLORA_ERR_TIMEOUT = -6,        /* device status: a bounded device-side wait ran out */
+    PLORA_ERR_UNSUPPORTED = -7     /* shape outside what the kernels handle (rank > 128, d not multiple of 8, ...) */
+};
+
+/* Which kernels plora_lora_delta uses. */
+enum {
+    PLORA_PATH_AUTO = 0,    /* fused BGMV for short segments, SGMV for long ones */
+    PLORA_PATH_UNFUSED = 1, /* BGMV shrink kernel then BGMV expand kernel, m in HBM workspace */
+    PLORA_PATH_FUSED = 2,   /* fused BGMV for every segment */
+    PLORA_PATH_SGMV = 3     /* tensor-core segmented GEMM for every segment */
+};
+
+/*
+ * Create a context on CUDA device `device`.  Allocates the bucketing buffers
+ * and kernel workspace for batches of up to `max_tokens` tokens over pools of up
+ * to `max_adapters` adapters.  Synchronous.  *out is set only on success.
+ */
+PLORA_API plora_status plora_create(plora_ctx **out, int device, int32_t max_tokens, int32_t max_adapters);
+
+/* Free everything the context owns (not the caller's slabs).  Synchronises the device. */
+PLORA_API plora_status plora_destroy(plora_ctx *ctx);
+
+/*
+ * Adapter-pool registry (the paper keeps each adapter as a matrix pair (A, B)
+ * attached to every injected weight of every layer, Sections II-A and VII-A; here
+ * one pool = all adapters of one (layer, projection)).
+ *
+ * plora_pool_desc describes one pool in the paper's logical layout.  All arrays
+ * are HOST arrays of length n_adapters; A[a] / B[a] point to bf16 matrices
+ * [d_in, ranks[a]] and [ranks[a], d_out], row-major contiguous, in host memory
+ * (ab_on_device = 0) or device memory (ab_on_device = 1).  Ranks must lie in
+ * [1, 128].  scales[a] is s_a (for instance alpha / r_a).
+ */
+typedef struct {
+    int32_t layer, proj;
+    int32_t d_in, d_out;
+    int32_t n_adapters;
+    int32_t ab_on_device;
+    const int32_t *ranks;
+    const float *scales;
+    const void *const *A;
+    const void *const *B;
+} plora_pool_desc;
+
+/*
+ * Bytes of device memory the library's private slab layout needs for this pool
+ * (only layer..n_adapters and ranks are read).  Returns 0 if the description is
+ * invalid or unsupported.  The caller allocates that much device memory,
+ * 256-byte aligned, and keeps it alive while the pool is registered.
+ */
+PLORA_API size_t plora_pool_slab_bytes(const plora_pool_desc *desc);
+
+/*
+ * Repack the pool into `slab_dev` (library-private tiled layout, ranks padded
+ * with zeros) and record its offset table under (layer, proj), replacing any
+ * earlier registration of that pair.  The source matrices are not needed after
+ * the call returns: it synchronises `stream` (registration is a set-up step).
+ * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE (slab_bytes too small or more
+ * adapters than the context allows), CUDA.
+ */
+PLORA_API plora_status plora_register_pool(plora_ctx *ctx, const plora_pool_desc *desc, void *slab_dev, size_t slab_bytes,
+                                 void *stream);
+
+/* Padded maximum rank of a registered pool: the leading dimension `ldm` that
+ * plora_shrink / plora_expand need at least.  Negative status on error. */
+PLORA_API int32_t plora_pool_max_rank(plora_ctx *ctx, int32_t layer, int32_t proj);
+
+/*
+ * Token bucketing (once per step; every layer and projection of the step reuses
+ * it).  The per-adapter request count B_i of the paper's cost model (Section
+ * VI-B) is the length of adapter i's segment.
+ *
+ * adapter_ids_dev: int32 [n_tok] on the device.  Produces, in context-owned
+ * device memory:
+ *   perm         int32 [n_tok]      token indices ordered by (id, token index), id -1 last
+ *   seg_adapter  int32 [cap]        ascending distinct ids >= 0 present; tail = -1
+ *   seg_start    int32 [cap + 1]    start of each segment in perm; entry n_seg and tail = n_active
+ *   n_seg, n_active  int32 scalars  segments, tokens with id >= 0
+ * with cap = min(n_tok, n_adapters).  The result is unique (stable order) and
+ * deterministic.  Errors: INVALID_ARG (null, n_tok < 0 or > max_tokens,
+ * n_adapters < 1 or > max_adapters).
+ */
+PLORA_API plora_status plora_bucket(plora_ctx *ctx, const int32_t *adapter_ids_dev, int32_t n_tok, int32_t n_adapters,
+                          void *stream);
+
+/* Device pointers to the current bucket's arrays (valid until the next plora_bucket
+ * or plora_destroy; written by work enqueued on the bucket's stream). */
+PLORA_API plora_status plora_bucket_view(plora_ctx *ctx, const int32_t **perm, const int32_t **seg_adapter,
+                               const int32_t **seg_start, const int32_t **n_seg, const int32_t **n_active);
+
+/*
+ * The LoRA delta of one projection (Section V-A, strategy E1):
+ *     y[t, :] += s_a * ((x[t, :] * A_a) * B_a),  a = adapter_ids[t]
+ * x_dev bf16 [n_tok, d_in], y_dev fp32 [n_tok, d_out] (holds the base projection
+ * output on entry), both on the device; d_in/d_out are the registered pool's.
+ * Uses the context's current bucket when plora_bucket was last called with this
+ * same (adapter_ids_dev, n_tok) and the pool's n_adapters; otherwise buckets
+ * first.  Every adapter present in the batch is read from HBM once per call,
+ * whatever its number of tokens (Section VI-B).  Each element of y receives
+ * exactly one addition, so results are bit-reproducible run to run.
+ * Errors: INVALID_ARG, NOT_REGISTERED, CUDA.
+ */
+PLORA_API plora_status plora_lora_delta(plora_ctx *ctx, const void *x_dev, const int32_t *adapter_ids_dev, int32_t n_tok,
+                              int32_t layer, int32_t proj, float *y_dev, void *stream);
+
+/*
+ * The two halves on their own (Section V-A, strategy E4: m = x A, then y = m B).
+ * m_dev is fp32 [n_tok, ldm] on the device, ldm >= plora_pool_max_rank.
+ * plora_shrink writes m[t, k] = sum_i x[t, i] A_a[i, k] (unscaled) for k < r_a and 0
+ * for the other columns and for tokens with id -1.  plora_expand computes
+ * y[t, :] += s_a * (m[t, :r_a] * B_a).  Same bucket rule and errors as above.
+ */
+PLORA_API plora_status plora_shrink(plora_ctx *ctx, const void *x_dev, const int32_t *adapter_ids_dev, int32_t n_tok,
+                          int32_t layer, int32_t proj, float *m_dev, int32_t ldm, void *stream);
+PLORA_API plora_status plora_expand(plora_ctx *ctx, const float *m_dev, int32_t ldm, const int32_t *adapter_ids_dev,
+                          int32_t n_tok, int32_t layer, int32_t proj, float *y_dev, void *stream);
+
+/*
+ * Same operation as plora_lora_delta with HOST buffers: copies x, ids and y to
+ * context-owned device staging buffers, buckets, runs the delta and copies y
+ * back, all on `stream`, then synchronises `stream`.  Pinned host memory makes
+ * the copies asynchronous to each other but is not required.
+ */
+PLORA_API plora_status plora_lora_delta_host(plora_ctx *ctx, const void *x_host, const int32_t *adapter_ids_host,
+                                   int32_t n_tok, int32_t layer, int32_t proj, float *y_host, void *stream);
+
+/* Choose the kernels plora_lora_delta uses (PLORA_PATH_*); takes effect at the next
+ * plora_bucket.  `sgmv_min_rows` (> 0) is the segment length from which AUTO sends a
+ * segment to the tensor-core path; pass 0 to keep the default. */
+PLORA_API plora_status plora_set_path(plora_ctx *ctx, int32_t path, int32_t sgmv_min_rows);
+
+/* Synchronise `stream`, copy the sticky device status word to *host_out (0 or a
+ * PLORA_ERR_* value) and clear it. */
+PLORA_API plora_status plora_device_status(plora_ctx *ctx, void *stream, int32_t *host_out);
+
+/* Kernels launched by this context since creation (host-side counter). */
+PLORA_API int64_t plora_launch_count(plora_ctx *ctx);
+
+PLORA_API const char *plora_status_string(plora_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PLORA_H_ */

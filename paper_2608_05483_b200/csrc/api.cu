@@ -1,0 +1,494 @@
+// C ABI of the library (declared in plora.h): context, adapter-pool registry,
+// bucketing and the delta entry points.  Host code only; the kernels live in
+// bucket.cu, registry.cu, bgmv.cu and sgmv.cu.
+#include <climits>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "plora_internal.cuh"
+
+using namespace plora;
+
+namespace {
+
+struct PoolRec {
+    int32_t layer, proj;
+    PoolDev dev;
+    AdapterEntry* table_dev;
+};
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+        if (prev == dev) prev = -1;
+    }
+    ~DeviceGuard() {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+constexpr int kDefaultSgmvMinRows = 1 << 30;   // tensor-core path not wired in yet
+
+}  // namespace
+
+struct plora_ctx {
+    int device = 0;
+    int32_t max_tokens = 0, max_adapters = 0;
+    int sm_count = 0;
+    // bucket
+    void* bucket_block = nullptr;
+    BucketDev bk{};
+    int32_t* status_dev = nullptr;
+    const int32_t* cur_ids = nullptr;
+    int32_t cur_ntok = -1, cur_nadapters = -1;
+    bool bucket_valid = false;
+    int32_t path = PLORA_PATH_AUTO;
+    int32_t sgmv_min_rows = kDefaultSgmvMinRows;
+    int32_t bucket_sgmv_min = INT_MAX;   // threshold the current bucket was built with
+    // workspace for the unfused path's m
+    float* m_ws = nullptr;
+    // staging for the host-buffer entry point
+    void* x_stage = nullptr;
+    float* y_stage = nullptr;
+    int32_t* ids_stage = nullptr;
+    size_t x_stage_bytes = 0, y_stage_bytes = 0;
+    std::vector<PoolRec> pools;
+    int64_t launches = 0;
+};
+
+namespace {
+
+inline cudaStream_t as_stream(void* s) { return static_cast<cudaStream_t>(s); }
+
+PoolRec* find_pool(plora_ctx* ctx, int32_t layer, int32_t proj) {
+    for (auto& p : ctx->pools)
+        if (p.layer == layer && p.proj == proj) return &p;
+    return nullptr;
+}
+
+bool desc_shape_ok(const plora_pool_desc* d, plora_status* why) {
+    if (!d || !d->ranks || d->n_adapters < 1 || d->d_in < 1 || d->d_out < 1) { *why = PLORA_ERR_INVALID_ARG; return false; }
+    if ((d->d_in & 7) || (d->d_out & 7)) { *why = PLORA_ERR_UNSUPPORTED; return false; }
+    for (int a = 0; a < d->n_adapters; ++a) {
+        if (d->ranks[a] < 1) { *why = PLORA_ERR_INVALID_ARG; return false; }
+        if (d->ranks[a] > kMaxRank) { *why = PLORA_ERR_UNSUPPORTED; return false; }
+    }
+    return true;
+}
+
+// Fills the offset table (host copy) and returns the slab size.
+size_t layout_pool(const plora_pool_desc* d, std::vector<AdapterEntry>* table, int* max_rp, int* uniform_rp = nullptr) {
+    size_t off = 0;
+    int mrp = 0, urp = -1;
+    if (table) table->resize(d->n_adapters);
+    for (int a = 0; a < d->n_adapters; ++a) {
+        const int rp = pad_rank(d->ranks[a]);
+        const size_t tb = (size_t)tile_bytes(rp);
+        AdapterEntry e{};
+        e.offA = off;
+        off += tb * tiles_for(d->d_in, rp);
+        e.offB = off;
+        off += tb * tiles_for(d->d_out, rp);
+        e.r = d->ranks[a];
+        e.rp = rp;
+        e.scale = d->scales ? d->scales[a] : 1.0f;
+        if (table) (*table)[a] = e;
+        if (rp > mrp) mrp = rp;
+        urp = (urp == -1 || urp == rp) ? rp : 0;
+    }
+    if (max_rp) *max_rp = mrp;
+    if (uniform_rp) *uniform_rp = urp > 0 ? urp : 0;
+    return off;
+}
+
+int32_t effective_sgmv_min(const plora_ctx* ctx) {
+    switch (ctx->path) {
+        case PLORA_PATH_SGMV: return 1;
+        case PLORA_PATH_AUTO: return ctx->sgmv_min_rows;
+        default: return INT_MAX;
+    }
+}
+
+plora_status do_bucket(plora_ctx* ctx, const int32_t* ids, int32_t n_tok, int32_t n_adapters, cudaStream_t st) {
+    const int32_t thr = effective_sgmv_min(ctx);
+    int nl = 0;
+    cudaError_t e = launch_bucket(ids, n_tok, n_adapters, thr, ctx->bk, ctx->status_dev, st, &nl);
+    ctx->launches += nl;
+    if (e != cudaSuccess) { ctx->bucket_valid = false; return PLORA_ERR_CUDA; }
+    ctx->cur_ids = ids;
+    ctx->cur_ntok = n_tok;
+    ctx->cur_nadapters = n_adapters;
+    ctx->bucket_sgmv_min = thr;
+    ctx->bucket_valid = true;
+    return PLORA_OK;
+}
+
+plora_status ensure_bucket(plora_ctx* ctx, const int32_t* ids, int32_t n_tok, int32_t n_adapters, cudaStream_t st) {
+    if (ctx->bucket_valid && ctx->cur_ids == ids && ctx->cur_ntok == n_tok && ctx->cur_nadapters == n_adapters &&
+        ctx->bucket_sgmv_min == effective_sgmv_min(ctx))
+        return PLORA_OK;
+    return do_bucket(ctx, ids, n_tok, n_adapters, st);
+}
+
+plora_status check_call(plora_ctx* ctx, const void* a, const void* ids, int32_t n_tok, const void* b) {
+    if (!ctx || n_tok < 0 || n_tok > ctx->max_tokens) return PLORA_ERR_INVALID_ARG;
+    if (n_tok > 0 && (!a || !ids || !b)) return PLORA_ERR_INVALID_ARG;
+    if (((uintptr_t)a & 15) || ((uintptr_t)b & 15) || ((uintptr_t)ids & 3)) return PLORA_ERR_INVALID_ARG;
+    return PLORA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+PLORA_API const char* plora_status_string(plora_status s) {
+    switch (s) {
+        case PLORA_OK: return "ok";
+        case PLORA_ERR_INVALID_ARG: return "invalid argument";
+        case PLORA_ERR_NOT_REGISTERED: return "no pool registered for (layer, proj)";
+        case PLORA_ERR_BAD_ADAPTER_ID: return "adapter id out of range";
+        case PLORA_ERR_WORKSPACE: return "slab or workspace too small";
+        case PLORA_ERR_CUDA: return "CUDA runtime error";
+        case PLORA_ERR_TIMEOUT: return "bounded device wait ran out";
+        case PLORA_ERR_UNSUPPORTED: return "unsupported shape";
+        default: return "unknown status";
+    }
+}
+
+PLORA_API plora_status plora_create(plora_ctx** out, int device, int32_t max_tokens, int32_t max_adapters) {
+    if (!out || max_tokens < 1 || max_adapters < 1) return PLORA_ERR_INVALID_ARG;
+    if (max_adapters > bucket_max_adapters()) return PLORA_ERR_UNSUPPORTED;
+    int n_dev = 0;
+    if (cudaGetDeviceCount(&n_dev) != cudaSuccess) return PLORA_ERR_CUDA;
+    if (device < 0 || device >= n_dev) return PLORA_ERR_INVALID_ARG;
+    DeviceGuard g(device);
+    if (!g.ok) return PLORA_ERR_CUDA;
+    plora_ctx* ctx = new (std::nothrow) plora_ctx();
+    if (!ctx) return PLORA_ERR_WORKSPACE;
+    ctx->device = device;
+    ctx->max_tokens = max_tokens;
+    ctx->max_adapters = max_adapters;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return PLORA_ERR_CUDA; }
+    ctx->sm_count = prop.multiProcessorCount;
+    if (prop.major < 10) { delete ctx; return PLORA_ERR_UNSUPPORTED; }
+
+    const size_t T = (size_t)max_tokens;
+    const size_t cap = T < (size_t)max_adapters ? T : (size_t)max_adapters;
+    auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
+    const size_t o_perm = 0;
+    const size_t o_sega = o_perm + up(T * 4);
+    const size_t o_segs = o_sega + up((cap + 1) * 4);
+    const size_t o_scal = o_segs + up((cap + 2) * 4);
+    const size_t o_bg = o_scal + 256;
+    const size_t o_sg = o_bg + up(T * sizeof(WorkUnit));
+    const size_t o_m = o_sg + up(T * sizeof(WorkUnit));
+    const size_t total = o_m + up(T * kMaxRank * 4);
+    uint8_t* blk = nullptr;
+    if (cudaMalloc(&blk, total) != cudaSuccess) { delete ctx; return PLORA_ERR_WORKSPACE; }
+    if (cudaMemset(blk, 0, total) != cudaSuccess) { cudaFree(blk); delete ctx; return PLORA_ERR_CUDA; }
+    ctx->bucket_block = blk;
+    ctx->bk.perm = (int32_t*)(blk + o_perm);
+    ctx->bk.seg_adapter = (int32_t*)(blk + o_sega);
+    ctx->bk.seg_start = (int32_t*)(blk + o_segs);
+    int32_t* scal = (int32_t*)(blk + o_scal);
+    ctx->bk.n_seg = scal + 0;
+    ctx->bk.n_active = scal + 1;
+    ctx->bk.n_bgmv_units = scal + 2;
+    ctx->bk.n_sgmv_tiles = scal + 3;
+    ctx->status_dev = scal + 8;
+    ctx->bk.bgmv_units = (WorkUnit*)(blk + o_bg);
+    ctx->bk.sgmv_tiles = (WorkUnit*)(blk + o_sg);
+    ctx->m_ws = (float*)(blk + o_m);
+    if (bucket_configure() != cudaSuccess || bgmv_configure() != cudaSuccess || sgmv_configure() != cudaSuccess ||
+        cudaDeviceSynchronize() != cudaSuccess) {
+        cudaFree(blk);
+        delete ctx;
+        return PLORA_ERR_CUDA;
+    }
+    *out = ctx;
+    return PLORA_OK;
+}
+
+PLORA_API plora_status plora_destroy(plora_ctx* ctx) {
+    if (!ctx) return PLORA_ERR_INVALID_ARG;
+    DeviceGuard g(ctx->device);
+    cudaDeviceSynchronize();
+    for (auto& p : ctx->pools) cudaFree(p.table_dev);
+    cudaFree(ctx->bucket_block);
+    cudaFree(ctx->x_stage);
+    cudaFree(ctx->y_stage);
+    cudaFree(ctx->ids_stage);
+    delete ctx;
+    return PLORA_OK;
+}
+
+PLORA_API size_t plora_pool_slab_bytes(const plora_pool_desc* desc) {
+    plora_status why;
+    if (!desc_shape_ok(desc, &why)) return 0;
+    return layout_pool(desc, nullptr, nullptr);
+}
+
+PLORA_API plora_status plora_register_pool(plora_ctx* ctx, const plora_pool_desc* d, void* slab_dev, size_t slab_bytes,
+                                 void* stream) {
+    if (!ctx || !d || !slab_dev || !d->A || !d->B) return PLORA_ERR_INVALID_ARG;
+    plora_status why;
+    if (!desc_shape_ok(d, &why)) return why;
+    if (d->n_adapters > ctx->max_adapters) return PLORA_ERR_WORKSPACE;
+    if ((uintptr_t)slab_dev & 255) return PLORA_ERR_INVALID_ARG;
+    for (int a = 0; a < d->n_adapters; ++a)
+        if (!d->A[a] || !d->B[a]) return PLORA_ERR_INVALID_ARG;
+    std::vector<AdapterEntry> table;
+    int max_rp = 0, uniform_rp = 0;
+    const size_t need = layout_pool(d, &table, &max_rp, &uniform_rp);
+    if (slab_bytes < need) return PLORA_ERR_WORKSPACE;
+
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return PLORA_ERR_CUDA;
+    cudaStream_t st = as_stream(stream);
+    const int N = d->n_adapters;
+    AdapterEntry* table_dev = nullptr;
+    const void** ptrs_dev = nullptr;   // [2N]: A pointers then B pointers
+    uint8_t* staging = nullptr;
+    plora_status rc = PLORA_OK;
+    std::vector<const void*> ptrs(2 * (size_t)N);
+    do {
+        if (cudaMalloc(&table_dev, sizeof(AdapterEntry) * N) != cudaSuccess ||
+            cudaMalloc(&ptrs_dev, sizeof(void*) * 2 * N) != cudaSuccess) { rc = PLORA_ERR_WORKSPACE; break; }
+        if (d->ab_on_device) {
+            for (int a = 0; a < N; ++a) { ptrs[a] = d->A[a]; ptrs[N + a] = d->B[a]; }
+        } else {
+            // stage the logical matrices on the device, then repack from there
+            size_t bytes = 0;
+            for (int a = 0; a < N; ++a) bytes += ((size_t)d->ranks[a] * (d->d_in + d->d_out) * 2 + 15) & ~(size_t)15;
+            if (cudaMalloc(&staging, bytes) != cudaSuccess) { rc = PLORA_ERR_WORKSPACE; break; }
+            size_t off = 0;
+            bool bad = false;
+            for (int a = 0; a < N && !bad; ++a) {
+                const size_t ba = (size_t)d->ranks[a] * d->d_in * 2, bb = (size_t)d->ranks[a] * d->d_out * 2;
+                bad |= cudaMemcpyAsync(staging + off, d->A[a], ba, cudaMemcpyHostToDevice, st) != cudaSuccess;
+                ptrs[a] = staging + off;
+                bad |= cudaMemcpyAsync(staging + off + ba, d->B[a], bb, cudaMemcpyHostToDevice, st) != cudaSuccess;
+                ptrs[N + a] = staging + off + ba;
+                off += (ba + bb + 15) & ~(size_t)15;
+            }
+            if (bad) { rc = PLORA_ERR_CUDA; break; }
+        }
+        if (cudaMemcpyAsync(table_dev, table.data(), sizeof(AdapterEntry) * N, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+            cudaMemcpyAsync(ptrs_dev, ptrs.data(), sizeof(void*) * 2 * N, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+            rc = PLORA_ERR_CUDA;
+            break;
+        }
+        int nl = 0;
+        cudaError_t e = launch_repack(table_dev, ptrs_dev, ptrs_dev + N, N, d->d_in, d->d_out, (uint8_t*)slab_dev, st, &nl);
+        ctx->launches += nl;
+        if (e != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess) { rc = PLORA_ERR_CUDA; break; }
+    } while (0);
+    cudaFree(staging);
+    cudaFree(ptrs_dev);
+    if (rc != PLORA_OK) {
+        cudaFree(table_dev);
+        cudaGetLastError();
+        return rc;
+    }
+    PoolRec rec{};
+    rec.layer = d->layer;
+    rec.proj = d->proj;
+    rec.table_dev = table_dev;
+    rec.dev.slab = (const uint8_t*)slab_dev;
+    rec.dev.table = table_dev;
+    rec.dev.d_in = d->d_in;
+    rec.dev.d_out = d->d_out;
+    rec.dev.n_adapters = N;
+    rec.dev.max_rp = max_rp;
+    rec.dev.uniform_rp = uniform_rp;
+    if (PoolRec* old = find_pool(ctx, d->layer, d->proj)) {
+        cudaStreamSynchronize(st);
+        cudaFree(old->table_dev);
+        *old = rec;
+    } else {
+        ctx->pools.push_back(rec);
+    }
+    return PLORA_OK;
+}
+
+PLORA_API int32_t plora_pool_max_rank(plora_ctx* ctx, int32_t layer, int32_t proj) {
+    if (!ctx) return PLORA_ERR_INVALID_ARG;
+    PoolRec* p = find_pool(ctx, layer, proj);
+    return p ? p->dev.max_rp : PLORA_ERR_NOT_REGISTERED;
+}
+
+PLORA_API plora_status plora_bucket(plora_ctx* ctx, const int32_t* ids, int32_t n_tok, int32_t n_adapters, void* stream) {
+    if (!ctx || n_tok < 0 || n_tok > ctx->max_tokens || n_adapters < 1 || n_adapters > ctx->max_adapters)
+        return PLORA_ERR_INVALID_ARG;
+    if (n_tok > 0 && !ids) return PLORA_ERR_INVALID_ARG;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return PLORA_ERR_CUDA;
+    return do_bucket(ctx, ids, n_tok, n_adapters, as_stream(stream));
+}
+
+PLORA_API plora_status plora_bucket_view(plora_ctx* ctx, const int32_t** perm, const int32_t** seg_adapter,
+                               const int32_t** seg_start, const int32_t** n_seg, const int32_t** n_active) {
+    if (!ctx || !ctx->bucket_valid) return PLORA_ERR_INVALID_ARG;
+    if (perm) *perm = ctx->bk.perm;
+    if (seg_adapter) *seg_adapter = ctx->bk.seg_adapter;
+    if (seg_start) *seg_start = ctx->bk.seg_start;
+    if (n_seg) *n_seg = ctx->bk.n_seg;
+    if (n_active) *n_active = ctx->bk.n_active;
+    return PLORA_OK;
+}
+
+PLORA_API plora_status plora_set_path(plora_ctx* ctx, int32_t path, int32_t sgmv_min_rows) {
+    if (!ctx || path < PLORA_PATH_AUTO || path > PLORA_PATH_SGMV || sgmv_min_rows < 0) return PLORA_ERR_INVALID_ARG;
+    ctx->path = path;
+    ctx->sgmv_min_rows = sgmv_min_rows > 0 ? sgmv_min_rows : kDefaultSgmvMinRows;
+    return PLORA_OK;
+}
+
+PLORA_API plora_status plora_lora_delta(plora_ctx* ctx, const void* x, const int32_t* ids, int32_t n_tok, int32_t layer,
+                              int32_t proj, float* y, void* stream) {
+    plora_status rc = check_call(ctx, x, ids, n_tok, y);
+    if (rc != PLORA_OK) return rc;
+    PoolRec* pool = find_pool(ctx, layer, proj);
+    if (!pool) return PLORA_ERR_NOT_REGISTERED;
+    if (n_tok == 0) return PLORA_OK;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return PLORA_ERR_CUDA;
+    cudaStream_t st = as_stream(stream);
+    rc = ensure_bucket(ctx, ids, n_tok, pool->dev.n_adapters, st);
+    if (rc != PLORA_OK) return rc;
+    int nl = 0;
+    cudaError_t e = cudaSuccess;
+    if (ctx->path == PLORA_PATH_UNFUSED) {
+        e = launch_bgmv(kShrinkOnly, pool->dev, ctx->bk, n_tok, x, nullptr, ctx->m_ws, pool->dev.max_rp, ctx->status_dev,
+                        ctx->sm_count, st, &nl);
+        if (e == cudaSuccess)
+            e = launch_bgmv(kExpandOnly, pool->dev, ctx->bk, n_tok, nullptr, y, ctx->m_ws, pool->dev.max_rp,
+                            ctx->status_dev, ctx->sm_count, st, &nl);
+    } else {
+        // a batch shorter than the threshold cannot hold a segment for the tensor-core path
+        const bool may_bgmv = ctx->path != PLORA_PATH_SGMV;
+        const bool may_sgmv = ctx->path == PLORA_PATH_SGMV || (ctx->path == PLORA_PATH_AUTO && n_tok >= ctx->sgmv_min_rows);
+        if (may_bgmv)
+            e = launch_bgmv(kFused, pool->dev, ctx->bk, n_tok, x, y, nullptr, 0, ctx->status_dev, ctx->sm_count, st, &nl);
+        if (e == cudaSuccess && may_sgmv)
+            e = launch_sgmv(pool->dev, ctx->bk, n_tok, x, y, ctx->status_dev, ctx->sm_count, st, &nl);
+    }
+    ctx->launches += nl;
+    return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
+}
+
+PLORA_API plora_status plora_shrink(plora_ctx* ctx, const void* x, const int32_t* ids, int32_t n_tok, int32_t layer, int32_t proj,
+                          float* m, int32_t ldm, void* stream) {
+    plora_status rc = check_call(ctx, x, ids, n_tok, m);
+    if (rc != PLORA_OK) return rc;
+    PoolRec* pool = find_pool(ctx, layer, proj);
+    if (!pool) return PLORA_ERR_NOT_REGISTERED;
+    if (ldm < pool->dev.max_rp || (ldm & 3)) return PLORA_ERR_INVALID_ARG;
+    if (n_tok == 0) return PLORA_OK;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return PLORA_ERR_CUDA;
+    cudaStream_t st = as_stream(stream);
+    // the split entry points always take the BGMV kernels: bucket with no tensor-core segments
+    const int32_t saved = ctx->path;
+    ctx->path = PLORA_PATH_UNFUSED;
+    rc = ensure_bucket(ctx, ids, n_tok, pool->dev.n_adapters, st);
+    ctx->path = saved;
+    if (rc != PLORA_OK) return rc;
+    int nl = 0;
+    cudaError_t e = launch_bgmv(kShrinkOnly, pool->dev, ctx->bk, n_tok, x, nullptr, m, ldm, ctx->status_dev,
+                                ctx->sm_count, st, &nl);
+    ctx->launches += nl;
+    return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
+}
+
+PLORA_API plora_status plora_expand(plora_ctx* ctx, const float* m, int32_t ldm, const int32_t* ids, int32_t n_tok,
+                          int32_t layer, int32_t proj, float* y, void* stream) {
+    plora_status rc = check_call(ctx, m, ids, n_tok, y);
+    if (rc != PLORA_OK) return rc;
+    PoolRec* pool = find_pool(ctx, layer, proj);
+    if (!pool) return PLORA_ERR_NOT_REGISTERED;
+    if (ldm < pool->dev.max_rp || (ldm & 3)) return PLORA_ERR_INVALID_ARG;
+    if (n_tok == 0) return PLORA_OK;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return PLORA_ERR_CUDA;
+    cudaStream_t st = as_stream(stream);
+    const int32_t saved = ctx->path;
+    ctx->path = PLORA_PATH_UNFUSED;
+    rc = ensure_bucket(ctx, ids, n_tok, pool->dev.n_adapters, st);
+    ctx->path = saved;
+    if (rc != PLORA_OK) return rc;
+    int nl = 0;
+    cudaError_t e = launch_bgmv(kExpandOnly, pool->dev, ctx->bk, n_tok, nullptr, y, const_cast<float*>(m), ldm,
+                                ctx->status_dev, ctx->sm_count, st, &nl);
+    ctx->launches += nl;
+    return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
+}
+
+PLORA_API plora_status plora_lora_delta_host(plora_ctx* ctx, const void* x_host, const int32_t* ids_host, int32_t n_tok,
+                                   int32_t layer, int32_t proj, float* y_host, void* stream) {
+    if (!ctx || n_tok < 0 || n_tok > ctx->max_tokens) return PLORA_ERR_INVALID_ARG;
+    if (n_tok > 0 && (!x_host || !ids_host || !y_host)) return PLORA_ERR_INVALID_ARG;
+    PoolRec* pool = find_pool(ctx, layer, proj);
+    if (!pool) return PLORA_ERR_NOT_REGISTERED;
+    if (n_tok == 0) return PLORA_OK;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return PLORA_ERR_CUDA;
+    cudaStream_t st = as_stream(stream);
+    const size_t xb = (size_t)ctx->max_tokens * pool->dev.d_in * 2, yb = (size_t)ctx->max_tokens * pool->dev.d_out * 4;
+    if (xb > ctx->x_stage_bytes) {
+        cudaStreamSynchronize(st);
+        cudaFree(ctx->x_stage);
+        ctx->x_stage = nullptr;
+        ctx->x_stage_bytes = 0;
+        if (cudaMalloc(&ctx->x_stage, xb) != cudaSuccess) return PLORA_ERR_WORKSPACE;
+        ctx->x_stage_bytes = xb;
+    }
+    if (yb > ctx->y_stage_bytes) {
+        cudaStreamSynchronize(st);
+        cudaFree(ctx->y_stage);
+        ctx->y_stage = nullptr;
+        ctx->y_stage_bytes = 0;
+        if (cudaMalloc(&ctx->y_stage, yb) != cudaSuccess) return PLORA_ERR_WORKSPACE;
+        ctx->y_stage_bytes = yb;
+    }
+    if (!ctx->ids_stage && cudaMalloc(&ctx->ids_stage, (size_t)ctx->max_tokens * 4) != cudaSuccess)
+        return PLORA_ERR_WORKSPACE;
+    const size_t nx = (size_t)n_tok * pool->dev.d_in * 2, ny = (size_t)n_tok * pool->dev.d_out * 4;
+    if (cudaMemcpyAsync(ctx->ids_stage, ids_host, (size_t)n_tok * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(ctx->x_stage, x_host, nx, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(ctx->y_stage, y_host, ny, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return PLORA_ERR_CUDA;
+    ctx->bucket_valid = false;   // the staged ids changed under the same pointer
+    plora_status rc = plora_lora_delta(ctx, ctx->x_stage, ctx->ids_stage, n_tok, layer, proj, ctx->y_stage, stream);
+    ctx->bucket_valid = false;
+    if (rc != PLORA_OK) return rc;
+    if (cudaMemcpyAsync(y_host, ctx->y_stage, ny, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess)
+        return PLORA_ERR_CUDA;
+    return PLORA_OK;
+}
+
+PLORA_API plora_status plora_device_status(plora_ctx* ctx, void* stream, int32_t* host_out) {
+    if (!ctx || !host_out) return PLORA_ERR_INVALID_ARG;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return PLORA_ERR_CUDA;
+    cudaStream_t st = as_stream(stream);
+    int32_t v = 0;
+    if (cudaMemcpyAsync(&v, ctx->status_dev, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess)
+        return PLORA_ERR_CUDA;
+    if (v != 0 && (cudaMemsetAsync(ctx->status_dev, 0, 4, st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess))
+        return PLORA_ERR_CUDA;
+    *host_out = v;
+    return PLORA_OK;
+}
+
+PLORA_API int64_t plora_launch_count(plora_ctx* ctx) { return ctx ? ctx->launches : -1; }
+
+}  // extern "C"

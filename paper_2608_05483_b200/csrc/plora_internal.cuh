@@ -1,0 +1,104 @@
+// Internal declarations shared by the library's translation units (not part of the ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "plora.h"
+
+namespace plora {
+
+// ---------------------------------------------------------------------------------
+// Slab layout (private).  Per adapter, A is stored transposed as rp rows (one per
+// rank index k, rp = rank padded to a power of two >= 8, zero rows beyond r) of d_in
+// values; B as rp rows of d_out values.  Each is cut along the long dimension into
+// tiles of TILE_COLS(rp) columns; a tile is nsub sub-tiles of [rp rows][64 columns]
+// (128-byte rows), sub-tiles back to back, and inside a sub-tile the 16-byte chunk c
+// of row k sits at chunk position c ^ (k & 7).  A tile is therefore one contiguous
+// block of rp * TILE_COLS * 2 bytes (16 KiB, 8 KiB for rp = 8): one bulk copy brings
+// it into shared memory, lanes that read one chunk per row at consecutive rows, or
+// consecutive chunks of one row, touch distinct banks, and a [rp][64] sub-tile has
+// the row pitch and chunk permutation of the tensor core's 128-byte-swizzled operand.
+// Columns beyond d_in / d_out in the last tile are zero.
+// ---------------------------------------------------------------------------------
+constexpr int kMaxRank = 128;
+constexpr int kSubCols = 64;                 // columns of one sub-tile (128 bytes of bf16)
+constexpr int kMaxSubPerTile = 8;            // at most 512 columns per tile
+constexpr int kTileBytesMax = 16384;
+
+__host__ __device__ inline int pad_rank(int r) {
+    int rp = 8;
+    while (rp < r) rp <<= 1;
+    return rp;
+}
+__host__ __device__ inline int subs_per_tile(int rp) {
+    int n = kMaxRank / rp;
+    return n > kMaxSubPerTile ? kMaxSubPerTile : n;
+}
+__host__ __device__ inline int tile_cols(int rp) { return subs_per_tile(rp) * kSubCols; }
+__host__ __device__ inline int tile_bytes(int rp) { return rp * tile_cols(rp) * 2; }
+__host__ __device__ inline int tiles_for(int d, int rp) { return (d + tile_cols(rp) - 1) / tile_cols(rp); }
+
+// One row of the per-pool offset table (device resident).
+struct AdapterEntry {
+    uint64_t offA;   // byte offset of the adapter's A tiles in the slab
+    uint64_t offB;   // byte offset of its B tiles
+    int32_t r;       // rank
+    int32_t rp;      // padded rank
+    float scale;     // s_a
+    int32_t pad_;
+};
+static_assert(sizeof(AdapterEntry) == 32, "table row is 32 bytes");
+
+struct PoolDev {
+    const uint8_t* slab;
+    const AdapterEntry* table;
+    int32_t d_in, d_out, n_adapters, max_rp;
+    int32_t uniform_rp;   // the padded rank if all adapters share it, else 0
+    int32_t pad_;
+};
+
+// ---------------------------------------------------------------------------------
+// Bucket (device resident, owned by the context).
+// ---------------------------------------------------------------------------------
+constexpr int kTokChunk = 4;      // tokens of one segment a BGMV work unit handles
+constexpr int kSgmvRows = 64;     // rows of one SGMV tile
+
+struct WorkUnit {   // 16 bytes
+    int32_t adapter;
+    int32_t pos0;   // first position in perm
+    int32_t cnt;    // tokens (<= kTokChunk for BGMV, <= kSgmvRows for SGMV)
+    int32_t seg;
+};
+
+struct BucketDev {
+    int32_t* perm;
+    int32_t* seg_adapter;
+    int32_t* seg_start;
+    int32_t* n_seg;
+    int32_t* n_active;
+    WorkUnit* bgmv_units;
+    int32_t* n_bgmv_units;
+    WorkUnit* sgmv_tiles;
+    int32_t* n_sgmv_tiles;
+};
+
+// Launchers (each returns the cudaError_t of its launch).
+cudaError_t launch_bucket(const int32_t* ids, int n_tok, int n_adapters, int sgmv_min_rows, BucketDev bk,
+                          int32_t* status, cudaStream_t stream, int* n_launches);
+cudaError_t launch_repack(const AdapterEntry* table_dev, const void* const* A_dev, const void* const* B_dev,
+                          int n_adapters, int d_in, int d_out, uint8_t* slab, cudaStream_t stream, int* n_launches);
+
+enum BgmvMode { kFused = 0, kShrinkOnly = 1, kExpandOnly = 2 };
+// x: bf16 [n_tok, d_in]; y: fp32 [n_tok, d_out] (accumulated); m: fp32 [n_tok, ldm]
+cudaError_t launch_bgmv(BgmvMode mode, const PoolDev& pool, const BucketDev& bk, int n_tok, const void* x, float* y,
+                        float* m, int ldm, int32_t* status, int sm_count, cudaStream_t stream, int* n_launches);
+cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, const void* x, float* y,
+                        int32_t* status, int sm_count, cudaStream_t stream, int* n_launches);
+// per-device function attributes (dynamic shared memory); called by plora_create
+cudaError_t bucket_configure();
+cudaError_t bgmv_configure();
+cudaError_t sgmv_configure();
+int bucket_max_adapters();      // largest pool the single-CTA bucketing kernel handles
+
+}  // namespace plora

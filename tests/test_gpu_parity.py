@@ -1,0 +1,186 @@
+"""GPU LoRA delta vs the float64 oracle, element by element, through the C ABI.
+
+Contract: max|gpu - ref| <= 5e-3 * max|ref| (bf16 inputs, fp32 accumulation).  The
+BGMV paths keep m in fp32, so they are also held to 1e-4: an indexing mistake that
+moves a few elements cannot hide under the contract's tolerance.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2608_05483_b200 as P
+from gpu_util import DEV, Runner, bits_to_dev
+from helpers import TOL_CONTRACT, TOL_FP32_PATH, random_problem, rel_err
+from workloads import gen_adapter, gen_x, gen_y_in, make_workload
+
+pytestmark = pytest.mark.gpu
+
+BGMV_PATHS = [P.PATH_FUSED, P.PATH_UNFUSED]
+
+
+def _oracle(p, y_in=None, ids=None):
+    return oracle.lora_delta(p["x"], p["ids"] if ids is None else ids, p["ranks"], p["scales"], p["A"], p["B"],
+                             p["d_out"], y_in)
+
+
+def _problem_from_workload(wl, pool):
+    AB = [gen_adapter(wl, pool, a) for a in range(wl.n_adapters)]
+    return dict(T=wl.n_tok, d_in=pool.d_in, d_out=pool.d_out, N=wl.n_adapters, ranks=wl.ranks, scales=wl.scales,
+                ids=wl.ids, x=gen_x(wl, pool), A=[ab[0] for ab in AB], B=[ab[1] for ab in AB],
+                y_in=gen_y_in(wl, pool))
+
+
+def _check_paths(p, paths=BGMV_PATHS, tol=TOL_FP32_PATH, on_device=False):
+    r = Runner(p, on_device=on_device)
+    try:
+        ref0 = _oracle(p)
+        ref1 = _oracle(p, y_in=p["y_in"])
+        for path in paths:
+            got0 = r.delta(path)
+            assert rel_err(got0, ref0) <= min(tol, TOL_CONTRACT), (path, rel_err(got0, ref0))
+            got1 = r.delta(path, y_in=p["y_in"])
+            # y_in enters with one fp32 rounding of the sum
+            assert np.max(np.abs(got1 - ref1)) <= tol * np.max(np.abs(ref0)) + 1e-6 * np.max(np.abs(ref1)), path
+            again = r.delta(path, y_in=p["y_in"])
+            assert again.tobytes() == got1.tobytes(), "not bit-reproducible"
+        assert r.ctx.device_status() == 0
+    finally:
+        r.close()
+
+
+def test_tiny_config():
+    wl = make_workload(1)
+    _check_paths(_problem_from_workload(wl, wl.pools[0]))
+
+
+def test_tiny_config_device_resident_sources():
+    wl = make_workload(1)
+    _check_paths(_problem_from_workload(wl, wl.pools[0]), on_device=True)
+
+
+@pytest.mark.parametrize("cfg,kw", [
+    (2, dict(n_adapters=200, d_model=1024, n_layers=1)),          # decode, Zipf ids, several tiles per matrix
+    (3, dict(n_adapters=100, d_model=640, d_ff=1728, n_layers=1, n_tok=128)),   # rectangular projections, rank 64
+    (4, dict(n_adapters=50, d_model=512, n_layers=1, n_tok=1024)),  # long contiguous segments
+    (5, dict(n_adapters=60, d_model=1024, n_layers=1, n_tok=512)),  # mixed ranks, mixed segment lengths
+])
+def test_reduced_benchmark_configs(cfg, kw):
+    wl = make_workload(cfg, **kw)
+    seen = set()
+    for pool in wl.pools:
+        if (pool.d_in, pool.d_out) in seen:
+            continue
+        seen.add((pool.d_in, pool.d_out))
+        _check_paths(_problem_from_workload(wl, pool))
+
+
+@pytest.mark.parametrize("r", [1, 2, 7, 8, 9, 16, 31, 33, 63, 64, 100, 128])
+def test_odd_ranks(r):
+    p = random_problem(100 + r, T=37, d_in=328, d_out=264, ranks=[r, max(1, r - 1), r], with_minus_one=True)
+    _check_paths(p)
+
+
+@pytest.mark.parametrize("d_in,d_out", [(8, 8), (64, 72), (520, 1032), (1048, 504), (2056, 4104)])
+def test_ragged_dims(d_in, d_out):
+    p = random_problem(d_in + d_out, T=19, d_in=d_in, d_out=d_out, ranks=[8, 16, 32, 64, 128, 4], with_minus_one=True)
+    _check_paths(p)
+
+
+@pytest.mark.parametrize("T", [1, 2, 3, 4, 5, 8, 9, 63, 257])
+def test_token_counts_and_hot_adapter(T):
+    p = random_problem(T, T=T, d_in=512, d_out=512, ranks=[16, 16, 8])
+    p["ids"][: max(1, T // 2)] = 1      # one hot adapter: many units share its matrices
+    _check_paths(p)
+
+
+def test_empty_and_all_minus_one():
+    p = random_problem(1, T=0, d_in=64, d_out=64, ranks=[8])
+    r = Runner(p, max_tokens=8)
+    assert r.delta(P.PATH_FUSED).shape == (0, 64)
+    r.close()
+    p = random_problem(2, T=9, d_in=64, d_out=64, ranks=[8, 8])
+    p["ids"][:] = -1
+    r = Runner(p)
+    for path in BGMV_PATHS:
+        got = r.delta(path, y_in=p["y_in"])
+        assert np.array_equal(got, p["y_in"])
+    r.close()
+
+
+def test_shrink_and_expand_entry_points():
+    p = random_problem(77, T=45, d_in=776, d_out=520, ranks=[8, 24, 64, 5], with_minus_one=True)
+    r = Runner(p)
+    try:
+        ldm = r.ctx.pool_max_rank(0, 0)
+        assert ldm == 64
+        m = torch.full((p["T"], ldm), 7.0, dtype=torch.float32, device=DEV)
+        r.ctx.shrink(r.x, r.ids, 0, 0, m)
+        torch.cuda.synchronize()
+        m_ref = oracle.shrink(p["x"], p["ids"], p["ranks"], p["A"], ldm=ldm)
+        assert rel_err(m.cpu().numpy(), m_ref) <= TOL_FP32_PATH
+        assert np.all(m.cpu().numpy()[m_ref == 0] == 0)      # padding columns and id -1 rows are exact zeros
+        y = torch.from_numpy(p["y_in"]).to(DEV)
+        r.ctx.expand(m, r.ids, 0, 0, y)
+        torch.cuda.synchronize()
+        y_ref = oracle.expand(m.cpu().numpy().astype(np.float64), p["ids"], p["ranks"], p["scales"], p["B"], p["d_out"],
+                              p["y_in"])
+        delta_scale = np.max(np.abs(y_ref - p["y_in"]))
+        assert np.max(np.abs(y.cpu().numpy() - y_ref)) <= TOL_FP32_PATH * delta_scale + 1e-6 * np.max(np.abs(y_ref))
+    finally:
+        r.close()
+
+
+def test_out_of_range_id_is_skipped_and_flagged():
+    p = random_problem(5, T=12, d_in=256, d_out=256, ranks=[8, 16])
+    ids = p["ids"].copy()
+    ids[4] = 2          # == n_adapters
+    r = Runner(p)
+    got = r.delta(P.PATH_FUSED, y_in=p["y_in"], ids=ids)
+    assert r.ctx.device_status() == P.ERR_BAD_ADAPTER_ID
+    ids_ref = ids.copy(); ids_ref[4] = -1
+    ref = _oracle(p, y_in=p["y_in"], ids=ids_ref)
+    assert np.array_equal(got[4], p["y_in"][4])
+    assert np.max(np.abs(got - ref)) <= 1e-4 * np.max(np.abs(ref))
+    r.close()
+
+
+def test_host_buffer_entry_point():
+    p = random_problem(6, T=33, d_in=512, d_out=384, ranks=[16, 8, 32])
+    r = Runner(p, max_tokens=64)
+    r.ctx.set_path(P.PATH_FUSED)
+    x_h = torch.from_numpy(p["x"].view(np.int16)).pin_memory()
+    ids_h = torch.from_numpy(p["ids"]).pin_memory()
+    y_h = torch.from_numpy(p["y_in"].copy()).pin_memory()
+    r.ctx.lora_delta_host(x_h, ids_h, 0, 0, y_h)
+    ref = _oracle(p, y_in=p["y_in"])
+    assert np.max(np.abs(y_h.numpy() - ref)) <= 1e-4 * np.max(np.abs(ref))
+    # numpy (pageable) buffers work too
+    y_np = p["y_in"].copy()
+    r.ctx.lora_delta_host(p["x"], p["ids"], 0, 0, y_np)
+    assert y_np.tobytes() == y_h.numpy().tobytes()
+    r.close()
+
+
+def test_two_pools_and_bucket_reuse():
+    wl = make_workload(2, n_adapters=64, d_model=512, n_layers=2, n_tok=96)
+    ctx = P.Context(wl.n_tok, wl.n_adapters)
+    ids = torch.from_numpy(wl.ids).to(DEV)
+    probs = {}
+    for pool in wl.pools:
+        pr = _problem_from_workload(wl, pool)
+        probs[(pool.layer, pool.proj)] = pr
+        ctx.register_pool(pool.layer, pool.proj, pool.d_in, pool.d_out, wl.ranks, wl.scales, pr["A"], pr["B"])
+    ctx.set_path(P.PATH_FUSED)
+    ctx.bucket(ids, wl.n_adapters)
+    before = ctx.launch_count()
+    ys = {}
+    for key, pr in probs.items():
+        y = torch.zeros((wl.n_tok, pr["d_out"]), dtype=torch.float32, device=DEV)
+        ctx.lora_delta(bits_to_dev(pr["x"]), ids, key[0], key[1], y)
+        ys[key] = y
+    torch.cuda.synchronize()
+    assert ctx.launch_count() - before == len(probs)    # one kernel per call, the bucket is reused
+    for key, pr in probs.items():
+        assert rel_err(ys[key].cpu().numpy(), _oracle(pr)) <= TOL_FP32_PATH
+    ctx.close()
