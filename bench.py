@@ -1,0 +1,424 @@
+#!/usr/bin/env python
+"""Benchmark of the batched LoRA-delta hot path on B200.
+
+One step = one pass of the whole hot path over one batch: bucket the batch's
+adapter ids once, then apply the LoRA delta of every (layer, projection) pool
+of the workload (for the default decode workload: 32 layers x q/k/v/o = 128
+calls over a 33.6 GB pool of 1000 rank-16 adapters per projection).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                  [--config 2|3|4|5] [--layers L] [--graph 0|1]
+
+Prints ONE JSON line (rank 0).  `value` is tokens per second through the whole
+step with inputs resident in HBM; `e2e` is the same step through the host-buffer
+entry point (pinned host memory, copies inside the timed region); `roofline`
+compares the dominant kernel's algorithmic bytes per launch with the measured
+HBM copy bandwidth; `cpu_baseline` is the float64 oracle timed on this machine's
+host cores on a bounded sample.  --impl reference times the oracle alone.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+import numpy as np
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+from workloads import gen_pool_device, make_workload  # noqa: E402
+
+FALLBACK_HBM_GBS = 6650.0   # used only when MEASURED_PEAKS.json is absent
+
+# DRAM bytes per launch of the dominant kernel from the committed ncu captures
+# (profiles/*.md say which capture each number comes from); None = not captured.
+NCU_TRAFFIC_BYTES = {}
+
+
+# ----------------------------------------------------------------------------------
+# accounting (the paper's cost model, Section VI-B: the memory term of strategy E1
+# counts every adapter present once, 2 bytes per value; generalised to d_in != d_out)
+# ----------------------------------------------------------------------------------
+def algorithmic_bytes(ids: np.ndarray, ranks: np.ndarray, d_in: int, d_out: int) -> dict:
+    act = ids[ids >= 0]
+    distinct = np.unique(act)
+    adapter = int(sum((d_in + d_out) * int(ranks[a]) * 2 for a in distinct))
+    x_bytes = int(len(ids) * d_in * 2)
+    y_bytes = int(len(act) * d_out * 8)   # fp32 read + write
+    return dict(adapter=adapter, x=x_bytes, y=y_bytes, total=adapter + x_bytes + y_bytes, distinct=int(len(distinct)))
+
+
+def algorithmic_flops(ids: np.ndarray, ranks: np.ndarray, d_in: int, d_out: int) -> int:
+    act = ids[ids >= 0]
+    return int(2 * sum(int(ranks[a]) for a in act) * (d_in + d_out))
+
+
+def hbm_floor_ms(n_bytes: float, gbs: float) -> float:
+    return n_bytes / (gbs * 1e9) * 1e3
+
+
+def measured_peaks() -> dict:
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        d = json.loads(p.read_text())
+        return dict(hbm_gbs=float(d["hbm_gbs"]), source="measured")
+    return dict(hbm_gbs=FALLBACK_HBM_GBS, source="fallback")
+
+
+# ----------------------------------------------------------------------------------
+# clocks sampling during the timed region
+# ----------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for r in self.rows:
+            c = [v.strip() for v in r.split(",")]
+            if len(c) < 7:
+                continue
+            try:
+                sm.append(float(c[0])); mx.append(float(c[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, c[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    samples=len(sm), reasons=sorted(reasons))
+
+
+# ----------------------------------------------------------------------------------
+# workload set-up on the device
+# ----------------------------------------------------------------------------------
+class DeviceWorkload:
+    """Pools registered in a library context plus per-call activations, all resident in HBM."""
+
+    def __init__(self, wl, device_index: int, max_tokens=None):
+        import torch
+        import paper_2608_05483_b200 as P
+        self.P, self.torch, self.wl = P, torch, wl
+        self.dev = f"cuda:{device_index}"
+        torch.cuda.set_device(device_index)
+        self.ctx = P.Context(max_tokens or wl.n_tok, wl.n_adapters, device=device_index)
+        self.ids = torch.from_numpy(wl.ids).to(self.dev)
+        g = torch.Generator(device=self.dev)
+        g.manual_seed(wl.seed)
+        self.x = {}
+        self.y = {}
+        for pool in wl.pools:
+            A, B = gen_pool_device(wl, pool, self.dev)
+            self.ctx.register_pool(pool.layer, pool.proj, pool.d_in, pool.d_out, wl.ranks, wl.scales, A, B)
+            del A, B
+            key = (pool.layer, pool.x_group)
+            if key not in self.x:
+                self.x[key] = torch.randn((wl.n_tok, pool.d_in), generator=g, device=self.dev,
+                                          dtype=torch.float32).to(torch.bfloat16)
+            self.y[(pool.layer, pool.proj)] = torch.randn((wl.n_tok, pool.d_out), generator=g, device=self.dev,
+                                                          dtype=torch.float32)
+        torch.cuda.synchronize()
+
+    def step(self):
+        """bucket once, then every (layer, proj) delta; enqueue only."""
+        ctx, wl = self.ctx, self.wl
+        ctx.bucket(self.ids, wl.n_adapters)
+        for pool in wl.pools:
+            ctx.lora_delta(self.x[(pool.layer, pool.x_group)], self.ids, pool.layer, pool.proj,
+                           self.y[(pool.layer, pool.proj)])
+
+    def host_adapters(self, pool, adapters):
+        """Logical A/B bit patterns of `adapters` of `pool`, regenerated on the device and copied to the host."""
+        A, B = gen_pool_device(self.wl, pool, self.dev)
+        outA = [None] * self.wl.n_adapters
+        outB = [None] * self.wl.n_adapters
+        for a in adapters:
+            outA[int(a)] = A[int(a)].contiguous().view(self.torch.int16).cpu().numpy().view(np.uint16)
+            outB[int(a)] = B[int(a)].contiguous().view(self.torch.int16).cpu().numpy().view(np.uint16)
+        return outA, outB
+
+    def close(self):
+        self.ctx.close()
+
+
+def bits_of(t):
+    import torch
+    return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+# ----------------------------------------------------------------------------------
+# the CPU oracle on a bounded sample (also a full-size parity check of sampled pools)
+# ----------------------------------------------------------------------------------
+def oracle_sample(dw: DeviceWorkload, n_pools: int, check_gpu: bool):
+    import oracle
+    wl = dw.wl
+    torch = dw.torch
+    pools = wl.pools[:: max(1, len(wl.pools) // n_pools)][:n_pools]
+    distinct = wl.distinct_adapters()
+    cpu_s, max_err = 0.0, 0.0
+    for pool in pools:
+        A, B = dw.host_adapters(pool, distinct)
+        x = bits_of(dw.x[(pool.layer, pool.x_group)])
+        y_in = dw.y[(pool.layer, pool.proj)].cpu().numpy().copy()
+        t0 = time.perf_counter()
+        ref = oracle.lora_delta(x, wl.ids, wl.ranks, wl.scales, A, B, pool.d_out, y_in)
+        cpu_s += time.perf_counter() - t0
+        if check_gpu:
+            y = dw.y[(pool.layer, pool.proj)].clone()
+            dw.ctx.lora_delta(dw.x[(pool.layer, pool.x_group)], dw.ids, pool.layer, pool.proj, y)
+            torch.cuda.synchronize()
+            delta_scale = float(np.max(np.abs(ref - y_in)))
+            max_err = max(max_err, float(np.max(np.abs(y.cpu().numpy() - ref)) / delta_scale))
+    return pools, cpu_s, max_err, oracle.threads()
+
+
+# ----------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2608_05483_b200 as P
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    torch.cuda.set_device(local)
+
+    wl = make_workload(args.config, n_layers=args.layers)
+    dw = DeviceWorkload(wl, local)
+    ctx = dw.ctx
+    ctx.set_path(P.PATH_AUTO)
+    n_calls = len(wl.pools)
+
+    # full-size parity on sampled pools + the oracle's time, before anything is timed (rank 0)
+    cpu = None
+    parity = None
+    if rank == 0 and not args.no_cpu:
+        pools, cpu_s, parity, threads = oracle_sample(dw, args.cpu_pools, check_gpu=True)
+        scaled = cpu_s * n_calls / len(pools)
+        cpu = dict(value=wl.n_tok / scaled, unit="tokens/s", cores=threads, kind="oracle",
+                   sample=f"{len(pools)} of {n_calls} (layer, proj) calls at full size ({wl.n_tok} tokens), "
+                          f"{cpu_s:.2f} s of oracle time scaled to the whole step")
+
+    stream = torch.cuda.current_stream()
+    graph = None
+    if args.graph:
+        s = torch.cuda.Stream()
+        s.wait_stream(stream)
+        with torch.cuda.stream(s):
+            dw.step()
+        stream.wait_stream(s)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            dw.step()
+
+    def one_step():
+        if graph is not None:
+            graph.replay()
+        else:
+            dw.step()
+
+    for _ in range(max(3, args.warmup)):
+        one_step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    l0 = ctx.launch_count()
+    ev[0].record()
+    for k in range(args.steps):
+        one_step()
+        ev[k + 1].record()
+    torch.cuda.synchronize()
+    launches = ctx.launch_count() - l0
+    if graph is not None:
+        launches = args.steps * (n_calls + 1)
+    total_ms = ev[0].elapsed_time(ev[-1])
+    clocks = sampler.stop()
+    if world > 1:
+        t = torch.tensor([total_ms], device=f"cuda:{local}")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+        dist.barrier()
+    ms_per_step = total_ms / args.steps
+
+    # kernel-only timing for the roofline: the delta calls of one step without the bucket kernel
+    ctx.bucket(dw.ids, wl.n_adapters)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = max(3, args.steps)
+    e0.record()
+    for _ in range(reps):
+        for pool in wl.pools:
+            ctx.lora_delta(dw.x[(pool.layer, pool.x_group)], dw.ids, pool.layer, pool.proj, dw.y[(pool.layer, pool.proj)])
+    e1.record()
+    torch.cuda.synchronize()
+    kernel_ms = e0.elapsed_time(e1) / (reps * n_calls)
+
+    per_call = [algorithmic_bytes(wl.ids, wl.ranks, p.d_in, p.d_out) for p in wl.pools]
+    step_bytes = sum(b["total"] for b in per_call)
+    step_adapter_bytes = sum(b["adapter"] for b in per_call)
+    peaks = measured_peaks()
+    achieved = step_bytes / n_calls / (kernel_ms * 1e-3) / 1e9
+    roofline = dict(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s", frac=achieved / peaks["hbm_gbs"],
+                    traffic=NCU_TRAFFIC_BYTES.get(wl.name), kernel="bgmv_kernel (fused shrink+expand)",
+                    peak_source=peaks["source"], avg_launch_us=kernel_ms * 1e3,
+                    algorithmic_bytes_per_launch=step_bytes / n_calls,
+                    adapter_bytes_only_gbs=step_adapter_bytes / n_calls / (kernel_ms * 1e-3) / 1e9,
+                    step_gbs=step_bytes / (ms_per_step * 1e-3) / 1e9)
+
+    # end to end through the host-buffer entry point (pinned host memory, copies timed)
+    e2e = None
+    if not args.no_e2e:
+        xh = {k: v.cpu().pin_memory() for k, v in list(dw.x.items())}
+        yh = {k: v.cpu().pin_memory() for k, v in list(dw.y.items())}
+        idh = dw.ids.cpu().pin_memory()
+
+        def host_step():
+            for pool in wl.pools:
+                ctx.lora_delta_host(xh[(pool.layer, pool.x_group)], idh, pool.layer, pool.proj, yh[(pool.layer, pool.proj)])
+
+        host_step()
+        torch.cuda.synchronize()
+        n_e2e = max(1, min(args.steps, 3))
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            host_step()
+        torch.cuda.synchronize()
+        e2e_s = (time.perf_counter() - t0) / n_e2e
+        if world > 1:
+            t = torch.tensor([e2e_s], device=f"cuda:{local}")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_s = float(t.item())
+        h2d = sum(wl.n_tok * p.d_in * 2 + wl.n_tok * 4 + wl.n_tok * p.d_out * 4 for p in wl.pools)
+        d2h = sum(wl.n_tok * p.d_out * 4 for p in wl.pools)
+        e2e = dict(value=world * wl.n_tok / e2e_s, unit="tokens/s", h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
+                   ms_per_step=e2e_s * 1e3, steps=n_e2e)
+
+    status = ctx.device_status()
+    if rank == 0:
+        out = dict(metric="LoRA-delta tokens/sec at 1000 adapters (whole step: bucket + every layer x projection delta)",
+                   value=world * wl.n_tok / (ms_per_step * 1e-3), unit="tokens/s", n_gpus=world, steps=args.steps,
+                   warmup=max(3, args.warmup), ms_per_step=ms_per_step, higher_is_better=True, scaling="weak",
+                   vs_baseline=None, dtype="bf16 in, fp32 accumulate", data="synthetic",
+                   config=dict(workload=f"config {args.config} ({wl.name})", n_tok=wl.n_tok, n_adapters=wl.n_adapters,
+                               layers=len({p.layer for p in wl.pools}), calls_per_step=n_calls,
+                               ranks=sorted({int(r) for r in wl.ranks}), ids=wl.meta.get("ids"),
+                               distinct_adapters=per_call[0]["distinct"], path="auto", cuda_graph=bool(args.graph),
+                               l2="inputs larger than L2: a step streams %.2f GB through %d distinct slabs"
+                                  % (step_bytes / 1e9, n_calls),
+                               multi_gpu="replicas: every rank runs its own batch, no data-path collective"),
+                   clocks=clocks, e2e=e2e, gpu_launches=int(launches), roofline=roofline, cpu_baseline=cpu,
+                   tokens_per_s_per_call=wl.n_tok / (kernel_ms * 1e-3), parity_max_rel_err=parity,
+                   device_status=status)
+        print(json.dumps(out))
+    dw.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_reference(args):
+    """The oracle, as it stands, on the host cores: each step a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from workloads import gen_adapter, gen_x, gen_y_in
+    wl = make_workload(args.config, n_layers=args.layers)
+    n_calls = len(wl.pools)
+    pools = wl.pools[: max(1, args.cpu_pools // 2)]
+    distinct = wl.distinct_adapters()
+    data = []
+    for pool in pools:   # host-generated logical matrices for the adapters the batch touches
+        A = [None] * wl.n_adapters
+        B = [None] * wl.n_adapters
+        for a in distinct:
+            A[int(a)], B[int(a)] = gen_adapter(wl, pool, int(a))
+        data.append((pool, gen_x(wl, pool), A, B, gen_y_in(wl, pool)))
+
+    def sample_step():
+        for pool, x, A, B, y_in in data:
+            oracle.lora_delta(x, wl.ids, wl.ranks, wl.scales, A, B, pool.d_out, y_in)
+
+    for _ in range(min(args.warmup, 1)):
+        sample_step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        sample_step()
+    s = (time.perf_counter() - t0) / args.steps
+    step_s = s * n_calls / len(pools)
+    value = wl.n_tok / step_s
+    sample = f"{len(pools)} of {n_calls} (layer, proj) calls per step at full size, scaled to the whole step"
+    out = dict(impl="reference", metric="LoRA-delta tokens/sec at 1000 adapters (whole step: bucket + every layer x projection delta)",
+               value=value, unit="tokens/s", n_gpus=1, steps=args.steps, warmup=min(args.warmup, 1), ms_per_step=step_s * 1e3,
+               higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
+               config=dict(workload=f"config {args.config} ({wl.name})", n_tok=wl.n_tok, n_adapters=wl.n_adapters,
+                           calls_per_step=n_calls),
+               cpu_baseline=dict(value=value, unit="tokens/s", cores=oracle.threads(), kind="oracle", sample=sample),
+               e2e=dict(value=value, unit="tokens/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
+    print(json.dumps(out))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4, 5])
+    ap.add_argument("--layers", type=int, default=None)
+    ap.add_argument("--graph", type=int, default=0)
+    ap.add_argument("--cpu-pools", type=int, default=8, dest="cpu_pools")
+    ap.add_argument("--no-cpu", action="store_true", dest="no_cpu")
+    ap.add_argument("--no-e2e", action="store_true", dest="no_e2e")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
