@@ -59,6 +59,9 @@ struct plora_ctx {
     size_t x_stage_bytes = 0, y_stage_bytes = 0;
     std::vector<PoolRec> pools;
     int64_t launches = 0;
+    // kernels launched through this context since the bucket kernel: from the second one on, the
+    // bucket tables were complete before the kernel preceding it in the stream started
+    int32_t launches_since_bucket = 0;
 };
 
 namespace {
@@ -82,9 +85,10 @@ bool desc_shape_ok(const plora_pool_desc* d, plora_status* why) {
 }
 
 // Fills the offset table (host copy) and returns the slab size.
-size_t layout_pool(const plora_pool_desc* d, std::vector<AdapterEntry>* table, int* max_rp, int* uniform_rp = nullptr) {
+size_t layout_pool(const plora_pool_desc* d, std::vector<AdapterEntry>* table, int* max_rp, int* uniform_rp = nullptr,
+                   int* min_rp = nullptr) {
     size_t off = 0;
-    int mrp = 0, urp = -1;
+    int mrp = 0, urp = -1, lrp = kMaxRank;
     if (table) table->resize(d->n_adapters);
     for (int a = 0; a < d->n_adapters; ++a) {
         const int rp = pad_rank(d->ranks[a]);
@@ -99,10 +103,12 @@ size_t layout_pool(const plora_pool_desc* d, std::vector<AdapterEntry>* table, i
         e.scale = d->scales ? d->scales[a] : 1.0f;
         if (table) (*table)[a] = e;
         if (rp > mrp) mrp = rp;
+        if (rp < lrp) lrp = rp;
         urp = (urp == -1 || urp == rp) ? rp : 0;
     }
     if (max_rp) *max_rp = mrp;
     if (uniform_rp) *uniform_rp = urp > 0 ? urp : 0;
+    if (min_rp) *min_rp = lrp;
     return off;
 }
 
@@ -125,6 +131,7 @@ plora_status do_bucket(plora_ctx* ctx, const int32_t* ids, int32_t n_tok, int32_
     ctx->cur_nadapters = n_adapters;
     ctx->bucket_sgmv_min = thr;
     ctx->bucket_valid = true;
+    ctx->launches_since_bucket = 0;
     return PLORA_OK;
 }
 
@@ -188,7 +195,9 @@ PLORA_API plora_status plora_create(plora_ctx** out, int device, int32_t max_tok
     const size_t o_bg = o_scal + 256;
     const size_t o_sg = o_bg + up(T * sizeof(WorkUnit));
     const size_t o_m = o_sg + up(T * sizeof(WorkUnit));
-    const size_t total = o_m + up(T * kMaxRank * 4);
+    const size_t o_part = o_m + up(T * kMaxRank * 4);
+    const size_t part_bytes = up(T * 8192 > ((size_t)16 << 20) ? T * 8192 : ((size_t)16 << 20));
+    const size_t total = o_part + part_bytes;
     uint8_t* blk = nullptr;
     if (cudaMalloc(&blk, total) != cudaSuccess) { delete ctx; return PLORA_ERR_WORKSPACE; }
     if (cudaMemset(blk, 0, total) != cudaSuccess) { cudaFree(blk); delete ctx; return PLORA_ERR_CUDA; }
@@ -205,6 +214,18 @@ PLORA_API plora_status plora_create(plora_ctx** out, int device, int32_t max_tok
     ctx->bk.bgmv_units = (WorkUnit*)(blk + o_bg);
     ctx->bk.sgmv_tiles = (WorkUnit*)(blk + o_sg);
     ctx->m_ws = (float*)(blk + o_m);
+    ctx->bk.m_part = (unsigned long long*)(blk + o_part);
+    ctx->bk.m_part_bytes = part_bytes;
+    ctx->bk.epoch = (uint32_t*)(scal + 16);
+    ctx->bk.exit_count = (uint32_t*)(scal + 17);
+    {
+        const uint32_t one = 1;
+        if (cudaMemcpy(ctx->bk.epoch, &one, 4, cudaMemcpyHostToDevice) != cudaSuccess) {
+            cudaFree(blk);
+            delete ctx;
+            return PLORA_ERR_CUDA;
+        }
+    }
     if (bucket_configure() != cudaSuccess || bgmv_configure() != cudaSuccess || sgmv_configure() != cudaSuccess ||
         cudaDeviceSynchronize() != cudaSuccess) {
         cudaFree(blk);
@@ -244,8 +265,8 @@ PLORA_API plora_status plora_register_pool(plora_ctx* ctx, const plora_pool_desc
     for (int a = 0; a < d->n_adapters; ++a)
         if (!d->A[a] || !d->B[a]) return PLORA_ERR_INVALID_ARG;
     std::vector<AdapterEntry> table;
-    int max_rp = 0, uniform_rp = 0;
-    const size_t need = layout_pool(d, &table, &max_rp, &uniform_rp);
+    int max_rp = 0, uniform_rp = 0, min_rp = 0;
+    const size_t need = layout_pool(d, &table, &max_rp, &uniform_rp, &min_rp);
     if (slab_bytes < need) return PLORA_ERR_WORKSPACE;
 
     DeviceGuard g(ctx->device);
@@ -307,6 +328,7 @@ PLORA_API plora_status plora_register_pool(plora_ctx* ctx, const plora_pool_desc
     rec.dev.n_adapters = N;
     rec.dev.max_rp = max_rp;
     rec.dev.uniform_rp = uniform_rp;
+    rec.dev.min_rp = min_rp;
     if (PoolRec* old = find_pool(ctx, d->layer, d->proj)) {
         cudaStreamSynchronize(st);
         cudaFree(old->table_dev);
@@ -366,16 +388,16 @@ PLORA_API plora_status plora_lora_delta(plora_ctx* ctx, const void* x, const int
     cudaError_t e = cudaSuccess;
     if (ctx->path == PLORA_PATH_UNFUSED) {
         e = launch_bgmv(kShrinkOnly, pool->dev, ctx->bk, n_tok, x, nullptr, ctx->m_ws, pool->dev.max_rp, ctx->status_dev,
-                        ctx->sm_count, st, &nl);
+                        ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl);
         if (e == cudaSuccess)
             e = launch_bgmv(kExpandOnly, pool->dev, ctx->bk, n_tok, nullptr, y, ctx->m_ws, pool->dev.max_rp,
-                            ctx->status_dev, ctx->sm_count, st, &nl);
+                            ctx->status_dev, ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl);
     } else {
         // a batch shorter than the threshold cannot hold a segment for the tensor-core path
         const bool may_bgmv = ctx->path != PLORA_PATH_SGMV;
         const bool may_sgmv = ctx->path == PLORA_PATH_SGMV || (ctx->path == PLORA_PATH_AUTO && n_tok >= ctx->sgmv_min_rows);
         if (may_bgmv)
-            e = launch_bgmv(kFused, pool->dev, ctx->bk, n_tok, x, y, nullptr, 0, ctx->status_dev, ctx->sm_count, st, &nl);
+            e = launch_bgmv(kFused, pool->dev, ctx->bk, n_tok, x, y, nullptr, 0, ctx->status_dev, ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl);
         if (e == cudaSuccess && may_sgmv)
             e = launch_sgmv(pool->dev, ctx->bk, n_tok, x, y, ctx->status_dev, ctx->sm_count, st, &nl);
     }
@@ -402,7 +424,7 @@ PLORA_API plora_status plora_shrink(plora_ctx* ctx, const void* x, const int32_t
     if (rc != PLORA_OK) return rc;
     int nl = 0;
     cudaError_t e = launch_bgmv(kShrinkOnly, pool->dev, ctx->bk, n_tok, x, nullptr, m, ldm, ctx->status_dev,
-                                ctx->sm_count, st, &nl);
+                                ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl);
     ctx->launches += nl;
     return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
 }
@@ -425,7 +447,7 @@ PLORA_API plora_status plora_expand(plora_ctx* ctx, const float* m, int32_t ldm,
     if (rc != PLORA_OK) return rc;
     int nl = 0;
     cudaError_t e = launch_bgmv(kExpandOnly, pool->dev, ctx->bk, n_tok, nullptr, y, const_cast<float*>(m), ldm,
-                                ctx->status_dev, ctx->sm_count, st, &nl);
+                                ctx->status_dev, ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl);
     ctx->launches += nl;
     return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
 }

@@ -55,7 +55,7 @@ __device__ __forceinline__ int units_of(int cnt, int per) { return (cnt + per - 
 
 // Fill one work list: unit u belongs to the last bin b with ustart[b] <= u.
 __device__ void write_units(WorkUnit* out, int n_units, const int* ustart, const int* start, const int* total,
-                            const int* segidx, int n_bins, int per) {
+                            const int* segidx, int n_bins, int per, const int32_t* perm) {
     for (int u = threadIdx.x; u < n_units; u += kThreads) {
         int lo = 0, hi = n_bins;   // find first b with ustart[b] > u
         while (lo < hi) {
@@ -69,6 +69,8 @@ __device__ void write_units(WorkUnit* out, int n_units, const int* ustart, const
         wu.pos0 = start[b] + k * per;
         wu.cnt = min(per, total[b] - k * per);
         wu.seg = segidx[b];
+#pragma unroll
+        for (int t = 0; t < kTokChunk; ++t) wu.tok[t] = t < wu.cnt ? perm[wu.pos0 + t] : 0;
         out[u] = wu;
     }
 }
@@ -167,8 +169,9 @@ bucket_kernel(const int32_t* __restrict__ ids, int T, int N, int nch, int sgmv_m
         *bk.n_bgmv_units = n_bg;
         *bk.n_sgmv_tiles = n_sg;
     }
-    write_units(bk.bgmv_units, n_bg, ubg, start, total, segidx, N, kTokChunk);
-    write_units(bk.sgmv_tiles, n_sg, usg, start, total, segidx, N, kSgmvRows);
+    __syncthreads();   // perm is complete (written by this block) before the units quote it
+    write_units(bk.bgmv_units, n_bg, ubg, start, total, segidx, N, kTokChunk, bk.perm);
+    write_units(bk.sgmv_tiles, n_sg, usg, start, total, segidx, N, kSgmvRows, bk.perm);
 }
 
 constexpr size_t kBucketSmemLimit = 200 * 1024;

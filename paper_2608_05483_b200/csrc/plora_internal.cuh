@@ -55,7 +55,7 @@ struct PoolDev {
     const AdapterEntry* table;
     int32_t d_in, d_out, n_adapters, max_rp;
     int32_t uniform_rp;   // the padded rank if all adapters share it, else 0
-    int32_t pad_;
+    int32_t min_rp;
 };
 
 // ---------------------------------------------------------------------------------
@@ -64,12 +64,16 @@ struct PoolDev {
 constexpr int kTokChunk = 4;      // tokens of one segment a BGMV work unit handles
 constexpr int kSgmvRows = 64;     // rows of one SGMV tile
 
-struct WorkUnit {   // 16 bytes
+struct WorkUnit {   // 32 bytes
     int32_t adapter;
     int32_t pos0;   // first position in perm
     int32_t cnt;    // tokens (<= kTokChunk for BGMV, <= kSgmvRows for SGMV)
     int32_t seg;
+    int32_t tok[kTokChunk];   // the first min(cnt, kTokChunk) token indices, perm[pos0 ...]
 };
+static_assert(sizeof(WorkUnit) == 32 && kTokChunk == 4, "work unit is two 16-byte words");
+
+constexpr int kMaxRuns = 8;       // a unit's shrink (or expand) is cut into at most this many tasks
 
 struct BucketDev {
     int32_t* perm;
@@ -81,6 +85,12 @@ struct BucketDev {
     int32_t* n_bgmv_units;
     WorkUnit* sgmv_tiles;
     int32_t* n_sgmv_tiles;
+    // cross-CTA hand-over of the fused BGMV kernel: every partial m value travels as one
+    // 64-bit word {value, launch epoch}, so a reader can tell on its own whether it has arrived
+    unsigned long long* m_part;
+    size_t m_part_bytes;
+    uint32_t* epoch;        // launch epoch, advanced by the last CTA of every fused launch (starts at 1)
+    uint32_t* exit_count;   // CTAs of the running launch that have finished
 };
 
 // Launchers (each returns the cudaError_t of its launch).
@@ -92,7 +102,8 @@ cudaError_t launch_repack(const AdapterEntry* table_dev, const void* const* A_de
 enum BgmvMode { kFused = 0, kShrinkOnly = 1, kExpandOnly = 2 };
 // x: bf16 [n_tok, d_in]; y: fp32 [n_tok, d_out] (accumulated); m: fp32 [n_tok, ldm]
 cudaError_t launch_bgmv(BgmvMode mode, const PoolDev& pool, const BucketDev& bk, int n_tok, const void* x, float* y,
-                        float* m, int ldm, int32_t* status, int sm_count, cudaStream_t stream, int* n_launches);
+                        float* m, int ldm, int32_t* status, int sm_count, bool early_tables, cudaStream_t stream,
+                        int* n_launches);
 cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, const void* x, float* y,
                         int32_t* status, int sm_count, cudaStream_t stream, int* n_launches);
 // per-device function attributes (dynamic shared memory); called by plora_create
