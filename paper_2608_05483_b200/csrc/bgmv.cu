@@ -41,7 +41,9 @@ namespace {
 
 constexpr int kConsumerWarps = 8;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kThreads = kConsumerThreads + 32;   // + one producer warp
+constexpr int kProducerWarp = kConsumerWarps;       // issues the copies
+constexpr int kGatherWarp = kConsumerWarps + 1;     // fused mode: assembles the m of the expand tasks
+constexpr int kThreads = kConsumerThreads + 64;
 #ifndef PLORA_EXP_STAGES
 #define PLORA_EXP_STAGES 4
 #endif
@@ -50,8 +52,14 @@ constexpr int kXBytesPerTok = kMaxSubPerTile * kSubCols * 2;             // x pi
 constexpr int kHdrOffset = kTileBytesMax + kTokChunk * kXBytesPerTok;
 constexpr int kSlotBytes = kHdrOffset + 128;                             // tile + x pieces + stage header
 constexpr int kPartFloats = kConsumerWarps * kTokChunk * kMaxRank;       // two buffers when the rank is <= 64
-constexpr int kSmemBytes = kStages * kSlotBytes + kPartFloats * 4 + (2 * kStages + 1) * 8 + 16;
+// m of the expand tasks in flight (fused mode): a ring filled by the gather warp and drained by
+// the consumers, with a full / empty barrier pair per entry.
+constexpr int kMRing = 4;
+constexpr int kMRingBytes = kTokChunk * kMaxRank * 4;
+constexpr int kNumBarriers = 2 * kStages + 2 * kMRing + 1;
+constexpr int kSmemBytes = kStages * kSlotBytes + kPartFloats * 4 + kMRing * kMRingBytes + kNumBarriers * 8 + 16;
 constexpr int kPrefetchTasks = 8;   // tasks per CTA whose tiles are prefetched to L2 before the stream-order wait
+constexpr uint32_t kSuspendHintNs = 20000;   // a waiting thread may sleep this long inside one try_wait
 constexpr long long kWaitCycles = 4000000000ll;   // about two seconds of SM clock
 
 struct Params {
@@ -86,10 +94,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(bar), "r"(parity)
+        : "r"(bar), "r"(parity), "r"(kSuspendHintNs)
         : "memory");
     return ok != 0;
 }
@@ -146,12 +154,37 @@ __device__ __forceinline__ void unpack8(const uint4& v, float* f) {
     f[4] = bf_lo(v.z); f[5] = bf_hi(v.z); f[6] = bf_lo(v.w); f[7] = bf_hi(v.w);
 }
 
+#ifdef PLORA_TRACE
+__device__ long long g_trace[8 * 1024];
+__device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+__device__ long long g_trace3[320 * 8];
+#define CYC_DECL(v) long long v = 0
+#define CYC_T0(v) const long long v = clock64()
+#define CYC_ADD(acc, t0) acc += clock64() - (t0)
+#define CYC_OUT(k, v) g_trace3[blockIdx.x * 8 + (k)] = (v)
+#define TRACE(slot) g_trace[blockIdx.x * 8 + (slot)] = gtime()
+#define g_trace_n(n) g_trace[blockIdx.x * 8 + 6] = (n)
+__device__ long long g_trace2[320 * 16 * 4];
+#define TRACE2(stage, k) do { if ((stage) < 16) g_trace2[(blockIdx.x * 16 + (stage)) * 4 + (k)] = gtime(); } while (0)
+#else
+#define TRACE(slot)
+#define CYC_DECL(v)
+#define CYC_T0(v)
+#define CYC_ADD(acc, t0)
+#define CYC_OUT(k, v)
+#define g_trace_n(n)
+#define TRACE2(stage, k)
+#endif
+
 struct Smem {
     uint32_t slots;      // shared address of stage 0
     uint32_t full;       // full[kStages] barriers
     uint32_t empty;      // empty[kStages]
     float* part;         // per-warp partial m of a shrink task
     volatile int* abort_flag;
+    uint32_t m_ring;     // shared address of the m ring (fused mode): kMRing entries of kMRingBytes
+    uint32_t m_full;     // m_full[kMRing]: the gather warp has written the entry
+    uint32_t m_empty;    // m_empty[kMRing]: every consumer warp is done with the entry
     uint32_t sync_bar;   // barrier of the consumer warps (one arrival per warp)
     int32_t* status;
     uint32_t epoch;      // this launch's epoch (fused mode)
@@ -161,6 +194,9 @@ struct Smem {
 struct Ctl {
     int pbuf;             // which half of part[] the next shrink task uses
     uint32_t sync_phase;  // parity of the next consumer_sync
+#ifdef PLORA_TRACE
+    long long c_tile = 0, c_fin = 0, c_finw = 0;
+#endif
 };
 
 // Barrier over the consumer warps, built on an mbarrier so that, like every other wait
@@ -181,14 +217,17 @@ struct StageHdr {
     int32_t tok[kTokChunk];
     int32_t rp, r;
     float scale;
+    int32_t m_seq;    // fused expand stages: running number of the expand task in this CTA (m-ring entry = m_seq % kMRing)
 };
 
 __device__ __forceinline__ StageHdr read_hdr(uint32_t a) {
     const uint4 q0 = lds128(a), q1 = lds128(a + 16), q2 = lds128(a + 32);
+    const uint32_t q3 = lds32(a + 48);
     StageHdr h;
     h.flags = (int)q0.x; h.unit = (int)q0.y; h.run = (int)q0.z; h.tile = (int)q0.w;
     h.cnt = (int)q1.x; h.tok[0] = (int)q1.y; h.tok[1] = (int)q1.z; h.tok[2] = (int)q1.w;
     h.tok[3] = (int)q2.x; h.rp = (int)q2.y; h.r = (int)q2.z; h.scale = __uint_as_float(q2.w);
+    h.m_seq = (int)q3;
     return h;
 }
 __device__ __forceinline__ void sts128(uint32_t a, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
@@ -234,29 +273,50 @@ struct ShrinkMap {
     }
 };
 
-template <int RP, bool CHECKED>
-__device__ __forceinline__ void shrink_chunks(const ShrinkMap<RP>& mp, int cnt, int cols_left, uint32_t tile,
+// CNT (tokens of the unit) is a template parameter: the loops unroll without branches, every
+// load of a chunk can be issued before the first use, and each (row, token, chunk) product
+// runs as two short chains (even / odd columns) instead of one long one.
+template <int RP, int CNT, bool CHECKED>
+__device__ __forceinline__ void shrink_chunks(const ShrinkMap<RP>& mp, int cols_left, uint32_t tile,
                                               float (&acc)[kMaxRowsPerLane][kTokChunk]) {
     using M = ShrinkMap<RP>;
     const uint32_t xs = tile + kTileBytesMax;
 #pragma unroll
     for (int q = 0; q < M::CPL; ++q) {
         if (!CHECKED || mp.col0 + q * M::G * 8 < cols_left) {
+            uint4 araw[M::RPL], xraw[CNT];
+#pragma unroll
+            for (int rr = 0; rr < M::RPL; ++rr) araw[rr] = lds128(tile + mp.a_off[q][rr]);
+#pragma unroll
+            for (int t = 0; t < CNT; ++t) xraw[t] = lds128(xs + t * kXBytesPerTok + mp.x_off[q]);
             float af[M::RPL][8];
 #pragma unroll
-            for (int rr = 0; rr < M::RPL; ++rr) unpack8(lds128(tile + mp.a_off[q][rr]), af[rr]);
+            for (int rr = 0; rr < M::RPL; ++rr) unpack8(araw[rr], af[rr]);
 #pragma unroll
-            for (int t = 0; t < kTokChunk; ++t)
-                if (t < cnt) {
-                    float xf[8];
-                    unpack8(lds128(xs + t * kXBytesPerTok + mp.x_off[q]), xf);
+            for (int t = 0; t < CNT; ++t) {
+                float xf[8];
+                unpack8(xraw[t], xf);
 #pragma unroll
-                    for (int rr = 0; rr < M::RPL; ++rr)
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) acc[rr][t] = fmaf(xf[j], af[rr][j], acc[rr][t]);
+                for (int rr = 0; rr < M::RPL; ++rr) {
+                    float e = xf[0] * af[rr][0], o = xf[1] * af[rr][1];
+                    e = fmaf(xf[2], af[rr][2], e); o = fmaf(xf[3], af[rr][3], o);
+                    e = fmaf(xf[4], af[rr][4], e); o = fmaf(xf[5], af[rr][5], o);
+                    e = fmaf(xf[6], af[rr][6], e); o = fmaf(xf[7], af[rr][7], o);
+                    acc[rr][t] += e + o;
                 }
+            }
         }
     }
+}
+
+template <int RP, int CNT>
+__device__ __forceinline__ void shrink_tile_cnt(const Params& p, const StageHdr& h, const ShrinkMap<RP>& mp,
+                                                uint32_t tile, float (&acc)[kMaxRowsPerLane][kTokChunk]) {
+    const int cols_left = p.pool.d_in - h.tile * ShrinkMap<RP>::C;   // only the last tile can be ragged
+    if (cols_left >= ShrinkMap<RP>::C)
+        shrink_chunks<RP, CNT, false>(mp, cols_left, tile, acc);
+    else
+        shrink_chunks<RP, CNT, true>(mp, cols_left, tile, acc);
 }
 
 template <int RP>
@@ -265,11 +325,12 @@ __device__ __forceinline__ void shrink_tile(const Params& p, const StageHdr& h, 
 #ifdef PLORA_EXP_NOCOMPUTE
     return;
 #endif
-    const int cols_left = p.pool.d_in - h.tile * ShrinkMap<RP>::C;   // only the last tile can be ragged
-    if (cols_left >= ShrinkMap<RP>::C)
-        shrink_chunks<RP, false>(mp, h.cnt, cols_left, tile, acc);
-    else
-        shrink_chunks<RP, true>(mp, h.cnt, cols_left, tile, acc);
+    switch (h.cnt) {
+        case 1: shrink_tile_cnt<RP, 1>(p, h, mp, tile, acc); break;
+        case 2: shrink_tile_cnt<RP, 2>(p, h, mp, tile, acc); break;
+        case 3: shrink_tile_cnt<RP, 3>(p, h, mp, tile, acc); break;
+        default: shrink_tile_cnt<RP, 4>(p, h, mp, tile, acc); break;
+    }
 }
 
 // ---- shrink: end of a task: the CTA's partial m leaves for the workspace (or the caller's m) ----
@@ -347,60 +408,82 @@ struct ExpandMap {
     }
 };
 
-template <int MODE, int RP>
-__device__ __forceinline__ void expand_tile(const Params& p, const StageHdr& h, const ExpandMap<RP>& mp, uint32_t tile,
-                                            uint32_t empty_bar, int lane) {
+template <int MODE, int RP, int CNT>
+__device__ __forceinline__ void expand_tile_cnt(const Params& p, const Smem& sm, const StageHdr& h,
+                                                const ExpandMap<RP>& mp, uint32_t tile, uint32_t empty_bar, int lane) {
     using M = ExpandMap<RP>;
     const uint32_t b0 = tile + mp.b_off;
-    const uint32_t mb = tile + mp.m_off;
-    float acc[kTokChunk][2];
+    const int m_slot = h.m_seq % kMRing;
+    if (MODE == kFused && (h.flags & kFlagFirst))   // the gather warp has assembled this task's m
+        mbar_wait(sm.m_full + m_slot * 8, (h.m_seq / kMRing) & 1, sm.abort_flag, sm.status);
+    // m[t][k], RP floats per token: in the m ring (fused) or in the stage next to the tile (expand-only)
+    const uint32_t mb = (MODE == kFused ? sm.m_ring + m_slot * kMRingBytes : tile + kTileBytesMax) + mp.rg * M::RPG * 4;
+    float acc[2][CNT][2];   // [even / odd rank row][token][column]
 #pragma unroll
-    for (int t = 0; t < kTokChunk; ++t) acc[t][0] = acc[t][1] = 0.f;
+    for (int t = 0; t < CNT; ++t) acc[0][t][0] = acc[0][t][1] = acc[1][t][0] = acc[1][t][1] = 0.f;
 #pragma unroll
     for (int kk = 0; kk < M::RPG; kk += 4) {
-        uint4 mv[kTokChunk];
+        uint4 mv[CNT];
+        uint32_t braw[4];
 #pragma unroll
-        for (int t = 0; t < kTokChunk; ++t)
-            if (t < h.cnt) {
-                mv[t] = lds128(mb + t * (RP * 4) + kk * 4);
-                if (MODE == kExpandOnly && h.r < RP) {
-                    // the caller's m may hold anything beyond the adapter's rank
-                    const int k0 = mp.rg * M::RPG + kk;
-                    if (k0 + 0 >= h.r) mv[t].x = 0u;
-                    if (k0 + 1 >= h.r) mv[t].y = 0u;
-                    if (k0 + 2 >= h.r) mv[t].z = 0u;
-                    if (k0 + 3 >= h.r) mv[t].w = 0u;
-                }
+        for (int q = 0; q < 4; ++q) braw[q] = lds32((b0 ^ (((kk + q) & 7) << 4)) + (kk + q) * 128);
+#pragma unroll
+        for (int t = 0; t < CNT; ++t) {
+            mv[t] = lds128(mb + t * (RP * 4) + kk * 4);
+            if (MODE == kExpandOnly && h.r < RP) {
+                // the caller's m may hold anything beyond the adapter's rank
+                const int k0 = mp.rg * M::RPG + kk;
+                if (k0 + 0 >= h.r) mv[t].x = 0u;
+                if (k0 + 1 >= h.r) mv[t].y = 0u;
+                if (k0 + 2 >= h.r) mv[t].z = 0u;
+                if (k0 + 3 >= h.r) mv[t].w = 0u;
             }
+        }
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-            const int k = kk + q;   // row inside the group; its swizzle class is k & 7
-            const uint32_t b = lds32((b0 ^ ((k & 7) << 4)) + k * 128);
-            const float blo = bf_lo(b), bhi = bf_hi(b);
+            const float blo = bf_lo(braw[q]), bhi = bf_hi(braw[q]);
 #pragma unroll
-            for (int t = 0; t < kTokChunk; ++t)
-                if (t < h.cnt) {
-                    const float mk = __uint_as_float(q == 0 ? mv[t].x : q == 1 ? mv[t].y : q == 2 ? mv[t].z : mv[t].w);
-                    acc[t][0] = fmaf(mk, blo, acc[t][0]);
-                    acc[t][1] = fmaf(mk, bhi, acc[t][1]);
-                }
+            for (int t = 0; t < CNT; ++t) {
+                const float mk = __uint_as_float(q == 0 ? mv[t].x : q == 1 ? mv[t].y : q == 2 ? mv[t].z : mv[t].w);
+                acc[q & 1][t][0] = fmaf(mk, blo, acc[q & 1][t][0]);
+                acc[q & 1][t][1] = fmaf(mk, bhi, acc[q & 1][t][1]);
+            }
         }
     }
     __syncwarp();
-    if (lane == 0) mbar_arrive(empty_bar);
+    if (lane == 0) {
+        mbar_arrive(empty_bar);
+        if (MODE == kFused && (h.flags & kFlagLast)) mbar_arrive(sm.m_empty + m_slot * 8);
+    }
+    float out[CNT][2];
+#pragma unroll
+    for (int t = 0; t < CNT; ++t) {
+        out[t][0] = acc[0][t][0] + acc[1][t][0];
+        out[t][1] = acc[0][t][1] + acc[1][t][1];
+    }
 #pragma unroll
     for (int d = M::P; d < 32; d <<= 1)
 #pragma unroll
-        for (int t = 0; t < kTokChunk; ++t) {
-            acc[t][0] += __shfl_xor_sync(0xffffffffu, acc[t][0], d);
-            acc[t][1] += __shfl_xor_sync(0xffffffffu, acc[t][1], d);
+        for (int t = 0; t < CNT; ++t) {
+            out[t][0] += __shfl_xor_sync(0xffffffffu, out[t][0], d);
+            out[t][1] += __shfl_xor_sync(0xffffffffu, out[t][1], d);
         }
     const int col = h.tile * M::C + mp.colw;
     if (mp.rg == 0 && col < p.pool.d_out) {
 #pragma unroll
-        for (int t = 0; t < kTokChunk; ++t)
-            if (t < h.cnt)
-                red_add_v2(p.y + (size_t)h.tok[t] * p.pool.d_out + col, acc[t][0] * h.scale, acc[t][1] * h.scale);
+        for (int t = 0; t < CNT; ++t)
+            red_add_v2(p.y + (size_t)h.tok[t] * p.pool.d_out + col, out[t][0] * h.scale, out[t][1] * h.scale);
+    }
+}
+
+template <int MODE, int RP>
+__device__ __forceinline__ void expand_tile(const Params& p, const Smem& sm, const StageHdr& h, const ExpandMap<RP>& mp,
+                                            uint32_t tile, uint32_t empty_bar, int lane) {
+    switch (h.cnt) {
+        case 1: expand_tile_cnt<MODE, RP, 1>(p, sm, h, mp, tile, empty_bar, lane); break;
+        case 2: expand_tile_cnt<MODE, RP, 2>(p, sm, h, mp, tile, empty_bar, lane); break;
+        case 3: expand_tile_cnt<MODE, RP, 3>(p, sm, h, mp, tile, empty_bar, lane); break;
+        default: expand_tile_cnt<MODE, RP, 4>(p, sm, h, mp, tile, empty_bar, lane); break;
     }
 }
 
@@ -428,14 +511,18 @@ __device__ __forceinline__ void consume_stage(const Params& p, const Smem& sm, c
 #pragma unroll
                     for (int t = 0; t < kTokChunk; ++t) acc[rr][t] = 0.f;
             }
+            CYC_T0(t_a);
             shrink_tile<RP>(p, h, maps.s, tile, acc);
             __syncwarp();
             if (lane == 0) mbar_arrive(empty_bar);
+            CYC_ADD(ctl.c_tile, t_a);
+            CYC_T0(t_b);
             if (h.flags & kFlagLast) shrink_finish<MODE, RP>(p, sm, h, acc, ctl, warp, lane);
+            CYC_ADD(ctl.c_fin, t_b);
         }
     } else {
         if (MODE != kShrinkOnly) {
-            expand_tile<MODE, RP>(p, h, maps.e, tile, empty_bar, lane);
+            expand_tile<MODE, RP>(p, sm, h, maps.e, tile, empty_bar, lane);
         }
     }
 }
@@ -452,38 +539,47 @@ __device__ __noinline__ void stage_of_rank(const Params& p, const Smem& sm, cons
 
 // ---- producer side: the m of an expand task ---------------------------------------------------
 // A unit's m has cnt * rp values; lane l of the producer warp owns the values l, l + 32, ...
-constexpr int kMPerLane = kTokChunk * kMaxRank / 32;
-
-struct MVals {
-    float v[kMPerLane];
-    bool ok;   // every partial read so far carried this launch's epoch
-};
-
-// Read the runs_a partials of every owned value and sum them in run order.  Nothing here
-// waits; `ok` tells whether every word carried this launch's epoch.
-__device__ __forceinline__ void load_m(const Params& p, uint32_t epoch, int unit, int cnt, int rp, int lane, MVals& out) {
-    out.ok = true;
-    const int n = cnt * rp;
-#pragma unroll
-    for (int q = 0; q < kMPerLane; ++q) {
-        const int idx = lane + 32 * q;
-        float s = 0.f;
-        if (idx < n) {
-            const int t = idx / rp, k = idx - t * rp;
-            unsigned long long w[kMaxRuns];
-#pragma unroll
-            for (int j = 0; j < kMaxRuns; ++j)
-                w[j] = j < p.runs_a ? ldg_cg_u64(p.bk.m_part + part_index(p, unit, j, t) + k)
-                                    : ((unsigned long long)epoch << 32);
-#pragma unroll
-            for (int j = 0; j < kMaxRuns; ++j) {
-                out.ok = out.ok && (uint32_t)(w[j] >> 32) == epoch;
-                s += __uint_as_float((uint32_t)w[j]);
-            }
-        }
-        out.v[q] = s;
-    }
+// For every owned value the runs_a partial words are read, checked for this launch's epoch,
+// summed in run order and the sum stored into the m-ring entry.  Nothing here waits: the
+// return value tells whether every word had arrived (if not, the next attempt rewrites the
+// entry).  rp is a power of two.
+__device__ __forceinline__ const unsigned long long* partial_src(const Params& p, int unit, int idx, int rp) {
+    const int sh = __ffs(rp) - 1;
+    const int t = idx >> sh, k = idx & (rp - 1);
+    return p.bk.m_part + part_index(p, unit, 0, t) + k;
 }
+__device__ __forceinline__ void partial_load(const Params& p, uint32_t epoch, const unsigned long long* src,
+                                             unsigned long long (&w)[kMaxRuns]) {
+    const size_t run_stride = (size_t)kTokChunk * p.pool.max_rp;
+#pragma unroll
+    for (int j = 0; j < kMaxRuns; ++j)
+        w[j] = j < p.runs_a ? ldg_cg_u64(src + j * run_stride) : ((unsigned long long)epoch << 32);
+}
+__device__ __forceinline__ bool partial_sum(uint32_t epoch, const unsigned long long (&w)[kMaxRuns], uint32_t dst) {
+    bool ok = true;
+    float s = 0.f;
+#pragma unroll
+    for (int j = 0; j < kMaxRuns; ++j) {
+        ok = ok && (uint32_t)(w[j] >> 32) == epoch;
+        s += __uint_as_float((uint32_t)w[j]);
+    }
+    asm volatile("st.shared.f32 [%0], %1;" ::"r"(dst), "f"(s) : "memory");
+    return ok;
+}
+__device__ __forceinline__ bool gather_m(const Params& p, uint32_t epoch, int unit, int cnt, int rp, int lane,
+                                         uint32_t mdst) {
+    bool ok = true;
+    const int n = cnt * rp;
+    for (int idx = lane; idx < n; idx += 32) {
+        unsigned long long w[kMaxRuns];
+        partial_load(p, epoch, partial_src(p, unit, idx, rp), w);
+        ok = partial_sum(epoch, w, mdst + idx * 4) && ok;
+    }
+    return ok;
+}
+// Units with at most this many m values have their partials requested one task ahead: the
+// words travel while the producer issues the current task's stages.
+constexpr int kPrefetchM = 64;
 
 // A task: one run of tiles of one unit in one phase.
 struct Task {
@@ -515,14 +611,18 @@ __global__ void __launch_bounds__(kThreads, 2) bgmv_kernel(const Params p) {
     Smem sm;
     sm.slots = smem_u32(smem_raw);
     sm.part = reinterpret_cast<float*>(smem_raw + kStages * kSlotBytes);
-    uint8_t* bars = reinterpret_cast<uint8_t*>(sm.part + kPartFloats);
+    sm.m_ring = smem_u32(sm.part + kPartFloats);
+    uint8_t* bars = reinterpret_cast<uint8_t*>(sm.part + kPartFloats) + kMRing * kMRingBytes;
     sm.full = smem_u32(bars);
     sm.empty = sm.full + kStages * 8;
-    sm.sync_bar = sm.empty + kStages * 8;
-    sm.abort_flag = reinterpret_cast<volatile int*>(bars + (2 * kStages + 1) * 8);
+    sm.m_full = sm.empty + kStages * 8;
+    sm.m_empty = sm.m_full + kMRing * 8;
+    sm.sync_bar = sm.m_empty + kMRing * 8;
+    sm.abort_flag = reinterpret_cast<volatile int*>(bars + kNumBarriers * 8);
     sm.status = p.status;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) TRACE(0);
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(sm.full + s * 8, 1);
@@ -531,6 +631,10 @@ __global__ void __launch_bounds__(kThreads, 2) bgmv_kernel(const Params p) {
             sts128(sm.slots + s * kSlotBytes + kHdrOffset, (uint32_t)kFlagEnd, 0u, 0u, 0u);
         }
         mbar_init(sm.sync_bar, kConsumerWarps);
+        for (int e = 0; e < kMRing; ++e) {
+            mbar_init(sm.m_full + e * 8, 1);
+            mbar_init(sm.m_empty + e * 8, kConsumerWarps);
+        }
         *sm.abort_flag = 0;
         fence_barrier_init();
     }
@@ -540,12 +644,13 @@ __global__ void __launch_bounds__(kThreads, 2) bgmv_kernel(const Params p) {
     // producer warp delays that wait: the slab is never written by a kernel, and bucket tables
     // older than the previous kernel are complete, so it fetches its first task descriptors and
     // pulls its first tiles into L2 while the previous kernel drains.
-    if (warp != kConsumerWarps) {
+    if (warp != kProducerWarp) {
         grid_dependency_wait();
         // Signalled only after this CTA has seen the previous kernel complete: when the next kernel
         // of the stream starts, everything older than this kernel is therefore complete.
         grid_launch_dependents();
         sm.epoch = MODE == kFused ? *p.bk.epoch : 0u;
+        if (tid == 0) TRACE(1);
     }
 
     if (MODE == kShrinkOnly) {
@@ -558,11 +663,14 @@ __global__ void __launch_bounds__(kThreads, 2) bgmv_kernel(const Params p) {
         }
     }
 
-    if (warp == kConsumerWarps) {
+    if (warp == kProducerWarp) {
         // ------------------------------- producer warp -------------------------------
-        // The warp fetches the descriptors of its next 32 tasks in one go (lane l owns the
-        // l-th of them), then walks them: lane 0 drives the barriers, writes the stage
-        // header and copies the tile; lane t < cnt copies token t's piece of x.
+        // The warp fetches the descriptors of its next 32 tasks in one go; lane l owns the l-th
+        // of them and works out everything about it (tile range, source address, header words)
+        // in parallel with the other lanes.  The lanes then take turns, in task order: the owner
+        // alone waits for free stages, writes the headers and issues the copies of its task, so
+        // the serial part of the producer is a few dozen instructions per stage.  In fused mode
+        // the whole warp first gathers an expand task's m into the m ring.
         bool waited = false;
         if (!p.early_tables) {
             grid_dependency_wait();
@@ -572,107 +680,159 @@ __global__ void __launch_bounds__(kThreads, 2) bgmv_kernel(const Params p) {
         const int n_shrink = MODE == kExpandOnly ? 0 : n_units * p.runs_a;
         const int n_tasks = n_shrink + (MODE == kShrinkOnly ? 0 : n_units * p.runs_b);
         const int stride = gridDim.x;
-        uint32_t it = 0;
+        const unsigned full = 0xffffffffu;
+        uint32_t it_base = 0;
+        uint32_t m_count = 0;   // expand tasks issued so far (fused mode)
+        CYC_DECL(p_batch); CYC_DECL(p_gather); CYC_DECL(p_wait); CYC_DECL(p_issue);
+        CYC_T0(p_begin);
         for (int base = blockIdx.x; base < n_tasks; base += 32 * stride) {
+            CYC_T0(tb0);
             const int my_task = base + lane * stride;
-            Task mine = decode_task(my_task < n_tasks ? my_task : base, n_shrink, p.runs_a, p.runs_b);
+            const bool has = my_task < n_tasks;
+            const Task mine = decode_task(has ? my_task : base, n_shrink, p.runs_a, p.runs_b);
             const WorkUnit mu = p.bk.bgmv_units[mine.unit];
             const AdapterEntry me = p.pool.table[mu.adapter];
             const int in_batch = min(32, (n_tasks - base + stride - 1) / stride);
+            const int C = tile_cols(me.rp);
+            const uint32_t tb = (uint32_t)tile_bytes(me.rp);
+            const int d = mine.phase ? p.pool.d_out : p.pool.d_in;
+            const int runs = mine.phase ? p.runs_b : p.runs_a;
+            const int nT = tiles_for(d, me.rp);
+            const int lo = has ? mine.run * nT / runs : 0, hi = has ? (mine.run + 1) * nT / runs : 0;
+            const uint8_t* src = p.pool.slab + (mine.phase ? me.offB : me.offA);
             if (!waited) {
-                // lane l pulls the tiles of this CTA's l-th task towards L2, then the warp joins the stream order
-                if (my_task < n_tasks && lane < kPrefetchTasks) {
-                    const int d = mine.phase ? p.pool.d_out : p.pool.d_in;
-                    const int runs = mine.phase ? p.runs_b : p.runs_a;
-                    const int nT = tiles_for(d, me.rp);
-                    const uint32_t tb = (uint32_t)tile_bytes(me.rp);
-                    const uint8_t* src = p.pool.slab + (mine.phase ? me.offB : me.offA);
-                    for (int i = mine.run * nT / runs; i < (mine.run + 1) * nT / runs; ++i)
-                        prefetch_l2(src + (size_t)i * tb, tb);
-                }
+                // pull the tiles of this CTA's first tasks towards L2, then join the stream order
+                if (lane < kPrefetchTasks)
+                    for (int i = lo; i < hi; ++i) prefetch_l2(src + (size_t)i * tb, tb);
+                if (lane == 0) TRACE(2);
                 grid_dependency_wait();
                 waited = true;
+                if (lane == 0) TRACE(3);
             }
             if (base == (int)blockIdx.x) sm.epoch = MODE == kFused ? *p.bk.epoch : 0u;
-            for (int b = 0; b < in_batch; ++b) {
-                const unsigned full = 0xffffffffu;
-                const int phase = __shfl_sync(full, mine.phase, b), unit = __shfl_sync(full, mine.unit, b);
-                const int run = __shfl_sync(full, mine.run, b), cnt = __shfl_sync(full, mu.cnt, b);
-                const int tok0 = __shfl_sync(full, mu.tok[0], b), tok1 = __shfl_sync(full, mu.tok[1], b);
-                const int tok2 = __shfl_sync(full, mu.tok[2], b), tok3 = __shfl_sync(full, mu.tok[3], b);
-                const int rp = __shfl_sync(full, me.rp, b), r = __shfl_sync(full, me.r, b);
-                const uint32_t scale_bits = __shfl_sync(full, __float_as_uint(me.scale), b);
-                const unsigned long long off = __shfl_sync(full, phase ? me.offB : me.offA, b);
-                const int C = tile_cols(rp);
-                const uint32_t tb = (uint32_t)tile_bytes(rp);
-                const int d = phase ? p.pool.d_out : p.pool.d_in;
-                const int runs = phase ? p.runs_b : p.runs_a;
-                const int nT = tiles_for(d, rp);
-                const int lo = run * nT / runs, hi = (run + 1) * nT / runs;
-                const uint8_t* src = p.pool.slab + off;
-                const int my_tok = lane == 1 ? tok1 : lane == 2 ? tok2 : lane == 3 ? tok3 : tok0;
-                const uint16_t* xrow = p.x + (size_t)my_tok * p.pool.d_in;
-                const uint16_t* mrow = reinterpret_cast<const uint16_t*>(p.m + (size_t)my_tok * p.ldm);
-                MVals mv;
-                if (MODE == kFused && phase) {
-                    load_m(p, sm.epoch, unit, cnt, rp, lane, mv);
-                    if (!__all_sync(full, mv.ok)) {
-                        // some shrink task of this unit has not delivered yet: read again, for a bounded time
-                        const long long t0 = clock64();
-                        for (;;) {
-                            __nanosleep(100);
-                            load_m(p, sm.epoch, unit, cnt, rp, lane, mv);
-                            if (__all_sync(full, mv.ok) || *sm.abort_flag) break;
-                            if (clock64() - t0 > kWaitCycles) {
-                                if (lane == 0) give_up(sm.abort_flag, p.status);
-                                break;
-                            }
-                        }
-                    }
-                }
-                // bytes a token adds to the stage besides the tile: its x piece (shrink) or its m row (expand-only)
-                const uint32_t mbytes = (MODE == kExpandOnly) ? (uint32_t)rp * 4u : 0u;
-                for (int i = lo; i < hi; ++i, ++it) {
-                    const uint32_t slot = it % kStages;
-                    const uint32_t dst = sm.slots + slot * kSlotBytes;
-                    const uint32_t bar = sm.full + slot * 8;
-                    const uint32_t tbytes = phase ? mbytes : (uint32_t)min(C, d - i * C) * 2u;
-                    if (lane == 0) {
-                        mbar_wait(sm.empty + slot * 8, ((it / kStages) & 1) ^ 1, sm.abort_flag, p.status);
-                        const int flags = (phase ? kFlagExpand : 0) | (i == lo ? kFlagFirst : 0) | (i == hi - 1 ? kFlagLast : 0);
-                        sts128(dst + kHdrOffset, (uint32_t)flags, (uint32_t)unit, (uint32_t)run, (uint32_t)i);
-                        sts128(dst + kHdrOffset + 16, (uint32_t)cnt, (uint32_t)tok0, (uint32_t)tok1, (uint32_t)tok2);
-                        sts128(dst + kHdrOffset + 32, (uint32_t)tok3, (uint32_t)rp, (uint32_t)r, scale_bits);
-                    }
-                    __syncwarp();   // the stage is free before anyone writes into it
-                    if (MODE == kFused && phase) {
-                        // m[t][k] of the unit (unscaled) rides in the stage's x area
+            // first stage number of every lane's task: exclusive prefix sum of the stage counts
+            int incl = hi - lo;
 #pragma unroll
-                        for (int q = 0; q < kMPerLane; ++q)
-                            if (lane + 32 * q < cnt * rp)
-                                asm volatile("st.shared.f32 [%0], %1;" ::"r"(dst + kTileBytesMax + (lane + 32 * q) * 4),
-                                             "f"(mv.v[q]) : "memory");
-                        __syncwarp();
-                    }
-                    if (lane == 0) {
+            for (int dlt = 1; dlt < 32; dlt <<= 1) {
+                const int v = __shfl_up_sync(full, incl, dlt);
+                if (lane >= dlt) incl += v;
+            }
+            const uint32_t my_it0 = it_base + (uint32_t)(incl - (hi - lo));
+            it_base += (uint32_t)__shfl_sync(full, incl, 31);
+            CYC_ADD(p_batch, tb0);
+
+            for (int b = 0; b < in_batch; ++b) {
+                // fused mode: the running number of this expand task tells the consumers where its m is
+                const uint32_t m_seq = m_count;
+                if (MODE == kFused && __shfl_sync(full, mine.phase, b)) ++m_count;
+                CYC_T0(tg0);
+                CYC_ADD(p_gather, tg0);
+                if (lane == b) {
+                    const int cnt = mu.cnt;
+                    // bytes a token adds to a stage besides the tile: its x piece (shrink) or its m row (expand-only)
+                    const uint32_t mbytes = (MODE == kExpandOnly) ? (uint32_t)me.rp * 4u : 0u;
+                    uint32_t it = my_it0;
+                    for (int i = lo; i < hi; ++i, ++it) {
+                        const uint32_t slot = it % kStages;
+                        const uint32_t dst = sm.slots + slot * kSlotBytes;
+                        const uint32_t bar = sm.full + slot * 8;
+                        const uint32_t tbytes = mine.phase ? mbytes : (uint32_t)min(C, d - i * C) * 2u;
+                        TRACE2(it, 0);
+                        CYC_T0(tpw);
+                        mbar_wait(sm.empty + slot * 8, ((it / kStages) & 1) ^ 1, sm.abort_flag, p.status);
+                        CYC_ADD(p_wait, tpw);
+                        CYC_T0(tpi);
+                        const int flags = (mine.phase ? kFlagExpand : 0) | (i == lo ? kFlagFirst : 0) | (i == hi - 1 ? kFlagLast : 0);
+                        sts128(dst + kHdrOffset, (uint32_t)flags, (uint32_t)mine.unit, (uint32_t)mine.run, (uint32_t)i);
+                        sts128(dst + kHdrOffset + 16, (uint32_t)cnt, (uint32_t)mu.tok[0], (uint32_t)mu.tok[1], (uint32_t)mu.tok[2]);
+                        sts128(dst + kHdrOffset + 32, (uint32_t)mu.tok[3], (uint32_t)me.rp, (uint32_t)me.r, __float_as_uint(me.scale));
+                        sts128(dst + kHdrOffset + 48, m_seq, 0u, 0u, 0u);
+#ifdef PLORA_EXP_NOLOAD
+                        mbar_arrive(bar);
+                        continue;
+#endif
                         mbar_arrive_expect_tx(bar, tb + (uint32_t)cnt * tbytes);
                         bulk_g2s(dst, src + (size_t)i * tb, tb, bar);
-                    }
-                    if (lane < cnt) {
-                        if (!phase)
-                            bulk_g2s(dst + kTileBytesMax + lane * kXBytesPerTok, xrow + (size_t)i * C, tbytes, bar);
-                        else if (MODE == kExpandOnly)   // the caller's m row, rp floats, lands as m[t][0..rp)
-                            bulk_g2s(dst + kTileBytesMax + lane * mbytes, mrow, mbytes, bar);
+                        if (!mine.phase) {
+#pragma unroll
+                            for (int t = 0; t < kTokChunk; ++t)
+                                if (t < cnt)
+                                    bulk_g2s(dst + kTileBytesMax + t * kXBytesPerTok,
+                                             p.x + (size_t)mu.tok[t] * p.pool.d_in + (size_t)i * C, tbytes, bar);
+                        } else if (MODE == kExpandOnly) {
+#pragma unroll
+                            for (int t = 0; t < kTokChunk; ++t)   // the caller's m row, rp floats, lands as m[t][0..rp)
+                                if (t < cnt)
+                                    bulk_g2s(dst + kTileBytesMax + t * mbytes, p.m + (size_t)mu.tok[t] * p.ldm, mbytes, bar);
+                        }
+                        TRACE2(it, 1);
+                        CYC_ADD(p_issue, tpi);
                     }
                 }
+                __syncwarp();
             }
         }
+#ifdef PLORA_TRACE
+        for (int dlt = 16; dlt > 0; dlt >>= 1) {
+            p_wait += __shfl_xor_sync(0xffffffffu, p_wait, dlt);
+            p_issue += __shfl_xor_sync(0xffffffffu, p_issue, dlt);
+        }
+        if (lane == 0) { CYC_OUT(6, p_issue); CYC_OUT(7, clock64() - p_begin); }
+#endif
         if (!waited) grid_dependency_wait();
         if (lane == 0) {   // tell the consumers that nothing follows
+            const uint32_t it = it_base;
             const uint32_t slot = it % kStages;
             mbar_wait(sm.empty + slot * 8, ((it / kStages) & 1) ^ 1, sm.abort_flag, p.status);
             sts128(sm.slots + slot * kSlotBytes + kHdrOffset, (uint32_t)kFlagEnd, 0u, 0u, 0u);
             mbar_arrive(sm.full + slot * 8);
+        }
+        return;
+    }
+
+    if (warp == kGatherWarp) {
+        // ------------------------------- gather warp (fused mode) -------------------------------
+        // Walks this CTA's expand tasks in order, ahead of the consumers: reads the partial words
+        // of the unit (again and again, for a bounded time, until all of them carry this launch's
+        // epoch), sums them in run order into the next m-ring entry and publishes the entry.
+        if (MODE != kFused) return;
+        const int n_units = *p.bk.n_bgmv_units;
+        const int n_shrink = n_units * p.runs_a;
+        const int n_tasks = n_shrink + n_units * p.runs_b;
+        const int stride = gridDim.x;
+        const unsigned full = 0xffffffffu;
+        // this CTA's first expand task
+        int t = blockIdx.x;
+        if (t < n_shrink) t += (n_shrink - t + stride - 1) / stride * stride;
+        uint32_t seq = 0;
+        for (int base = t; base < n_tasks; base += 32 * stride) {
+            const int my_task = base + lane * stride;
+            const bool has = my_task < n_tasks;
+            const int my_unit = (has ? my_task - n_shrink : base - n_shrink) / p.runs_b;
+            const WorkUnit mu = p.bk.bgmv_units[my_unit];
+            const int my_rp = p.pool.table[mu.adapter].rp;
+            const int in_batch = min(32, (n_tasks - base + stride - 1) / stride);
+            for (int b = 0; b < in_batch; ++b, ++seq) {
+                const int unit_b = __shfl_sync(full, my_unit, b), cnt_b = __shfl_sync(full, mu.cnt, b);
+                const int rp_b = __shfl_sync(full, my_rp, b);
+                const uint32_t e = seq % kMRing;
+                if (lane == 0) mbar_wait(sm.m_empty + e * 8, ((seq / kMRing) & 1) ^ 1, sm.abort_flag, p.status);
+                __syncwarp();
+                const uint32_t mdst = sm.m_ring + e * kMRingBytes;
+                if (!__all_sync(full, gather_m(p, sm.epoch, unit_b, cnt_b, rp_b, lane, mdst))) {
+                    const long long t0 = clock64();
+                    for (;;) {
+                        __nanosleep(100);
+                        if (__all_sync(full, gather_m(p, sm.epoch, unit_b, cnt_b, rp_b, lane, mdst)) || *sm.abort_flag) break;
+                        if (clock64() - t0 > kWaitCycles) {
+                            if (lane == 0) give_up(sm.abort_flag, p.status);
+                            break;
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(sm.m_full + e * 8);
+            }
         }
         return;
     }
@@ -684,13 +844,21 @@ __global__ void __launch_bounds__(kThreads, 2) bgmv_kernel(const Params p) {
     ctl.sync_phase = 0;
     LaneMaps<RPK == 0 ? 8 : RPK> maps;   // per-lane constants, computed once when the rank is uniform
     if constexpr (RPK != 0) maps.init(warp, lane);
+    CYC_DECL(c_wait); CYC_DECL(c_hdr); CYC_DECL(c_work);
     for (uint32_t it = 0;; ++it) {
         const uint32_t slot = it % kStages;
+        CYC_T0(tw);
         mbar_wait(sm.full + slot * 8, (it / kStages) & 1, sm.abort_flag, p.status);
+        CYC_ADD(c_wait, tw);
+        CYC_T0(th);
         const uint32_t tile = sm.slots + slot * kSlotBytes;
         const StageHdr h = read_hdr(tile + kHdrOffset);
-        if ((h.flags & kFlagEnd) || *sm.abort_flag) break;
+        CYC_ADD(c_hdr, th);
+        if (tid == 0 && it == 0) TRACE(4);
+        if (tid == 0) TRACE2(it, 2);
+        if ((h.flags & kFlagEnd) || *sm.abort_flag) { if (tid == 0) { TRACE(5); g_trace_n(it); CYC_OUT(0, c_wait); CYC_OUT(1, c_hdr); CYC_OUT(2, c_work); CYC_OUT(3, ctl.c_tile); CYC_OUT(4, ctl.c_fin); CYC_OUT(5, ctl.c_finw); } break; }
         const uint32_t empty_bar = sm.empty + slot * 8;
+        CYC_T0(tc);
         if constexpr (RPK != 0) {
             consume_stage<MODE, RPK>(p, sm, h, maps, tile, empty_bar, acc, ctl, warp, lane);
         } else {
@@ -702,6 +870,8 @@ __global__ void __launch_bounds__(kThreads, 2) bgmv_kernel(const Params p) {
                 default: stage_of_rank<MODE, 128>(p, sm, h, tile, empty_bar, acc, ctl, warp, lane); break;
             }
         }
+        CYC_ADD(c_work, tc);
+        if (tid == 0) TRACE2(it, 3);
     }
     if (MODE == kFused && tid == 0) {
         // the last CTA to finish opens the next epoch: words written by this launch can never
@@ -738,6 +908,18 @@ KernelFn pick_kernel(BgmvMode mode, int uniform_rp) {
 int clamp_runs(int tiles) { return tiles < 1 ? 1 : (tiles > kMaxRuns ? kMaxRuns : tiles); }
 
 }  // namespace
+
+#ifdef PLORA_TRACE
+extern "C" __attribute__((visibility("default"))) int plora_debug_trace(long long* host, int n) {
+    return (int)cudaMemcpyFromSymbol(host, g_trace, sizeof(long long) * n);
+}
+extern "C" __attribute__((visibility("default"))) int plora_debug_trace3(long long* host, int n) {
+    return (int)cudaMemcpyFromSymbol(host, g_trace3, sizeof(long long) * n);
+}
+extern "C" __attribute__((visibility("default"))) int plora_debug_trace2(long long* host, int n) {
+    return (int)cudaMemcpyFromSymbol(host, g_trace2, sizeof(long long) * n);
+}
+#endif
 
 cudaError_t bgmv_configure() {
     const int modes[3] = {kFused, kShrinkOnly, kExpandOnly};
