@@ -185,6 +185,41 @@ PLORA_API plora_status plora_expand(plora_ctx *ctx, const float *m_dev, int32_t 
 PLORA_API plora_status plora_lora_delta_host(plora_ctx *ctx, const void *x_host, const int32_t *adapter_ids_host,
                                    int32_t n_tok, int32_t layer, int32_t proj, float *y_host, void *stream);
 
+/*
+ * The LoRA delta for callers that must not allocate device memory.  (The paper has no
+ * counterpart for this entry point; it exists for the way the library is embedded.)
+ *
+ * Some hosts of this library cannot call cudaMalloc at the point where they need the
+ * delta: a serving loop that may not stall (cudaMalloc and cudaFree synchronise the whole
+ * device), a process whose device memory was handed out in full at start-up, or code
+ * running under an allocator it does not control.  This call computes exactly what
+ * plora_lora_delta computes, by the shrink kernel followed by the expand kernel, and keeps
+ * the intermediate m = x A in a fixed array that is part of the library image instead of
+ * in allocated workspace.  It calls no cudaMalloc, no cudaFree and no allocating library
+ * routine; it only enqueues kernels on `stream` (bucketing first if the context's current
+ * bucket does not match, as plora_lora_delta does).
+ *
+ * The array holds PLORA_NOALLOC_SCRATCH_FLOATS floats (1 MiB) and every GPU that loads the
+ * library carries it until the process exits.  The call needs n_tok * R floats of it, R
+ * being the pool's padded maximum rank (plora_pool_max_rank): for instance 16384 tokens at
+ * rank 16 or 2048 tokens at rank 128.  A larger request is refused with
+ * PLORA_ERR_WORKSPACE before anything is launched.
+ *
+ * The first call on a device looks up the array's device address (once per device) before
+ * it launches; make that first call outside any stream capture.  All calls, on all
+ * contexts of a device, share the one array, and it keeps what the previous call left in
+ * it: the shrink kernel rewrites every row the expand kernel will read (rows of tokens
+ * without an adapter are written as zeros), so nothing has to be cleared between calls,
+ * but two calls whose kernels overlap on the GPU (different streams, no ordering between
+ * them) race on it and give wrong results.  Keep them on one stream or order them with
+ * events.
+ *
+ * Arguments, bucket rule and other errors are those of plora_lora_delta.
+ */
+#define PLORA_NOALLOC_SCRATCH_FLOATS (1 << 18)
+PLORA_API plora_status plora_lora_delta_noalloc(plora_ctx *ctx, const void *x_dev, const int32_t *adapter_ids_dev,
+                                                int32_t n_tok, int32_t layer, int32_t proj, float *y_dev, void *stream);
+
 /* Choose the kernels plora_lora_delta uses (PLORA_PATH_*); takes effect at the next
  * plora_bucket.  `sgmv_min_rows` (> 0) is the segment length from which AUTO sends a
  * segment to the tensor-core path; pass 0 to keep the default. */

@@ -30,7 +30,7 @@ PATH_AUTO, PATH_UNFUSED, PATH_FUSED, PATH_SGMV = 0, 1, 2, 3
 EXPORTS = (
     "plora_create", "plora_destroy", "plora_pool_slab_bytes", "plora_register_pool", "plora_pool_max_rank",
     "plora_bucket", "plora_bucket_view", "plora_lora_delta", "plora_shrink", "plora_expand",
-    "plora_lora_delta_host", "plora_set_path", "plora_device_status", "plora_launch_count", "plora_status_string",
+    "plora_lora_delta_host", "plora_lora_delta_noalloc", "plora_set_path", "plora_device_status", "plora_launch_count", "plora_status_string",
 )
 
 
@@ -81,6 +81,7 @@ def load(build_if_missing: bool = True):
         "plora_shrink": (i32, [vp, vp, vp, i32, i32, i32, vp, i32, vp]),
         "plora_expand": (i32, [vp, vp, i32, vp, i32, i32, i32, vp, vp]),
         "plora_lora_delta_host": (i32, [vp, vp, vp, i32, i32, i32, vp, vp]),
+        "plora_lora_delta_noalloc": (i32, [vp, vp, vp, i32, i32, i32, vp, vp]),
         "plora_set_path": (i32, [vp, i32, i32]),
         "plora_device_status": (i32, [vp, vp, ctypes.POINTER(i32)]),
         "plora_launch_count": (i64, [vp]),
@@ -144,6 +145,10 @@ def plora_expand(ctx, m_ptr, ldm, ids_ptr, n_tok, layer, proj, y_ptr, stream=0):
 
 def plora_lora_delta_host(ctx, x_host_ptr, ids_host_ptr, n_tok, layer, proj, y_host_ptr, stream=0):
     return load().plora_lora_delta_host(ctx, x_host_ptr, ids_host_ptr, n_tok, layer, proj, y_host_ptr, stream)
+
+
+def plora_lora_delta_noalloc(ctx, x_ptr, ids_ptr, n_tok, layer, proj, y_ptr, stream=0):
+    return load().plora_lora_delta_noalloc(ctx, x_ptr, ids_ptr, n_tok, layer, proj, y_ptr, stream)
 
 
 def plora_set_path(ctx, path: int, sgmv_min_rows: int = 0):
@@ -298,6 +303,12 @@ class Context:
         n_tok = int(ids_host.shape[0])
         _check(plora_lora_delta_host(self._h, _data_ptr(x_host), _data_ptr(ids_host), n_tok, layer, proj,
                                      _data_ptr(y_host), _stream_handle(stream)), "plora_lora_delta_host")
+
+    def lora_delta_noalloc(self, x, ids, layer, proj, y, stream=None):
+        """The delta for callers that must not allocate: same result as lora_delta, with the
+        intermediate m in the library's fixed scratch array (see plora_lora_delta_noalloc)."""
+        _check(plora_lora_delta_noalloc(self._h, x.data_ptr(), ids.data_ptr(), int(ids.numel()), layer, proj,
+                                        y.data_ptr(), _stream_handle(stream)), "plora_lora_delta_noalloc")
 
     def set_path(self, path: int, sgmv_min_rows: int = 0):
         _check(plora_set_path(self._h, path, sgmv_min_rows), "plora_set_path")

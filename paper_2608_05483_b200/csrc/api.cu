@@ -514,3 +514,65 @@ PLORA_API plora_status plora_device_status(plora_ctx* ctx, void* stream, int32_t
 PLORA_API int64_t plora_launch_count(plora_ctx* ctx) { return ctx ? ctx->launches : -1; }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------
+// The delta without any allocation: m = x A lives in an array of the library image.
+// ---------------------------------------------------------------------------------
+namespace {
+
+// Part of the library image on every device that loads it.  In host code this name is only
+// a handle for cudaGetSymbolAddress: it is NOT a device address and must never be passed to
+// a kernel as it is.
+static __device__ __align__(256) float g_noalloc_scratch[PLORA_NOALLOC_SCRATCH_FLOATS];
+
+constexpr int kMaxDevicesTracked = 64;
+float* g_noalloc_scratch_addr[kMaxDevicesTracked] = {};   // per device, filled on first use
+
+// Device address of the scratch array on `device`, which must be the current device.
+cudaError_t noalloc_scratch_address(int device, float** out) {
+    if (device < 0 || device >= kMaxDevicesTracked) return cudaErrorInvalidDevice;
+    if (!g_noalloc_scratch_addr[device]) {
+        void* addr = nullptr;
+        const cudaError_t e = cudaGetSymbolAddress(&addr, g_noalloc_scratch);
+        if (e != cudaSuccess) return e;
+        g_noalloc_scratch_addr[device] = static_cast<float*>(addr);
+    }
+    *out = g_noalloc_scratch_addr[device];
+    return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" {
+
+PLORA_API plora_status plora_lora_delta_noalloc(plora_ctx* ctx, const void* x, const int32_t* ids, int32_t n_tok,
+                                                int32_t layer, int32_t proj, float* y, void* stream) {
+    plora_status rc = check_call(ctx, x, ids, n_tok, y);
+    if (rc != PLORA_OK) return rc;
+    PoolRec* pool = find_pool(ctx, layer, proj);
+    if (!pool) return PLORA_ERR_NOT_REGISTERED;
+    if (n_tok == 0) return PLORA_OK;
+    const int32_t ldm = pool->dev.max_rp;
+    if ((size_t)n_tok * (size_t)ldm > (size_t)PLORA_NOALLOC_SCRATCH_FLOATS) return PLORA_ERR_WORKSPACE;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return PLORA_ERR_CUDA;
+    float* m = nullptr;
+    if (noalloc_scratch_address(ctx->device, &m) != cudaSuccess) return PLORA_ERR_CUDA;
+    cudaStream_t st = as_stream(stream);
+    // the two BGMV kernels take every segment: bucket with no tensor-core segments
+    const int32_t saved = ctx->path;
+    ctx->path = PLORA_PATH_UNFUSED;
+    rc = ensure_bucket(ctx, ids, n_tok, pool->dev.n_adapters, st);
+    ctx->path = saved;
+    if (rc != PLORA_OK) return rc;
+    int nl = 0;
+    cudaError_t e = launch_bgmv(kShrinkOnly, pool->dev, ctx->bk, n_tok, x, nullptr, m, ldm, ctx->status_dev,
+                                ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl);
+    if (e == cudaSuccess)
+        e = launch_bgmv(kExpandOnly, pool->dev, ctx->bk, n_tok, nullptr, y, m, ldm, ctx->status_dev, ctx->sm_count,
+                        ctx->launches_since_bucket++ > 0, st, &nl);
+    ctx->launches += nl;
+    return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
+}
+
+}  // extern "C"
