@@ -32,7 +32,8 @@ struct DeviceGuard {
     }
 };
 
-constexpr int kDefaultSgmvMinRows = 1 << 30;   // tensor-core path not wired in yet
+constexpr int kDefaultSgmvMinRows = 32;   // AUTO: segments at least this long take the tensor-core path ...
+constexpr int kSgmvMinBatch = 512;        // ... in batches at least this large (a decode batch stays one launch)
 
 }  // namespace
 
@@ -112,16 +113,16 @@ size_t layout_pool(const plora_pool_desc* d, std::vector<AdapterEntry>* table, i
     return off;
 }
 
-int32_t effective_sgmv_min(const plora_ctx* ctx) {
+int32_t effective_sgmv_min(const plora_ctx* ctx, int32_t n_tok) {
     switch (ctx->path) {
         case PLORA_PATH_SGMV: return 1;
-        case PLORA_PATH_AUTO: return ctx->sgmv_min_rows;
+        case PLORA_PATH_AUTO: return n_tok >= kSgmvMinBatch ? ctx->sgmv_min_rows : INT_MAX;
         default: return INT_MAX;
     }
 }
 
 plora_status do_bucket(plora_ctx* ctx, const int32_t* ids, int32_t n_tok, int32_t n_adapters, cudaStream_t st) {
-    const int32_t thr = effective_sgmv_min(ctx);
+    const int32_t thr = effective_sgmv_min(ctx, n_tok);
     int nl = 0;
     cudaError_t e = launch_bucket(ids, n_tok, n_adapters, thr, ctx->bk, ctx->status_dev, st, &nl);
     ctx->launches += nl;
@@ -137,7 +138,7 @@ plora_status do_bucket(plora_ctx* ctx, const int32_t* ids, int32_t n_tok, int32_
 
 plora_status ensure_bucket(plora_ctx* ctx, const int32_t* ids, int32_t n_tok, int32_t n_adapters, cudaStream_t st) {
     if (ctx->bucket_valid && ctx->cur_ids == ids && ctx->cur_ntok == n_tok && ctx->cur_nadapters == n_adapters &&
-        ctx->bucket_sgmv_min == effective_sgmv_min(ctx))
+        ctx->bucket_sgmv_min == effective_sgmv_min(ctx, n_tok))
         return PLORA_OK;
     return do_bucket(ctx, ids, n_tok, n_adapters, st);
 }
@@ -395,11 +396,11 @@ PLORA_API plora_status plora_lora_delta(plora_ctx* ctx, const void* x, const int
     } else {
         // a batch shorter than the threshold cannot hold a segment for the tensor-core path
         const bool may_bgmv = ctx->path != PLORA_PATH_SGMV;
-        const bool may_sgmv = ctx->path == PLORA_PATH_SGMV || (ctx->path == PLORA_PATH_AUTO && n_tok >= ctx->sgmv_min_rows);
+        const bool may_sgmv = ctx->bucket_sgmv_min != INT_MAX;
         if (may_bgmv)
             e = launch_bgmv(kFused, pool->dev, ctx->bk, n_tok, x, y, nullptr, 0, ctx->status_dev, ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl);
         if (e == cudaSuccess && may_sgmv)
-            e = launch_sgmv(pool->dev, ctx->bk, n_tok, x, y, ctx->status_dev, ctx->sm_count, st, &nl);
+            e = launch_sgmv(pool->dev, ctx->bk, n_tok, ctx->bucket_sgmv_min, x, y, ctx->status_dev, ctx->sm_count, st, &nl);
     }
     ctx->launches += nl;
     return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;

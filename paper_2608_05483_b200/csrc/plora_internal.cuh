@@ -104,7 +104,7 @@ enum BgmvMode { kFused = 0, kShrinkOnly = 1, kExpandOnly = 2 };
 cudaError_t launch_bgmv(BgmvMode mode, const PoolDev& pool, const BucketDev& bk, int n_tok, const void* x, float* y,
                         float* m, int ldm, int32_t* status, int sm_count, bool early_tables, cudaStream_t stream,
                         int* n_launches);
-cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, const void* x, float* y,
+cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, int sgmv_min_rows, const void* x, float* y,
                         int32_t* status, int sm_count, cudaStream_t stream, int* n_launches);
 // per-device function attributes (dynamic shared memory); called by plora_create
 cudaError_t bucket_configure();

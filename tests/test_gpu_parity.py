@@ -17,6 +17,8 @@ from workloads import gen_adapter, gen_x, gen_y_in, make_workload
 pytestmark = pytest.mark.gpu
 
 BGMV_PATHS = [P.PATH_FUSED, P.PATH_UNFUSED]
+# SGMV carries m as bf16 hi + lo (about 2^-17 relative), still far inside the fp32-path bound
+ALL_PATHS = [P.PATH_FUSED, P.PATH_UNFUSED, P.PATH_SGMV, P.PATH_AUTO]
 
 
 def _oracle(p, y_in=None, ids=None):
@@ -31,7 +33,7 @@ def _problem_from_workload(wl, pool):
                 y_in=gen_y_in(wl, pool))
 
 
-def _check_paths(p, paths=BGMV_PATHS, tol=TOL_FP32_PATH, on_device=False):
+def _check_paths(p, paths=ALL_PATHS, tol=TOL_FP32_PATH, on_device=False):
     r = Runner(p, on_device=on_device)
     try:
         ref0 = _oracle(p)
@@ -64,6 +66,7 @@ def test_tiny_config_device_resident_sources():
     (3, dict(n_adapters=100, d_model=640, d_ff=1728, n_layers=1, n_tok=128)),   # rectangular projections, rank 64
     (4, dict(n_adapters=50, d_model=512, n_layers=1, n_tok=1024)),  # long contiguous segments
     (5, dict(n_adapters=60, d_model=1024, n_layers=1, n_tok=512)),  # mixed ranks, mixed segment lengths
+    (5, dict(n_adapters=200, d_model=512, n_layers=1, n_tok=2048)),  # AUTO sends long segments to SGMV, short ones to BGMV
 ])
 def test_reduced_benchmark_configs(cfg, kw):
     wl = make_workload(cfg, **kw)
@@ -94,6 +97,34 @@ def test_token_counts_and_hot_adapter(T):
     _check_paths(p)
 
 
+def test_auto_dispatch_uses_both_kernels():
+    wl = make_workload(5, n_adapters=200, d_model=512, n_layers=1, n_tok=2048)
+    p = _problem_from_workload(wl, wl.pools[0])
+    lens = np.bincount(wl.ids, minlength=wl.n_adapters)
+    assert (lens >= 32).any() and ((lens > 0) & (lens < 32)).any()
+    r = Runner(p)
+    try:
+        r.ctx.set_path(P.PATH_AUTO)
+        ids = r.ids
+        y = torch.zeros((p["T"], p["d_out"]), dtype=torch.float32, device=DEV)
+        r.ctx.bucket(ids, p["N"])
+        n0 = r.ctx.launch_count()
+        r.ctx.lora_delta(r.x, ids, 0, 0, y)
+        torch.cuda.synchronize()
+        assert r.ctx.launch_count() - n0 == 2        # one BGMV launch + one SGMV launch
+        assert rel_err(y.cpu().numpy(), _oracle(p)) <= TOL_FP32_PATH
+        # a decode-sized batch stays a single launch
+        small = torch.from_numpy(wl.ids[:256].copy()).to(DEV)
+        y2 = torch.zeros((256, p["d_out"]), dtype=torch.float32, device=DEV)
+        r.ctx.bucket(small, p["N"])
+        n0 = r.ctx.launch_count()
+        r.ctx.lora_delta(r.x[:256], small, 0, 0, y2)
+        torch.cuda.synchronize()
+        assert r.ctx.launch_count() - n0 == 1
+    finally:
+        r.close()
+
+
 def test_empty_and_all_minus_one():
     p = random_problem(1, T=0, d_in=64, d_out=64, ranks=[8])
     r = Runner(p, max_tokens=8)
@@ -102,7 +133,7 @@ def test_empty_and_all_minus_one():
     p = random_problem(2, T=9, d_in=64, d_out=64, ranks=[8, 8])
     p["ids"][:] = -1
     r = Runner(p)
-    for path in BGMV_PATHS:
+    for path in ALL_PATHS:
         got = r.delta(path, y_in=p["y_in"])
         assert np.array_equal(got, p["y_in"])
     r.close()
