@@ -224,7 +224,7 @@ def run_ours(args):
     wl = make_workload(args.config, n_layers=args.layers)
     dw = DeviceWorkload(wl, local)
     ctx = dw.ctx
-    ctx.set_path(P.PATH_AUTO)
+    ctx.set_path({"auto": P.PATH_AUTO, "fused": P.PATH_FUSED, "unfused": P.PATH_UNFUSED, "sgmv": P.PATH_SGMV}[args.path])
     n_calls = len(wl.pools)
 
     # full-size parity on sampled pools + the oracle's time, before anything is timed (rank 0)
@@ -364,7 +364,7 @@ def run_ours(args):
                    config=dict(workload=f"config {args.config} ({wl.name})", n_tok=wl.n_tok, n_adapters=wl.n_adapters,
                                layers=len({p.layer for p in wl.pools}), calls_per_step=n_calls,
                                ranks=sorted({int(r) for r in wl.ranks}), ids=wl.meta.get("ids"),
-                               distinct_adapters=per_call[0]["distinct"], path="auto", cuda_graph=bool(args.graph),
+                               distinct_adapters=per_call[0]["distinct"], path=args.path, cuda_graph=bool(args.graph),
                                l2="inputs larger than L2: a step streams %.2f GB through %d distinct slabs"
                                   % (step_bytes / 1e9, n_calls),
                                multi_gpu="replicas: every rank runs its own batch, no data-path collective"),
@@ -429,6 +429,7 @@ def main():
     ap.add_argument("--layers", type=int, default=None)
     ap.add_argument("--graph", type=int, default=1)
     ap.add_argument("--cpu-pools", type=int, default=8, dest="cpu_pools")
+    ap.add_argument("--path", default="auto", choices=["auto", "fused", "unfused", "sgmv"])
     ap.add_argument("--no-cpu", action="store_true", dest="no_cpu")
     ap.add_argument("--no-e2e", action="store_true", dest="no_e2e")
     args = ap.parse_args()

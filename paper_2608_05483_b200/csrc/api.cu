@@ -34,6 +34,7 @@ struct DeviceGuard {
 
 constexpr int kDefaultSgmvMinRows = 32;   // AUTO: segments at least this long take the tensor-core path ...
 constexpr int kSgmvMinBatch = 512;        // ... in batches at least this large (a decode batch stays one launch)
+constexpr int kSgmvMinTiles = 128;        // ... and only if they make at least this many 64-row tiles together
 
 }  // namespace
 
@@ -86,10 +87,10 @@ bool desc_shape_ok(const plora_pool_desc* d, plora_status* why) {
 }
 
 // Fills the offset table (host copy) and returns the slab size.
-size_t layout_pool(const plora_pool_desc* d, std::vector<AdapterEntry>* table, int* max_rp, int* uniform_rp = nullptr,
+size_t layout_pool(const plora_pool_desc* d, std::vector<AdapterEntry>* table, int* max_rp, int* rp_mask = nullptr,
                    int* min_rp = nullptr) {
     size_t off = 0;
-    int mrp = 0, urp = -1, lrp = kMaxRank;
+    int mrp = 0, mask = 0, lrp = kMaxRank;
     if (table) table->resize(d->n_adapters);
     for (int a = 0; a < d->n_adapters; ++a) {
         const int rp = pad_rank(d->ranks[a]);
@@ -105,10 +106,10 @@ size_t layout_pool(const plora_pool_desc* d, std::vector<AdapterEntry>* table, i
         if (table) (*table)[a] = e;
         if (rp > mrp) mrp = rp;
         if (rp < lrp) lrp = rp;
-        urp = (urp == -1 || urp == rp) ? rp : 0;
+        mask |= rp;
     }
     if (max_rp) *max_rp = mrp;
-    if (uniform_rp) *uniform_rp = urp > 0 ? urp : 0;
+    if (rp_mask) *rp_mask = mask;
     if (min_rp) *min_rp = lrp;
     return off;
 }
@@ -124,7 +125,8 @@ int32_t effective_sgmv_min(const plora_ctx* ctx, int32_t n_tok) {
 plora_status do_bucket(plora_ctx* ctx, const int32_t* ids, int32_t n_tok, int32_t n_adapters, cudaStream_t st) {
     const int32_t thr = effective_sgmv_min(ctx, n_tok);
     int nl = 0;
-    cudaError_t e = launch_bucket(ids, n_tok, n_adapters, thr, ctx->bk, ctx->status_dev, st, &nl);
+    cudaError_t e = launch_bucket(ids, n_tok, n_adapters, thr, ctx->path == PLORA_PATH_AUTO ? kSgmvMinTiles : 0, ctx->bk,
+                                  ctx->status_dev, st, &nl);
     ctx->launches += nl;
     if (e != cudaSuccess) { ctx->bucket_valid = false; return PLORA_ERR_CUDA; }
     ctx->cur_ids = ids;
@@ -266,8 +268,8 @@ PLORA_API plora_status plora_register_pool(plora_ctx* ctx, const plora_pool_desc
     for (int a = 0; a < d->n_adapters; ++a)
         if (!d->A[a] || !d->B[a]) return PLORA_ERR_INVALID_ARG;
     std::vector<AdapterEntry> table;
-    int max_rp = 0, uniform_rp = 0, min_rp = 0;
-    const size_t need = layout_pool(d, &table, &max_rp, &uniform_rp, &min_rp);
+    int max_rp = 0, rp_mask = 0, min_rp = 0;
+    const size_t need = layout_pool(d, &table, &max_rp, &rp_mask, &min_rp);
     if (slab_bytes < need) return PLORA_ERR_WORKSPACE;
 
     DeviceGuard g(ctx->device);
@@ -328,7 +330,7 @@ PLORA_API plora_status plora_register_pool(plora_ctx* ctx, const plora_pool_desc
     rec.dev.d_out = d->d_out;
     rec.dev.n_adapters = N;
     rec.dev.max_rp = max_rp;
-    rec.dev.uniform_rp = uniform_rp;
+    rec.dev.rp_mask = rp_mask;
     rec.dev.min_rp = min_rp;
     if (PoolRec* old = find_pool(ctx, d->layer, d->proj)) {
         cudaStreamSynchronize(st);

@@ -527,16 +527,6 @@ __device__ __forceinline__ void consume_stage(const Params& p, const Smem& sm, c
     }
 }
 
-// Pools of mixed ranks: the lane constants are rebuilt for every stage.
-template <int MODE, int RP>
-__device__ __noinline__ void stage_of_rank(const Params& p, const Smem& sm, const StageHdr& h, uint32_t tile,
-                                           uint32_t empty_bar, float (&acc)[kMaxRowsPerLane][kTokChunk], Ctl& ctl,
-                                           int warp, int lane) {
-    LaneMaps<RP> maps;
-    maps.init(warp, lane);
-    consume_stage<MODE, RP>(p, sm, h, maps, tile, empty_bar, acc, ctl, warp, lane);
-}
-
 // ---- producer side: the m of an expand task ---------------------------------------------------
 // A unit's m has cnt * rp values; lane l of the producer warp owns the values l, l + 32, ...
 // For every owned value the runs_a partial words are read, checked for this launch's epoch,
@@ -603,8 +593,9 @@ __device__ __forceinline__ Task decode_task(int t, int n_shrink_tasks, int runs_
     return k;
 }
 
-// RPK = the padded rank when every adapter of the pool has the same one (no dispatch
-// inside the stage loop), 0 for a pool of mixed ranks.
+// One instantiation per padded rank RPK.  The kernel handles the units whose adapter has that
+// padded rank and skips the others: a pool of mixed ranks is served by one launch per rank
+// class present in it, each with loops specialised (and registers allocated) for its rank.
 template <int MODE, int RPK>
 __global__ void __launch_bounds__(kThreads, 2) bgmv_kernel(const Params p) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -688,10 +679,11 @@ __global__ void __launch_bounds__(kThreads, 2) bgmv_kernel(const Params p) {
         for (int base = blockIdx.x; base < n_tasks; base += 32 * stride) {
             CYC_T0(tb0);
             const int my_task = base + lane * stride;
-            const bool has = my_task < n_tasks;
-            const Task mine = decode_task(has ? my_task : base, n_shrink, p.runs_a, p.runs_b);
+            const bool in_range = my_task < n_tasks;
+            const Task mine = decode_task(in_range ? my_task : base, n_shrink, p.runs_a, p.runs_b);
             const WorkUnit mu = p.bk.bgmv_units[mine.unit];
             const AdapterEntry me = p.pool.table[mu.adapter];
+            const bool has = in_range && me.rp == RPK;   // units of other rank classes belong to other launches
             const int in_batch = min(32, (n_tasks - base + stride - 1) / stride);
             const int C = tile_cols(me.rp);
             const uint32_t tb = (uint32_t)tile_bytes(me.rp);
@@ -724,7 +716,7 @@ __global__ void __launch_bounds__(kThreads, 2) bgmv_kernel(const Params p) {
             for (int b = 0; b < in_batch; ++b) {
                 // fused mode: the running number of this expand task tells the consumers where its m is
                 const uint32_t m_seq = m_count;
-                if (MODE == kFused && __shfl_sync(full, mine.phase, b)) ++m_count;
+                if (MODE == kFused && __shfl_sync(full, (int)(has && mine.phase), b)) ++m_count;
                 CYC_T0(tg0);
                 CYC_ADD(p_gather, tg0);
                 if (lane == b) {
@@ -807,14 +799,15 @@ __global__ void __launch_bounds__(kThreads, 2) bgmv_kernel(const Params p) {
         uint32_t seq = 0;
         for (int base = t; base < n_tasks; base += 32 * stride) {
             const int my_task = base + lane * stride;
-            const bool has = my_task < n_tasks;
-            const int my_unit = (has ? my_task - n_shrink : base - n_shrink) / p.runs_b;
+            const bool in_range = my_task < n_tasks;
+            const int my_unit = (in_range ? my_task - n_shrink : base - n_shrink) / p.runs_b;
             const WorkUnit mu = p.bk.bgmv_units[my_unit];
             const int my_rp = p.pool.table[mu.adapter].rp;
             const int in_batch = min(32, (n_tasks - base + stride - 1) / stride);
-            for (int b = 0; b < in_batch; ++b, ++seq) {
-                const int unit_b = __shfl_sync(full, my_unit, b), cnt_b = __shfl_sync(full, mu.cnt, b);
+            for (int b = 0; b < in_batch; ++b) {
                 const int rp_b = __shfl_sync(full, my_rp, b);
+                if (rp_b != RPK) continue;   // another launch's unit
+                const int unit_b = __shfl_sync(full, my_unit, b), cnt_b = __shfl_sync(full, mu.cnt, b);
                 const uint32_t e = seq % kMRing;
                 if (lane == 0) mbar_wait(sm.m_empty + e * 8, ((seq / kMRing) & 1) ^ 1, sm.abort_flag, p.status);
                 __syncwarp();
@@ -832,6 +825,7 @@ __global__ void __launch_bounds__(kThreads, 2) bgmv_kernel(const Params p) {
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(sm.m_full + e * 8);
+                ++seq;
             }
         }
         return;
@@ -842,8 +836,8 @@ __global__ void __launch_bounds__(kThreads, 2) bgmv_kernel(const Params p) {
     Ctl ctl;
     ctl.pbuf = 0;
     ctl.sync_phase = 0;
-    LaneMaps<RPK == 0 ? 8 : RPK> maps;   // per-lane constants, computed once when the rank is uniform
-    if constexpr (RPK != 0) maps.init(warp, lane);
+    LaneMaps<RPK> maps;   // per-lane constants of both phases
+    maps.init(warp, lane);
     CYC_DECL(c_wait); CYC_DECL(c_hdr); CYC_DECL(c_work);
     for (uint32_t it = 0;; ++it) {
         const uint32_t slot = it % kStages;
@@ -859,17 +853,7 @@ __global__ void __launch_bounds__(kThreads, 2) bgmv_kernel(const Params p) {
         if ((h.flags & kFlagEnd) || *sm.abort_flag) { if (tid == 0) { TRACE(5); g_trace_n(it); CYC_OUT(0, c_wait); CYC_OUT(1, c_hdr); CYC_OUT(2, c_work); CYC_OUT(3, ctl.c_tile); CYC_OUT(4, ctl.c_fin); CYC_OUT(5, ctl.c_finw); } break; }
         const uint32_t empty_bar = sm.empty + slot * 8;
         CYC_T0(tc);
-        if constexpr (RPK != 0) {
-            consume_stage<MODE, RPK>(p, sm, h, maps, tile, empty_bar, acc, ctl, warp, lane);
-        } else {
-            switch (h.rp) {
-                case 8: stage_of_rank<MODE, 8>(p, sm, h, tile, empty_bar, acc, ctl, warp, lane); break;
-                case 16: stage_of_rank<MODE, 16>(p, sm, h, tile, empty_bar, acc, ctl, warp, lane); break;
-                case 32: stage_of_rank<MODE, 32>(p, sm, h, tile, empty_bar, acc, ctl, warp, lane); break;
-                case 64: stage_of_rank<MODE, 64>(p, sm, h, tile, empty_bar, acc, ctl, warp, lane); break;
-                default: stage_of_rank<MODE, 128>(p, sm, h, tile, empty_bar, acc, ctl, warp, lane); break;
-            }
-        }
+        consume_stage<MODE, RPK>(p, sm, h, maps, tile, empty_bar, acc, ctl, warp, lane);
         CYC_ADD(c_work, tc);
         if (tid == 0) TRACE2(it, 3);
     }
@@ -886,22 +870,21 @@ __global__ void __launch_bounds__(kThreads, 2) bgmv_kernel(const Params p) {
 using KernelFn = void (*)(const Params);
 
 template <int MODE>
-KernelFn pick_rank(int uniform_rp) {
-    switch (uniform_rp) {
+KernelFn pick_rank(int rp) {
+    switch (rp) {
         case 8: return bgmv_kernel<MODE, 8>;
         case 16: return bgmv_kernel<MODE, 16>;
         case 32: return bgmv_kernel<MODE, 32>;
         case 64: return bgmv_kernel<MODE, 64>;
-        case 128: return bgmv_kernel<MODE, 128>;
-        default: return bgmv_kernel<MODE, 0>;
+        default: return bgmv_kernel<MODE, 128>;
     }
 }
 
-KernelFn pick_kernel(BgmvMode mode, int uniform_rp) {
+KernelFn pick_kernel(BgmvMode mode, int rp) {
     switch (mode) {
-        case kFused: return pick_rank<kFused>(uniform_rp);
-        case kShrinkOnly: return pick_rank<kShrinkOnly>(uniform_rp);
-        default: return pick_rank<kExpandOnly>(uniform_rp);
+        case kFused: return pick_rank<kFused>(rp);
+        case kShrinkOnly: return pick_rank<kShrinkOnly>(rp);
+        default: return pick_rank<kExpandOnly>(rp);
     }
 }
 
@@ -923,7 +906,7 @@ extern "C" __attribute__((visibility("default"))) int plora_debug_trace2(long lo
 
 cudaError_t bgmv_configure() {
     const int modes[3] = {kFused, kShrinkOnly, kExpandOnly};
-    const int rps[6] = {0, 8, 16, 32, 64, 128};
+    const int rps[5] = {8, 16, 32, 64, 128};
     for (int m : modes)
         for (int rp : rps) {
             cudaError_t e = cudaFuncSetAttribute(pick_kernel((BgmvMode)m, rp),
@@ -946,35 +929,40 @@ cudaError_t launch_bgmv(BgmvMode mode, const PoolDev& pool, const BucketDev& bk,
     p.n_tok = n_tok;
     p.status = status;
     p.early_tables = early_tables ? 1 : 0;
-    // Every adapter has at least tiles_for(d, min_rp) tiles, so each unit can be cut into that many runs.
-    p.runs_a = mode == kShrinkOnly ? 1 : clamp_runs(tiles_for(pool.d_in, pool.min_rp));
-    // an expand task pays one round trip for its m before its first tile: give it at least two tiles
-    p.runs_b = clamp_runs(tiles_for(pool.d_out, pool.min_rp) / (mode == kFused ? 2 : 1));
-    if (mode == kFused) {
-        // the partial-m workspace holds n_units * runs_a * kTokChunk * max_rp words, n_units <= n_tok
-        const size_t per_run = (size_t)n_tok * kTokChunk * pool.max_rp * sizeof(unsigned long long);
-        while (p.runs_a > 1 && per_run * p.runs_a > bk.m_part_bytes) --p.runs_a;
-        if (per_run * p.runs_a > bk.m_part_bytes) return cudaErrorMemoryAllocation;
-    }
-    // persistent grid: two CTAs per SM, never more CTAs than there can be tasks
-    const long long max_tasks = (long long)n_tok * (p.runs_a + p.runs_b);
-    int grid = 2 * sm_count;
-    if (grid > max_tasks) grid = (int)max_tasks;
-    if (grid < 1) grid = 1;
-
-    cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = kSmemBytes;
-    cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, pick_kernel(mode, pool.uniform_rp), p);
-    ++*n_launches;
-    return e;
+    // one launch per padded-rank class present in the pool
+    for (int rp = 8; rp <= kMaxRank; rp <<= 1) {
+        if (!(pool.rp_mask & rp)) continue;
+        // a unit of this class has tiles_for(d, rp) tiles per phase: cut each phase into runs
+        p.runs_a = mode == kShrinkOnly ? 1 : clamp_runs(tiles_for(pool.d_in, rp));
+        // an expand task pays one round trip for its m before its first tile: give it at least two tiles
+        p.runs_b = clamp_runs(tiles_for(pool.d_out, rp) / (mode == kFused ? 2 : 1));
+        if (mode == kFused) {
+            // the partial-m workspace holds n_units * runs_a * kTokChunk * max_rp words, n_units <= n_tok
+            const size_t per_run = (size_t)n_tok * kTokChunk * pool.max_rp * sizeof(unsigned long long);
+            while (p.runs_a > 1 && per_run * p.runs_a > bk.m_part_bytes) --p.runs_a;
+            if (per_run * p.runs_a > bk.m_part_bytes) return cudaErrorMemoryAllocation;
+        }
+        // persistent grid: two CTAs per SM, never more CTAs than there can be tasks
+        const long long max_tasks = (long long)n_tok * (p.runs_a + p.runs_b);
+        int grid = 2 * sm_count;
+        if (grid > max_tasks) grid = (int)max_tasks;
+        if (grid < 1) grid = 1;
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3(grid);
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = kSmemBytes;
+        cfg.stream = stream;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        const cudaError_t e = cudaLaunchKernelEx(&cfg, pick_kernel(mode, rp), p);
+        ++*n_launches;
+        if (e != cudaSuccess) return e;
+        p.early_tables = 1;   // the next class's launch follows a kernel that is not the bucket kernel
+    }
+    return cudaSuccess;
 }
 
 }  // namespace plora

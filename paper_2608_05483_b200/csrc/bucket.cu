@@ -76,8 +76,8 @@ __device__ void write_units(WorkUnit* out, int n_units, const int* ustart, const
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
-bucket_kernel(const int32_t* __restrict__ ids, int T, int N, int nch, int sgmv_min_rows, BucketDev bk,
-              int32_t* status) {
+bucket_kernel(const int32_t* __restrict__ ids, int T, int N, int nch, int sgmv_min_rows, int sgmv_min_tiles,
+              BucketDev bk, int32_t* status) {
     extern __shared__ int smem[];
     const int nb = N + 1;                 // bins: ids 0..N-1, then "no adapter"
     int* cnt = smem;                      // [nch][nb]   per-chunk counts, later per-chunk cursors
@@ -118,16 +118,24 @@ bucket_kernel(const int32_t* __restrict__ ids, int T, int N, int nch, int sgmv_m
         total[b] = run;
         start[b] = run;
         segidx[b] = (b < N && run > 0) ? 1 : 0;
-        const bool sg = run >= sgmv_min_rows;
-        ubg[b] = (b < N && run > 0 && !sg) ? units_of(run, kTokChunk) : 0;
-        usg[b] = (b < N && run > 0 && sg) ? units_of(run, kSgmvRows) : 0;
+        usg[b] = (b < N && run > 0 && run >= sgmv_min_rows) ? units_of(run, kSgmvRows) : 0;
     }
     __syncthreads();
     block_exclusive_scan(start, nb, wsum);
     if (tid == 0) start[nb] = T;
     const int n_seg = block_exclusive_scan(segidx, nb, wsum);
+    // Long segments go to the tensor-core path only if together they make enough tiles to occupy
+    // the GPU; a handful of tiles would each be one long serial job, so they stay with BGMV.
+    const int n_sg_cand = block_exclusive_scan(usg, nb, wsum);
+    const bool use_sg = n_sg_cand >= sgmv_min_tiles;
+    const int n_sg = use_sg ? n_sg_cand : 0;
+    for (int b = tid; b < nb; b += kThreads) {
+        const int run = total[b];
+        const bool sg = use_sg && run >= sgmv_min_rows;
+        ubg[b] = (b < N && run > 0 && !sg) ? units_of(run, kTokChunk) : 0;
+    }
+    __syncthreads();
     const int n_bg = block_exclusive_scan(ubg, nb, wsum);
-    const int n_sg = block_exclusive_scan(usg, nb, wsum);
     const int n_active = start[N];
 
     // stable scatter: each warp walks its chunk in order, 32 tokens at a time
@@ -190,13 +198,13 @@ int bucket_max_adapters() {
     return n;
 }
 
-cudaError_t launch_bucket(const int32_t* ids, int n_tok, int n_adapters, int sgmv_min_rows, BucketDev bk,
-                          int32_t* status, cudaStream_t stream, int* n_launches) {
+cudaError_t launch_bucket(const int32_t* ids, int n_tok, int n_adapters, int sgmv_min_rows, int sgmv_min_tiles,
+                          BucketDev bk, int32_t* status, cudaStream_t stream, int* n_launches) {
     int nch = kWarps;
     while (nch > 1 && bucket_smem_bytes(n_adapters, nch) > kBucketSmemLimit) nch >>= 1;
     const size_t smem = bucket_smem_bytes(n_adapters, nch);
     if (smem > kBucketSmemLimit) return cudaErrorInvalidValue;
-    bucket_kernel<<<1, kThreads, smem, stream>>>(ids, n_tok, n_adapters, nch, sgmv_min_rows, bk, status);
+    bucket_kernel<<<1, kThreads, smem, stream>>>(ids, n_tok, n_adapters, nch, sgmv_min_rows, sgmv_min_tiles, bk, status);
     ++*n_launches;
     return cudaGetLastError();
 }

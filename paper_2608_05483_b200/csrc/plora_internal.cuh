@@ -54,7 +54,7 @@ struct PoolDev {
     const uint8_t* slab;
     const AdapterEntry* table;
     int32_t d_in, d_out, n_adapters, max_rp;
-    int32_t uniform_rp;   // the padded rank if all adapters share it, else 0
+    int32_t rp_mask;      // OR of the padded ranks present in the pool (each a power of two, 8..128)
     int32_t min_rp;
 };
 
@@ -94,8 +94,8 @@ struct BucketDev {
 };
 
 // Launchers (each returns the cudaError_t of its launch).
-cudaError_t launch_bucket(const int32_t* ids, int n_tok, int n_adapters, int sgmv_min_rows, BucketDev bk,
-                          int32_t* status, cudaStream_t stream, int* n_launches);
+cudaError_t launch_bucket(const int32_t* ids, int n_tok, int n_adapters, int sgmv_min_rows, int sgmv_min_tiles,
+                          BucketDev bk, int32_t* status, cudaStream_t stream, int* n_launches);
 cudaError_t launch_repack(const AdapterEntry* table_dev, const void* const* A_dev, const void* const* B_dev,
                           int n_adapters, int d_in, int d_out, uint8_t* slab, cudaStream_t stream, int* n_launches);
 

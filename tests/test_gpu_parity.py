@@ -98,29 +98,43 @@ def test_token_counts_and_hot_adapter(T):
 
 
 def test_auto_dispatch_uses_both_kernels():
-    wl = make_workload(5, n_adapters=200, d_model=512, n_layers=1, n_tok=2048)
-    p = _problem_from_workload(wl, wl.pools[0])
-    lens = np.bincount(wl.ids, minlength=wl.n_adapters)
-    assert (lens >= 32).any() and ((lens > 0) & (lens < 32)).any()
+    # 128 prefill runs of 64 tokens (>= 128 tensor-core tiles) followed by 300 single decode tokens
+    rng = np.random.default_rng(21)
+    N = 300
+    ids = np.concatenate([np.repeat(rng.permutation(N)[:128], 64), rng.integers(0, N, size=300)]).astype(np.int32)
+    p = random_problem(22, T=len(ids), d_in=256, d_out=320, ranks=rng.choice([8, 16, 32, 64], size=N))
+    p["ids"] = ids
+    lens = np.bincount(ids, minlength=N)
+    assert (lens >= 64).sum() >= 128 and ((lens > 0) & (lens < 32)).any()
     r = Runner(p)
     try:
         r.ctx.set_path(P.PATH_AUTO)
-        ids = r.ids
         y = torch.zeros((p["T"], p["d_out"]), dtype=torch.float32, device=DEV)
-        r.ctx.bucket(ids, p["N"])
+        r.ctx.bucket(r.ids, p["N"])
         n0 = r.ctx.launch_count()
-        r.ctx.lora_delta(r.x, ids, 0, 0, y)
+        r.ctx.lora_delta(r.x, r.ids, 0, 0, y)
         torch.cuda.synchronize()
-        assert r.ctx.launch_count() - n0 == 2        # one BGMV launch + one SGMV launch
+        n_classes = len(set(int(v) for v in p["ranks"]))   # ranks 8..64 are their own padded classes
+        assert r.ctx.launch_count() - n0 == n_classes + 1  # one BGMV launch per rank class + one SGMV launch
         assert rel_err(y.cpu().numpy(), _oracle(p)) <= TOL_FP32_PATH
-        # a decode-sized batch stays a single launch
-        small = torch.from_numpy(wl.ids[:256].copy()).to(DEV)
+        # a decode-sized batch stays with BGMV
+        small = torch.from_numpy(ids[-256:].copy()).to(DEV)
         y2 = torch.zeros((256, p["d_out"]), dtype=torch.float32, device=DEV)
         r.ctx.bucket(small, p["N"])
         n0 = r.ctx.launch_count()
-        r.ctx.lora_delta(r.x[:256], small, 0, 0, y2)
+        r.ctx.lora_delta(r.x[-256:], small, 0, 0, y2)
         torch.cuda.synchronize()
-        assert r.ctx.launch_count() - n0 == 1
+        assert r.ctx.launch_count() - n0 == n_classes
+        assert rel_err(y2.cpu().numpy(), _oracle(p, ids=ids)[-256:]) <= TOL_FP32_PATH
+        # few long segments: everything stays with BGMV although the batch is large
+        few = np.concatenate([np.repeat(np.arange(3), 200), rng.integers(0, N, size=200)]).astype(np.int32)
+        few_t = torch.from_numpy(few).to(DEV)
+        y3 = torch.zeros((len(few), p["d_out"]), dtype=torch.float32, device=DEV)
+        r.ctx.bucket(few_t, p["N"])
+        r.ctx.lora_delta(r.x[:len(few)], few_t, 0, 0, y3)
+        torch.cuda.synchronize()
+        p3 = dict(p, x=p["x"][:len(few)], ids=few)
+        assert rel_err(y3.cpu().numpy(), _oracle(p3)) <= TOL_FP32_PATH
     finally:
         r.close()
 
