@@ -209,6 +209,26 @@ def oracle_sample(dw: DeviceWorkload, n_pools: int, check_gpu: bool):
 
 
 # ----------------------------------------------------------------------------------
+# replicas: every rank runs its own batch on its own GPU; the only thing that crosses ranks is
+# the timing (max over ranks), never data of the path
+# ----------------------------------------------------------------------------------
+def max_over_ranks(value: float, device=None) -> float:
+    """Largest `value` over all ranks (the value itself when no process group is up)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device or "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tokens_per_s(n_tok_per_rank: int, world: int, ms_per_step_max: float) -> float:
+    """Weak scaling: the job processed world * n_tok tokens in the slowest rank's step time."""
+    return world * n_tok_per_rank / (ms_per_step_max * 1e-3)
+
+
+# ----------------------------------------------------------------------------------
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -277,10 +297,8 @@ def run_ours(args):
         launches = args.steps * (n_calls + 1)
     total_ms = ev[0].elapsed_time(ev[-1])
     clocks = sampler.stop()
+    total_ms = max_over_ranks(total_ms, f"cuda:{local}")
     if world > 1:
-        t = torch.tensor([total_ms], device=f"cuda:{local}")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
         dist.barrier()
     ms_per_step = total_ms / args.steps
 
@@ -346,10 +364,7 @@ def run_ours(args):
             host_step()
         torch.cuda.synchronize()
         e2e_s = (time.perf_counter() - t0) / n_e2e
-        if world > 1:
-            t = torch.tensor([e2e_s], device=f"cuda:{local}")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_s = float(t.item())
+        e2e_s = max_over_ranks(e2e_s, f"cuda:{local}")
         h2d = sum(wl.n_tok * p.d_in * 2 + wl.n_tok * 4 + wl.n_tok * p.d_out * 4 for p in wl.pools)
         d2h = sum(wl.n_tok * p.d_out * 4 for p in wl.pools)
         e2e = dict(value=world * wl.n_tok / e2e_s, unit="tokens/s", h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
@@ -358,7 +373,7 @@ def run_ours(args):
     status = ctx.device_status()
     if rank == 0:
         out = dict(metric="LoRA-delta tokens/sec at 1000 adapters (whole step: bucket + every layer x projection delta)",
-                   value=world * wl.n_tok / (ms_per_step * 1e-3), unit="tokens/s", n_gpus=world, steps=args.steps,
+                   value=whole_job_tokens_per_s(wl.n_tok, world, ms_per_step), unit="tokens/s", n_gpus=world, steps=args.steps,
                    warmup=max(3, args.warmup), ms_per_step=ms_per_step, higher_is_better=True, scaling="weak",
                    vs_baseline=None, dtype="bf16 in, fp32 accumulate", data="synthetic",
                    config=dict(workload=f"config {args.config} ({wl.name})", n_tok=wl.n_tok, n_adapters=wl.n_adapters,
