@@ -39,7 +39,10 @@ FALLBACK_HBM_GBS = 6650.0   # used only when MEASURED_PEAKS.json is absent
 
 # DRAM bytes per launch of the dominant kernel from the committed ncu captures
 # (profiles/*.md say which capture each number comes from); None = not captured.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    "decode7b": 40.45e6,   # profiles/bgmv_fused_config2_decode7b.md (2-layer capture, same launch shape)
+    "prefill": 628.6e6,    # profiles/sgmv_config4_prefill.md
+}
 
 
 # ----------------------------------------------------------------------------------
