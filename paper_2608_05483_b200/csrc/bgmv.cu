@@ -17,9 +17,11 @@
 //     into a ring of shared-memory stages, and runs ahead of the consumers across
 //     tiles and tasks; each stage carries a small header that tells the consumers
 //     what it holds, so they never wait on global memory for a descriptor;
-//   - eight consumer warps split every tile by columns.  Shrink: a lane owns rank
-//     rows, reads 16-byte chunks of A^T and broadcast chunks of x, accumulates in
-//     fp32; the task's partial m goes to an L2-resident workspace as 64-bit words
+//   - eight consumer warps work on every tile.  Shrink: the warps split the rank rows,
+//     the lanes of a warp split the tile's columns (16-byte chunks of A^T against the
+//     matching chunks of x, fp32 accumulation) and meet by shuffles at the end of the
+//     task, so a warp owns complete sums of its rows and no warp waits for another;
+//     the task's partial m goes to an L2-resident workspace as 64-bit words
 //     {value, launch epoch} with plain stores and no fence.  Expand: the producer
 //     warp of the CTA that owns the expand task loads the unit's partials (a word
 //     whose epoch matches has arrived, otherwise it is read again), sums them in a
@@ -51,13 +53,12 @@ constexpr int kStages = PLORA_EXP_STAGES;
 constexpr int kXBytesPerTok = kMaxSubPerTile * kSubCols * 2;             // x piece of one token for one tile
 constexpr int kHdrOffset = kTileBytesMax + kTokChunk * kXBytesPerTok;
 constexpr int kSlotBytes = kHdrOffset + 128;                             // tile + x pieces + stage header
-constexpr int kPartFloats = kConsumerWarps * kTokChunk * kMaxRank;       // two buffers when the rank is <= 64
 // m of the expand tasks in flight (fused mode): a ring filled by the gather warp and drained by
 // the consumers, with a full / empty barrier pair per entry.
 constexpr int kMRing = 4;
 constexpr int kMRingBytes = kTokChunk * kMaxRank * 4;
-constexpr int kNumBarriers = 2 * kStages + 2 * kMRing + 1;
-constexpr int kSmemBytes = kStages * kSlotBytes + kPartFloats * 4 + kMRing * kMRingBytes + kNumBarriers * 8 + 16;
+constexpr int kNumBarriers = 2 * kStages + 2 * kMRing;
+constexpr int kSmemBytes = kStages * kSlotBytes + kMRing * kMRingBytes + kNumBarriers * 8 + 16;
 constexpr int kPrefetchTasks = 8;   // tasks per CTA whose tiles are prefetched to L2 before the stream-order wait
 constexpr uint32_t kSuspendHintNs = 20000;   // a waiting thread may sleep this long inside one try_wait
 constexpr long long kWaitCycles = 4000000000ll;   // about two seconds of SM clock
@@ -180,33 +181,20 @@ struct Smem {
     uint32_t slots;      // shared address of stage 0
     uint32_t full;       // full[kStages] barriers
     uint32_t empty;      // empty[kStages]
-    float* part;         // per-warp partial m of a shrink task
     volatile int* abort_flag;
     uint32_t m_ring;     // shared address of the m ring (fused mode): kMRing entries of kMRingBytes
     uint32_t m_full;     // m_full[kMRing]: the gather warp has written the entry
     uint32_t m_empty;    // m_empty[kMRing]: every consumer warp is done with the entry
-    uint32_t sync_bar;   // barrier of the consumer warps (one arrival per warp)
     int32_t* status;
     uint32_t epoch;      // this launch's epoch (fused mode)
 };
 
-// Per-thread state of the consumer loop.
+// Per-thread state of the consumer loop (only the experiment build keeps any).
 struct Ctl {
-    int pbuf;             // which half of part[] the next shrink task uses
-    uint32_t sync_phase;  // parity of the next consumer_sync
 #ifdef PLORA_TRACE
     long long c_tile = 0, c_fin = 0, c_finw = 0;
 #endif
 };
-
-// Barrier over the consumer warps, built on an mbarrier so that, like every other wait
-// in this kernel, it gives up after a bounded time instead of hanging.
-__device__ __forceinline__ void consumer_sync(const Smem& sm, Ctl& ctl) {
-    __syncwarp();
-    if ((threadIdx.x & 31) == 0) mbar_arrive(sm.sync_bar);
-    mbar_wait(sm.sync_bar, ctl.sync_phase, sm.abort_flag, sm.status);
-    ctl.sync_phase ^= 1;
-}
 
 // What a stage holds (written by the producer into the stage, read by every consumer warp).
 constexpr int kFlagExpand = 1, kFlagFirst = 2, kFlagLast = 4, kFlagEnd = 8;
@@ -243,65 +231,74 @@ __device__ __forceinline__ size_t part_index(const Params& p, int unit, int run,
 constexpr int kMaxRowsPerLane = kMaxRank / 32;
 
 // ---- shrink: one tile of A^T against the unit's x pieces --------------------------------
-// Lane mapping: for RP <= 32 a lane owns one rank row and CPL of the warp's chunks (lane
-// groups that share the rows take different chunks); for RP > 32 it owns RP/32 rows and
-// all of the warp's chunks.  A 16-byte chunk is 8 consecutive columns.
+// Work split: warp w owns the rank rows [w * RP/8, (w + 1) * RP/8).  Inside the warp the lanes
+// split the tile's 16-byte chunks (8 columns each); when the tile has fewer than 32 chunks
+// (RP >= 64) lane groups also split the warp's rows.  Every lane ends up with 32 products per
+// token and tile (16 for RP = 8, whose tile is half as large).
 template <int RP>
 struct ShrinkMap {
     static constexpr int NSUB = (kMaxRank / RP > kMaxSubPerTile) ? kMaxSubPerTile : kMaxRank / RP;
-    static constexpr int C = NSUB * kSubCols;           // columns per tile
-    static constexpr int RPL = RP <= 32 ? 1 : RP / 32;  // rank rows per lane
-    static constexpr int G = RP <= 32 ? 32 / RP : 1;    // lane groups that share the rows
-    static constexpr int CPL = NSUB / G;                // chunks per lane per tile
+    static constexpr int C = NSUB * kSubCols;            // columns per tile
+    static constexpr int CH = 8 * NSUB;                  // chunks per tile
+    static constexpr int CHL = CH < 32 ? CH : 32;        // lanes that split the chunks
+    static constexpr int LG = 32 / CHL;                  // lane groups that split the warp's rows
+    static constexpr int CPL = CH / CHL;                 // chunks per lane
+    static constexpr int RW = RP / 8;                    // rows per warp
+    static constexpr int RPL = RW / LG;                  // rows per lane
+    static_assert(RPL >= 1 && RPL <= kMaxRowsPerLane, "row split");
     uint32_t a_off[CPL][RPL];   // byte offset of (row, chunk) inside the tile, swizzle applied
     uint32_t x_off[CPL];        // byte offset of the chunk inside a token's x piece
     int col0;                   // first column (inside the tile) of this lane's first chunk
+    int row0;                   // first rank row of this lane
     __device__ __forceinline__ void init(int warp, int lane) {
-        const int row = RP <= 32 ? (lane % RP) : lane;
-        const int g = RP <= 32 ? (lane / RP) : 0;
+        const int cl = lane % CHL, rg = lane / CHL;
+        row0 = warp * RW + rg * RPL;
 #pragma unroll
         for (int q = 0; q < CPL; ++q) {
-            const int c = warp * NSUB + g + q * G;
+            const int c = cl + q * CHL;
             x_off[q] = c * 16;
 #pragma unroll
             for (int rr = 0; rr < RPL; ++rr) {
-                const int k = row + 32 * rr;
+                const int k = row0 + rr;
                 a_off[q][rr] = (c >> 3) * (RP * 128) + k * 128 + (((c & 7) ^ (k & 7)) << 4);
             }
         }
-        col0 = (warp * NSUB + g) * 8;
+        col0 = cl * 8;
     }
 };
 
 // CNT (tokens of the unit) is a template parameter: the loops unroll without branches, every
-// load of a chunk can be issued before the first use, and each (row, token, chunk) product
+// load of the tile is issued before the first use, and each (row, token, chunk) product
 // runs as two short chains (even / odd columns) instead of one long one.
 template <int RP, int CNT, bool CHECKED>
 __device__ __forceinline__ void shrink_chunks(const ShrinkMap<RP>& mp, int cols_left, uint32_t tile,
                                               float (&acc)[kMaxRowsPerLane][kTokChunk]) {
     using M = ShrinkMap<RP>;
     const uint32_t xs = tile + kTileBytesMax;
+    uint4 araw[M::CPL][M::RPL], xraw[M::CPL][CNT];
 #pragma unroll
     for (int q = 0; q < M::CPL; ++q) {
-        if (!CHECKED || mp.col0 + q * M::G * 8 < cols_left) {
-            uint4 araw[M::RPL], xraw[CNT];
 #pragma unroll
-            for (int rr = 0; rr < M::RPL; ++rr) araw[rr] = lds128(tile + mp.a_off[q][rr]);
+        for (int rr = 0; rr < M::RPL; ++rr) araw[q][rr] = lds128(tile + mp.a_off[q][rr]);
 #pragma unroll
-            for (int t = 0; t < CNT; ++t) xraw[t] = lds128(xs + t * kXBytesPerTok + mp.x_off[q]);
-            float af[M::RPL][8];
+        for (int t = 0; t < CNT; ++t) xraw[q][t] = lds128(xs + t * kXBytesPerTok + mp.x_off[q]);
+    }
 #pragma unroll
-            for (int rr = 0; rr < M::RPL; ++rr) unpack8(araw[rr], af[rr]);
+    for (int q = 0; q < M::CPL; ++q) {
+        if (!CHECKED || mp.col0 + q * M::CHL * 8 < cols_left) {
+            float xf[CNT][8];
 #pragma unroll
-            for (int t = 0; t < CNT; ++t) {
-                float xf[8];
-                unpack8(xraw[t], xf);
+            for (int t = 0; t < CNT; ++t) unpack8(xraw[q][t], xf[t]);
 #pragma unroll
-                for (int rr = 0; rr < M::RPL; ++rr) {
-                    float e = xf[0] * af[rr][0], o = xf[1] * af[rr][1];
-                    e = fmaf(xf[2], af[rr][2], e); o = fmaf(xf[3], af[rr][3], o);
-                    e = fmaf(xf[4], af[rr][4], e); o = fmaf(xf[5], af[rr][5], o);
-                    e = fmaf(xf[6], af[rr][6], e); o = fmaf(xf[7], af[rr][7], o);
+            for (int rr = 0; rr < M::RPL; ++rr) {
+                float af[8];
+                unpack8(araw[q][rr], af);
+#pragma unroll
+                for (int t = 0; t < CNT; ++t) {
+                    float e = xf[t][0] * af[0], o = xf[t][1] * af[1];
+                    e = fmaf(xf[t][2], af[2], e); o = fmaf(xf[t][3], af[3], o);
+                    e = fmaf(xf[t][4], af[4], e); o = fmaf(xf[t][5], af[5], o);
+                    e = fmaf(xf[t][6], af[6], e); o = fmaf(xf[t][7], af[7], o);
                     acc[rr][t] += e + o;
                 }
             }
@@ -333,54 +330,87 @@ __device__ __forceinline__ void shrink_tile(const Params& p, const StageHdr& h, 
     }
 }
 
-// ---- shrink: end of a task: the CTA's partial m leaves for the workspace (or the caller's m) ----
-template <int MODE, int RP>
-__device__ __forceinline__ void shrink_finish(const Params& p, const Smem& sm, const StageHdr& h,
-                                              float (&acc)[kMaxRowsPerLane][kTokChunk], Ctl& ctl, int warp, int lane) {
-    constexpr int RPL = RP <= 32 ? 1 : RP / 32;
-    constexpr bool kTwoBuffers = RP <= 64;
-    const int row = RP <= 32 ? (lane % RP) : lane;
-    const int g = RP <= 32 ? (lane / RP) : 0;
-    const int tid = warp * 32 + lane;
-    // lanes of different groups hold partial sums of the same rows
+// ---- shrink: end of a task ---------------------------------------------------------------
+// The lanes that split the chunks meet by shuffles; every (row, token) sum of the warp's rows
+// is then complete and one lane per value sends it off: to the workspace as a {value, epoch}
+// word (fused) or to the caller's m (shrink-only).  No warp waits for another.
+//
+// CNT is the token count rounded up to a power of two (tokens beyond the unit's count hold
+// zeros and are not written).  The butterfly runs over the CHL lanes that split the chunks;
+// while a lane holds more than one value each step also halves them (partners swap halves),
+// so a step costs one shuffle per surviving value instead of one per value.
+template <int MODE, int RP, int CNT>
+__device__ __forceinline__ void shrink_finish_cnt(const Params& p, const Smem& sm, const StageHdr& h,
+                                                  const ShrinkMap<RP>& mp, float (&acc)[kMaxRowsPerLane][kTokChunk],
+                                                  int lane) {
+    using M = ShrinkMap<RP>;
+    constexpr int V = M::RPL * CNT;   // values per lane; value v = (row v / CNT, token v % CNT)
+    constexpr int kLog2V = V >= 16 ? 4 : V >= 8 ? 3 : V >= 4 ? 2 : V >= 2 ? 1 : 0;
+    constexpr int kLog2L = M::CHL >= 32 ? 5 : M::CHL >= 16 ? 4 : 3;
+    constexpr int kHalvings = kLog2V < kLog2L ? kLog2V : kLog2L;
+    constexpr int kLeft = V >> kHalvings;                 // values per lane at the end
+    constexpr int kLanesPerValue = M::CHL >> kHalvings;   // lanes that end up with the same values
+    float val[V];
 #pragma unroll
-    for (int d = RP; d < 32; d <<= 1)
+    for (int v = 0; v < V; ++v) val[v] = acc[v / CNT][v % CNT];
+    const int cl = lane % M::CHL;
+    int idx = 0;   // first value this lane holds
 #pragma unroll
-        for (int rr = 0; rr < RPL; ++rr)
+    for (int s = 0; s < kLog2L; ++s) {
+        const int d = M::CHL >> (s + 1);
+        if (s < kHalvings) {
+            const int n = V >> s;                 // values held before this step
+            const bool upper = (cl & d) != 0;     // lower lanes keep the first half, upper lanes the second
 #pragma unroll
-            for (int t = 0; t < kTokChunk; ++t) acc[rr][t] += __shfl_xor_sync(0xffffffffu, acc[rr][t], d);
-    float* part = sm.part + (kTwoBuffers ? ctl.pbuf * (kConsumerWarps * kTokChunk * RP) : 0);
-    if (g == 0) {
-#pragma unroll
-        for (int rr = 0; rr < RPL; ++rr)
-#pragma unroll
-            for (int t = 0; t < kTokChunk; ++t)
-                if (t < h.cnt) part[(warp * kTokChunk + t) * RP + row + 32 * rr] = acc[rr][t];
-    }
-    consumer_sync(sm, ctl);
-    // fixed-order sum over the warps' column slices
-    const int n = h.cnt * RP;
-    for (int idx = tid; idx < n; idx += kConsumerThreads) {
-        const int t = idx / RP, k = idx % RP;
-        float s = 0.f;
-#pragma unroll
-        for (int w = 0; w < kConsumerWarps; ++w) s += part[(w * kTokChunk + t) * RP + k];
-        if (MODE == kFused) {
-            // value and epoch leave in one 64-bit store: no fence, nobody waits for it here
-            p.bk.m_part[part_index(p, h.unit, h.run, t) + k] =
-                ((unsigned long long)sm.epoch << 32) | (unsigned long long)__float_as_uint(s);
+            for (int v = 0; v < V / 2; ++v) {
+                if (v < n / 2) {
+                    const float keep = upper ? val[v + n / 2] : val[v];
+                    const float give = upper ? val[v] : val[v + n / 2];
+                    val[v] = keep + __shfl_xor_sync(0xffffffffu, give, d);
+                }
+            }
+            if (upper) idx += n / 2;
         } else {
-            p.m[(size_t)tok_at(h, t) * p.ldm + k] = s;
+#pragma unroll
+            for (int v = 0; v < kLeft; ++v) val[v] += __shfl_xor_sync(0xffffffffu, val[v], d);
         }
     }
+    // the lane holds the values idx .. idx + kLeft - 1, complete; one lane of each group of equals writes
+    if ((cl & (kLanesPerValue - 1)) == 0) {
+#pragma unroll
+        for (int j = 0; j < kLeft; ++j) {
+            const int rr = (idx + j) / CNT, t = (idx + j) % CNT;
+            if (t < h.cnt) {
+                const int k = mp.row0 + rr;
+                if (MODE == kFused) {
+                    // value and epoch leave in one 64-bit store: no fence, nobody waits for it here
+                    p.bk.m_part[part_index(p, h.unit, h.run, t) + k] =
+                        ((unsigned long long)sm.epoch << 32) | (unsigned long long)__float_as_uint(val[j]);
+                } else {
+                    p.m[(size_t)tok_at(h, t) * p.ldm + k] = val[j];
+                }
+            }
+        }
+    }
+}
+
+template <int MODE, int RP>
+__device__ __forceinline__ void shrink_finish(const Params& p, const Smem& sm, const StageHdr& h,
+                                              const ShrinkMap<RP>& mp, float (&acc)[kMaxRowsPerLane][kTokChunk],
+                                              int warp, int lane) {
+    switch (h.cnt) {
+        case 1: shrink_finish_cnt<MODE, RP, 1>(p, sm, h, mp, acc, lane); break;
+        case 2: shrink_finish_cnt<MODE, RP, 2>(p, sm, h, mp, acc, lane); break;
+        default: shrink_finish_cnt<MODE, RP, 4>(p, sm, h, mp, acc, lane); break;
+    }
     if (MODE != kFused) {
+        // columns beyond this adapter's padded rank are zeros
         const int extra = p.ldm - RP;
-        for (int idx = tid; idx < h.cnt * extra; idx += kConsumerThreads) {
+        for (int idx = warp * 32 + lane; idx < h.cnt * extra; idx += kConsumerThreads) {
             const int t = idx / extra, k = RP + idx % extra;
             p.m[(size_t)tok_at(h, t) * p.ldm + k] = 0.f;
         }
     }
-    if (kTwoBuffers) ctl.pbuf ^= 1; else consumer_sync(sm, ctl);   // the next task must not overwrite what is still being summed
 }
 
 // ---- expand: one tile of B; the result goes straight to y ------------------------------------------
@@ -517,7 +547,7 @@ __device__ __forceinline__ void consume_stage(const Params& p, const Smem& sm, c
             if (lane == 0) mbar_arrive(empty_bar);
             CYC_ADD(ctl.c_tile, t_a);
             CYC_T0(t_b);
-            if (h.flags & kFlagLast) shrink_finish<MODE, RP>(p, sm, h, acc, ctl, warp, lane);
+            if (h.flags & kFlagLast) shrink_finish<MODE, RP>(p, sm, h, maps.s, acc, warp, lane);
             CYC_ADD(ctl.c_fin, t_b);
         }
     } else {
@@ -601,14 +631,12 @@ __global__ void __launch_bounds__(kThreads, 2) bgmv_kernel(const Params p) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     Smem sm;
     sm.slots = smem_u32(smem_raw);
-    sm.part = reinterpret_cast<float*>(smem_raw + kStages * kSlotBytes);
-    sm.m_ring = smem_u32(sm.part + kPartFloats);
-    uint8_t* bars = reinterpret_cast<uint8_t*>(sm.part + kPartFloats) + kMRing * kMRingBytes;
+    sm.m_ring = smem_u32(smem_raw + kStages * kSlotBytes);
+    uint8_t* bars = smem_raw + kStages * kSlotBytes + kMRing * kMRingBytes;
     sm.full = smem_u32(bars);
     sm.empty = sm.full + kStages * 8;
     sm.m_full = sm.empty + kStages * 8;
     sm.m_empty = sm.m_full + kMRing * 8;
-    sm.sync_bar = sm.m_empty + kMRing * 8;
     sm.abort_flag = reinterpret_cast<volatile int*>(bars + kNumBarriers * 8);
     sm.status = p.status;
 
@@ -621,7 +649,6 @@ __global__ void __launch_bounds__(kThreads, 2) bgmv_kernel(const Params p) {
             // a stage that was never filled reads as "nothing follows"
             sts128(sm.slots + s * kSlotBytes + kHdrOffset, (uint32_t)kFlagEnd, 0u, 0u, 0u);
         }
-        mbar_init(sm.sync_bar, kConsumerWarps);
         for (int e = 0; e < kMRing; ++e) {
             mbar_init(sm.m_full + e * 8, 1);
             mbar_init(sm.m_empty + e * 8, kConsumerWarps);
@@ -834,8 +861,6 @@ __global__ void __launch_bounds__(kThreads, 2) bgmv_kernel(const Params p) {
     // ------------------------------- consumer warps -------------------------------
     float acc[kMaxRowsPerLane][kTokChunk];
     Ctl ctl;
-    ctl.pbuf = 0;
-    ctl.sync_phase = 0;
     LaneMaps<RPK> maps;   // per-lane constants of both phases
     maps.init(warp, lane);
     CYC_DECL(c_wait); CYC_DECL(c_hdr); CYC_DECL(c_work);
@@ -850,7 +875,7 @@ __global__ void __launch_bounds__(kThreads, 2) bgmv_kernel(const Params p) {
         CYC_ADD(c_hdr, th);
         if (tid == 0 && it == 0) TRACE(4);
         if (tid == 0) TRACE2(it, 2);
-        if ((h.flags & kFlagEnd) || *sm.abort_flag) { if (tid == 0) { TRACE(5); g_trace_n(it); CYC_OUT(0, c_wait); CYC_OUT(1, c_hdr); CYC_OUT(2, c_work); CYC_OUT(3, ctl.c_tile); CYC_OUT(4, ctl.c_fin); CYC_OUT(5, ctl.c_finw); } break; }
+        if ((h.flags & kFlagEnd) || lds32(smem_u32(const_cast<int*>(sm.abort_flag)))) { if (tid == 0) { TRACE(5); g_trace_n(it); CYC_OUT(0, c_wait); CYC_OUT(1, c_hdr); CYC_OUT(2, c_work); CYC_OUT(3, ctl.c_tile); CYC_OUT(4, ctl.c_fin); CYC_OUT(5, ctl.c_finw); } break; }
         const uint32_t empty_bar = sm.empty + slot * 8;
         CYC_T0(tc);
         consume_stage<MODE, RPK>(p, sm, h, maps, tile, empty_bar, acc, ctl, warp, lane);
