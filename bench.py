@@ -146,6 +146,8 @@ class DeviceWorkload:
         g.manual_seed(wl.seed)
         self.x = {}
         self.y = {}
+        self.grouped = True
+        self._groups = None
         for pool in wl.pools:
             A, B = gen_pool_device(wl, pool, self.dev)
             self.ctx.register_pool(pool.layer, pool.proj, pool.d_in, pool.d_out, wl.ranks, wl.scales, A, B)
@@ -158,13 +160,31 @@ class DeviceWorkload:
                                                           dtype=torch.float32)
         torch.cuda.synchronize()
 
+    def groups(self):
+        """The calls of one step: projections of a layer that do not depend on one another go
+        together (q/k/v read the same activations, so do up/gate); o and down stand alone."""
+        if self._groups is None:
+            by = {}
+            for pool in self.wl.pools:
+                by.setdefault((pool.layer, pool.x_group), []).append(pool)
+            self._groups = [by[k] for k in sorted(by)]
+        return self._groups
+
+    def deltas(self):
+        """Every (layer, proj) delta of the step; enqueue only."""
+        ctx = self.ctx
+        for grp in self.groups():
+            if self.grouped and len(grp) > 1:
+                ctx.lora_delta_group([self.x[(p.layer, p.x_group)] for p in grp], self.ids, [p.layer for p in grp],
+                                     [p.proj for p in grp], [self.y[(p.layer, p.proj)] for p in grp])
+            else:
+                for p in grp:
+                    ctx.lora_delta(self.x[(p.layer, p.x_group)], self.ids, p.layer, p.proj, self.y[(p.layer, p.proj)])
+
     def step(self):
         """bucket once, then every (layer, proj) delta; enqueue only."""
-        ctx, wl = self.ctx, self.wl
-        ctx.bucket(self.ids, wl.n_adapters)
-        for pool in wl.pools:
-            ctx.lora_delta(self.x[(pool.layer, pool.x_group)], self.ids, pool.layer, pool.proj,
-                           self.y[(pool.layer, pool.proj)])
+        self.ctx.bucket(self.ids, self.wl.n_adapters)
+        self.deltas()
 
     def host_adapters(self, pool, adapters):
         """Logical A/B bit patterns of `adapters` of `pool`, regenerated on the device and copied to the host."""
@@ -246,6 +266,7 @@ def run_ours(args):
 
     wl = make_workload(args.config, n_layers=args.layers)
     dw = DeviceWorkload(wl, local)
+    dw.grouped = not args.no_group
     ctx = dw.ctx
     ctx.set_path({"auto": P.PATH_AUTO, "fused": P.PATH_FUSED, "unfused": P.PATH_UNFUSED, "sgmv": P.PATH_SGMV}[args.path])
     n_calls = len(wl.pools)
@@ -270,8 +291,10 @@ def run_ours(args):
         stream.wait_stream(s)
         torch.cuda.synchronize()
         graph = torch.cuda.CUDAGraph()
+        lc0 = ctx.launch_count()
         with torch.cuda.graph(graph):
             dw.step()
+        launches_per_step = ctx.launch_count() - lc0   # kernels recorded in the graph = launched per replay
 
     def one_step():
         if graph is not None:
@@ -297,7 +320,7 @@ def run_ours(args):
     torch.cuda.synchronize()
     launches = ctx.launch_count() - l0
     if graph is not None:
-        launches = args.steps * (n_calls + 1)
+        launches = args.steps * launches_per_step
     total_ms = ev[0].elapsed_time(ev[-1])
     clocks = sampler.stop()
     total_ms = max_over_ranks(total_ms, f"cuda:{local}")
@@ -308,8 +331,7 @@ def run_ours(args):
     # kernel-only timing for the roofline: the delta calls of one step without the bucket kernel,
     # replayed from a CUDA graph like the step itself so that host launch cost does not pace them
     def deltas_only():
-        for pool in wl.pools:
-            ctx.lora_delta(dw.x[(pool.layer, pool.x_group)], dw.ids, pool.layer, pool.proj, dw.y[(pool.layer, pool.proj)])
+        dw.deltas()
 
     ctx.bucket(dw.ids, wl.n_adapters)
     torch.cuda.synchronize()
@@ -334,7 +356,7 @@ def run_ours(args):
         kgraph.replay() if kgraph is not None else deltas_only()
     e1.record()
     torch.cuda.synchronize()
-    kernel_ms = e0.elapsed_time(e1) / (reps * n_calls)
+    kernel_ms = e0.elapsed_time(e1) / (reps * n_calls)   # per (layer, proj) delta, however they are grouped
 
     per_call = [algorithmic_bytes(wl.ids, wl.ranks, p.d_in, p.d_out) for p in wl.pools]
     step_bytes = sum(b["total"] for b in per_call)
@@ -382,7 +404,7 @@ def run_ours(args):
                    config=dict(workload=f"config {args.config} ({wl.name})", n_tok=wl.n_tok, n_adapters=wl.n_adapters,
                                layers=len({p.layer for p in wl.pools}), calls_per_step=n_calls,
                                ranks=sorted({int(r) for r in wl.ranks}), ids=wl.meta.get("ids"),
-                               distinct_adapters=per_call[0]["distinct"], path=args.path, cuda_graph=bool(args.graph),
+                               distinct_adapters=per_call[0]["distinct"], path=args.path, cuda_graph=bool(args.graph), grouped_calls=not args.no_group,
                                l2="inputs larger than L2: a step streams %.2f GB through %d distinct slabs"
                                   % (step_bytes / 1e9, n_calls),
                                multi_gpu="replicas: every rank runs its own batch, no data-path collective"),
@@ -448,6 +470,8 @@ def main():
     ap.add_argument("--graph", type=int, default=1)
     ap.add_argument("--cpu-pools", type=int, default=8, dest="cpu_pools")
     ap.add_argument("--path", default="auto", choices=["auto", "fused", "unfused", "sgmv"])
+    ap.add_argument("--no-group", action="store_true", dest="no_group",
+                    help="one call per projection instead of grouping q/k/v and up/gate")
     ap.add_argument("--no-cpu", action="store_true", dest="no_cpu")
     ap.add_argument("--no-e2e", action="store_true", dest="no_e2e")
     args = ap.parse_args()

@@ -166,6 +166,21 @@ PLORA_API plora_status plora_lora_delta(plora_ctx *ctx, const void *x_dev, const
                               int32_t layer, int32_t proj, float *y_dev, void *stream);
 
 /*
+ * The LoRA delta of several projections that do not depend on one another, in one call (the
+ * paper attaches adapters to the query, key and value generation, the output projection and
+ * the FFN weights of every layer, Section II-A: q, k and v of a layer read the same activations
+ * and can run together, and so can up and gate).  Equivalent to n calls of plora_lora_delta;
+ * projections whose pools have the same shape (d_in, d_out, adapter count, largest rank) share
+ * one kernel launch, which matters at decode sizes where a launch is only a few microseconds
+ * of work.  x_dev[g], layers[g], projs[g], y_dev[g] describe projection g; the arrays are HOST
+ * arrays of length n, 1 <= n <= 4; the x_dev[g] may or may not be the same buffer; the y_dev[g]
+ * must be distinct.  Same bucket rule and errors as plora_lora_delta.
+ */
+PLORA_API plora_status plora_lora_delta_group(plora_ctx *ctx, int32_t n, const void *const *x_dev,
+                                              const int32_t *adapter_ids_dev, int32_t n_tok, const int32_t *layers,
+                                              const int32_t *projs, float *const *y_dev, void *stream);
+
+/*
  * The two halves on their own (Section V-A, strategy E4: m = x A, then y = m B).
  * m_dev is fp32 [n_tok, ldm] on the device, ldm >= plora_pool_max_rank.
  * plora_shrink writes m[t, k] = sum_i x[t, i] A_a[i, k] (unscaled) for k < r_a and 0

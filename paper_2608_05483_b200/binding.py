@@ -29,7 +29,7 @@ PATH_AUTO, PATH_UNFUSED, PATH_FUSED, PATH_SGMV = 0, 1, 2, 3
 
 EXPORTS = (
     "plora_create", "plora_destroy", "plora_pool_slab_bytes", "plora_register_pool", "plora_pool_max_rank",
-    "plora_bucket", "plora_bucket_view", "plora_lora_delta", "plora_shrink", "plora_expand",
+    "plora_bucket", "plora_bucket_view", "plora_lora_delta", "plora_lora_delta_group", "plora_shrink", "plora_expand",
     "plora_lora_delta_host", "plora_lora_delta_noalloc", "plora_set_path", "plora_device_status", "plora_launch_count", "plora_status_string",
 )
 
@@ -78,6 +78,7 @@ def load(build_if_missing: bool = True):
         "plora_bucket": (i32, [vp, vp, i32, i32, vp]),
         "plora_bucket_view": (i32, [vp] + [ctypes.POINTER(vp)] * 5),
         "plora_lora_delta": (i32, [vp, vp, vp, i32, i32, i32, vp, vp]),
+        "plora_lora_delta_group": (i32, [vp, i32, vp, vp, i32, vp, vp, vp, vp]),
         "plora_shrink": (i32, [vp, vp, vp, i32, i32, i32, vp, i32, vp]),
         "plora_expand": (i32, [vp, vp, i32, vp, i32, i32, i32, vp, vp]),
         "plora_lora_delta_host": (i32, [vp, vp, vp, i32, i32, i32, vp, vp]),
@@ -133,6 +134,18 @@ def plora_bucket_view(ctx):
 
 def plora_lora_delta(ctx, x_ptr: int, ids_ptr: int, n_tok: int, layer: int, proj: int, y_ptr: int, stream: int = 0):
     return load().plora_lora_delta(ctx, x_ptr, ids_ptr, n_tok, layer, proj, y_ptr, stream)
+
+
+def plora_lora_delta_group(ctx, x_ptrs, ids_ptr, n_tok, layers, projs, y_ptrs, stream=0):
+    """x_ptrs / y_ptrs: sequences of device pointers; layers / projs: sequences of ints (all of length n)."""
+    n = len(x_ptrs)
+    xs = (ctypes.c_void_p * n)(*x_ptrs)
+    ys = (ctypes.c_void_p * n)(*y_ptrs)
+    ls = (ctypes.c_int32 * n)(*layers)
+    ps = (ctypes.c_int32 * n)(*projs)
+    return load().plora_lora_delta_group(ctx, n, ctypes.cast(xs, ctypes.c_void_p), ids_ptr, n_tok,
+                                         ctypes.cast(ls, ctypes.c_void_p), ctypes.cast(ps, ctypes.c_void_p),
+                                         ctypes.cast(ys, ctypes.c_void_p), stream)
 
 
 def plora_shrink(ctx, x_ptr, ids_ptr, n_tok, layer, proj, m_ptr, ldm, stream=0):
@@ -289,6 +302,12 @@ class Context:
     def lora_delta(self, x, ids, layer, proj, y, stream=None):
         _check(plora_lora_delta(self._h, x.data_ptr(), ids.data_ptr(), int(ids.numel()), layer, proj, y.data_ptr(),
                                 _stream_handle(stream)), "plora_lora_delta")
+
+    def lora_delta_group(self, xs, ids, layers, projs, ys, stream=None):
+        """Independent projections (q/k/v of a layer, up/gate) in one call; same-shape pools share a launch."""
+        _check(plora_lora_delta_group(self._h, [t.data_ptr() for t in xs], ids.data_ptr(), int(ids.numel()),
+                                      list(layers), list(projs), [t.data_ptr() for t in ys], _stream_handle(stream)),
+               "plora_lora_delta_group")
 
     def shrink(self, x, ids, layer, proj, m, stream=None):
         _check(plora_shrink(self._h, x.data_ptr(), ids.data_ptr(), int(ids.numel()), layer, proj, m.data_ptr(),

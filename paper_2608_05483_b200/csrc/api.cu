@@ -145,6 +145,14 @@ plora_status ensure_bucket(plora_ctx* ctx, const int32_t* ids, int32_t n_tok, in
     return do_bucket(ctx, ids, n_tok, n_adapters, st);
 }
 
+cudaError_t launch_bgmv_one(BgmvMode mode, const PoolDev& pool, const BucketDev& bk, int n_tok, const void* x, float* y,
+                            float* m, int ldm, int32_t* status, int sm_count, bool early_tables, cudaStream_t stream,
+                            int* n_launches) {
+    const void* xs[1] = {x};
+    float* ys[1] = {y};
+    return launch_bgmv(mode, &pool, 1, bk, n_tok, xs, ys, m, ldm, status, sm_count, early_tables, stream, n_launches);
+}
+
 plora_status check_call(plora_ctx* ctx, const void* a, const void* ids, int32_t n_tok, const void* b) {
     if (!ctx || n_tok < 0 || n_tok > ctx->max_tokens) return PLORA_ERR_INVALID_ARG;
     if (n_tok > 0 && (!a || !ids || !b)) return PLORA_ERR_INVALID_ARG;
@@ -390,20 +398,61 @@ PLORA_API plora_status plora_lora_delta(plora_ctx* ctx, const void* x, const int
     int nl = 0;
     cudaError_t e = cudaSuccess;
     if (ctx->path == PLORA_PATH_UNFUSED) {
-        e = launch_bgmv(kShrinkOnly, pool->dev, ctx->bk, n_tok, x, nullptr, ctx->m_ws, pool->dev.max_rp, ctx->status_dev,
+        e = launch_bgmv_one(kShrinkOnly, pool->dev, ctx->bk, n_tok, x, nullptr, ctx->m_ws, pool->dev.max_rp, ctx->status_dev,
                         ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl);
         if (e == cudaSuccess)
-            e = launch_bgmv(kExpandOnly, pool->dev, ctx->bk, n_tok, nullptr, y, ctx->m_ws, pool->dev.max_rp,
+            e = launch_bgmv_one(kExpandOnly, pool->dev, ctx->bk, n_tok, nullptr, y, ctx->m_ws, pool->dev.max_rp,
                             ctx->status_dev, ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl);
     } else {
         // a batch shorter than the threshold cannot hold a segment for the tensor-core path
         const bool may_bgmv = ctx->path != PLORA_PATH_SGMV;
         const bool may_sgmv = ctx->bucket_sgmv_min != INT_MAX;
         if (may_bgmv)
-            e = launch_bgmv(kFused, pool->dev, ctx->bk, n_tok, x, y, nullptr, 0, ctx->status_dev, ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl);
+            e = launch_bgmv_one(kFused, pool->dev, ctx->bk, n_tok, x, y, nullptr, 0, ctx->status_dev, ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl);
         if (e == cudaSuccess && may_sgmv)
             e = launch_sgmv(pool->dev, ctx->bk, n_tok, ctx->bucket_sgmv_min, x, y, ctx->status_dev, ctx->sm_count, st, &nl);
     }
+    ctx->launches += nl;
+    return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
+}
+
+PLORA_API plora_status plora_lora_delta_group(plora_ctx* ctx, int32_t n, const void* const* x, const int32_t* ids,
+                                              int32_t n_tok, const int32_t* layers, const int32_t* projs, float* const* y,
+                                              void* stream) {
+    if (!ctx || n < 1 || n > kMaxGroupPools || !x || !y || !layers || !projs) return PLORA_ERR_INVALID_ARG;
+    PoolRec* recs[kMaxGroupPools];
+    for (int g = 0; g < n; ++g) {
+        plora_status rc = check_call(ctx, x[g], ids, n_tok, y[g]);
+        if (rc != PLORA_OK) return rc;
+        recs[g] = find_pool(ctx, layers[g], projs[g]);
+        if (!recs[g]) return PLORA_ERR_NOT_REGISTERED;
+    }
+    if (n_tok == 0) return PLORA_OK;
+    bool same = true;
+    for (int g = 1; g < n; ++g)
+        same = same && recs[g]->dev.d_in == recs[0]->dev.d_in && recs[g]->dev.d_out == recs[0]->dev.d_out &&
+               recs[g]->dev.n_adapters == recs[0]->dev.n_adapters && recs[g]->dev.max_rp == recs[0]->dev.max_rp;
+    if (!same || ctx->path == PLORA_PATH_UNFUSED || ctx->path == PLORA_PATH_SGMV) {
+        // pools of different shape, or a path without a grouped kernel: one projection after the other
+        for (int g = 0; g < n; ++g) {
+            plora_status rc = plora_lora_delta(ctx, x[g], ids, n_tok, layers[g], projs[g], y[g], stream);
+            if (rc != PLORA_OK) return rc;
+        }
+        return PLORA_OK;
+    }
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return PLORA_ERR_CUDA;
+    cudaStream_t st = as_stream(stream);
+    plora_status rc = ensure_bucket(ctx, ids, n_tok, recs[0]->dev.n_adapters, st);
+    if (rc != PLORA_OK) return rc;
+    PoolDev pools[kMaxGroupPools];
+    for (int g = 0; g < n; ++g) pools[g] = recs[g]->dev;
+    int nl = 0;
+    cudaError_t e = launch_bgmv(kFused, pools, n, ctx->bk, n_tok, x, y, nullptr, 0, ctx->status_dev, ctx->sm_count,
+                                ctx->launches_since_bucket++ > 0, st, &nl);
+    if (e == cudaSuccess && ctx->bucket_sgmv_min != INT_MAX)
+        for (int g = 0; g < n && e == cudaSuccess; ++g)
+            e = launch_sgmv(pools[g], ctx->bk, n_tok, ctx->bucket_sgmv_min, x[g], y[g], ctx->status_dev, ctx->sm_count, st, &nl);
     ctx->launches += nl;
     return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
 }
@@ -426,7 +475,7 @@ PLORA_API plora_status plora_shrink(plora_ctx* ctx, const void* x, const int32_t
     ctx->path = saved;
     if (rc != PLORA_OK) return rc;
     int nl = 0;
-    cudaError_t e = launch_bgmv(kShrinkOnly, pool->dev, ctx->bk, n_tok, x, nullptr, m, ldm, ctx->status_dev,
+    cudaError_t e = launch_bgmv_one(kShrinkOnly, pool->dev, ctx->bk, n_tok, x, nullptr, m, ldm, ctx->status_dev,
                                 ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl);
     ctx->launches += nl;
     return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
@@ -449,7 +498,7 @@ PLORA_API plora_status plora_expand(plora_ctx* ctx, const float* m, int32_t ldm,
     ctx->path = saved;
     if (rc != PLORA_OK) return rc;
     int nl = 0;
-    cudaError_t e = launch_bgmv(kExpandOnly, pool->dev, ctx->bk, n_tok, nullptr, y, const_cast<float*>(m), ldm,
+    cudaError_t e = launch_bgmv_one(kExpandOnly, pool->dev, ctx->bk, n_tok, nullptr, y, const_cast<float*>(m), ldm,
                                 ctx->status_dev, ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl);
     ctx->launches += nl;
     return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
@@ -569,10 +618,10 @@ PLORA_API plora_status plora_lora_delta_noalloc(plora_ctx* ctx, const void* x, c
     ctx->path = saved;
     if (rc != PLORA_OK) return rc;
     int nl = 0;
-    cudaError_t e = launch_bgmv(kShrinkOnly, pool->dev, ctx->bk, n_tok, x, nullptr, m, ldm, ctx->status_dev,
+    cudaError_t e = launch_bgmv_one(kShrinkOnly, pool->dev, ctx->bk, n_tok, x, nullptr, m, ldm, ctx->status_dev,
                                 ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl);
     if (e == cudaSuccess)
-        e = launch_bgmv(kExpandOnly, pool->dev, ctx->bk, n_tok, nullptr, y, m, ldm, ctx->status_dev, ctx->sm_count,
+        e = launch_bgmv_one(kExpandOnly, pool->dev, ctx->bk, n_tok, nullptr, y, m, ldm, ctx->status_dev, ctx->sm_count,
                         ctx->launches_since_bucket++ > 0, st, &nl);
     ctx->launches += nl;
     return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;

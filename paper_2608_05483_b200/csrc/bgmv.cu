@@ -46,6 +46,10 @@ constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kProducerWarp = kConsumerWarps;       // issues the copies
 constexpr int kGatherWarp = kConsumerWarps + 1;     // fused mode: assembles the m of the expand tasks
 constexpr int kThreads = kConsumerThreads + 64;
+#ifndef PLORA_EXP_CTAS
+#define PLORA_EXP_CTAS 2
+#endif
+constexpr int kCtasPerSm = PLORA_EXP_CTAS;   // persistent CTAs per SM
 #ifndef PLORA_EXP_STAGES
 #define PLORA_EXP_STAGES 4
 #endif
@@ -63,11 +67,19 @@ constexpr int kPrefetchTasks = 8;   // tasks per CTA whose tiles are prefetched 
 constexpr uint32_t kSuspendHintNs = 20000;   // a waiting thread may sleep this long inside one try_wait
 constexpr long long kWaitCycles = 4000000000ll;   // about two seconds of SM clock
 
+// Projections that do not depend on one another (q, k and v of a layer; up and gate) can share a
+// launch: the task list simply runs over "virtual units" (group, unit).  The pools of a group have
+// the same shape.
+constexpr int kMaxGroup = kMaxGroupPools;
+
 struct Params {
-    PoolDev pool;
+    PoolDev pool;                                // shape (d_in, d_out, max_rp) shared by the group
     BucketDev bk;
-    const uint16_t* x;
-    float* y;
+    int32_t n_groups;
+    const uint8_t* slab_g[kMaxGroup];
+    const AdapterEntry* table_g[kMaxGroup];
+    const uint16_t* x_g[kMaxGroup];
+    float* y_g[kMaxGroup];
     float* m;
     int32_t ldm;
     int32_t n_tok;
@@ -206,16 +218,18 @@ struct StageHdr {
     int32_t rp, r;
     float scale;
     int32_t m_seq;    // fused expand stages: running number of the expand task in this CTA (m-ring entry = m_seq % kMRing)
+    int32_t group;    // which projection of the launch's group (unit = group * n_units + bucket unit)
 };
 
 __device__ __forceinline__ StageHdr read_hdr(uint32_t a) {
     const uint4 q0 = lds128(a), q1 = lds128(a + 16), q2 = lds128(a + 32);
-    const uint32_t q3 = lds32(a + 48);
+    const uint32_t q3 = lds32(a + 48), q4 = lds32(a + 52);
     StageHdr h;
     h.flags = (int)q0.x; h.unit = (int)q0.y; h.run = (int)q0.z; h.tile = (int)q0.w;
     h.cnt = (int)q1.x; h.tok[0] = (int)q1.y; h.tok[1] = (int)q1.z; h.tok[2] = (int)q1.w;
     h.tok[3] = (int)q2.x; h.rp = (int)q2.y; h.r = (int)q2.z; h.scale = __uint_as_float(q2.w);
     h.m_seq = (int)q3;
+    h.group = (int)q4;
     return h;
 }
 __device__ __forceinline__ void sts128(uint32_t a, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
@@ -502,7 +516,7 @@ __device__ __forceinline__ void expand_tile_cnt(const Params& p, const Smem& sm,
     if (mp.rg == 0 && col < p.pool.d_out) {
 #pragma unroll
         for (int t = 0; t < CNT; ++t)
-            red_add_v2(p.y + (size_t)h.tok[t] * p.pool.d_out + col, out[t][0] * h.scale, out[t][1] * h.scale);
+            red_add_v2(p.y_g[h.group] + (size_t)h.tok[t] * p.pool.d_out + col, out[t][0] * h.scale, out[t][1] * h.scale);
     }
 }
 
@@ -627,7 +641,7 @@ __device__ __forceinline__ Task decode_task(int t, int n_shrink_tasks, int runs_
 // padded rank and skips the others: a pool of mixed ranks is served by one launch per rank
 // class present in it, each with loops specialised (and registers allocated) for its rank.
 template <int MODE, int RPK>
-__global__ void __launch_bounds__(kThreads, 2) bgmv_kernel(const Params p) {
+__global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params p) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     Smem sm;
     sm.slots = smem_u32(smem_raw);
@@ -695,8 +709,9 @@ __global__ void __launch_bounds__(kThreads, 2) bgmv_kernel(const Params p) {
             waited = true;
         }
         const int n_units = *p.bk.n_bgmv_units;
-        const int n_shrink = MODE == kExpandOnly ? 0 : n_units * p.runs_a;
-        const int n_tasks = n_shrink + (MODE == kShrinkOnly ? 0 : n_units * p.runs_b);
+        const int n_vunits = n_units * p.n_groups;   // (group, unit) pairs
+        const int n_shrink = MODE == kExpandOnly ? 0 : n_vunits * p.runs_a;
+        const int n_tasks = n_shrink + (MODE == kShrinkOnly ? 0 : n_vunits * p.runs_b);
         const int stride = gridDim.x;
         const unsigned full = 0xffffffffu;
         uint32_t it_base = 0;
@@ -708,8 +723,9 @@ __global__ void __launch_bounds__(kThreads, 2) bgmv_kernel(const Params p) {
             const int my_task = base + lane * stride;
             const bool in_range = my_task < n_tasks;
             const Task mine = decode_task(in_range ? my_task : base, n_shrink, p.runs_a, p.runs_b);
-            const WorkUnit mu = p.bk.bgmv_units[mine.unit];
-            const AdapterEntry me = p.pool.table[mu.adapter];
+            const int my_group = mine.unit / max(n_units, 1);
+            const WorkUnit mu = p.bk.bgmv_units[mine.unit - my_group * n_units];
+            const AdapterEntry me = p.table_g[my_group][mu.adapter];
             const bool has = in_range && me.rp == RPK;   // units of other rank classes belong to other launches
             const int in_batch = min(32, (n_tasks - base + stride - 1) / stride);
             const int C = tile_cols(me.rp);
@@ -718,7 +734,8 @@ __global__ void __launch_bounds__(kThreads, 2) bgmv_kernel(const Params p) {
             const int runs = mine.phase ? p.runs_b : p.runs_a;
             const int nT = tiles_for(d, me.rp);
             const int lo = has ? mine.run * nT / runs : 0, hi = has ? (mine.run + 1) * nT / runs : 0;
-            const uint8_t* src = p.pool.slab + (mine.phase ? me.offB : me.offA);
+            const uint8_t* src = p.slab_g[my_group] + (mine.phase ? me.offB : me.offA);
+            const uint16_t* my_x = p.x_g[my_group];
             if (!waited) {
                 // pull the tiles of this CTA's first tasks towards L2, then join the stream order
                 if (lane < kPrefetchTasks)
@@ -765,7 +782,7 @@ __global__ void __launch_bounds__(kThreads, 2) bgmv_kernel(const Params p) {
                         sts128(dst + kHdrOffset, (uint32_t)flags, (uint32_t)mine.unit, (uint32_t)mine.run, (uint32_t)i);
                         sts128(dst + kHdrOffset + 16, (uint32_t)cnt, (uint32_t)mu.tok[0], (uint32_t)mu.tok[1], (uint32_t)mu.tok[2]);
                         sts128(dst + kHdrOffset + 32, (uint32_t)mu.tok[3], (uint32_t)me.rp, (uint32_t)me.r, __float_as_uint(me.scale));
-                        sts128(dst + kHdrOffset + 48, m_seq, 0u, 0u, 0u);
+                        sts128(dst + kHdrOffset + 48, m_seq, (uint32_t)my_group, 0u, 0u);
 #ifdef PLORA_EXP_NOLOAD
                         mbar_arrive(bar);
                         continue;
@@ -777,7 +794,7 @@ __global__ void __launch_bounds__(kThreads, 2) bgmv_kernel(const Params p) {
                             for (int t = 0; t < kTokChunk; ++t)
                                 if (t < cnt)
                                     bulk_g2s(dst + kTileBytesMax + t * kXBytesPerTok,
-                                             p.x + (size_t)mu.tok[t] * p.pool.d_in + (size_t)i * C, tbytes, bar);
+                                             my_x + (size_t)mu.tok[t] * p.pool.d_in + (size_t)i * C, tbytes, bar);
                         } else if (MODE == kExpandOnly) {
 #pragma unroll
                             for (int t = 0; t < kTokChunk; ++t)   // the caller's m row, rp floats, lands as m[t][0..rp)
@@ -816,8 +833,9 @@ __global__ void __launch_bounds__(kThreads, 2) bgmv_kernel(const Params p) {
         // epoch), sums them in run order into the next m-ring entry and publishes the entry.
         if (MODE != kFused) return;
         const int n_units = *p.bk.n_bgmv_units;
-        const int n_shrink = n_units * p.runs_a;
-        const int n_tasks = n_shrink + n_units * p.runs_b;
+        const int n_vunits = n_units * p.n_groups;
+        const int n_shrink = n_vunits * p.runs_a;
+        const int n_tasks = n_shrink + n_vunits * p.runs_b;
         const int stride = gridDim.x;
         const unsigned full = 0xffffffffu;
         // this CTA's first expand task
@@ -828,8 +846,9 @@ __global__ void __launch_bounds__(kThreads, 2) bgmv_kernel(const Params p) {
             const int my_task = base + lane * stride;
             const bool in_range = my_task < n_tasks;
             const int my_unit = (in_range ? my_task - n_shrink : base - n_shrink) / p.runs_b;
-            const WorkUnit mu = p.bk.bgmv_units[my_unit];
-            const int my_rp = p.pool.table[mu.adapter].rp;
+            const int my_group = my_unit / max(n_units, 1);
+            const WorkUnit mu = p.bk.bgmv_units[my_unit - my_group * n_units];
+            const int my_rp = p.table_g[my_group][mu.adapter].rp;
             const int in_batch = min(32, (n_tasks - base + stride - 1) / stride);
             for (int b = 0; b < in_batch; ++b) {
                 const int rp_b = __shfl_sync(full, my_rp, b);
@@ -941,14 +960,24 @@ cudaError_t bgmv_configure() {
     return cudaSuccess;
 }
 
-cudaError_t launch_bgmv(BgmvMode mode, const PoolDev& pool, const BucketDev& bk, int n_tok, const void* x, float* y,
-                        float* m, int ldm, int32_t* status, int sm_count, bool early_tables, cudaStream_t stream,
-                        int* n_launches) {
+cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const BucketDev& bk, int n_tok,
+                        const void* const* x, float* const* y, float* m, int ldm, int32_t* status, int sm_count,
+                        bool early_tables, cudaStream_t stream, int* n_launches) {
+    if (n_groups < 1 || n_groups > kMaxGroup || (mode != kFused && n_groups != 1)) return cudaErrorInvalidValue;
+    const PoolDev& pool = pools[0];
     Params p;
     p.pool = pool;
     p.bk = bk;
-    p.x = static_cast<const uint16_t*>(x);
-    p.y = y;
+    p.n_groups = n_groups;
+    int rp_mask = 0;
+    for (int g = 0; g < kMaxGroup; ++g) {
+        const int gg = g < n_groups ? g : 0;
+        p.slab_g[g] = pools[gg].slab;
+        p.table_g[g] = pools[gg].table;
+        p.x_g[g] = static_cast<const uint16_t*>(x ? x[gg] : nullptr);
+        p.y_g[g] = y ? y[gg] : nullptr;
+        if (g < n_groups) rp_mask |= pools[g].rp_mask;
+    }
     p.m = m;
     p.ldm = ldm;
     p.n_tok = n_tok;
@@ -959,20 +988,20 @@ cudaError_t launch_bgmv(BgmvMode mode, const PoolDev& pool, const BucketDev& bk,
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     // one launch per padded-rank class present in the pool
     for (int rp = 8; rp <= kMaxRank; rp <<= 1) {
-        if (!(pool.rp_mask & rp)) continue;
+        if (!(rp_mask & rp)) continue;
         // a unit of this class has tiles_for(d, rp) tiles per phase: cut each phase into runs
         p.runs_a = mode == kShrinkOnly ? 1 : clamp_runs(tiles_for(pool.d_in, rp));
         // an expand task pays one round trip for its m before its first tile: give it at least two tiles
         p.runs_b = clamp_runs(tiles_for(pool.d_out, rp) / (mode == kFused ? 2 : 1));
         if (mode == kFused) {
             // the partial-m workspace holds n_units * runs_a * kTokChunk * max_rp words, n_units <= n_tok
-            const size_t per_run = (size_t)n_tok * kTokChunk * pool.max_rp * sizeof(unsigned long long);
+            const size_t per_run = (size_t)n_tok * n_groups * kTokChunk * pool.max_rp * sizeof(unsigned long long);
             while (p.runs_a > 1 && per_run * p.runs_a > bk.m_part_bytes) --p.runs_a;
             if (per_run * p.runs_a > bk.m_part_bytes) return cudaErrorMemoryAllocation;
         }
         // persistent grid: two CTAs per SM, never more CTAs than there can be tasks
-        const long long max_tasks = (long long)n_tok * (p.runs_a + p.runs_b);
-        int grid = 2 * sm_count;
+        const long long max_tasks = (long long)n_tok * n_groups * (p.runs_a + p.runs_b);
+        int grid = kCtasPerSm * sm_count;
         if (grid > max_tasks) grid = (int)max_tasks;
         if (grid < 1) grid = 1;
         cudaLaunchConfig_t cfg{};

@@ -101,9 +101,12 @@ cudaError_t launch_repack(const AdapterEntry* table_dev, const void* const* A_de
 
 enum BgmvMode { kFused = 0, kShrinkOnly = 1, kExpandOnly = 2 };
 // x: bf16 [n_tok, d_in]; y: fp32 [n_tok, d_out] (accumulated); m: fp32 [n_tok, ldm]
-cudaError_t launch_bgmv(BgmvMode mode, const PoolDev& pool, const BucketDev& bk, int n_tok, const void* x, float* y,
-                        float* m, int ldm, int32_t* status, int sm_count, bool early_tables, cudaStream_t stream,
-                        int* n_launches);
+// pools[0 .. n_groups): projections of one launch (same shape; more than one only in fused mode);
+// x / y: per-projection pointers (x unused by the expand-only mode, y by the shrink-only mode)
+constexpr int kMaxGroupPools = 4;
+cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const BucketDev& bk, int n_tok,
+                        const void* const* x, float* const* y, float* m, int ldm, int32_t* status, int sm_count,
+                        bool early_tables, cudaStream_t stream, int* n_launches);
 cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, int sgmv_min_rows, const void* x, float* y,
                         int32_t* status, int sm_count, cudaStream_t stream, int* n_launches);
 // per-device function attributes (dynamic shared memory); called by plora_create

@@ -207,6 +207,45 @@ def test_host_buffer_entry_point():
     r.close()
 
 
+def test_grouped_projections_share_a_launch():
+    # q, k, v of one layer read the same x; o has its own.  Grouped q/k/v = one launch, bit-identical
+    # to three separate calls (every y element still receives exactly one addition).
+    wl = make_workload(2, n_adapters=64, d_model=768, n_layers=1, n_tok=200)
+    ctx = P.Context(wl.n_tok, wl.n_adapters)
+    ids = torch.from_numpy(wl.ids).to(DEV)
+    probs = {}
+    for pool in wl.pools:
+        pr = _problem_from_workload(wl, pool)
+        probs[pool.proj] = pr
+        ctx.register_pool(pool.layer, pool.proj, pool.d_in, pool.d_out, wl.ranks, wl.scales, pr["A"], pr["B"])
+    ctx.set_path(P.PATH_AUTO)
+    ctx.bucket(ids, wl.n_adapters)
+    x_qkv = bits_to_dev(probs[0]["x"])
+    x_o = bits_to_dev(probs[3]["x"])
+    y_sep = {}
+    for proj in (0, 1, 2, 3):
+        y_sep[proj] = torch.from_numpy(probs[proj]["y_in"]).to(DEV)
+        ctx.lora_delta(x_qkv if proj < 3 else x_o, ids, 0, proj, y_sep[proj])
+    y_grp = {proj: torch.from_numpy(probs[proj]["y_in"]).to(DEV) for proj in (0, 1, 2, 3)}
+    n0 = ctx.launch_count()
+    ctx.lora_delta_group([x_qkv, x_qkv, x_qkv], ids, [0, 0, 0], [0, 1, 2], [y_grp[0], y_grp[1], y_grp[2]])
+    assert ctx.launch_count() - n0 == 1
+    ctx.lora_delta_group([x_o], ids, [0], [3], [y_grp[3]])
+    torch.cuda.synchronize()
+    for proj in (0, 1, 2, 3):
+        assert y_grp[proj].cpu().numpy().tobytes() == y_sep[proj].cpu().numpy().tobytes(), proj
+        ref = _oracle(probs[proj], y_in=probs[proj]["y_in"])
+        delta = np.max(np.abs(ref - probs[proj]["y_in"]))
+        assert np.max(np.abs(y_grp[proj].cpu().numpy() - ref)) <= TOL_FP32_PATH * delta + 1e-6 * np.max(np.abs(ref))
+    assert ctx.device_status() == 0
+    # pools of different shape fall back to one launch each; bad arguments are refused
+    assert P.plora_lora_delta_group(ctx.handle, [x_qkv.data_ptr()] * 5, ids.data_ptr(), wl.n_tok, [0] * 5, [0] * 5,
+                                    [y_grp[0].data_ptr()] * 5) == P.ERR_INVALID_ARG
+    assert P.plora_lora_delta_group(ctx.handle, [x_qkv.data_ptr()], ids.data_ptr(), wl.n_tok, [7], [0],
+                                    [y_grp[0].data_ptr()]) == P.ERR_NOT_REGISTERED
+    ctx.close()
+
+
 def test_two_pools_and_bucket_reuse():
     wl = make_workload(2, n_adapters=64, d_model=512, n_layers=2, n_tok=96)
     ctx = P.Context(wl.n_tok, wl.n_adapters)
