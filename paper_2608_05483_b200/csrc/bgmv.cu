@@ -685,11 +685,14 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
         if (tid == 0) TRACE(1);
     }
 
-    if (MODE == kShrinkOnly) {
-        // tokens without an adapter get a zero row of m
+    if (MODE == kShrinkOnly && warp != kProducerWarp) {
+        // tokens without an adapter get a zero row of m (by the warps that have already joined the
+        // stream order: an earlier kernel may still be reading m)
         const int n_active = *p.bk.n_active;
         const long long total = (long long)(p.n_tok - n_active) * p.ldm;
-        for (long long i = (long long)blockIdx.x * kThreads + tid; i < total; i += (long long)gridDim.x * kThreads) {
+        const int wtid = warp < kProducerWarp ? tid : tid - 32;   // index among the threads that take part
+        for (long long i = (long long)blockIdx.x * (kThreads - 32) + wtid; i < total;
+             i += (long long)gridDim.x * (kThreads - 32)) {
             const int pos = n_active + (int)(i / p.ldm);
             p.m[(size_t)p.bk.perm[pos] * p.ldm + (int)(i % p.ldm)] = 0.f;
         }
