@@ -46,14 +46,8 @@ constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kProducerWarp = kConsumerWarps;       // issues the copies
 constexpr int kGatherWarp = kConsumerWarps + 1;     // fused mode: assembles the m of the expand tasks
 constexpr int kThreads = kConsumerThreads + 64;
-#ifndef PLORA_EXP_CTAS
-#define PLORA_EXP_CTAS 2
-#endif
-constexpr int kCtasPerSm = PLORA_EXP_CTAS;   // persistent CTAs per SM
-#ifndef PLORA_EXP_STAGES
-#define PLORA_EXP_STAGES 4
-#endif
-constexpr int kStages = PLORA_EXP_STAGES;
+constexpr int kCtasPerSm = 2;   // persistent CTAs per SM
+constexpr int kStages = 5;
 constexpr int kXBytesPerTok = kMaxSubPerTile * kSubCols * 2;             // x piece of one token for one tile
 constexpr int kHdrOffset = kTileBytesMax + kTokChunk * kXBytesPerTok;
 constexpr int kSlotBytes = kHdrOffset + 128;                             // tile + x pieces + stage header
@@ -63,7 +57,6 @@ constexpr int kMRing = 4;
 constexpr int kMRingBytes = kTokChunk * kMaxRank * 4;
 constexpr int kNumBarriers = 2 * kStages + 2 * kMRing;
 constexpr int kSmemBytes = kStages * kSlotBytes + kMRing * kMRingBytes + kNumBarriers * 8 + 16;
-constexpr int kPrefetchTasks = 8;   // tasks per CTA whose tiles are prefetched to L2 before the stream-order wait
 constexpr uint32_t kSuspendHintNs = 20000;   // a waiting thread may sleep this long inside one try_wait
 constexpr long long kWaitCycles = 4000000000ll;   // about two seconds of SM clock
 
@@ -131,9 +124,6 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
     give_up(abort_flag, status);
 }
-__device__ __forceinline__ void prefetch_l2(const void* src, uint32_t bytes) {
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
-}
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                  "l"(src), "r"(bytes), "r"(bar)
@@ -167,28 +157,6 @@ __device__ __forceinline__ void unpack8(const uint4& v, float* f) {
     f[4] = bf_lo(v.z); f[5] = bf_hi(v.z); f[6] = bf_lo(v.w); f[7] = bf_hi(v.w);
 }
 
-#ifdef PLORA_TRACE
-__device__ long long g_trace[8 * 1024];
-__device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
-__device__ long long g_trace3[320 * 8];
-#define CYC_DECL(v) long long v = 0
-#define CYC_T0(v) const long long v = clock64()
-#define CYC_ADD(acc, t0) acc += clock64() - (t0)
-#define CYC_OUT(k, v) g_trace3[blockIdx.x * 8 + (k)] = (v)
-#define TRACE(slot) g_trace[blockIdx.x * 8 + (slot)] = gtime()
-#define g_trace_n(n) g_trace[blockIdx.x * 8 + 6] = (n)
-__device__ long long g_trace2[320 * 16 * 4];
-#define TRACE2(stage, k) do { if ((stage) < 16) g_trace2[(blockIdx.x * 16 + (stage)) * 4 + (k)] = gtime(); } while (0)
-#else
-#define TRACE(slot)
-#define CYC_DECL(v)
-#define CYC_T0(v)
-#define CYC_ADD(acc, t0)
-#define CYC_OUT(k, v)
-#define g_trace_n(n)
-#define TRACE2(stage, k)
-#endif
-
 struct Smem {
     uint32_t slots;      // shared address of stage 0
     uint32_t full;       // full[kStages] barriers
@@ -199,13 +167,6 @@ struct Smem {
     uint32_t m_empty;    // m_empty[kMRing]: every consumer warp is done with the entry
     int32_t* status;
     uint32_t epoch;      // this launch's epoch (fused mode)
-};
-
-// Per-thread state of the consumer loop (only the experiment build keeps any).
-struct Ctl {
-#ifdef PLORA_TRACE
-    long long c_tile = 0, c_fin = 0, c_finw = 0;
-#endif
 };
 
 // What a stage holds (written by the producer into the stage, read by every consumer warp).
@@ -333,9 +294,6 @@ __device__ __forceinline__ void shrink_tile_cnt(const Params& p, const StageHdr&
 template <int RP>
 __device__ __forceinline__ void shrink_tile(const Params& p, const StageHdr& h, const ShrinkMap<RP>& mp, uint32_t tile,
                                             float (&acc)[kMaxRowsPerLane][kTokChunk]) {
-#ifdef PLORA_EXP_NOCOMPUTE
-    return;
-#endif
     switch (h.cnt) {
         case 1: shrink_tile_cnt<RP, 1>(p, h, mp, tile, acc); break;
         case 2: shrink_tile_cnt<RP, 2>(p, h, mp, tile, acc); break;
@@ -546,7 +504,7 @@ struct LaneMaps {
 template <int MODE, int RP>
 __device__ __forceinline__ void consume_stage(const Params& p, const Smem& sm, const StageHdr& h,
                                               const LaneMaps<RP>& maps, uint32_t tile, uint32_t empty_bar,
-                                              float (&acc)[kMaxRowsPerLane][kTokChunk], Ctl& ctl, int warp, int lane) {
+                                              float (&acc)[kMaxRowsPerLane][kTokChunk], int warp, int lane) {
     if (!(h.flags & kFlagExpand)) {
         if (MODE != kExpandOnly) {
             if (h.flags & kFlagFirst) {
@@ -555,14 +513,10 @@ __device__ __forceinline__ void consume_stage(const Params& p, const Smem& sm, c
 #pragma unroll
                     for (int t = 0; t < kTokChunk; ++t) acc[rr][t] = 0.f;
             }
-            CYC_T0(t_a);
             shrink_tile<RP>(p, h, maps.s, tile, acc);
             __syncwarp();
             if (lane == 0) mbar_arrive(empty_bar);
-            CYC_ADD(ctl.c_tile, t_a);
-            CYC_T0(t_b);
             if (h.flags & kFlagLast) shrink_finish<MODE, RP>(p, sm, h, maps.s, acc, warp, lane);
-            CYC_ADD(ctl.c_fin, t_b);
         }
     } else {
         if (MODE != kShrinkOnly) {
@@ -655,7 +609,6 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
     sm.status = p.status;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    if (tid == 0) TRACE(0);
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(sm.full + s * 8, 1);
@@ -674,15 +627,15 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
     // Everything above may overlap the previous kernel of the stream.  Its results (x, y, m,
     // the epoch, possibly the bucket tables) are read only after grid_dependency_wait().  The
     // producer warp delays that wait: the slab is never written by a kernel, and bucket tables
-    // older than the previous kernel are complete, so it fetches its first task descriptors and
-    // pulls its first tiles into L2 while the previous kernel drains.
+    // older than the previous kernel are complete, so it fetches its first task descriptors while
+    // the previous kernel drains.  (Pulling the first tiles towards L2 at that point was tried
+    // and was slower: it competes with the draining kernel's own loads.)
     if (warp != kProducerWarp) {
         grid_dependency_wait();
         // Signalled only after this CTA has seen the previous kernel complete: when the next kernel
         // of the stream starts, everything older than this kernel is therefore complete.
         grid_launch_dependents();
         sm.epoch = MODE == kFused ? *p.bk.epoch : 0u;
-        if (tid == 0) TRACE(1);
     }
 
     if (MODE == kShrinkOnly && warp != kProducerWarp) {
@@ -719,10 +672,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
         const unsigned full = 0xffffffffu;
         uint32_t it_base = 0;
         uint32_t m_count = 0;   // expand tasks issued so far (fused mode)
-        CYC_DECL(p_batch); CYC_DECL(p_gather); CYC_DECL(p_wait); CYC_DECL(p_issue);
-        CYC_T0(p_begin);
         for (int base = blockIdx.x; base < n_tasks; base += 32 * stride) {
-            CYC_T0(tb0);
             const int my_task = base + lane * stride;
             const bool in_range = my_task < n_tasks;
             const Task mine = decode_task(in_range ? my_task : base, n_shrink, p.runs_a, p.runs_b);
@@ -740,13 +690,9 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
             const uint8_t* src = p.slab_g[my_group] + (mine.phase ? me.offB : me.offA);
             const uint16_t* my_x = p.x_g[my_group];
             if (!waited) {
-                // pull the tiles of this CTA's first tasks towards L2, then join the stream order
-                if (lane < kPrefetchTasks)
-                    for (int i = lo; i < hi; ++i) prefetch_l2(src + (size_t)i * tb, tb);
-                if (lane == 0) TRACE(2);
+                // this CTA's first descriptors are in registers: join the stream order
                 grid_dependency_wait();
                 waited = true;
-                if (lane == 0) TRACE(3);
             }
             if (base == (int)blockIdx.x) sm.epoch = MODE == kFused ? *p.bk.epoch : 0u;
             // first stage number of every lane's task: exclusive prefix sum of the stage counts
@@ -758,14 +704,11 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
             }
             const uint32_t my_it0 = it_base + (uint32_t)(incl - (hi - lo));
             it_base += (uint32_t)__shfl_sync(full, incl, 31);
-            CYC_ADD(p_batch, tb0);
 
             for (int b = 0; b < in_batch; ++b) {
                 // fused mode: the running number of this expand task tells the consumers where its m is
                 const uint32_t m_seq = m_count;
                 if (MODE == kFused && __shfl_sync(full, (int)(has && mine.phase), b)) ++m_count;
-                CYC_T0(tg0);
-                CYC_ADD(p_gather, tg0);
                 if (lane == b) {
                     const int cnt = mu.cnt;
                     // bytes a token adds to a stage besides the tile: its x piece (shrink) or its m row (expand-only)
@@ -776,20 +719,12 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
                         const uint32_t dst = sm.slots + slot * kSlotBytes;
                         const uint32_t bar = sm.full + slot * 8;
                         const uint32_t tbytes = mine.phase ? mbytes : (uint32_t)min(C, d - i * C) * 2u;
-                        TRACE2(it, 0);
-                        CYC_T0(tpw);
                         mbar_wait(sm.empty + slot * 8, ((it / kStages) & 1) ^ 1, sm.abort_flag, p.status);
-                        CYC_ADD(p_wait, tpw);
-                        CYC_T0(tpi);
                         const int flags = (mine.phase ? kFlagExpand : 0) | (i == lo ? kFlagFirst : 0) | (i == hi - 1 ? kFlagLast : 0);
                         sts128(dst + kHdrOffset, (uint32_t)flags, (uint32_t)mine.unit, (uint32_t)mine.run, (uint32_t)i);
                         sts128(dst + kHdrOffset + 16, (uint32_t)cnt, (uint32_t)mu.tok[0], (uint32_t)mu.tok[1], (uint32_t)mu.tok[2]);
                         sts128(dst + kHdrOffset + 32, (uint32_t)mu.tok[3], (uint32_t)me.rp, (uint32_t)me.r, __float_as_uint(me.scale));
                         sts128(dst + kHdrOffset + 48, m_seq, (uint32_t)my_group, 0u, 0u);
-#ifdef PLORA_EXP_NOLOAD
-                        mbar_arrive(bar);
-                        continue;
-#endif
                         mbar_arrive_expect_tx(bar, tb + (uint32_t)cnt * tbytes);
                         bulk_g2s(dst, src + (size_t)i * tb, tb, bar);
                         if (!mine.phase) {
@@ -804,20 +739,11 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
                                 if (t < cnt)
                                     bulk_g2s(dst + kTileBytesMax + t * mbytes, p.m + (size_t)mu.tok[t] * p.ldm, mbytes, bar);
                         }
-                        TRACE2(it, 1);
-                        CYC_ADD(p_issue, tpi);
                     }
                 }
                 __syncwarp();
             }
         }
-#ifdef PLORA_TRACE
-        for (int dlt = 16; dlt > 0; dlt >>= 1) {
-            p_wait += __shfl_xor_sync(0xffffffffu, p_wait, dlt);
-            p_issue += __shfl_xor_sync(0xffffffffu, p_issue, dlt);
-        }
-        if (lane == 0) { CYC_OUT(6, p_issue); CYC_OUT(7, clock64() - p_begin); }
-#endif
         if (!waited) grid_dependency_wait();
         if (lane == 0) {   // tell the consumers that nothing follows
             const uint32_t it = it_base;
@@ -882,27 +808,16 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
 
     // ------------------------------- consumer warps -------------------------------
     float acc[kMaxRowsPerLane][kTokChunk];
-    Ctl ctl;
     LaneMaps<RPK> maps;   // per-lane constants of both phases
     maps.init(warp, lane);
-    CYC_DECL(c_wait); CYC_DECL(c_hdr); CYC_DECL(c_work);
     for (uint32_t it = 0;; ++it) {
         const uint32_t slot = it % kStages;
-        CYC_T0(tw);
         mbar_wait(sm.full + slot * 8, (it / kStages) & 1, sm.abort_flag, p.status);
-        CYC_ADD(c_wait, tw);
-        CYC_T0(th);
         const uint32_t tile = sm.slots + slot * kSlotBytes;
         const StageHdr h = read_hdr(tile + kHdrOffset);
-        CYC_ADD(c_hdr, th);
-        if (tid == 0 && it == 0) TRACE(4);
-        if (tid == 0) TRACE2(it, 2);
-        if ((h.flags & kFlagEnd) || lds32(smem_u32(const_cast<int*>(sm.abort_flag)))) { if (tid == 0) { TRACE(5); g_trace_n(it); CYC_OUT(0, c_wait); CYC_OUT(1, c_hdr); CYC_OUT(2, c_work); CYC_OUT(3, ctl.c_tile); CYC_OUT(4, ctl.c_fin); CYC_OUT(5, ctl.c_finw); } break; }
+        if ((h.flags & kFlagEnd) || lds32(smem_u32(const_cast<int*>(sm.abort_flag)))) break;
         const uint32_t empty_bar = sm.empty + slot * 8;
-        CYC_T0(tc);
-        consume_stage<MODE, RPK>(p, sm, h, maps, tile, empty_bar, acc, ctl, warp, lane);
-        CYC_ADD(c_work, tc);
-        if (tid == 0) TRACE2(it, 3);
+        consume_stage<MODE, RPK>(p, sm, h, maps, tile, empty_bar, acc, warp, lane);
     }
     if (MODE == kFused && tid == 0) {
         // the last CTA to finish opens the next epoch: words written by this launch can never
@@ -938,18 +853,6 @@ KernelFn pick_kernel(BgmvMode mode, int rp) {
 int clamp_runs(int tiles) { return tiles < 1 ? 1 : (tiles > kMaxRuns ? kMaxRuns : tiles); }
 
 }  // namespace
-
-#ifdef PLORA_TRACE
-extern "C" __attribute__((visibility("default"))) int plora_debug_trace(long long* host, int n) {
-    return (int)cudaMemcpyFromSymbol(host, g_trace, sizeof(long long) * n);
-}
-extern "C" __attribute__((visibility("default"))) int plora_debug_trace3(long long* host, int n) {
-    return (int)cudaMemcpyFromSymbol(host, g_trace3, sizeof(long long) * n);
-}
-extern "C" __attribute__((visibility("default"))) int plora_debug_trace2(long long* host, int n) {
-    return (int)cudaMemcpyFromSymbol(host, g_trace2, sizeof(long long) * n);
-}
-#endif
 
 cudaError_t bgmv_configure() {
     const int modes[3] = {kFused, kShrinkOnly, kExpandOnly};
