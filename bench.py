@@ -39,8 +39,9 @@ FALLBACK_HBM_GBS = 6650.0   # used only when MEASURED_PEAKS.json is absent
 
 # DRAM bytes per launch of the dominant kernel from the committed ncu captures
 # (profiles/*.md say which capture each number comes from); None = not captured.
+# Per (layer, proj) delta; the roofline entry scales it to the average launch (a launch may carry a group).
 NCU_TRAFFIC_BYTES = {
-    "decode7b": 40.45e6,   # profiles/bgmv_fused_config2_decode7b.md (2-layer capture, same launch shape)
+    "decode7b": 40.19e6,   # profiles/bgmv_fused_config2_decode7b.md: (116.47 + 3.81 + 40.37 + 0.12) MB over q/k/v + o
     "prefill": 628.6e6,    # profiles/sgmv_config4_prefill.md
 }
 
@@ -356,17 +357,28 @@ def run_ours(args):
         kgraph.replay() if kgraph is not None else deltas_only()
     e1.record()
     torch.cuda.synchronize()
-    kernel_ms = e0.elapsed_time(e1) / (reps * n_calls)   # per (layer, proj) delta, however they are grouped
+    deltas_ms = e0.elapsed_time(e1) / reps               # all delta launches of one step
+    kernel_ms = deltas_ms / n_calls                        # per (layer, proj) delta, however they are grouped
+    lc1 = ctx.launch_count()
+    deltas_only()
+    torch.cuda.synchronize()
+    delta_launches = ctx.launch_count() - lc1              # kernel launches that carry the step's deltas
 
     per_call = [algorithmic_bytes(wl.ids, wl.ranks, p.d_in, p.d_out) for p in wl.pools]
     step_bytes = sum(b["total"] for b in per_call)
     step_adapter_bytes = sum(b["adapter"] for b in per_call)
     peaks = measured_peaks()
-    achieved = step_bytes / n_calls / (kernel_ms * 1e-3) / 1e9
+    # algorithmic bytes per launch / average launch duration, over the step's delta launches (a launch
+    # carries one projection or a group of independent ones): equal to step bytes / their total time
+    bytes_per_launch = step_bytes / delta_launches
+    launch_us = deltas_ms * 1e3 / delta_launches
+    achieved = bytes_per_launch / (launch_us * 1e-6) / 1e9
+    traffic = NCU_TRAFFIC_BYTES.get(wl.name)
     roofline = dict(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s", frac=achieved / peaks["hbm_gbs"],
-                    traffic=NCU_TRAFFIC_BYTES.get(wl.name), kernel="bgmv_kernel (fused shrink+expand)",
-                    peak_source=peaks["source"], avg_launch_us=kernel_ms * 1e3,
-                    algorithmic_bytes_per_launch=step_bytes / n_calls,
+                    traffic=None if traffic is None else traffic * n_calls / delta_launches,
+                    kernel="sgmv_kernel (tensor-core segmented GEMM)" if wl.name == "prefill" else "bgmv_kernel (fused shrink+expand)",
+                    peak_source=peaks["source"], avg_launch_us=launch_us, launches_per_step=delta_launches,
+                    per_projection_us=kernel_ms * 1e3, algorithmic_bytes_per_launch=bytes_per_launch,
                     adapter_bytes_only_gbs=step_adapter_bytes / n_calls / (kernel_ms * 1e-3) / 1e9,
                     step_gbs=step_bytes / (ms_per_step * 1e-3) / 1e9)
 
