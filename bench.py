@@ -93,7 +93,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except Exception:
@@ -209,27 +209,36 @@ def bits_of(t):
 # ----------------------------------------------------------------------------------
 # the CPU oracle on a bounded sample (also a full-size parity check of sampled pools)
 # ----------------------------------------------------------------------------------
-def oracle_sample(dw: DeviceWorkload, n_pools: int, check_gpu: bool):
+def oracle_sample(dw: DeviceWorkload, n_pools: int, check_gpu: bool, target_s: float = 0.0):
+    """Times the oracle on `n_pools` (layer, proj) calls of the step at full size.  When one pass
+    over them takes less than `target_s`, every call is repeated (same inputs) so that the whole
+    sample is about `target_s` of CPU work; returns the time of ONE pass (the mean)."""
     import oracle
     wl = dw.wl
     torch = dw.torch
     pools = wl.pools[:: max(1, len(wl.pools) // n_pools)][:n_pools]
     distinct = wl.distinct_adapters()
-    cpu_s, max_err = 0.0, 0.0
-    for pool in pools:
+    cpu_s, max_err, repeats = 0.0, 0.0, 1
+    for i, pool in enumerate(pools):
         A, B = dw.host_adapters(pool, distinct)
         x = bits_of(dw.x[(pool.layer, pool.x_group)])
         y_in = dw.y[(pool.layer, pool.proj)].cpu().numpy().copy()
         t0 = time.perf_counter()
         ref = oracle.lora_delta(x, wl.ids, wl.ranks, wl.scales, A, B, pool.d_out, y_in)
-        cpu_s += time.perf_counter() - t0
+        first = time.perf_counter() - t0
+        if i == 0 and target_s > 0:
+            repeats = int(max(1, min(200, round(target_s / max(first * len(pools), 1e-6)))))
+        t0 = time.perf_counter()
+        for _ in range(repeats - 1):
+            oracle.lora_delta(x, wl.ids, wl.ranks, wl.scales, A, B, pool.d_out, y_in)
+        cpu_s += (first + time.perf_counter() - t0) / repeats
         if check_gpu:
             y = dw.y[(pool.layer, pool.proj)].clone()
             dw.ctx.lora_delta(dw.x[(pool.layer, pool.x_group)], dw.ids, pool.layer, pool.proj, y)
             torch.cuda.synchronize()
             delta_scale = float(np.max(np.abs(ref - y_in)))
             max_err = max(max_err, float(np.max(np.abs(y.cpu().numpy() - ref)) / delta_scale))
-    return pools, cpu_s, max_err, oracle.threads()
+    return pools, cpu_s, max_err, oracle.threads(), repeats
 
 
 # ----------------------------------------------------------------------------------
@@ -276,11 +285,12 @@ def run_ours(args):
     cpu = None
     parity = None
     if rank == 0 and not args.no_cpu:
-        pools, cpu_s, parity, threads = oracle_sample(dw, args.cpu_pools, check_gpu=True)
+        pools, cpu_s, parity, threads, repeats = oracle_sample(dw, args.cpu_pools, check_gpu=True,
+                                                               target_s=args.cpu_seconds)
         scaled = cpu_s * n_calls / len(pools)
         cpu = dict(value=wl.n_tok / scaled, unit="tokens/s", cores=threads, kind="oracle",
                    sample=f"{len(pools)} of {n_calls} (layer, proj) calls at full size ({wl.n_tok} tokens), "
-                          f"{cpu_s:.2f} s of oracle time scaled to the whole step")
+                          f"each run {repeats}x: {cpu_s * repeats:.1f} s of oracle time, mean pass scaled to the whole step")
 
     stream = torch.cuda.current_stream()
     graph = None
@@ -351,7 +361,7 @@ def run_ours(args):
         kgraph.replay() if kgraph is not None else deltas_only()
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    reps = max(3, args.steps)
+    reps = max(3, min(args.steps, 50))
     e0.record()
     for _ in range(reps):
         kgraph.replay() if kgraph is not None else deltas_only()
@@ -474,13 +484,15 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4, 5])
     ap.add_argument("--layers", type=int, default=None)
     ap.add_argument("--graph", type=int, default=1)
-    ap.add_argument("--cpu-pools", type=int, default=8, dest="cpu_pools")
+    ap.add_argument("--cpu-pools", type=int, default=64, dest="cpu_pools")
+    ap.add_argument("--cpu-seconds", type=float, default=10.0, dest="cpu_seconds",
+                    help="target CPU time of the oracle sample (cpu_baseline leg)")
     ap.add_argument("--path", default="auto", choices=["auto", "fused", "unfused", "sgmv"])
     ap.add_argument("--no-group", action="store_true", dest="no_group",
                     help="one call per projection instead of grouping q/k/v and up/gate")
