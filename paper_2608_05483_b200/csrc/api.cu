@@ -208,7 +208,8 @@ PLORA_API plora_status plora_create(plora_ctx** out, int device, int32_t max_tok
     const size_t o_m = o_sg + up(T * sizeof(WorkUnit));
     const size_t o_part = o_m + up(T * kMaxRank * 4);
     const size_t part_bytes = up(T * 8192 > ((size_t)16 << 20) ? T * 8192 : ((size_t)16 << 20));
-    const size_t total = o_part + part_bytes;
+    const size_t o_cls = o_part + part_bytes;
+    const size_t total = o_cls + up(T * kMaxGroupPools * 4);
     uint8_t* blk = nullptr;
     if (cudaMalloc(&blk, total) != cudaSuccess) { delete ctx; return PLORA_ERR_WORKSPACE; }
     if (cudaMemset(blk, 0, total) != cudaSuccess) { cudaFree(blk); delete ctx; return PLORA_ERR_CUDA; }
@@ -229,6 +230,8 @@ PLORA_API plora_status plora_create(plora_ctx** out, int device, int32_t max_tok
     ctx->bk.m_part_bytes = part_bytes;
     ctx->bk.epoch = (uint32_t*)(scal + 16);
     ctx->bk.exit_count = (uint32_t*)(scal + 17);
+    ctx->bk.cls_start = scal + 24;
+    ctx->bk.cls_list = (int32_t*)(blk + o_cls);
     {
         const uint32_t one = 1;
         if (cudaMemcpy(ctx->bk.epoch, &one, 4, cudaMemcpyHostToDevice) != cudaSuccess) {

@@ -78,6 +78,7 @@ struct Params {
     int32_t n_tok;
     int32_t runs_a, runs_b;   // tasks per unit in the shrink / expand phase
     int32_t early_tables;     // the bucket tables were complete before the previous kernel of the stream began
+    int32_t by_class;         // the launch walks its class's part of bk.cls_list (pools of mixed ranks)
     int32_t* status;
 };
 
@@ -554,14 +555,21 @@ __device__ __forceinline__ bool partial_sum(uint32_t epoch, const unsigned long 
     asm volatile("st.shared.f32 [%0], %1;" ::"r"(dst), "f"(s) : "memory");
     return ok;
 }
+// The words of up to kGatherDepth values per lane are requested before the first of them is
+// used: a unit's m costs one round trip to L2 per 32 * kGatherDepth values, not one per 32.
+constexpr int kGatherDepth = 1;
 __device__ __forceinline__ bool gather_m(const Params& p, uint32_t epoch, int unit, int cnt, int rp, int lane,
                                          uint32_t mdst) {
     bool ok = true;
     const int n = cnt * rp;
-    for (int idx = lane; idx < n; idx += 32) {
-        unsigned long long w[kMaxRuns];
-        partial_load(p, epoch, partial_src(p, unit, idx, rp), w);
-        ok = partial_sum(epoch, w, mdst + idx * 4) && ok;
+    for (int i0 = lane; i0 < n; i0 += 32 * kGatherDepth) {
+        unsigned long long w[kGatherDepth][kMaxRuns];
+#pragma unroll
+        for (int q = 0; q < kGatherDepth; ++q)
+            if (i0 + q * 32 < n) partial_load(p, epoch, partial_src(p, unit, i0 + q * 32, rp), w[q]);
+#pragma unroll
+        for (int q = 0; q < kGatherDepth; ++q)
+            if (i0 + q * 32 < n) ok = partial_sum(epoch, w[q], mdst + (i0 + q * 32) * 4) && ok;
     }
     return ok;
 }
@@ -589,6 +597,96 @@ __device__ __forceinline__ Task decode_task(int t, int n_shrink_tasks, int runs_
         k.run = t - k.unit * runs_b;
     }
     return k;
+}
+
+// The (group, unit) pairs a launch walks: all of them (pools of one rank), or its class's part
+// of the list the classify pass wrote.  An entry is group * n_units + unit.
+struct ClassList {
+    const int32_t* list;   // nullptr: the identity
+    int n;
+    __device__ __forceinline__ int at(int i) const { return list ? list[i] : i; }
+};
+template <int RPK>
+__device__ __forceinline__ ClassList class_list(const Params& p, int n_units) {
+    constexpr int kClass = RPK == 8 ? 0 : RPK == 16 ? 1 : RPK == 32 ? 2 : RPK == 64 ? 3 : 4;
+    ClassList c;
+    if (p.by_class) {
+        const int lo = p.bk.cls_start[kClass], hi = p.bk.cls_start[kClass + 1];
+        c.list = p.bk.cls_list + lo;
+        c.n = hi - lo;
+    } else {
+        c.list = nullptr;
+        c.n = n_units * p.n_groups;
+    }
+    return c;
+}
+
+// Classify pass (pools of mixed ranks): sorts the (group, unit) pairs of a call by the padded
+// rank of the unit's adapter in that group's pool, keeping their order inside a class, so
+// that every class launch gets a dense list and an even share of work per CTA.  One CTA.
+constexpr int kClassifyThreads = 1024;
+__device__ __forceinline__ int class_of(const Params& p, int v, int n_units) {
+    const int g = v / n_units, u = v - g * n_units;
+    const int rp = p.table_g[g][p.bk.bgmv_units[u].adapter].rp;
+    return __ffs(rp) - 4;   // 8 -> 0, 16 -> 1, ...
+}
+__global__ void __launch_bounds__(kClassifyThreads) classify_kernel(const Params p) {
+    __shared__ int total[kRankClasses], base[kRankClasses];
+    __shared__ int warp_cnt[kClassifyThreads / 32][kRankClasses];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    grid_dependency_wait();
+    grid_launch_dependents();
+    const int n_units = *p.bk.n_bgmv_units;
+    const int n_v = n_units * p.n_groups;
+    if (tid < kRankClasses) total[tid] = 0;
+    __syncthreads();
+    int local[kRankClasses] = {0, 0, 0, 0, 0};
+    for (int v = tid; v < n_v; v += kClassifyThreads) {
+        const int c = class_of(p, v, n_units);
+#pragma unroll
+        for (int cc = 0; cc < kRankClasses; ++cc) local[cc] += (c == cc);
+    }
+#pragma unroll
+    for (int cc = 0; cc < kRankClasses; ++cc) {
+        int s = local[cc];
+        for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
+        if (lane == 0 && s) atomicAdd(&total[cc], s);
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int run = 0;
+        for (int cc = 0; cc < kRankClasses; ++cc) {
+            base[cc] = run;
+            p.bk.cls_start[cc] = run;
+            run += total[cc];
+        }
+        p.bk.cls_start[kRankClasses] = run;
+    }
+    __syncthreads();
+    for (int v0 = 0; v0 < n_v; v0 += kClassifyThreads) {
+        const int v = v0 + tid;
+        const int c = v < n_v ? class_of(p, v, n_units) : -1;
+        int rank = 0;
+#pragma unroll
+        for (int cc = 0; cc < kRankClasses; ++cc) {
+            const unsigned mask = __ballot_sync(0xffffffffu, c == cc);
+            if (lane == 0) warp_cnt[warp][cc] = __popc(mask);
+            if (c == cc) rank = __popc(mask & ((1u << lane) - 1u));
+        }
+        __syncthreads();
+        if (c >= 0) {
+            int before = 0;
+            for (int w = 0; w < warp; ++w) before += warp_cnt[w][c];
+            p.bk.cls_list[base[c] + before + rank] = v;
+        }
+        __syncthreads();
+        if (tid < kRankClasses) {
+            int add = 0;
+            for (int w = 0; w < kClassifyThreads / 32; ++w) add += warp_cnt[w][tid];
+            base[tid] += add;
+        }
+        __syncthreads();
+    }
 }
 
 // One instantiation per padded rank RPK.  The kernel handles the units whose adapter has that
@@ -665,7 +763,8 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
             waited = true;
         }
         const int n_units = *p.bk.n_bgmv_units;
-        const int n_vunits = n_units * p.n_groups;   // (group, unit) pairs
+        const ClassList cl = class_list<RPK>(p, n_units);   // the (group, unit) pairs of this launch
+        const int n_vunits = cl.n;
         const int n_shrink = MODE == kExpandOnly ? 0 : n_vunits * p.runs_a;
         const int n_tasks = n_shrink + (MODE == kShrinkOnly ? 0 : n_vunits * p.runs_b);
         const int stride = gridDim.x;
@@ -675,7 +774,8 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
         for (int base = blockIdx.x; base < n_tasks; base += 32 * stride) {
             const int my_task = base + lane * stride;
             const bool in_range = my_task < n_tasks;
-            const Task mine = decode_task(in_range ? my_task : base, n_shrink, p.runs_a, p.runs_b);
+            Task mine = decode_task(in_range ? my_task : base, n_shrink, p.runs_a, p.runs_b);
+            mine.unit = cl.at(mine.unit);   // group * n_units + unit
             const int my_group = mine.unit / max(n_units, 1);
             const WorkUnit mu = p.bk.bgmv_units[mine.unit - my_group * n_units];
             const AdapterEntry me = p.table_g[my_group][mu.adapter];
@@ -762,7 +862,8 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
         // epoch), sums them in run order into the next m-ring entry and publishes the entry.
         if (MODE != kFused) return;
         const int n_units = *p.bk.n_bgmv_units;
-        const int n_vunits = n_units * p.n_groups;
+        const ClassList cl = class_list<RPK>(p, n_units);
+        const int n_vunits = cl.n;
         const int n_shrink = n_vunits * p.runs_a;
         const int n_tasks = n_shrink + n_vunits * p.runs_b;
         const int stride = gridDim.x;
@@ -774,7 +875,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
         for (int base = t; base < n_tasks; base += 32 * stride) {
             const int my_task = base + lane * stride;
             const bool in_range = my_task < n_tasks;
-            const int my_unit = (in_range ? my_task - n_shrink : base - n_shrink) / p.runs_b;
+            const int my_unit = cl.at((in_range ? my_task - n_shrink : base - n_shrink) / p.runs_b);
             const int my_group = my_unit / max(n_units, 1);
             const WorkUnit mu = p.bk.bgmv_units[my_unit - my_group * n_units];
             const int my_rp = p.table_g[my_group][mu.adapter].rp;
@@ -892,6 +993,20 @@ cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
+    p.by_class = (rp_mask & (rp_mask - 1)) != 0;   // more than one rank class in the call's pools
+    p.runs_a = p.runs_b = 1;
+    if (p.by_class) {
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3(1);
+        cfg.blockDim = dim3(kClassifyThreads);
+        cfg.stream = stream;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        const cudaError_t e = cudaLaunchKernelEx(&cfg, classify_kernel, p);
+        ++*n_launches;
+        if (e != cudaSuccess) return e;
+        p.early_tables = 0;   // the first class launch reads what the classify pass has just written
+    }
     // one launch per padded-rank class present in the pool
     for (int rp = 8; rp <= kMaxRank; rp <<= 1) {
         if (!(rp_mask & rp)) continue;

@@ -91,7 +91,12 @@ struct BucketDev {
     size_t m_part_bytes;
     uint32_t* epoch;        // launch epoch, advanced by the last CTA of every fused launch (starts at 1)
     uint32_t* exit_count;   // CTAs of the running launch that have finished
+    // pools of mixed ranks: the (projection, unit) pairs of a call sorted by padded-rank class, so
+    // that the launch of a class walks only its own units (written by the classify pass)
+    int32_t* cls_list;      // kMaxGroupPools * max_tokens entries: projection * n_units + unit
+    int32_t* cls_start;     // kRankClasses + 1 offsets into cls_list
 };
+constexpr int kRankClasses = 5;   // padded ranks 8, 16, 32, 64, 128
 
 // Launchers (each returns the cudaError_t of its launch).
 cudaError_t launch_bucket(const int32_t* ids, int n_tok, int n_adapters, int sgmv_min_rows, int sgmv_min_tiles,
