@@ -6,68 +6,166 @@
 //     m [rows, rp]    = X [rows, d_in] * A          bf16 x bf16 -> fp32   (K = d_in)
 //     y [rows, d_out] += s * m * B                  fp32 m carried as bf16 hi + lo, two products
 //
-// The path is bound by HBM traffic on the activations (x read once, y updated once), not by the
-// tensor pipe, so the kernel is organised around keeping copies in flight: a multi-stage cp.async
-// ring feeds warp-level mma.sync (m16n8k16, bf16 in, fp32 accumulate) from shared memory in the
-// slab's swizzled sub-tile layout, and y is updated with one vector reduction per element.
-// The intermediate m never leaves the SM: it is reduced in shared memory, scaled in fp32 and
-// split into bf16 hi + lo (error ~2^-17 relative), which become the A operand of the expand.
+// Both GEMMs are issued as tcgen05.mma (M = 128, accumulators in tensor memory) by one thread
+// of the CTA; the operands reach shared memory without passing through registers:
+//
+//   - the x rows of a tile are gathered by token index with the tensor-map copy in gather mode
+//     (four rows of 64 columns per instruction) straight into the 128-byte-swizzled K-major
+//     operand layout; the matching [rp][64] sub-tile of A^T, stored in the slab in that very
+//     layout, arrives with one bulk copy;
+//   - in the expand the [rp][64] sub-tiles of B are the MN-major operand, again as they sit in
+//     the slab;
+//   - four epilogue warps read the shrink result from tensor memory, scale it, split it into
+//     bf16 hi + lo (error ~2^-17 relative) and store it as the K-major operand of the expand;
+//     they then drain every 64-column block of the expand result: transposed through a small
+//     per-warp staging buffer so that a warp adds whole 256-byte row pieces to y with vector
+//     reductions (one addition per element of y, so the result is bit-reproducible).
+//
+// Roles: warp 0 issues the copies, warp 1 owns the tensor memory and issues the MMAs, warps 2-5
+// are the epilogue.  Stages (x block + weight sub-tile) cycle through a ring guarded by
+// full / empty mbarriers; the MMA thread releases a stage with tcgen05.commit.  The path is
+// bound by HBM traffic on the activations (x read once, y updated once), not by the tensor
+// pipe.  Every wait is bounded: when one runs out the kernel records PLORA_ERR_TIMEOUT, every
+// role leaves its loop, and the tensor memory is freed before the CTA exits.
+#include <cuda.h>
+
 #include "plora_internal.cuh"
 
 namespace plora {
 
 namespace {
 
-constexpr int kRows = kSgmvRows;          // rows of a tile (64)
-constexpr int kWarps = 8;
-constexpr int kThreads = kWarps * 32;
-constexpr int kStages = 4;
+constexpr int kRows = kSgmvRows;          // rows of a tile = M of the MMAs (128)
 constexpr int kKC = kSubCols;             // K (or N) columns per stage = one slab sub-tile (64)
-constexpr int kXStageBytes = kRows * kKC * 2;              // 8 KiB of x per stage
-// Shared memory is sized for the pool's largest padded rank R (at least 16):
-//   kStages x (x stage + one [R][64] weight sub-tile), m hi and m lo [64][R] bf16 with a padded
-//   row pitch, and the tile's token indices.
-__host__ __device__ inline int w_stage_bytes(int R) { return R * kKC * 2; }
+constexpr int kXStageBytes = kRows * kKC * 2;              // 16 KiB of x per stage
+constexpr int kThreads = 6 * 32;
+constexpr int kProducerWarp = 0, kMmaWarp = 1, kEpiWarps = 4;   // warps 2..5 are the epilogue
+constexpr int kMaxStages = 8;
+constexpr int kD2Bufs = 4;                // expand accumulators in flight (64 columns each)
+constexpr int kTmemCols = 512;            // columns [0, 128): shrink result; [128, 384): expand blocks
+constexpr int kTmemD2 = 128;
+constexpr int kStagePitch = kKC * 4 + 16;                  // row pitch of the epilogue staging buffer
+constexpr int kStagingBytes = kEpiWarps * 32 * kStagePitch;
+constexpr int kSmemBudget = 227 * 1024;
+constexpr long long kWaitCycles = 4000000000ll;            // about two seconds of SM clock
+
+// Shared memory, sized for R = max(16, largest padded rank of the pool):
+//   ring of n_stages x (x block 16 KiB + weight sub-tile R x 128 B)      1024-byte aligned
+//   m hi, m lo: (R / 8) column chunks x 128 rows x 16 B each             no-swizzle K-major operand
+//   staging buffer of the epilogue, token indices of the tile, barriers
+__host__ __device__ inline int w_stage_bytes(int R) { return R * 128; }
 __host__ __device__ inline int stage_bytes(int R) { return kXStageBytes + w_stage_bytes(R); }
-__host__ __device__ inline int m_pitch(int R) { return R * 2 + 16; }
-__host__ __device__ inline int m_bytes(int R) { return kRows * m_pitch(R); }
-__host__ __device__ inline int smem_bytes(int R) { return kStages * stage_bytes(R) + 2 * m_bytes(R) + kRows * 4; }
+__host__ __device__ inline int m_bytes(int R) { return (R / 8) * kRows * 16; }
+constexpr int kTailBytes = kStagingBytes + kRows * 4 + 256;
+__host__ __device__ inline int stages_for(int R) {
+    const int n = (kSmemBudget - 1024 - kTailBytes - 2 * m_bytes(R)) / stage_bytes(R);
+    return n > kMaxStages ? kMaxStages : n;
+}
+__host__ __device__ inline int smem_bytes(int R) {
+    return 1024 + stages_for(R) * stage_bytes(R) + 2 * m_bytes(R) + kTailBytes;
+}
 
 struct Params {
     PoolDev pool;
     BucketDev bk;
-    const uint16_t* x;
     float* y;
     int32_t* status;
-    int32_t R;   // max(16, largest padded rank of the pool): sizes the shared-memory layout
+    int32_t R;          // max(16, largest padded rank of the pool): sizes the shared-memory layout
+    int32_t n_stages;
 };
 
+// ---- PTX wrappers -----------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-// 16-byte asynchronous copy; src_bytes = 0 writes zeros (used for columns beyond the matrix)
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-__device__ __forceinline__ void ldmatrix_x4(uint32_t a, uint32_t (&r)[4]) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void ldmatrix_x2(uint32_t a, uint32_t (&r)[2]) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0,%1}, [%2];" : "=r"(r[0]), "=r"(r[1]) : "r"(a));
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t a, uint32_t (&r)[4]) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
 }
-__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+// Bounded wait on an mbarrier phase; false when the CTA has given up (here or elsewhere).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitCycles) break;
+    }
+    *abort_flag = 1;
+    __threadfence_block();
+    atomicCAS(status, 0, PLORA_ERR_TIMEOUT);
+    return false;
 }
-__device__ __forceinline__ void red_add_v2(float* p, float a, float b) {
-    asm volatile("red.global.add.v2.f32 [%0], {%1, %2};" ::"l"(p), "f"(a), "f"(b) : "memory");
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+// Rows r0..r3 of the 2-D tensor, 64 columns from `col`, land as four consecutive 128-byte rows.
+__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap* tm, int col, int r0, int r1, int r2, int r3,
+                                            uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%2, %3, %4, %5, %6}], [%7];" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(tm)), "r"(col), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory"); }
+
+// Shared-memory matrix descriptor of tcgen05.mma: start address, leading and stride byte
+// offsets (all in 16-byte units), descriptor version 1, layout type (0 none, 2 128-byte swizzle).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout) {
+    return (uint64_t)((saddr >> 4) & 0x3fffu) | ((uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16) |
+           ((uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32) | ((uint64_t)1 << 46) | ((uint64_t)layout << 61);
+}
+// Instruction descriptor: fp32 accumulate, bf16 operands, A K-major, B K- or MN-major, M = 128.
+__device__ __forceinline__ uint32_t instr_desc(int n, bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) | ((uint32_t)(n >> 3) << 17) |
+           ((uint32_t)(kRows >> 4) << 24);
+}
+__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, bool accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"((uint32_t)accumulate)
+        : "memory");
+}
+// The mbarrier gets one arrival when every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 32 consecutive columns of this thread's lane of tensor memory.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void red_add_v4(float* p, float a, float b, float c, float d) {
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
 // fp32 -> bf16, round to nearest even, on the bit pattern
 __device__ __forceinline__ uint32_t f32_to_bf16_bits(float f) {
@@ -75,199 +173,280 @@ __device__ __forceinline__ uint32_t f32_to_bf16_bits(float f) {
     return (u + 0x7fffu + ((u >> 16) & 1u)) >> 16;
 }
 
-// One tile: up to kRows tokens of one adapter.  RP = padded rank of that adapter.
-template <int RP>
-__device__ void sgmv_tile(const Params& p, const WorkUnit& wu, const AdapterEntry& e, uint8_t* smem, int* tok_s) {
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int d_in = p.pool.d_in, d_out = p.pool.d_out;
-    const int cnt = wu.cnt;
-    const int kStageBytes = stage_bytes(p.R), kMPitch = m_pitch(p.R);
-    uint8_t* stages = smem;
-    uint8_t* m_hi = smem + kStages * kStageBytes;
-    uint8_t* m_lo = m_hi + m_bytes(p.R);
-    const uint32_t stages_a = smem_u32(stages);
+struct Smem {
+    uint32_t ring;        // stage 0 (1024-byte aligned); stage = x block, then the weight sub-tile
+    uint32_t m_hi, m_lo;  // K-major operand of the expand, chunk kc (8 columns) of row r at kc * 2048 + r * 16
+    uint32_t staging;     // epilogue staging, one 32-row block per epilogue warp
+    int* tok;             // token index of every row of the tile
+    uint32_t full, empty; // [kMaxStages] each
+    uint32_t d_full;      // the shrink accumulator is complete
+    uint32_t m_ready;     // the epilogue has stored m hi / lo (and is done with the shrink accumulator)
+    uint32_t d2_full, d2_empty;   // [kD2Bufs] each
+    volatile int* abort_flag;
+    uint32_t* tmem_slot;
+};
 
-    // token index of every row of the tile (rows beyond cnt repeat the last token: they are
-    // computed and thrown away, so every address stays inside the caller's buffers)
-    __syncthreads();   // the previous tile is completely done with shared memory
-    if (tid < kRows) tok_s[tid] = p.bk.perm[wu.pos0 + min(tid, cnt - 1)];
-    __syncthreads();
-
-    // ------------------------------------------------------------------ shrink
-    // stage = x[64 rows][64 cols] (chunk c of row r at c ^ (r & 7)) + the A^T sub-tile [RP][64] as it
-    // sits in the slab.  Warp (mi, kh): rows 16*mi..+16, k16 steps {2*kh, 2*kh+1} of every stage.
-    const int nK = (d_in + kKC - 1) / kKC;
-    const uint8_t* a_src = p.pool.slab + e.offA;
-    constexpr int NSUB = (kMaxRank / RP > kMaxSubPerTile) ? kMaxSubPerTile : kMaxRank / RP;
-    auto load_shrink_stage = [&](int kc) {
-        if (kc < nK) {
-            const uint32_t base = stages_a + (kc % kStages) * kStageBytes;
-            // x: 64 rows x 8 chunks
-            for (int j = tid; j < kRows * 8; j += kThreads) {
-                const int r = j >> 3, c = j & 7;
-                const int col = kc * kKC + c * 8;
-                const uint16_t* src = p.x + (size_t)tok_s[r] * d_in + (col < d_in ? col : 0);
-                cp_async16(base + r * 128 + ((c ^ (r & 7)) << 4), src, col < d_in ? 16 : 0);
-            }
-            // A^T sub-tile kc: tile kc / NSUB, sub-tile kc % NSUB, RP * 128 contiguous bytes
-            const uint8_t* src = a_src + (size_t)(kc / NSUB) * (RP * NSUB * 128) + (size_t)(kc % NSUB) * (RP * 128);
-            for (int j = tid; j < RP * 8; j += kThreads) cp_async16(base + kXStageBytes + j * 16, src + j * 16, 16);
-        }
-        cp_async_commit();
-    };
-
-    constexpr int NT = RP / 8;            // n8 tiles of the shrink output
-    float acc[NT][4];
-#pragma unroll
-    for (int n = 0; n < NT; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
-    const int mi = warp & 3, kh = warp >> 2;
-
-#pragma unroll
-    for (int s = 0; s < kStages - 1; ++s) load_shrink_stage(s);
-    for (int kc = 0; kc < nK; ++kc) {
-        cp_async_wait<kStages - 2>();
-        __syncthreads();
-        load_shrink_stage(kc + kStages - 1);
-        const uint32_t base = stages_a + (kc % kStages) * kStageBytes;
-#pragma unroll
-        for (int ks = 0; ks < 2; ++ks) {
-            const int kk = (kh * 2 + ks) * 16;                 // column of this k16 step inside the stage
-            uint32_t a[4];
-            {
-                const int r = mi * 16 + (lane & 15), c = (kk >> 3) + (lane >> 4);
-                ldmatrix_x4(base + r * 128 + ((c ^ (r & 7)) << 4), a);
-            }
-#pragma unroll
-            for (int n = 0; n < NT; ++n) {
-                uint32_t b[2];
-                const int r = n * 8 + (lane & 7), c = (kk >> 3) + ((lane >> 3) & 1);
-                ldmatrix_x2(base + kXStageBytes + r * 128 + ((c ^ (r & 7)) << 4), b);
-                mma_bf16(acc[n], a, b[0], b[1]);
-            }
-        }
-    }
-    cp_async_wait<0>();
-    __syncthreads();   // every warp is done with the stage buffers: reuse them for the reduction
-
-    // the two K-halves meet in shared memory: red[kh][64][RP] fp32 (at most 64 KiB, inside the stages)
-    float* red = reinterpret_cast<float*>(stages);
-    {
-        const int g = lane >> 2, q = lane & 3;
-#pragma unroll
-        for (int n = 0; n < NT; ++n) {
-            float* r0 = red + ((size_t)kh * kRows + mi * 16 + g) * RP + n * 8 + q * 2;
-            r0[0] = acc[n][0]; r0[1] = acc[n][1];
-            r0[8 * RP] = acc[n][2]; r0[8 * RP + 1] = acc[n][3];
-        }
-    }
-    __syncthreads();
-    // m = s * (half 0 + half 1), split into bf16 hi + lo, row pitch kMPitch
-    for (int j = tid; j < kRows * RP; j += kThreads) {
-        const int r = j / RP, k = j % RP;
-        const float v = (red[(size_t)r * RP + k] + red[((size_t)kRows + r) * RP + k]) * e.scale;
-        const uint32_t hi = f32_to_bf16_bits(v);
-        const float rest = v - __uint_as_float(hi << 16);
-        reinterpret_cast<uint16_t*>(m_hi + r * kMPitch)[k] = (uint16_t)hi;
-        reinterpret_cast<uint16_t*>(m_lo + r * kMPitch)[k] = (uint16_t)f32_to_bf16_bits(rest);
-    }
-    if (RP < 16) {   // the expand multiplies with K = 16: columns 8..15 of m are zero
-        for (int j = tid; j < kRows * 8; j += kThreads) {
-            const int r = j >> 3, k = 8 + (j & 7);
-            reinterpret_cast<uint16_t*>(m_hi + r * kMPitch)[k] = 0;
-            reinterpret_cast<uint16_t*>(m_lo + r * kMPitch)[k] = 0;
-        }
-    }
-    __syncthreads();
-
-    // ------------------------------------------------------------------ expand
-    // stage = the B sub-tile [RP][64 cols] as it sits in the slab.  Warp w: rows 16*(w & 3)..+16,
-    // columns 32*(w >> 2)..+32 of every 64-column chunk.
-    const int nN = (d_out + kKC - 1) / kKC;
-    const uint8_t* b_src = p.pool.slab + e.offB;
-    constexpr int KP = RP < 16 ? 16 : RP;      // K of the expand, padded to a multiple of 16
-    auto load_expand_stage = [&](int nc) {
-        if (nc < nN) {
-            const uint32_t base = stages_a + (nc % kStages) * kStageBytes;
-            const uint8_t* src = b_src + (size_t)(nc / NSUB) * (RP * NSUB * 128) + (size_t)(nc % NSUB) * (RP * 128);
-            for (int j = tid; j < RP * 8; j += kThreads) cp_async16(base + j * 16, src + j * 16, 16);
-            if (RP < 16)   // rows 8..15 do not exist in the slab: zeros (cp.async with no source bytes)
-                for (int j = tid; j < 8 * 8; j += kThreads) cp_async16(base + (RP * 8 + j) * 16, src, 0);
-        }
-        cp_async_commit();
-    };
-    // A operands (m hi / lo) of this warp's 16 rows stay in registers for the whole expand
-    uint32_t ah[KP / 16][4], al[KP / 16][4];
-#pragma unroll
-    for (int ks = 0; ks < KP / 16; ++ks) {
-        const int r = mi * 16 + (lane & 15), cb = ks * 32 + (lane >> 4) * 16;
-        ldmatrix_x4(smem_u32(m_hi) + r * kMPitch + cb, ah[ks]);
-        ldmatrix_x4(smem_u32(m_lo) + r * kMPitch + cb, al[ks]);
-    }
-    const int nh = warp >> 2;
-    const int g = lane >> 2, q = lane & 3;
-    const int row0 = mi * 16 + g;
-    const bool ok0 = row0 < cnt, ok1 = row0 + 8 < cnt;
-    float* y0 = p.y + (size_t)tok_s[row0] * d_out;
-    float* y1 = p.y + (size_t)tok_s[row0 + 8] * d_out;
-
-#pragma unroll
-    for (int s = 0; s < kStages - 1; ++s) load_expand_stage(s);
-    for (int nc = 0; nc < nN; ++nc) {
-        cp_async_wait<kStages - 2>();
-        __syncthreads();
-        load_expand_stage(nc + kStages - 1);
-        const uint32_t base = stages_a + (nc % kStages) * kStageBytes;
-        float c[4][4];
-#pragma unroll
-        for (int n = 0; n < 4; ++n) c[n][0] = c[n][1] = c[n][2] = c[n][3] = 0.f;
-#pragma unroll
-        for (int ks = 0; ks < KP / 16; ++ks) {
-#pragma unroll
-            for (int np = 0; np < 2; ++np) {
-                // two n8 tiles at once: matrices (k 0-7, n), (k 8-15, n), (k 0-7, n+8), (k 8-15, n+8)
-                uint32_t b[4];
-                const int r = ks * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
-                const int cch = nh * 4 + np * 2 + (lane >> 4);
-                ldmatrix_x4_trans(base + r * 128 + ((cch ^ (r & 7)) << 4), b);
-                mma_bf16(c[np * 2], ah[ks], b[0], b[1]);
-                mma_bf16(c[np * 2], al[ks], b[0], b[1]);
-                mma_bf16(c[np * 2 + 1], ah[ks], b[2], b[3]);
-                mma_bf16(c[np * 2 + 1], al[ks], b[2], b[3]);
-            }
-        }
-#pragma unroll
-        for (int n = 0; n < 4; ++n) {
-            const int col = nc * kKC + nh * 32 + n * 8 + q * 2;
-            if (col < d_out) {
-                if (ok0) red_add_v2(y0 + col, c[n][0], c[n][1]);
-                if (ok1) red_add_v2(y1 + col, c[n][2], c[n][3]);
-            }
-        }
-    }
-    cp_async_wait<0>();
+__device__ __forceinline__ Smem carve(uint8_t* raw, const Params& p) {
+    uint8_t* base = raw + ((1024u - (smem_u32(raw) & 1023u)) & 1023u);
+    uint8_t* m = base + p.n_stages * stage_bytes(p.R);
+    uint8_t* staging = m + 2 * m_bytes(p.R);
+    uint8_t* tok = staging + kStagingBytes;
+    uint8_t* bars = tok + kRows * 4;
+    Smem s;
+    s.ring = smem_u32(base);
+    s.m_hi = smem_u32(m);
+    s.m_lo = s.m_hi + m_bytes(p.R);
+    s.staging = smem_u32(staging);
+    s.tok = reinterpret_cast<int*>(tok);
+    s.full = smem_u32(bars);
+    s.empty = s.full + kMaxStages * 8;
+    s.d_full = s.empty + kMaxStages * 8;
+    s.m_ready = s.d_full + 8;
+    s.d2_full = s.m_ready + 8;
+    s.d2_empty = s.d2_full + kD2Bufs * 8;
+    s.abort_flag = reinterpret_cast<volatile int*>(bars + (2 * kMaxStages + 2 + 2 * kD2Bufs) * 8);
+    s.tmem_slot = reinterpret_cast<uint32_t*>(bars + (2 * kMaxStages + 2 + 2 * kD2Bufs) * 8 + 8);
+    return s;
 }
 
-__global__ void __launch_bounds__(kThreads, 2) sgmv_kernel(const Params p) {
-    extern __shared__ __align__(1024) uint8_t smem[];
-    int* tok_s = reinterpret_cast<int*>(smem + kStages * stage_bytes(p.R) + 2 * m_bytes(p.R));
-    const int n_tiles = *p.bk.n_sgmv_tiles;
+// ---- warp 0: copies ----------------------------------------------------------------------------
+// Lane g owns rows 4g .. 4g + 3 of every tile: one gather instruction per lane and stage.  Rows
+// beyond the tile's count repeat its last token (their results are never written); groups that
+// lie entirely beyond it are not copied at all.
+__device__ __forceinline__ void producer_warp(const Params& p, const Smem& sm, const CUtensorMap* tm_x, int n_tiles,
+                                              int lane) {
+    const int nK = (p.pool.d_in + kKC - 1) / kKC, nN = (p.pool.d_out + kKC - 1) / kKC;
+    const int stage = stage_bytes(p.R);
+    uint32_t it = 0;
     for (int t = blockIdx.x; t < n_tiles; t += gridDim.x) {
         const WorkUnit wu = p.bk.sgmv_tiles[t];
         const AdapterEntry e = p.pool.table[wu.adapter];
-        switch (e.rp) {
-            case 8: sgmv_tile<8>(p, wu, e, smem, tok_s); break;
-            case 16: sgmv_tile<16>(p, wu, e, smem, tok_s); break;
-            case 32: sgmv_tile<32>(p, wu, e, smem, tok_s); break;
-            case 64: sgmv_tile<64>(p, wu, e, smem, tok_s); break;
-            default: sgmv_tile<128>(p, wu, e, smem, tok_s); break;
+        const int cnt = wu.cnt;
+        int r[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) r[j] = p.bk.perm[wu.pos0 + min(4 * lane + j, cnt - 1)];
+        const bool active = 4 * lane < cnt;
+        const uint32_t xbytes = (uint32_t)((cnt + 3) / 4) * 512u, wbytes = (uint32_t)e.rp * 128u;
+        const uint8_t* a_src = p.pool.slab + e.offA;
+        const uint8_t* b_src = p.pool.slab + e.offB;
+        for (int c = 0; c < nK + nN; ++c, ++it) {
+            const uint32_t slot = it % p.n_stages;
+            const uint32_t dst = sm.ring + slot * stage, bar = sm.full + slot * 8;
+            const bool shrink = c < nK;
+            int ok = 1;
+            if (lane == 0) {
+                ok = mbar_wait(sm.empty + slot * 8, ((it / p.n_stages) & 1) ^ 1, sm.abort_flag, p.status);
+                if (ok) {
+                    mbar_arrive_expect_tx(bar, wbytes + (shrink ? xbytes : 0u));
+                    bulk_g2s(dst + kXStageBytes, shrink ? a_src + (size_t)c * wbytes : b_src + (size_t)(c - nK) * wbytes,
+                             wbytes, bar);
+                }
+            }
+            if (!__shfl_sync(0xffffffffu, ok, 0)) return;
+            if (shrink && active) tma_gather4(dst + lane * 512, tm_x, c * kKC, r[0], r[1], r[2], r[3], bar);
         }
     }
+}
+
+// ---- warp 1, one lane: MMAs --------------------------------------------------------------------
+__device__ __forceinline__ void mma_thread(const Params& p, const Smem& sm, uint32_t tmem, int n_tiles) {
+    const int nK = (p.pool.d_in + kKC - 1) / kKC, nN = (p.pool.d_out + kKC - 1) / kKC;
+    const int stage = stage_bytes(p.R);
+    uint32_t it = 0, d2 = 0, tile_idx = 0;
+    for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++tile_idx) {
+        const WorkUnit wu = p.bk.sgmv_tiles[t];
+        const int rp = p.pool.table[wu.adapter].rp;
+        const int KP = rp < 16 ? 16 : rp;      // N of the shrink, K of the expand
+        // shrink: D[128, KP] (tensor-memory columns [0, KP)) = sum over stages of X[128, 64] * W[KP, 64]^T
+        const uint32_t idesc_s = instr_desc(KP, false);
+        for (int kc = 0; kc < nK; ++kc, ++it) {
+            const uint32_t slot = it % p.n_stages;
+            if (!mbar_wait(sm.full + slot * 8, (it / p.n_stages) & 1, sm.abort_flag, p.status)) return;
+            tc_fence_after();
+            const uint32_t xa = sm.ring + slot * stage, wa = xa + kXStageBytes;
+#pragma unroll
+            for (int k = 0; k < kKC / 16; ++k)   // 16 columns = 32 bytes further along the swizzled rows
+                umma(tmem, smem_desc(xa + k * 32, 16, 1024, 2), smem_desc(wa + k * 32, 16, 1024, 2), idesc_s, kc > 0 || k > 0);
+            umma_commit(sm.empty + slot * 8);
+        }
+        umma_commit(sm.d_full);
+        // expand: for every 64-column block, D2[128, 64] = (m_hi + m_lo)[128, KP] * B[KP, 64]
+        if (!mbar_wait(sm.m_ready, tile_idx & 1, sm.abort_flag, p.status)) return;
+        tc_fence_after();
+        const uint32_t idesc_e = instr_desc(kKC, true);
+        for (int nc = 0; nc < nN; ++nc, ++it, ++d2) {
+            const uint32_t slot = it % p.n_stages, b = d2 % kD2Bufs;
+            if (!mbar_wait(sm.full + slot * 8, (it / p.n_stages) & 1, sm.abort_flag, p.status)) return;
+            if (!mbar_wait(sm.d2_empty + b * 8, ((d2 / kD2Bufs) & 1) ^ 1, sm.abort_flag, p.status)) return;
+            tc_fence_after();
+            const uint32_t wa = sm.ring + slot * stage + kXStageBytes;
+            const uint32_t dst = tmem + kTmemD2 + b * kKC;
+            for (int k = 0; k < KP / 16; ++k) {
+                // 16 rank rows of the sub-tile = two 8-row groups of 1024 bytes; 16 columns of m = two chunks of 2048 bytes
+                const uint64_t bd = smem_desc(wa + k * 2048, 1024, 1024, 2);
+                umma(dst, smem_desc(sm.m_hi + k * 4096, 2048, 128, 0), bd, idesc_e, k > 0);
+                umma(dst, smem_desc(sm.m_lo + k * 4096, 2048, 128, 0), bd, idesc_e, true);
+            }
+            umma_commit(sm.empty + slot * 8);
+            umma_commit(sm.d2_full + b * 8);
+        }
+    }
+}
+
+// ---- warps 2-5: epilogue -----------------------------------------------------------------------
+// Thread (q, lane) owns row q * 32 + lane of the tile, q = warp % 4 being the quarter of the
+// tensor memory lanes its warp may read.  `alive` is kept uniform over the warp, and the two
+// barriers per tile are executed whatever happens, so a wait that ran out cannot strand a thread.
+__device__ __forceinline__ void epilogue_warp(const Params& p, const Smem& sm, uint32_t tmem, int n_tiles, int warp,
+                                              int lane) {
+    const int nN = (p.pool.d_out + kKC - 1) / kKC;
+    const int q = warp & 3, row = q * 32 + lane;
+    const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
+    const uint32_t stg = sm.staging + q * 32 * kStagePitch;
+    const unsigned full = 0xffffffffu;
+    uint32_t d2 = 0, tile_idx = 0;
+    bool alive = true;
+    for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++tile_idx) {
+        const WorkUnit wu = p.bk.sgmv_tiles[t];
+        const AdapterEntry e = p.pool.table[wu.adapter];
+        const int cnt = wu.cnt, KP = e.rp < 16 ? 16 : e.rp;
+        epi_barrier();   // every epilogue thread is done with the previous tile's token indices
+        sm.tok[row] = p.bk.perm[wu.pos0 + min(row, cnt - 1)];
+        epi_barrier();
+        if (alive) alive = __all_sync(full, mbar_wait(sm.d_full, tile_idx & 1, sm.abort_flag, p.status));
+        if (!alive) continue;
+        tc_fence_after();
+        // m = s * (x A), split into bf16 hi + lo; columns beyond the padded rank (rank 8 only) are zeros
+        for (int c0 = 0; c0 < KP; c0 += 32) {
+            uint32_t r[32];
+            tmem_ld32(lane_addr + c0, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int kc = 0; kc < 4; ++kc) {
+                if (c0 + kc * 8 < KP) {
+                    uint32_t hi[4], lo[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        uint32_t h2[2], l2[2];
+#pragma unroll
+                        for (int u = 0; u < 2; ++u) {
+                            const int k = c0 + kc * 8 + 2 * j + u;
+                            const float v = k < e.rp ? __uint_as_float(r[kc * 8 + 2 * j + u]) * e.scale : 0.f;
+                            h2[u] = f32_to_bf16_bits(v);
+                            l2[u] = f32_to_bf16_bits(v - __uint_as_float(h2[u] << 16));
+                        }
+                        hi[j] = h2[0] | (h2[1] << 16);
+                        lo[j] = l2[0] | (l2[1] << 16);
+                    }
+                    const uint32_t off = (uint32_t)(c0 / 8 + kc) * (kRows * 16) + row * 16;
+                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(sm.m_hi + off), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]), "r"(hi[3]) : "memory");
+                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(sm.m_lo + off), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]) : "memory");
+                }
+            }
+        }
+        fence_async_smem();   // the MMAs read m through the asynchronous proxy
+        tc_fence_before();
+        mbar_arrive(sm.m_ready);
+        // y += every 64-column block of the expand result
+        for (int nc = 0; nc < nN; ++nc, ++d2) {
+            const uint32_t b = d2 % kD2Bufs;
+            alive = __all_sync(full, mbar_wait(sm.d2_full + b * 8, (d2 / kD2Bufs) & 1, sm.abort_flag, p.status));
+            if (!alive) break;
+            tc_fence_after();
+            uint32_t r0[32], r1[32];
+            tmem_ld32(lane_addr + kTmemD2 + b * kKC, r0);
+            tmem_ld32(lane_addr + kTmemD2 + b * kKC + 32, r1);
+            tmem_ld_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(sm.d2_empty + b * 8);
+            // this thread's row goes to the staging buffer ...
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(stg + lane * kStagePitch + j * 16), "r"(r0[4 * j]), "r"(r0[4 * j + 1]), "r"(r0[4 * j + 2]), "r"(r0[4 * j + 3]) : "memory");
+                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(stg + lane * kStagePitch + 128 + j * 16), "r"(r1[4 * j]), "r"(r1[4 * j + 1]), "r"(r1[4 * j + 2]), "r"(r1[4 * j + 3]) : "memory");
+            }
+            __syncwarp();
+            // ... and leaves it two rows per instruction: 16 lanes cover the 256 bytes of a row piece
+            const int c = lane & 15, col = nc * kKC + c * 4;
+#pragma unroll 4
+            for (int i = 0; i < 16; ++i) {
+                const int rr = 2 * i + (lane >> 4), grow = q * 32 + rr;
+                float4 v;
+                asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(stg + rr * kStagePitch + c * 16));
+                if (grow < cnt && col < p.pool.d_out)
+                    red_add_v4(p.y + (size_t)sm.tok[grow] * p.pool.d_out + col, v.x, v.y, v.z, v.w);
+            }
+            __syncwarp();
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 1) sgmv_kernel(const __grid_constant__ CUtensorMap tm_x, const Params p) {
+    extern __shared__ uint8_t smem_raw[];
+    const Smem sm = carve(smem_raw, p);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        for (int s = 0; s < kMaxStages; ++s) {
+            mbar_init(sm.full + s * 8, 1);
+            mbar_init(sm.empty + s * 8, 1);
+        }
+        mbar_init(sm.d_full, 1);
+        mbar_init(sm.m_ready, kEpiWarps * 32);
+        for (int b = 0; b < kD2Bufs; ++b) {
+            mbar_init(sm.d2_full + b * 8, 1);
+            mbar_init(sm.d2_empty + b * 8, kEpiWarps);
+        }
+        *sm.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // The weight area of every stage starts as zeros: a rank-8 sub-tile fills 8 of the 16 rows
+    // the MMAs read, the others must hold finite values (zeros now, older weights later).
+    for (int s = 0; s < p.n_stages; ++s)
+        for (int i = tid * 16; i < w_stage_bytes(p.R); i += kThreads * 16)
+            asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(sm.ring + s * stage_bytes(p.R) + kXStageBytes + i), "r"(0u) : "memory");
+    fence_async_smem();
+    if (warp == kMmaWarp) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(sm.tmem_slot)), "r"((uint32_t)kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *sm.tmem_slot;
+    const int n_tiles = *p.bk.n_sgmv_tiles;
+
+    if (warp == kProducerWarp) {
+        producer_warp(p, sm, &tm_x, n_tiles, lane);
+    } else if (warp == kMmaWarp) {
+        if (lane == 0) mma_thread(p, sm, tmem, n_tiles);
+    } else {
+        epilogue_warp(p, sm, tmem, n_tiles, warp, lane);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kMmaWarp)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)kTmemCols) : "memory");
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled() {
+    static EncodeTiledFn fn = [] {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess) f = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(f);
+    }();
+    return fn;
 }
 
 }  // namespace
 
 cudaError_t sgmv_configure() {
-    return cudaFuncSetAttribute(sgmv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(kMaxRank));
+    if (!encode_tiled()) return cudaErrorNotSupported;
+    return cudaFuncSetAttribute(sgmv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
 }
 
 cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, int sgmv_min_rows, const void* x, float* y,
@@ -275,17 +454,28 @@ cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, int
     Params p;
     p.pool = pool;
     p.bk = bk;
-    p.x = static_cast<const uint16_t*>(x);
     p.y = y;
     p.status = status;
     p.R = pool.max_rp < 16 ? 16 : pool.max_rp;
+    p.n_stages = stages_for(p.R);
+    // x as a 2-D tensor [n_tok][d_in] of bf16; a gather instruction copies 64 columns of four rows,
+    // 128-byte swizzled (columns beyond d_in read as zeros)
+    CUtensorMap tm;
+    const cuuint64_t dims[2] = {(cuuint64_t)pool.d_in, (cuuint64_t)n_tok};
+    const cuuint64_t strides[1] = {(cuuint64_t)pool.d_in * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kKC, 1};
+    const cuuint32_t elem_strides[2] = {1, 1};
+    if (encode_tiled()(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(x), dims, strides, box, elem_strides,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return cudaErrorInvalidValue;
     // every tensor-core segment has at least sgmv_min_rows tokens: at most this many tiles
     const int min_rows = sgmv_min_rows < 1 ? 1 : sgmv_min_rows;
     long long max_tiles = (long long)n_tok / kRows + (long long)n_tok / min_rows + 1;
-    int grid = 2 * sm_count;
+    int grid = sm_count;   // one CTA per SM: the CTA holds all of the SM's tensor memory
     if (grid > max_tiles) grid = (int)max_tiles;
     if (grid < 1) grid = 1;
-    sgmv_kernel<<<grid, kThreads, smem_bytes(p.R), stream>>>(p);
+    sgmv_kernel<<<grid, kThreads, smem_bytes(p.R), stream>>>(tm, p);
     ++*n_launches;
     return cudaGetLastError();
 }
