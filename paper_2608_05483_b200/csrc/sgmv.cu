@@ -28,7 +28,6 @@
 // pipe.  Every wait is bounded: when one runs out the kernel records PLORA_ERR_TIMEOUT, every
 // role leaves its loop, and the tensor memory is freed before the CTA exits.
 #include <cuda.h>
-#include <cstdio>
 
 #include "plora_internal.cuh"
 
@@ -39,35 +38,12 @@ namespace {
 constexpr int kRows = kSgmvRows;          // rows of a tile = M of the MMAs (128)
 constexpr int kKC = kSubCols;             // K (or N) columns per stage = one slab sub-tile (64)
 constexpr int kXStageBytes = kRows * kKC * 2;              // 16 KiB of x per stage
-#ifndef PLORA_SGMV_EPI_GROUPS
-#define PLORA_SGMV_EPI_GROUPS 1
-#endif
-#ifndef PLORA_SGMV_DIRECT
-#define PLORA_SGMV_DIRECT 0
-#endif
-#ifndef PLORA_SGMV_RMW
-#define PLORA_SGMV_RMW 0
-#endif
-#ifndef PLORA_SGMV_PFX
-#define PLORA_SGMV_PFX 0
-#endif
-#ifndef PLORA_SGMV_PFY
-#define PLORA_SGMV_PFY 0
-#endif
-constexpr int kEpiGroups = PLORA_SGMV_EPI_GROUPS;   // groups of four epilogue warps; they take the expand blocks in turn
-constexpr bool kDirectRed = PLORA_SGMV_DIRECT != 0; // add to y straight from the registers (a thread adds pieces of its own row)
-// A tile owns its rows of y, so y can be updated with plain loads and stores instead of
-// reductions in L2; the loads of a block are issued before the block's MMAs are waited for.
-constexpr bool kYLoadStore = PLORA_SGMV_RMW != 0;
-// A stage touches only 128 bytes (x) or 256 bytes (y) of each of the tile's 128 rows, which sit
-// kilobytes apart: left alone, DRAM would serve the tile in row-buffer-unfriendly crumbs.  Both
-// streams are therefore pulled into L2 ahead of their use in pieces of kPrefetchBytes per row.
-constexpr bool kPrefetchX = PLORA_SGMV_PFX != 0, kPrefetchY = PLORA_SGMV_PFY != 0;
-constexpr int kPrefetchBytes = 2048;
+constexpr int kEpiGroups = 1;   // groups of four epilogue warps; with more than one they take the expand blocks in turn
 // The gather copy moves four rows per instruction and is paced by the copy engine's rate of
 // instructions; where 32 rows of a tile are consecutive tokens (a prefill request is a
 // contiguous run) one ordinary box copy brings all of them.
 constexpr int kBoxRows = 32;
+constexpr int kBoxLanes = kBoxRows / 4;   // lanes of the copy warp whose rows one box covers
 constexpr int kProducerWarp = 0, kMmaWarp = 1, kEpiWarps = 4 * kEpiGroups;   // warps 2.. are the epilogue
 constexpr int kThreads = (2 + kEpiWarps) * 32;
 constexpr int kMaxStages = 8;
@@ -75,7 +51,7 @@ constexpr int kD2Bufs = 4;                // expand accumulators in flight (64 c
 constexpr int kTmemCols = 512;            // columns [0, 128): shrink result; [128, 384): expand blocks
 constexpr int kTmemD2 = 128;
 constexpr int kStagePitch = kKC * 4 + 16;                  // row pitch of the epilogue staging buffer
-constexpr int kStagingBytes = kDirectRed ? 0 : kEpiWarps * 32 * kStagePitch;
+constexpr int kStagingBytes = kEpiWarps * 32 * kStagePitch;
 constexpr int kSmemBudget = 227 * 1024;
 constexpr long long kWaitCycles = 4000000000ll;            // about two seconds of SM clock
 
@@ -98,7 +74,6 @@ __host__ __device__ inline int smem_bytes(int R) {
 struct Params {
     PoolDev pool;
     BucketDev bk;
-    const uint16_t* x;
     float* y;
     int32_t* status;
     int32_t R;          // max(16, largest padded rank of the pool): sizes the shared-memory layout
@@ -156,15 +131,7 @@ __device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap* tm,
         "l"(reinterpret_cast<uint64_t>(tm)), "r"(col), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(bar)
         : "memory");
 }
-// Asks for `bytes` (a multiple of 16) from a 16-byte aligned global address to be brought into L2.
-__device__ __forceinline__ void prefetch_l2(const void* src, uint32_t bytes) {
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void prefetch_row_piece(const uint8_t* row, int row_bytes, int piece) {
-    const int off = piece * kPrefetchBytes;
-    if (off < row_bytes) prefetch_l2(row + off, (uint32_t)min(kPrefetchBytes, row_bytes - off));
-}
-// A box of kBoxRows consecutive rows x 64 columns of the 2-D tensor, rows 128 bytes apart, swizzled.
+// A box of kBoxRows consecutive rows x 64 columns of the 2-D tensor lands as 128-byte rows, swizzled.
 __device__ __forceinline__ void tma_box(uint32_t dst, const CUtensorMap* tm, int col, int row, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
@@ -262,7 +229,6 @@ __device__ __forceinline__ Smem carve(uint8_t* raw, const Params& p) {
 // lie entirely beyond it are not copied at all.
 __device__ __forceinline__ void producer_warp(const Params& p, const Smem& sm, const CUtensorMap* tm_x,
                                               const CUtensorMap* tm_box, int n_tiles, int lane) {
-    const uint8_t* x_bytes = reinterpret_cast<const uint8_t*>(p.x);
     const int nK = (p.pool.d_in + kKC - 1) / kKC, nN = (p.pool.d_out + kKC - 1) / kKC;
     const int stage = stage_bytes(p.R);
     uint32_t it = 0;
@@ -275,31 +241,16 @@ __device__ __forceinline__ void producer_warp(const Params& p, const Smem& sm, c
         for (int j = 0; j < 4; ++j) r[j] = p.bk.perm[wu.pos0 + min(4 * lane + j, cnt - 1)];
         const bool active = 4 * lane < cnt;
         // lanes 8j .. 8j + 7 hold rows 32j .. 32j + 31: one box copy if those are consecutive tokens
-        const int lead = lane & ~7;
+        const int lead = lane & ~(kBoxLanes - 1);
         const int first = __shfl_sync(0xffffffffu, r[0], lead);
         const bool in_run = 4 * lane + 3 < cnt && r[0] == first + 4 * (lane - lead) && r[1] == r[0] + 1 &&
                             r[2] == r[0] + 2 && r[3] == r[0] + 3;
-        const bool boxed = ((__ballot_sync(0xffffffffu, in_run) >> lead) & 0xffu) == 0xffu;
+        constexpr unsigned kBoxMask = kBoxLanes >= 32 ? 0xffffffffu : ((1u << kBoxLanes) - 1u);
+        const bool boxed = ((__ballot_sync(0xffffffffu, in_run) >> lead) & kBoxMask) == kBoxMask;
         const uint32_t xbytes = (uint32_t)((cnt + 3) / 4) * 512u, wbytes = (uint32_t)e.rp * 128u;
         const uint8_t* a_src = p.pool.slab + e.offA;
         const uint8_t* b_src = p.pool.slab + e.offB;
-        constexpr int kStagesPerPiece = kPrefetchBytes / (kKC * 2);
-        const int x_row_bytes = p.pool.d_in * 2;
-        if (kPrefetchX && active) {
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (4 * lane + j < cnt) {
-                    prefetch_row_piece(x_bytes + (size_t)r[j] * x_row_bytes, x_row_bytes, 0);
-                    prefetch_row_piece(x_bytes + (size_t)r[j] * x_row_bytes, x_row_bytes, 1);
-                }
-        }
         for (int c = 0; c < nK + nN; ++c, ++it) {
-            if (kPrefetchX && active && c < nK && c > 0 && c % kStagesPerPiece == 0) {
-#pragma unroll
-                for (int j = 0; j < 4; ++j)
-                    if (4 * lane + j < cnt)
-                        prefetch_row_piece(x_bytes + (size_t)r[j] * x_row_bytes, x_row_bytes, c / kStagesPerPiece + 1);
-            }
             const uint32_t slot = it % p.n_stages;
             const uint32_t dst = sm.ring + slot * stage, bar = sm.full + slot * 8;
             const bool shrink = c < nK;
@@ -386,18 +337,11 @@ __device__ __forceinline__ void epilogue_warp(const Params& p, const Smem& sm, u
         const WorkUnit wu = p.bk.sgmv_tiles[t];
         const AdapterEntry e = p.pool.table[wu.adapter];
         const int cnt = wu.cnt, KP = e.rp < 16 ? 16 : e.rp;
-#ifdef PLORA_SGMV_TRACE
-        unsigned long long tr0, tr1, tr2, tr3;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tr0));
-#endif
         epi_barrier();   // every epilogue thread is done with the previous tile's token indices
         sm.tok[row] = p.bk.perm[wu.pos0 + min(row, cnt - 1)];
         epi_barrier();
         if (alive) alive = __all_sync(full, mbar_wait(sm.d_full, tile_idx & 1, sm.abort_flag, p.status));
         if (!alive) continue;
-#ifdef PLORA_SGMV_TRACE
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tr1));
-#endif
         tc_fence_after();
         // m = s * (x A), split into bf16 hi + lo; columns beyond the padded rank (rank 8 only) are zeros
         for (int c0 = 0; c0 < KP; c0 += 32) {
@@ -430,35 +374,12 @@ __device__ __forceinline__ void epilogue_warp(const Params& p, const Smem& sm, u
         fence_async_smem();   // the MMAs read m through the asynchronous proxy
         tc_fence_before();
         mbar_arrive(sm.m_ready);
-#ifdef PLORA_SGMV_TRACE
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tr2));
-#endif
         // y += every 64-column block of the expand result
-        constexpr int kBlocksPerPiece = kPrefetchBytes / (kKC * 4);
-        const uint8_t* y_row = reinterpret_cast<const uint8_t*>(p.y + (size_t)sm.tok[row] * p.pool.d_out);
-        const int y_row_bytes = p.pool.d_out * 4;
-        if (kPrefetchY && grp == 0 && row < cnt) {
-            prefetch_row_piece(y_row, y_row_bytes, 0);
-            prefetch_row_piece(y_row, y_row_bytes, 1);
-        }
         for (int nc = 0; nc < nN; ++nc, ++d2) {
-            if (kPrefetchY && grp == 0 && row < cnt && nc > 0 && nc % kBlocksPerPiece == 0)
-                prefetch_row_piece(y_row, y_row_bytes, nc / kBlocksPerPiece + 1);
             const uint32_t b = d2 % kD2Bufs;
             if ((int)(d2 % kEpiGroups) != grp) continue;   // the other group's block
             // lane (h, c) handles the 16-byte piece c of rows 2i + h of its warp's 32 rows
             const int c = lane & 15, col = nc * kKC + c * 4;
-            float4 yv[16];
-            if (kYLoadStore && !kDirectRed) {
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const int grow = q * 32 + 2 * i + (lane >> 4);
-                    if (grow < cnt && col < p.pool.d_out) {
-                        const float* src = p.y + (size_t)sm.tok[grow] * p.pool.d_out + col;
-                        asm volatile("ld.global.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(yv[i].x), "=f"(yv[i].y), "=f"(yv[i].z), "=f"(yv[i].w) : "l"(src) : "memory");
-                    }
-                }
-            }
             alive = __all_sync(full, mbar_wait(sm.d2_full + b * 8, (d2 / kD2Bufs) & 1, sm.abort_flag, p.status));
             if (!alive) break;
             tc_fence_after();
@@ -469,21 +390,6 @@ __device__ __forceinline__ void epilogue_warp(const Params& p, const Smem& sm, u
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(sm.d2_empty + b * 8);
-            if (kDirectRed) {
-                if (row < cnt) {
-                    float* yr = p.y + (size_t)sm.tok[row] * p.pool.d_out + nc * kKC;
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        if (nc * kKC + 4 * j < p.pool.d_out)
-                            red_add_v4(yr + 4 * j, __uint_as_float(r0[4 * j]), __uint_as_float(r0[4 * j + 1]),
-                                       __uint_as_float(r0[4 * j + 2]), __uint_as_float(r0[4 * j + 3]));
-                        if (nc * kKC + 32 + 4 * j < p.pool.d_out)
-                            red_add_v4(yr + 32 + 4 * j, __uint_as_float(r1[4 * j]), __uint_as_float(r1[4 * j + 1]),
-                                       __uint_as_float(r1[4 * j + 2]), __uint_as_float(r1[4 * j + 3]));
-                    }
-                }
-                continue;
-            }
             // this thread's row goes to the staging buffer ...
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
@@ -499,25 +405,19 @@ __device__ __forceinline__ void epilogue_warp(const Params& p, const Smem& sm, u
                 asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(stg + rr * kStagePitch + c * 16));
                 if (grow < cnt && col < p.pool.d_out) {
                     float* dst = p.y + (size_t)sm.tok[grow] * p.pool.d_out + col;
-                    if (kYLoadStore)
-                        asm volatile("st.global.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(dst), "f"(yv[i].x + v.x), "f"(yv[i].y + v.y), "f"(yv[i].z + v.z), "f"(yv[i].w + v.w) : "memory");
-                    else
-                        red_add_v4(dst, v.x, v.y, v.z, v.w);
+                    red_add_v4(dst, v.x, v.y, v.z, v.w);
                 }
             }
             __syncwarp();
         }
-#ifdef PLORA_SGMV_TRACE
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tr3));
-        if ((blockIdx.x == 0 || blockIdx.x == 77) && warp == 2 && lane == 0)
-            printf("cta %d tile %d cnt %d: wait shrink %llu ns, m %llu ns, expand %llu ns\n", blockIdx.x, t, cnt, tr1 - tr0, tr2 - tr1, tr3 - tr2);
-#endif
     }
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
 sgmv_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_box, const Params p) {
     extern __shared__ uint8_t smem_raw[];
+    const int n_tiles = *p.bk.n_sgmv_tiles;
+    if ((int)blockIdx.x >= n_tiles) return;   // nothing for this CTA (often: no tensor-core segment in the batch)
     const Smem sm = carve(smem_raw, p);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
@@ -548,7 +448,6 @@ sgmv_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CU
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *sm.tmem_slot;
-    const int n_tiles = *p.bk.n_sgmv_tiles;
 
     if (warp == kProducerWarp) {
         producer_warp(p, sm, &tm_x, &tm_box, n_tiles, lane);
@@ -588,7 +487,6 @@ cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, int
     Params p;
     p.pool = pool;
     p.bk = bk;
-    p.x = static_cast<const uint16_t*>(x);
     p.y = y;
     p.status = status;
     p.R = pool.max_rp < 16 ? 16 : pool.max_rp;
