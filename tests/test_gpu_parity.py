@@ -140,6 +140,33 @@ def test_auto_dispatch_uses_both_kernels():
         r.close()
 
 
+def _ids_from_runs(runs, shuffle_seed=None):
+    """ids for consecutive runs [(adapter, length), ...]; optionally dealt out in a random order."""
+    ids = np.concatenate([np.full(n, a, np.int32) for a, n in runs])
+    if shuffle_seed is not None:
+        np.random.default_rng(shuffle_seed).shuffle(ids)
+    return ids
+
+
+@pytest.mark.parametrize("layout", ["contiguous", "shuffled", "broken_runs"])
+def test_sgmv_tile_shapes(layout):
+    # segment lengths around the 128-row tile and the 32-row copy box: whole tiles, ragged last tiles,
+    # a one-row tile, tokens that are consecutive (box copies), scattered (gather copies) or consecutive
+    # in pieces that end inside a box
+    lens = [128, 129, 33, 255, 300, 1, 31, 64]
+    ranks = [8, 16, 32, 64, 128, 24, 5, 16]
+    if layout == "broken_runs":
+        runs = []
+        for rep in range(3):      # every adapter's tokens come as three separate runs of uneven length
+            runs += [(a, n // 3 + (rep == 2) * (n % 3)) for a, n in enumerate(lens)]
+        ids = _ids_from_runs([r for r in runs if r[1] > 0])
+    else:
+        ids = _ids_from_runs(list(enumerate(lens)), shuffle_seed=5 if layout == "shuffled" else None)
+    p = random_problem(300, T=len(ids), d_in=328, d_out=264, ranks=ranks)
+    p["ids"] = ids
+    _check_paths(p, paths=[P.PATH_SGMV, P.PATH_AUTO])
+
+
 def test_empty_and_all_minus_one():
     p = random_problem(1, T=0, d_in=64, d_out=64, ranks=[8])
     r = Runner(p, max_tokens=8)
