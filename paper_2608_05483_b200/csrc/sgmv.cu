@@ -21,8 +21,8 @@
 //     per-warp staging buffer so that a warp adds whole 256-byte row pieces to y with vector
 //     reductions (one addition per element of y, so the result is bit-reproducible).
 //
-// Roles: warp 0 issues the copies, warp 1 owns the tensor memory and issues the MMAs, warps 2-5
-// are the epilogue.  Stages (x block + weight sub-tile) cycle through a ring guarded by
+// Roles: the first warps issue the copies (stage i belongs to copy warp i mod their number), the
+// next warp owns the tensor memory and issues the MMAs, the last four are the epilogue.  Stages (x block + weight sub-tile) cycle through a ring guarded by
 // full / empty mbarriers; the MMA thread releases a stage with tcgen05.commit.  The path is
 // bound by HBM traffic on the activations (x read once, y updated once), not by the tensor
 // pipe.  Every wait is bounded: when one runs out the kernel records PLORA_ERR_TIMEOUT, every
@@ -44,8 +44,12 @@ constexpr int kEpiGroups = 1;   // groups of four epilogue warps; with more than
 // contiguous run) one ordinary box copy brings all of them.
 constexpr int kBoxRows = 32;
 constexpr int kBoxLanes = kBoxRows / 4;   // lanes of the copy warp whose rows one box covers
-constexpr int kProducerWarp = 0, kMmaWarp = 1, kEpiWarps = 4 * kEpiGroups;   // warps 2.. are the epilogue
-constexpr int kThreads = (2 + kEpiWarps) * 32;
+// A thread gets a copy instruction out about every 45 ns and a stage takes up to five of them:
+// the stages are dealt out to two copy warps.  (The copy engine itself moves about 50 GB/s per
+// SM in boxes of this shape, which is what bounds the shrink phase.)
+constexpr int kProducerWarps = 2;
+constexpr int kMmaWarp = kProducerWarps, kFirstEpiWarp = kProducerWarps + 1, kEpiWarps = 4 * kEpiGroups;
+constexpr int kThreads = (kFirstEpiWarp + kEpiWarps) * 32;
 constexpr int kMaxStages = 8;
 constexpr int kD2Bufs = 4;                // expand accumulators in flight (64 columns each)
 constexpr int kTmemCols = 512;            // columns [0, 128): shrink result; [128, 384): expand blocks
@@ -223,12 +227,12 @@ __device__ __forceinline__ Smem carve(uint8_t* raw, const Params& p) {
     return s;
 }
 
-// ---- warp 0: copies ----------------------------------------------------------------------------
+// ---- copy warps ----------------------------------------------------------------------------
 // Lane g owns rows 4g .. 4g + 3 of every tile: one gather instruction per lane and stage.  Rows
 // beyond the tile's count repeat its last token (their results are never written); groups that
 // lie entirely beyond it are not copied at all.
 __device__ __forceinline__ void producer_warp(const Params& p, const Smem& sm, const CUtensorMap* tm_x,
-                                              const CUtensorMap* tm_box, int n_tiles, int lane) {
+                                              const CUtensorMap* tm_box, int n_tiles, int warp, int lane) {
     const int nK = (p.pool.d_in + kKC - 1) / kKC, nN = (p.pool.d_out + kKC - 1) / kKC;
     const int stage = stage_bytes(p.R);
     uint32_t it = 0;
@@ -251,6 +255,7 @@ __device__ __forceinline__ void producer_warp(const Params& p, const Smem& sm, c
         const uint8_t* a_src = p.pool.slab + e.offA;
         const uint8_t* b_src = p.pool.slab + e.offB;
         for (int c = 0; c < nK + nN; ++c, ++it) {
+            if ((int)(it % kProducerWarps) != warp) continue;   // another copy warp's stage
             const uint32_t slot = it % p.n_stages;
             const uint32_t dst = sm.ring + slot * stage, bar = sm.full + slot * 8;
             const bool shrink = c < nK;
@@ -274,7 +279,7 @@ __device__ __forceinline__ void producer_warp(const Params& p, const Smem& sm, c
     }
 }
 
-// ---- warp 1, one lane: MMAs --------------------------------------------------------------------
+// ---- MMA warp, one lane --------------------------------------------------------------------
 __device__ __forceinline__ void mma_thread(const Params& p, const Smem& sm, uint32_t tmem, int n_tiles) {
     const int nK = (p.pool.d_in + kKC - 1) / kKC, nN = (p.pool.d_out + kKC - 1) / kKC;
     const int stage = stage_bytes(p.R);
@@ -319,7 +324,7 @@ __device__ __forceinline__ void mma_thread(const Params& p, const Smem& sm, uint
     }
 }
 
-// ---- warps 2-5: epilogue -----------------------------------------------------------------------
+// ---- the last four warps: epilogue -----------------------------------------------------------------------
 // Thread (q, lane) owns row q * 32 + lane of the tile, q = warp % 4 being the quarter of the
 // tensor memory lanes its warp may read.  `alive` is kept uniform over the warp, and the two
 // barriers per tile are executed whatever happens, so a wait that ran out cannot strand a thread.
@@ -327,9 +332,9 @@ __device__ __forceinline__ void epilogue_warp(const Params& p, const Smem& sm, u
                                               int lane) {
     const int nN = (p.pool.d_out + kKC - 1) / kKC;
     const int q = warp & 3, row = q * 32 + lane;
-    const int grp = (warp - 2) >> 2;   // which group of four warps
+    const int grp = (warp - kFirstEpiWarp) >> 2;   // which group of four warps
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
-    const uint32_t stg = sm.staging + (warp - 2) * 32 * kStagePitch;
+    const uint32_t stg = sm.staging + (warp - kFirstEpiWarp) * 32 * kStagePitch;
     const unsigned full = 0xffffffffu;
     uint32_t d2 = 0, tile_idx = 0;
     bool alive = true;
@@ -449,8 +454,8 @@ sgmv_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CU
     tc_fence_after();
     const uint32_t tmem = *sm.tmem_slot;
 
-    if (warp == kProducerWarp) {
-        producer_warp(p, sm, &tm_x, &tm_box, n_tiles, lane);
+    if (warp < kProducerWarps) {
+        producer_warp(p, sm, &tm_x, &tm_box, n_tiles, warp, lane);
     } else if (warp == kMmaWarp) {
         if (lane == 0) mma_thread(p, sm, tmem, n_tiles);
     } else {
