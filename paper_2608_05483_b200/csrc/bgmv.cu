@@ -6,7 +6,7 @@
 // the adapters present, once per adapter whatever its batch), so the kernel is a
 // streaming pipeline:
 //
-//   - a unit's shrink is cut into up to kMaxRuns tasks (runs of consecutive A tiles)
+//   - a unit's shrink is cut into up to kMaxRunsA tasks (runs of consecutive A tiles)
 //     and its expand into up to kMaxRuns tasks (runs of B tiles); all shrink tasks
 //     come first in the task list and persistent CTAs take tasks round-robin, so
 //     the tiles of one adapter stream through many SMs at once and the load is
@@ -538,17 +538,17 @@ __device__ __forceinline__ const unsigned long long* partial_src(const Params& p
     return p.bk.m_part + part_index(p, unit, 0, t) + k;
 }
 __device__ __forceinline__ void partial_load(const Params& p, uint32_t epoch, const unsigned long long* src,
-                                             unsigned long long (&w)[kMaxRuns]) {
+                                             unsigned long long (&w)[kMaxRunsA]) {
     const size_t run_stride = (size_t)kTokChunk * p.pool.max_rp;
 #pragma unroll
-    for (int j = 0; j < kMaxRuns; ++j)
+    for (int j = 0; j < kMaxRunsA; ++j)
         w[j] = j < p.runs_a ? ldg_cg_u64(src + j * run_stride) : ((unsigned long long)epoch << 32);
 }
-__device__ __forceinline__ bool partial_sum(uint32_t epoch, const unsigned long long (&w)[kMaxRuns], uint32_t dst) {
+__device__ __forceinline__ bool partial_sum(uint32_t epoch, const unsigned long long (&w)[kMaxRunsA], uint32_t dst) {
     bool ok = true;
     float s = 0.f;
 #pragma unroll
-    for (int j = 0; j < kMaxRuns; ++j) {
+    for (int j = 0; j < kMaxRunsA; ++j) {
         ok = ok && (uint32_t)(w[j] >> 32) == epoch;
         s += __uint_as_float((uint32_t)w[j]);
     }
@@ -557,13 +557,13 @@ __device__ __forceinline__ bool partial_sum(uint32_t epoch, const unsigned long 
 }
 // The words of up to kGatherDepth values per lane are requested before the first of them is
 // used: a unit's m costs one round trip to L2 per 32 * kGatherDepth values, not one per 32.
-constexpr int kGatherDepth = 1;
+constexpr int kGatherDepth = 2;
 __device__ __forceinline__ bool gather_m(const Params& p, uint32_t epoch, int unit, int cnt, int rp, int lane,
                                          uint32_t mdst) {
     bool ok = true;
     const int n = cnt * rp;
     for (int i0 = lane; i0 < n; i0 += 32 * kGatherDepth) {
-        unsigned long long w[kGatherDepth][kMaxRuns];
+        unsigned long long w[kGatherDepth][kMaxRunsA];
 #pragma unroll
         for (int q = 0; q < kGatherDepth; ++q)
             if (i0 + q * 32 < n) partial_load(p, epoch, partial_src(p, unit, i0 + q * 32, rp), w[q]);
@@ -1014,6 +1014,10 @@ cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const
         p.runs_a = mode == kShrinkOnly ? 1 : clamp_runs(tiles_for(pool.d_in, rp));
         // an expand task pays one round trip for its m before its first tile: give it at least two tiles
         p.runs_b = clamp_runs(tiles_for(pool.d_out, rp) / (mode == kFused ? 2 : 1));
+        // every shrink task ends with a hand-over of its partial m (and every expand task reads all of
+        // them): at most kMaxRunsA shrink tasks per unit measured best (4: 0.764 of the roofline on the
+        // decode 7B shapes, 8: 0.748, 2: 0.757)
+        if (p.runs_a > kMaxRunsA) p.runs_a = kMaxRunsA;
         if (mode == kFused) {
             // the partial-m workspace holds n_units * runs_a * kTokChunk * max_rp words, n_units <= n_tok
             const size_t per_run = (size_t)n_tok * n_groups * kTokChunk * pool.max_rp * sizeof(unsigned long long);

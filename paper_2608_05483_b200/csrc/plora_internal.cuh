@@ -73,7 +73,8 @@ struct WorkUnit {   // 32 bytes
 };
 static_assert(sizeof(WorkUnit) == 32 && kTokChunk == 4, "work unit is two 16-byte words");
 
-constexpr int kMaxRuns = 8;       // a unit's shrink (or expand) is cut into at most this many tasks
+constexpr int kMaxRuns = 8;       // a unit's expand is cut into at most this many tasks
+constexpr int kMaxRunsA = 4;      // ... and its shrink into at most this many
 
 struct BucketDev {
     int32_t* perm;
