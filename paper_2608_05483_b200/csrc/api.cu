@@ -34,7 +34,7 @@ struct DeviceGuard {
 
 constexpr int kDefaultSgmvMinRows = 32;   // AUTO: segments at least this long take the tensor-core path ...
 constexpr int kSgmvMinBatch = 512;        // ... in batches at least this large (a decode batch stays one launch)
-constexpr int kSgmvMinTiles = 64;         // ... and only if they make at least this many 128-row tiles together
+constexpr int kSgmvMinTiles = 128;        // ... and only if they make at least this many 64-row tiles together
 
 }  // namespace
 

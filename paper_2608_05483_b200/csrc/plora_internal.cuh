@@ -62,7 +62,7 @@ struct PoolDev {
 // Bucket (device resident, owned by the context).
 // ---------------------------------------------------------------------------------
 constexpr int kTokChunk = 4;      // tokens of one segment a BGMV work unit handles
-constexpr int kSgmvRows = 128;    // rows of one SGMV tile (M of the tensor-core instruction)
+constexpr int kSgmvRows = 64;     // rows of one SGMV tile (M of the tensor-core instruction)
 
 struct WorkUnit {   // 32 bytes
     int32_t adapter;

@@ -6,7 +6,7 @@
 //     m [rows, rp]    = X [rows, d_in] * A          bf16 x bf16 -> fp32   (K = d_in)
 //     y [rows, d_out] += s * m * B                  fp32 m carried as bf16 hi + lo, two products
 //
-// Both GEMMs are issued as tcgen05.mma (M = 128, accumulators in tensor memory) by one thread
+// Both GEMMs are issued as tcgen05.mma (M = 64, accumulators in tensor memory) by one thread
 // of the CTA; the operands reach shared memory without passing through registers:
 //
 //   - the x rows of a tile are gathered by token index with the tensor-map copy in gather mode
@@ -35,9 +35,11 @@ namespace plora {
 
 namespace {
 
-constexpr int kRows = kSgmvRows;          // rows of a tile = M of the MMAs (128)
+constexpr int kRows = kSgmvRows;          // rows of a tile = M of the MMAs (64)
+constexpr int kRowsPerWarp = kRows / 4;   // M = 64: row r of the accumulator sits in tensor-memory lane 32 (r / 16) + r % 16
+static_assert(kRows == 64, "the epilogue's lane mapping is the one of M = 64");
 constexpr int kKC = kSubCols;             // K (or N) columns per stage = one slab sub-tile (64)
-constexpr int kXStageBytes = kRows * kKC * 2;              // 16 KiB of x per stage
+constexpr int kXStageBytes = kRows * kKC * 2;              // 8 KiB of x per stage
 constexpr int kEpiGroups = 1;   // groups of four epilogue warps; with more than one they take the expand blocks in turn
 // The gather copy moves four rows per instruction and is paced by the copy engine's rate of
 // instructions; where 32 rows of a tile are consecutive tokens (a prefill request is a
@@ -51,24 +53,26 @@ constexpr int kProducerWarps = 2;
 constexpr int kMmaWarp = kProducerWarps, kFirstEpiWarp = kProducerWarps + 1, kEpiWarps = 4 * kEpiGroups;
 constexpr int kThreads = (kFirstEpiWarp + kEpiWarps) * 32;
 constexpr int kMaxStages = 8;
-constexpr int kD2Bufs = 4;                // expand accumulators in flight (64 columns each)
-constexpr int kTmemCols = 512;            // columns [0, 128): shrink result; [128, 384): expand blocks
+constexpr int kD2Bufs = 2;                // expand accumulators in flight (64 columns each)
+constexpr int kTmemCols = 256;            // columns [0, 128): shrink result; [128, 256): expand blocks; two CTAs share an SM's 512
 constexpr int kTmemD2 = 128;
 constexpr int kStagePitch = kKC * 4 + 16;                  // row pitch of the epilogue staging buffer
-constexpr int kStagingBytes = kEpiWarps * 32 * kStagePitch;
-constexpr int kSmemBudget = 227 * 1024;
+constexpr int kStagingBytes = kEpiWarps * kRowsPerWarp * kStagePitch;
+constexpr int kSmemBudget = 227 * 1024;                    // of an SM
+constexpr int kSmemPerCta = kSmemBudget / 2 - 1024;        // two CTAs per SM, so that one tile's shrink overlaps another's expand
 constexpr long long kWaitCycles = 4000000000ll;            // about two seconds of SM clock
 
 // Shared memory, sized for R = max(16, largest padded rank of the pool):
-//   ring of n_stages x (x block 16 KiB + weight sub-tile R x 128 B)      1024-byte aligned
-//   m hi, m lo: (R / 8) column chunks x 128 rows x 16 B each             no-swizzle K-major operand
+//   ring of n_stages x (x block 8 KiB + weight sub-tile R x 128 B)       1024-byte aligned
+//   m hi, m lo: (R / 8) column chunks x 64 rows x 16 B each              no-swizzle K-major operand
 //   staging buffer of the epilogue, token indices of the tile, barriers
 __host__ __device__ inline int w_stage_bytes(int R) { return R * 128; }
 __host__ __device__ inline int stage_bytes(int R) { return kXStageBytes + w_stage_bytes(R); }
 __host__ __device__ inline int m_bytes(int R) { return (R / 8) * kRows * 16; }
 constexpr int kTailBytes = kStagingBytes + kRows * 4 + 256;
 __host__ __device__ inline int stages_for(int R) {
-    const int n = (kSmemBudget - 1024 - kTailBytes - 2 * m_bytes(R)) / stage_bytes(R);
+    int n = (kSmemPerCta - 1024 - kTailBytes - 2 * m_bytes(R)) / stage_bytes(R);
+    if (n < 3) n = (kSmemBudget - 1024 - kTailBytes - 2 * m_bytes(R)) / stage_bytes(R);   // rank 128: one CTA per SM
     return n > kMaxStages ? kMaxStages : n;
 }
 __host__ __device__ inline int smem_bytes(int R) {
@@ -313,10 +317,10 @@ __device__ __forceinline__ void mma_thread(const Params& p, const Smem& sm, uint
             const uint32_t wa = sm.ring + slot * stage + kXStageBytes;
             const uint32_t dst = tmem + kTmemD2 + b * kKC;
             for (int k = 0; k < KP / 16; ++k) {
-                // 16 rank rows of the sub-tile = two 8-row groups of 1024 bytes; 16 columns of m = two chunks of 2048 bytes
+                // 16 rank rows of the sub-tile = two 8-row groups of 1024 bytes; 16 columns of m = two chunks of kRows * 16 bytes
                 const uint64_t bd = smem_desc(wa + k * 2048, 1024, 1024, 2);
-                umma(dst, smem_desc(sm.m_hi + k * 4096, 2048, 128, 0), bd, idesc_e, k > 0);
-                umma(dst, smem_desc(sm.m_lo + k * 4096, 2048, 128, 0), bd, idesc_e, true);
+                umma(dst, smem_desc(sm.m_hi + k * (2 * kRows * 16), kRows * 16, 128, 0), bd, idesc_e, k > 0);
+                umma(dst, smem_desc(sm.m_lo + k * (2 * kRows * 16), kRows * 16, 128, 0), bd, idesc_e, true);
             }
             umma_commit(sm.empty + slot * 8);
             umma_commit(sm.d2_full + b * 8);
@@ -325,16 +329,18 @@ __device__ __forceinline__ void mma_thread(const Params& p, const Smem& sm, uint
 }
 
 // ---- the last four warps: epilogue -----------------------------------------------------------------------
-// Thread (q, lane) owns row q * 32 + lane of the tile, q = warp % 4 being the quarter of the
-// tensor memory lanes its warp may read.  `alive` is kept uniform over the warp, and the two
+// Thread (q, lane < 16) owns row 16 q + lane of the tile, q = warp % 4 being the quarter of the
+// tensor memory lanes its warp may read (with M = 64 a quarter holds 16 rows in its first 16
+// lanes; the other lanes of the warp take part in the loads and help in the write-out).  `alive` is kept uniform over the warp, and the two
 // barriers per tile are executed whatever happens, so a wait that ran out cannot strand a thread.
 __device__ __forceinline__ void epilogue_warp(const Params& p, const Smem& sm, uint32_t tmem, int n_tiles, int warp,
                                               int lane) {
     const int nN = (p.pool.d_out + kKC - 1) / kKC;
-    const int q = warp & 3, row = q * 32 + lane;
+    const int q = warp & 3, row = q * kRowsPerWarp + (lane & (kRowsPerWarp - 1));
+    const bool owner = lane < kRowsPerWarp;
     const int grp = (warp - kFirstEpiWarp) >> 2;   // which group of four warps
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
-    const uint32_t stg = sm.staging + (warp - kFirstEpiWarp) * 32 * kStagePitch;
+    const uint32_t stg = sm.staging + (warp - kFirstEpiWarp) * kRowsPerWarp * kStagePitch;
     const unsigned full = 0xffffffffu;
     uint32_t d2 = 0, tile_idx = 0;
     bool alive = true;
@@ -343,7 +349,7 @@ __device__ __forceinline__ void epilogue_warp(const Params& p, const Smem& sm, u
         const AdapterEntry e = p.pool.table[wu.adapter];
         const int cnt = wu.cnt, KP = e.rp < 16 ? 16 : e.rp;
         epi_barrier();   // every epilogue thread is done with the previous tile's token indices
-        sm.tok[row] = p.bk.perm[wu.pos0 + min(row, cnt - 1)];
+        if (owner) sm.tok[row] = p.bk.perm[wu.pos0 + min(row, cnt - 1)];
         epi_barrier();
         if (alive) alive = __all_sync(full, mbar_wait(sm.d_full, tile_idx & 1, sm.abort_flag, p.status));
         if (!alive) continue;
@@ -355,7 +361,7 @@ __device__ __forceinline__ void epilogue_warp(const Params& p, const Smem& sm, u
             tmem_ld_wait();
 #pragma unroll
             for (int kc = 0; kc < 4; ++kc) {
-                if (c0 + kc * 8 < KP && (kc % kEpiGroups) == grp) {   // the groups share the 8-column chunks
+                if (owner && c0 + kc * 8 < KP && (kc % kEpiGroups) == grp) {   // the groups share the 8-column chunks
                     uint32_t hi[4], lo[4];
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
@@ -396,16 +402,18 @@ __device__ __forceinline__ void epilogue_warp(const Params& p, const Smem& sm, u
             __syncwarp();
             if (lane == 0) mbar_arrive(sm.d2_empty + b * 8);
             // this thread's row goes to the staging buffer ...
+            if (owner) {
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(stg + lane * kStagePitch + j * 16), "r"(r0[4 * j]), "r"(r0[4 * j + 1]), "r"(r0[4 * j + 2]), "r"(r0[4 * j + 3]) : "memory");
-                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(stg + lane * kStagePitch + 128 + j * 16), "r"(r1[4 * j]), "r"(r1[4 * j + 1]), "r"(r1[4 * j + 2]), "r"(r1[4 * j + 3]) : "memory");
+                for (int j = 0; j < 8; ++j) {
+                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(stg + lane * kStagePitch + j * 16), "r"(r0[4 * j]), "r"(r0[4 * j + 1]), "r"(r0[4 * j + 2]), "r"(r0[4 * j + 3]) : "memory");
+                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(stg + lane * kStagePitch + 128 + j * 16), "r"(r1[4 * j]), "r"(r1[4 * j + 1]), "r"(r1[4 * j + 2]), "r"(r1[4 * j + 3]) : "memory");
+                }
             }
             __syncwarp();
             // ... and leaves it two rows per instruction: 16 lanes cover the 256 bytes of a row piece
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const int rr = 2 * i + (lane >> 4), grow = q * 32 + rr;
+            for (int i = 0; i < kRowsPerWarp / 2; ++i) {
+                const int rr = 2 * i + (lane >> 4), grow = q * kRowsPerWarp + rr;
                 float4 v;
                 asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(stg + rr * kStagePitch + c * 16));
                 if (grow < cnt && col < p.pool.d_out) {
@@ -418,7 +426,7 @@ __device__ __forceinline__ void epilogue_warp(const Params& p, const Smem& sm, u
     }
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)
 sgmv_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_box, const Params p) {
     extern __shared__ uint8_t smem_raw[];
     const int n_tiles = *p.bk.n_sgmv_tiles;
@@ -515,7 +523,7 @@ cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, int
     // every tensor-core segment has at least sgmv_min_rows tokens: at most this many tiles
     const int min_rows = sgmv_min_rows < 1 ? 1 : sgmv_min_rows;
     long long max_tiles = (long long)n_tok / kRows + (long long)n_tok / min_rows + 1;
-    int grid = sm_count;   // one CTA per SM: the CTA holds all of the SM's tensor memory
+    int grid = 2 * sm_count;   // two CTAs per SM, half of its tensor memory each
     if (grid > max_tiles) grid = (int)max_tiles;
     if (grid < 1) grid = 1;
     sgmv_kernel<<<grid, kThreads, smem_bytes(p.R), stream>>>(tm, tm_box, p);
