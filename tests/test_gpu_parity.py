@@ -150,11 +150,11 @@ def _ids_from_runs(runs, shuffle_seed=None):
 
 @pytest.mark.parametrize("layout", ["contiguous", "shuffled", "broken_runs"])
 def test_sgmv_tile_shapes(layout):
-    # segment lengths around the 128-row tile and the 32-row copy box: whole tiles, ragged last tiles,
+    # segment lengths around the 64-row tile and the 32-row copy box: whole tiles, ragged last tiles,
     # a one-row tile, tokens that are consecutive (box copies), scattered (gather copies) or consecutive
     # in pieces that end inside a box
-    lens = [128, 129, 33, 255, 300, 1, 31, 64]
-    ranks = [8, 16, 32, 64, 128, 24, 5, 16]
+    lens = [128, 129, 33, 255, 300, 1, 31, 64, 65, 63]
+    ranks = [8, 16, 32, 64, 128, 24, 5, 16, 32, 8]
     if layout == "broken_runs":
         runs = []
         for rep in range(3):      # every adapter's tokens come as three separate runs of uneven length
