@@ -41,8 +41,8 @@ FALLBACK_HBM_GBS = 6650.0   # used only when MEASURED_PEAKS.json is absent
 # (profiles/*.md say which capture each number comes from); None = not captured.
 # Per (layer, proj) delta; the roofline entry scales it to the average launch (a launch may carry a group).
 NCU_TRAFFIC_BYTES = {
-    "decode7b": 40.19e6,   # profiles/bgmv_fused_config2_decode7b.md: (116.47 + 3.81 + 40.37 + 0.12) MB over q/k/v + o
-    "prefill": 622.5e6,    # profiles/sgmv_config4_prefill.md
+    "decode7b": 40.17e6,   # profiles/bgmv_fused_config2_decode7b.md: (116.41 + 3.89 + 40.29 + 0.09) MB over q/k/v + o
+    "prefill": 622.7e6,    # profiles/sgmv_config4_prefill.md
 }
 
 
