@@ -7,7 +7,7 @@ of the workload (for the default decode workload: 32 layers x q/k/v/o = 128
 calls over a 33.6 GB pool of 1000 rank-16 adapters per projection).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                  [--config 2|3|4|5] [--layers L] [--graph 0|1]
+                  [--config 2|3|4|5|6] [--layers L] [--graph 0|1]
 
 Prints ONE JSON line (rank 0).  `value` is tokens per second through the whole
 step with inputs resident in HBM; `e2e` is the same step through the host-buffer
@@ -487,7 +487,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4, 5])
+    ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4, 5, 6])
     ap.add_argument("--layers", type=int, default=None)
     ap.add_argument("--graph", type=int, default=1)
     ap.add_argument("--cpu-pools", type=int, default=64, dest="cpu_pools")

@@ -207,7 +207,10 @@ PLORA_API plora_status plora_create(plora_ctx** out, int device, int32_t max_tok
     const size_t o_sg = o_bg + up(T * sizeof(WorkUnit));
     const size_t o_m = o_sg + up(T * sizeof(WorkUnit));
     const size_t o_part = o_m + up(T * kMaxRank * 4);
-    const size_t part_bytes = up(T * 8192 > ((size_t)16 << 20) ? T * 8192 : ((size_t)16 << 20));
+    // partial-m hand-over of the fused kernel: one 64-bit word per (projection of a grouped call, token,
+    // shrink run, rank row)
+    const size_t part_need = T * kMaxGroupPools * kMaxRunsA * kMaxRank * sizeof(unsigned long long);
+    const size_t part_bytes = up(part_need > ((size_t)16 << 20) ? part_need : ((size_t)16 << 20));
     const size_t o_cls = o_part + part_bytes;
     const size_t total = o_cls + up(T * kMaxGroupPools * 4);
     uint8_t* blk = nullptr;

@@ -79,6 +79,11 @@ struct Params {
     int32_t runs_a, runs_b;   // tasks per unit in the shrink / expand phase
     int32_t early_tables;     // the bucket tables were complete before the previous kernel of the stream began
     int32_t by_class;         // the launch walks its class's part of bk.cls_list (pools of mixed ranks)
+    // The class launches of one call work on different units: a later one need not wait for the
+    // one before it.  It joins the stream order only when its CTAs are done (so that its completion
+    // still implies the completion of everything before it) and leaves the epoch to the last of them.
+    int32_t defer_wait;
+    int32_t bump_epoch;
     int32_t* status;
 };
 
@@ -201,8 +206,12 @@ __device__ __forceinline__ int tok_at(const StageHdr& h, int t) {
     return t == 1 ? h.tok[1] : t == 2 ? h.tok[2] : t == 3 ? h.tok[3] : h.tok[0];
 }
 
-__device__ __forceinline__ size_t part_index(const Params& p, int unit, int run, int t) {
-    return (((size_t)unit * p.runs_a + run) * kTokChunk + t) * p.pool.max_rp;
+// Where the partial m of (run, token) lives: a token is named by its projection and its position in
+// the sorted order (row0 = projection * n_tok + position of the unit's first token).  The layout does
+// not depend on a launch's own number of runs or on its rank class: the class launches of one call
+// share an epoch, so their units must not meet in the workspace.
+__device__ __forceinline__ size_t part_index(const Params& p, int row0, int run, int t) {
+    return (((size_t)row0 + t) * kMaxRunsA + run) * p.pool.max_rp;
 }
 constexpr int kMaxRowsPerLane = kMaxRank / 32;
 
@@ -539,7 +548,7 @@ __device__ __forceinline__ const unsigned long long* partial_src(const Params& p
 }
 __device__ __forceinline__ void partial_load(const Params& p, uint32_t epoch, const unsigned long long* src,
                                              unsigned long long (&w)[kMaxRunsA]) {
-    const size_t run_stride = (size_t)kTokChunk * p.pool.max_rp;
+    const size_t run_stride = (size_t)p.pool.max_rp;
 #pragma unroll
     for (int j = 0; j < kMaxRunsA; ++j)
         w[j] = j < p.runs_a ? ldg_cg_u64(src + j * run_stride) : ((unsigned long long)epoch << 32);
@@ -729,9 +738,10 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
     // the previous kernel drains.  (Pulling the first tiles towards L2 at that point was tried
     // and was slower: it competes with the draining kernel's own loads.)
     if (warp != kProducerWarp) {
-        grid_dependency_wait();
-        // Signalled only after this CTA has seen the previous kernel complete: when the next kernel
-        // of the stream starts, everything older than this kernel is therefore complete.
+        if (!p.defer_wait) grid_dependency_wait();
+        // Signalled only after this CTA has seen the previous kernel complete (or, for a class launch
+        // that defers its wait, after the first class launch of the call has): when the next kernel of
+        // the stream starts, everything older than this call is therefore complete.
         grid_launch_dependents();
         sm.epoch = MODE == kFused ? *p.bk.epoch : 0u;
     }
@@ -757,8 +767,8 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
         // alone waits for free stages, writes the headers and issues the copies of its task, so
         // the serial part of the producer is a few dozen instructions per stage.  In fused mode
         // the whole warp first gathers an expand task's m into the m ring.
-        bool waited = false;
-        if (!p.early_tables) {
+        bool waited = p.defer_wait != 0;
+        if (!waited && !p.early_tables) {
             grid_dependency_wait();
             waited = true;
         }
@@ -821,7 +831,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
                         const uint32_t tbytes = mine.phase ? mbytes : (uint32_t)min(C, d - i * C) * 2u;
                         mbar_wait(sm.empty + slot * 8, ((it / kStages) & 1) ^ 1, sm.abort_flag, p.status);
                         const int flags = (mine.phase ? kFlagExpand : 0) | (i == lo ? kFlagFirst : 0) | (i == hi - 1 ? kFlagLast : 0);
-                        sts128(dst + kHdrOffset, (uint32_t)flags, (uint32_t)mine.unit, (uint32_t)mine.run, (uint32_t)i);
+                        sts128(dst + kHdrOffset, (uint32_t)flags, (uint32_t)(my_group * p.n_tok + mu.pos0), (uint32_t)mine.run, (uint32_t)i);
                         sts128(dst + kHdrOffset + 16, (uint32_t)cnt, (uint32_t)mu.tok[0], (uint32_t)mu.tok[1], (uint32_t)mu.tok[2]);
                         sts128(dst + kHdrOffset + 32, (uint32_t)mu.tok[3], (uint32_t)me.rp, (uint32_t)me.r, __float_as_uint(me.scale));
                         sts128(dst + kHdrOffset + 48, m_seq, (uint32_t)my_group, 0u, 0u);
@@ -883,7 +893,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
             for (int b = 0; b < in_batch; ++b) {
                 const int rp_b = __shfl_sync(full, my_rp, b);
                 if (rp_b != RPK) continue;   // another launch's unit
-                const int unit_b = __shfl_sync(full, my_unit, b), cnt_b = __shfl_sync(full, mu.cnt, b);
+                const int unit_b = __shfl_sync(full, my_group * p.n_tok + mu.pos0, b), cnt_b = __shfl_sync(full, mu.cnt, b);
                 const uint32_t e = seq % kMRing;
                 if (lane == 0) mbar_wait(sm.m_empty + e * 8, ((seq / kMRing) & 1) ^ 1, sm.abort_flag, p.status);
                 __syncwarp();
@@ -920,8 +930,9 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
         const uint32_t empty_bar = sm.empty + slot * 8;
         consume_stage<MODE, RPK>(p, sm, h, maps, tile, empty_bar, acc, warp, lane);
     }
-    if (MODE == kFused && tid == 0) {
-        // the last CTA to finish opens the next epoch: words written by this launch can never
+    if (tid == 0 && p.defer_wait) grid_dependency_wait();
+    if (MODE == kFused && tid == 0 && p.bump_epoch) {
+        // the last CTA to finish opens the next epoch: words written by this call can never
         // be mistaken for the next one's
         if (atomicAdd(p.bk.exit_count, 1u) == gridDim.x - 1) {
             *p.bk.exit_count = 0u;
@@ -990,6 +1001,8 @@ cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const
     p.n_tok = n_tok;
     p.status = status;
     p.early_tables = early_tables ? 1 : 0;
+    p.defer_wait = 0;
+    p.bump_epoch = 1;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -1008,8 +1021,12 @@ cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const
         p.early_tables = 0;   // the first class launch reads what the classify pass has just written
     }
     // one launch per padded-rank class present in the pool
+    int last_rp = 8;
+    for (int rp = 8; rp <= kMaxRank; rp <<= 1)
+        if (rp_mask & rp) last_rp = rp;
     for (int rp = 8; rp <= kMaxRank; rp <<= 1) {
         if (!(rp_mask & rp)) continue;
+        p.bump_epoch = rp == last_rp;
         // a unit of this class has tiles_for(d, rp) tiles per phase: cut each phase into runs
         p.runs_a = mode == kShrinkOnly ? 1 : clamp_runs(tiles_for(pool.d_in, rp));
         // an expand task pays one round trip for its m before its first tile: give it at least two tiles
@@ -1019,10 +1036,9 @@ cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const
         // decode 7B shapes, 8: 0.748, 2: 0.757)
         if (p.runs_a > kMaxRunsA) p.runs_a = kMaxRunsA;
         if (mode == kFused) {
-            // the partial-m workspace holds n_units * runs_a * kTokChunk * max_rp words, n_units <= n_tok
-            const size_t per_run = (size_t)n_tok * n_groups * kTokChunk * pool.max_rp * sizeof(unsigned long long);
-            while (p.runs_a > 1 && per_run * p.runs_a > bk.m_part_bytes) --p.runs_a;
-            if (per_run * p.runs_a > bk.m_part_bytes) return cudaErrorMemoryAllocation;
+            // the partial-m workspace holds n_groups * n_tok * kMaxRunsA * max_rp words
+            const size_t need = (size_t)n_tok * n_groups * kMaxRunsA * pool.max_rp * sizeof(unsigned long long);
+            if (need > bk.m_part_bytes) return cudaErrorMemoryAllocation;
         }
         // persistent grid: two CTAs per SM, never more CTAs than there can be tasks
         const long long max_tasks = (long long)n_tok * n_groups * (p.runs_a + p.runs_b);
@@ -1040,6 +1056,7 @@ cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const
         ++*n_launches;
         if (e != cudaSuccess) return e;
         p.early_tables = 1;   // the next class's launch follows a kernel that is not the bucket kernel
+        p.defer_wait = mode == kFused ? 1 : 0;
     }
     return cudaSuccess;
 }

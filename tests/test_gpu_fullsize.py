@@ -17,7 +17,7 @@ from workloads import make_workload
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("cfg", [2, 3, 4, 5])
+@pytest.mark.parametrize("cfg", [2, 3, 4, 5, 6])
 def test_sampled_rows_match_oracle(cfg):
     wl = make_workload(cfg, n_layers=1)
     dw = DeviceWorkload(wl, 0)

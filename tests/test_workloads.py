@@ -16,7 +16,8 @@ def test_bf16_round_to_nearest_even():
     assert np.array_equal(f32_to_bf16_bits(x), want)
 
 
-@pytest.mark.parametrize("cfg,T,N", [(1, 64, 16), (2, 256, 1000), (3, 512, 1000), (4, 16384, 1000), (5, 2048, 1000)])
+@pytest.mark.parametrize("cfg,T,N", [(1, 64, 16), (2, 256, 1000), (3, 512, 1000), (4, 16384, 1000), (5, 2048, 1000),
+                                      (6, 256, 1000)])
 def test_shapes_and_determinism(cfg, T, N):
     a, b = make_workload(cfg), make_workload(cfg)
     assert a.n_tok == T and a.n_adapters == N and a.ids.shape == (T,)
@@ -67,3 +68,18 @@ def test_adapter_regenerates_alone_with_right_variance():
     x = gen_x(wl, pool)
     assert np.array_equal(x, gen_x(wl, wl.pools[0]))  # q and k read the same activations
     assert not np.array_equal(x, gen_x(wl, wl.pools[3]))
+
+
+def test_skewed_mix_sends_four_fifths_of_the_requests_to_fifty_adapters():
+    # the paper's skewed request distribution (its workload table): 80 % of the requests go to 50 adapters
+    shares = []
+    for seed in range(20):
+        wl = make_workload(6, n_tok=4096, seed=1000 + seed)
+        counts = np.sort(np.bincount(wl.ids, minlength=wl.n_adapters))[::-1]
+        shares.append(counts[:50].sum() / wl.n_tok)
+        assert set(np.unique(wl.ranks)) <= {8, 16, 32, 64, 128}
+        assert np.allclose(wl.scales * wl.ranks, 32.0)
+    assert abs(np.mean(shares) - 0.8) < 0.01
+    wl = make_workload(6)
+    assert wl.n_tok == 256 and len(wl.pools) == 8 * 4 and {(p.d_in, p.d_out) for p in wl.pools} == {(4096, 4096)}
+    assert set(np.unique(wl.ranks)) == {8, 16, 32, 64, 128}

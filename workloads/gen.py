@@ -1,4 +1,4 @@
-"""Seeded generators for the five benchmark-shaped workloads.
+"""Seeded generators for the benchmark-shaped workloads.
 
 Every array is a pure function of (config number, overrides, seed): a test can
 regenerate any single adapter, activation block or id vector without building
@@ -21,6 +21,10 @@ projection shapes — Section VII-A and its workload table):
               length U[2,256] filling 1024 more tokens, request order shuffled,
               q/o 8192->8192, per-adapter rank ~ U{8,16,32,64}, ids ~ bounded
               Zipf(0.8), s_a = 32/r_a
+  6 skew7b    the paper's own skewed request mix on the decode shapes of 2: 256
+              one-token requests, 80 % of them to 50 hot adapters (uniform inside
+              the hot and inside the cold set), per-adapter rank ~ U{8,16,32,64,128}
+              (the evaluation's rank set), q/k/v/o 4096->4096, s_a = 32/r_a
 
 Distributions: x ~ N(0,1); A ~ N(0, 1/d_in) (variance); B ~ N(0, 1/r)
 (variance); y_in ~ N(0,1).  Bounded Zipf: p_k proportional to k^-alpha for
@@ -35,7 +39,7 @@ import numpy as np
 
 BASE_SEED = 20260805 * 10
 
-CONFIG_NAMES = {1: "tiny", 2: "decode7b", 3: "decode13b", 4: "prefill", 5: "mixed"}
+CONFIG_NAMES = {1: "tiny", 2: "decode7b", 3: "decode13b", 4: "prefill", 5: "mixed", 6: "skew7b"}
 
 PROJ_NAMES = ("q", "k", "v", "o", "up", "gate", "down")
 # projections that read the same activation tensor share an x group
@@ -178,6 +182,22 @@ def make_workload(cfg: int, *, n_layers: int | None = None, n_adapters: int | No
         req_ids = _zipf_ids(_rng(seed, _TAG_IDS), _rng(seed, _TAG_POP), n_req, N, 1.2)
         ids = np.repeat(req_ids, req_len).astype(np.int32)
         meta.update(ids="zipf(1.2) per request", n_requests=n_req, request_len=req_len)
+    elif cfg == 6:
+        T, N, D, L = n_tok or 256, n_adapters or 1000, d_model or 4096, n_layers or 8
+        pools = _pools(L, (0, 1, 2, 3), {p: (D, D) for p in range(4)})
+        if rank is None:
+            ranks = _rng(seed, _TAG_RANKS).choice(np.array([8, 16, 32, 64, 128], np.int32), size=N).astype(np.int32)
+        else:
+            ranks = np.full(N, rank, np.int32)
+        scales = (32.0 / ranks.astype(np.float64)).astype(np.float32)
+        n_hot = min(50, max(1, N // 20))
+        order = _rng(seed, _TAG_POP).permutation(N)           # the first n_hot of it are the hot adapters
+        draw = _rng(seed, _TAG_IDS)
+        to_hot = draw.random(T) < 0.8
+        pick_hot = draw.integers(0, n_hot, size=T)
+        pick_cold = draw.integers(n_hot, N, size=T) if N > n_hot else pick_hot
+        ids = order[np.where(to_hot, pick_hot, pick_cold)].astype(np.int32)
+        meta.update(ids="80 % of requests to 50 hot adapters", n_hot=int(n_hot))
     else:  # cfg == 5
         T, N, D, L = n_tok or 2048, n_adapters or 1000, d_model or 8192, n_layers or 1
         pools = _pools(L, (0, 3), {0: (D, D), 3: (D, D)})
