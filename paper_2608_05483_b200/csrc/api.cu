@@ -416,7 +416,7 @@ PLORA_API plora_status plora_lora_delta(plora_ctx* ctx, const void* x, const int
         if (may_bgmv)
             e = launch_bgmv_one(kFused, pool->dev, ctx->bk, n_tok, x, y, nullptr, 0, ctx->status_dev, ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl);
         if (e == cudaSuccess && may_sgmv)
-            e = launch_sgmv(pool->dev, ctx->bk, n_tok, ctx->bucket_sgmv_min, x, y, ctx->status_dev, ctx->sm_count, st, &nl);
+            e = launch_sgmv(pool->dev, ctx->bk, n_tok, ctx->bucket_sgmv_min, x, y, ctx->status_dev, ctx->sm_count, may_bgmv, st, &nl);
     }
     ctx->launches += nl;
     return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
@@ -458,7 +458,7 @@ PLORA_API plora_status plora_lora_delta_group(plora_ctx* ctx, int32_t n, const v
                                 ctx->launches_since_bucket++ > 0, st, &nl);
     if (e == cudaSuccess && ctx->bucket_sgmv_min != INT_MAX)
         for (int g = 0; g < n && e == cudaSuccess; ++g)
-            e = launch_sgmv(pools[g], ctx->bk, n_tok, ctx->bucket_sgmv_min, x[g], y[g], ctx->status_dev, ctx->sm_count, st, &nl);
+            e = launch_sgmv(pools[g], ctx->bk, n_tok, ctx->bucket_sgmv_min, x[g], y[g], ctx->status_dev, ctx->sm_count, true, st, &nl);
     ctx->launches += nl;
     return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
 }

@@ -113,8 +113,11 @@ constexpr int kMaxGroupPools = 4;
 cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const BucketDev& bk, int n_tok,
                         const void* const* x, float* const* y, float* m, int ldm, int32_t* status, int sm_count,
                         bool early_tables, cudaStream_t stream, int* n_launches);
+// after_bgmv_of_same_call: the launch follows fused BGMV launches of the same call (other tokens of the
+// same batch) and may overlap them
 cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, int sgmv_min_rows, const void* x, float* y,
-                        int32_t* status, int sm_count, cudaStream_t stream, int* n_launches);
+                        int32_t* status, int sm_count, bool after_bgmv_of_same_call, cudaStream_t stream,
+                        int* n_launches);
 // per-device function attributes (dynamic shared memory); called by plora_create
 cudaError_t bucket_configure();
 cudaError_t bgmv_configure();

@@ -86,6 +86,10 @@ struct Params {
     int32_t* status;
     int32_t R;          // max(16, largest padded rank of the pool): sizes the shared-memory layout
     int32_t n_stages;
+    // The launch follows the BGMV launches of the same call, which work on other tokens: it need not
+    // wait for them.  It joins the stream order only when its CTAs are done, so that its completion
+    // still implies the completion of everything before it.
+    int32_t defer_wait;
 };
 
 // ---- PTX wrappers -----------------------------------------------------------------
@@ -429,8 +433,16 @@ __device__ __forceinline__ void epilogue_warp(const Params& p, const Smem& sm, u
 __global__ void __launch_bounds__(kThreads, 2)
 sgmv_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_box, const Params p) {
     extern __shared__ uint8_t smem_raw[];
+    // Launched with programmatic stream serialisation: nothing of the stream's earlier work is read
+    // before this wait, unless the launch defers it (then the kernels it overlaps are those of its own
+    // call, and everything older is complete because the first of them has waited).
+    if (!p.defer_wait) asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int n_tiles = *p.bk.n_sgmv_tiles;
-    if ((int)blockIdx.x >= n_tiles) return;   // nothing for this CTA (often: no tensor-core segment in the batch)
+    if ((int)blockIdx.x >= n_tiles) {   // nothing for this CTA (often: no tensor-core segment in the batch)
+        if (p.defer_wait && threadIdx.x == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
+        return;
+    }
     const Smem sm = carve(smem_raw, p);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
@@ -473,6 +485,7 @@ sgmv_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CU
     __syncthreads();
     if (warp == kMmaWarp)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)kTmemCols) : "memory");
+    if (p.defer_wait && tid == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -496,7 +509,8 @@ cudaError_t sgmv_configure() {
 }
 
 cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, int sgmv_min_rows, const void* x, float* y,
-                        int32_t* status, int sm_count, cudaStream_t stream, int* n_launches) {
+                        int32_t* status, int sm_count, bool after_bgmv_of_same_call, cudaStream_t stream,
+                        int* n_launches) {
     Params p;
     p.pool = pool;
     p.bk = bk;
@@ -504,6 +518,7 @@ cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, int
     p.status = status;
     p.R = pool.max_rp < 16 ? 16 : pool.max_rp;
     p.n_stages = stages_for(p.R);
+    p.defer_wait = after_bgmv_of_same_call ? 1 : 0;
     // x as a 2-D tensor [n_tok][d_in] of bf16; a gather instruction copies 64 columns of four rows,
     // 128-byte swizzled (columns beyond d_in read as zeros)
     CUtensorMap tm, tm_box;
@@ -526,9 +541,19 @@ cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, int
     int grid = 2 * sm_count;   // two CTAs per SM, half of its tensor memory each
     if (grid > max_tiles) grid = (int)max_tiles;
     if (grid < 1) grid = 1;
-    sgmv_kernel<<<grid, kThreads, smem_bytes(p.R), stream>>>(tm, tm_box, p);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem_bytes(p.R);
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, sgmv_kernel, tm, tm_box, p);
     ++*n_launches;
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace plora
