@@ -250,6 +250,36 @@ PLORA_API int64_t plora_launch_count(plora_ctx *ctx);
 
 PLORA_API const char *plora_status_string(plora_status s);
 
+/* ---- Cost model of the LoRA computation (paper Section VI-B: the table of per-strategy cost terms
+ * and the equation T_LoRA = max{T_Base, T_LoRA_dev} + T_LoRA_GPU).  Host arithmetic only: nothing
+ * is launched, no context is needed.  The benchmark's roofline is strategy E1's memory term of this
+ * model (every adapter present is read once per step, S bytes per value) plus the activations.
+ *
+ * Hardware: throughputs in flop/s, bandwidths in byte/s, latency in seconds. */
+typedef struct {
+    double c_gpu, w_gpu;    /* GPU compute throughput and HBM bandwidth */
+    double c_dev, w_dram;   /* per-device near-data compute throughput and DRAM bandwidth */
+    double n_dev;           /* number of devices */
+    double l_link, w_link;  /* one-way link latency and link bandwidth */
+} plora_cost_hw;
+
+/* Per strategy j = 0..3 (the paper's E1..E4): GPU time, device compute time, device-to-GPU transfer
+ * time; then the sums over the strategies and the total. */
+typedef struct {
+    double t_gpu[4], t_dev_cpt[4], t_dev_trs[4];
+    double t_lora_gpu, t_lora_dev, t_lora;
+} plora_cost_terms;
+
+/* ranks: host [n_adapters], R_i >= 1.  batch: host [n_adapters][4] row-major, batch[i][j] = requests of
+ * adapter i served under strategy E(j+1), >= 0.  d: model dimension D.  value_bytes: S (2 under FP16).
+ * t_base: profiled base-model GPU time.  A strategy nobody uses contributes zero to every term; a
+ * memory argument sums only over the adapters that serve a request under that strategy.
+ * Returns PLORA_ERR_INVALID_ARG for null pointers, non-positive hardware parameters, d, value_bytes or
+ * ranks, or negative batch entries. */
+PLORA_API plora_status plora_cost_model(const plora_cost_hw *hw, int32_t n_adapters, const int32_t *ranks,
+                                        const double *batch, double d, double value_bytes, double t_base,
+                                        plora_cost_terms *out);
+
 #ifdef __cplusplus
 }
 #endif

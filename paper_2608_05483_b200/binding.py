@@ -31,6 +31,7 @@ EXPORTS = (
     "plora_create", "plora_destroy", "plora_pool_slab_bytes", "plora_register_pool", "plora_pool_max_rank",
     "plora_bucket", "plora_bucket_view", "plora_lora_delta", "plora_lora_delta_group", "plora_shrink", "plora_expand",
     "plora_lora_delta_host", "plora_lora_delta_noalloc", "plora_set_path", "plora_device_status", "plora_launch_count", "plora_status_string",
+    "plora_cost_model",
 )
 
 
@@ -42,6 +43,15 @@ class PoolDesc(ctypes.Structure):
         ("ranks", ctypes.c_void_p), ("scales", ctypes.c_void_p),
         ("A", ctypes.c_void_p), ("B", ctypes.c_void_p),
     ]
+
+
+class CostHw(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_double) for n in ("c_gpu", "w_gpu", "c_dev", "w_dram", "n_dev", "l_link", "w_link")]
+
+
+class CostTerms(ctypes.Structure):
+    _fields_ = [("t_gpu", ctypes.c_double * 4), ("t_dev_cpt", ctypes.c_double * 4), ("t_dev_trs", ctypes.c_double * 4),
+                ("t_lora_gpu", ctypes.c_double), ("t_lora_dev", ctypes.c_double), ("t_lora", ctypes.c_double)]
 
 
 class PloraError(RuntimeError):
@@ -87,6 +97,8 @@ def load(build_if_missing: bool = True):
         "plora_device_status": (i32, [vp, vp, ctypes.POINTER(i32)]),
         "plora_launch_count": (i64, [vp]),
         "plora_status_string": (ctypes.c_char_p, [i32]),
+        "plora_cost_model": (i32, [ctypes.POINTER(CostHw), i32, vp, vp, ctypes.c_double, ctypes.c_double, ctypes.c_double,
+                                   ctypes.POINTER(CostTerms)]),
     }
     for name in EXPORTS:
         fn = getattr(lib, name)  # AttributeError here = the library does not export what the header declares
@@ -108,6 +120,21 @@ def plora_create(device: int, max_tokens: int, max_adapters: int):
 
 def plora_destroy(ctx):
     return load().plora_destroy(ctx)
+
+
+def plora_cost_model(hw: dict, ranks, batch, d: float, value_bytes: float, t_base: float):
+    """(status, terms): the cost terms of the paper's four strategies (Section VI-B) as a dict of lists / floats.
+    hw: c_gpu, w_gpu, c_dev, w_dram, n_dev, l_link, w_link.  batch: [n_adapters][4] request counts."""
+    import numpy as np
+    r = np.ascontiguousarray(ranks, np.int32)
+    b = np.ascontiguousarray(batch, np.float64).reshape(len(r), 4)
+    chw = CostHw(**{k: float(v) for k, v in hw.items()})
+    out = CostTerms()
+    rc = load().plora_cost_model(ctypes.byref(chw), len(r), r.ctypes.data, b.ctypes.data, float(d), float(value_bytes),
+                                 float(t_base), ctypes.byref(out))
+    terms = dict(t_gpu=list(out.t_gpu), t_dev_cpt=list(out.t_dev_cpt), t_dev_trs=list(out.t_dev_trs),
+                 t_lora_gpu=out.t_lora_gpu, t_lora_dev=out.t_lora_dev, t_lora=out.t_lora)
+    return rc, terms
 
 
 def plora_pool_slab_bytes(desc: PoolDesc) -> int:
