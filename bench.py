@@ -422,11 +422,11 @@ def run_ours(args):
         out = dict(metric="LoRA-delta tokens/sec at 1000 adapters (whole step: bucket + every layer x projection delta)",
                    value=whole_job_tokens_per_s(wl.n_tok, world, ms_per_step), unit="tokens/s", n_gpus=world, steps=args.steps,
                    warmup=max(3, args.warmup), ms_per_step=ms_per_step, higher_is_better=True, scaling="weak",
-                   vs_baseline=None, dtype="bf16 in, fp32 accumulate", data="synthetic",
+                   vs_baseline=None, dtype="bf16", data="synthetic",
                    config=dict(workload=f"config {args.config} ({wl.name})", n_tok=wl.n_tok, n_adapters=wl.n_adapters,
                                layers=len({p.layer for p in wl.pools}), calls_per_step=n_calls,
                                ranks=sorted({int(r) for r in wl.ranks}), ids=wl.meta.get("ids"),
-                               distinct_adapters=per_call[0]["distinct"], path=args.path, cuda_graph=bool(args.graph), grouped_calls=not args.no_group,
+                               accumulate="fp32", y="fp32", distinct_adapters=per_call[0]["distinct"], path=args.path, cuda_graph=bool(args.graph), grouped_calls=not args.no_group,
                                l2="inputs larger than L2: a step streams %.2f GB through %d distinct slabs"
                                   % (step_bytes / 1e9, n_calls),
                                multi_gpu="replicas: every rank runs its own batch, no data-path collective"),
@@ -491,7 +491,7 @@ def main():
     ap.add_argument("--layers", type=int, default=None)
     ap.add_argument("--graph", type=int, default=1)
     ap.add_argument("--cpu-pools", type=int, default=64, dest="cpu_pools")
-    ap.add_argument("--cpu-seconds", type=float, default=10.0, dest="cpu_seconds",
+    ap.add_argument("--cpu-seconds", type=float, default=20.0, dest="cpu_seconds",
                     help="target CPU time of the oracle sample (cpu_baseline leg)")
     ap.add_argument("--path", default="auto", choices=["auto", "fused", "unfused", "sgmv"])
     ap.add_argument("--no-group", action="store_true", dest="no_group",
