@@ -185,6 +185,52 @@ def test_mixed_rank_calls_repeat_bit_for_bit():
         r.close()
 
 
+def test_cuda_graph_replay_of_a_mixed_call_sequence():
+    # bucket + two dependent deltas (AUTO: classify, overlapping class launches, SGMV) captured once and
+    # replayed: every replay must give the bits of the eager run
+    rng = np.random.default_rng(31)
+    N = 200
+    ids = np.concatenate([np.repeat(rng.permutation(N)[:130], 64), rng.integers(0, N, size=300)]).astype(np.int32)
+    p = random_problem(32, T=len(ids), d_in=256, d_out=320, ranks=rng.choice([8, 16, 32, 64, 128], size=N))
+    p["ids"] = ids
+    r = Runner(p)
+    try:
+        r.ctx.set_path(P.PATH_AUTO, sgmv_min_rows=32)
+        y_in = torch.from_numpy(p["y_in"]).to(DEV)
+        y = y_in.clone()
+
+        def step():
+            r.ctx.bucket(r.ids, p["N"])
+            r.ctx.lora_delta(r.x, r.ids, 0, 0, y)       # y += delta(x)
+            r.ctx.lora_delta(r.x, r.ids, 0, 0, y)       # and once more: depends on the first through y
+
+        n0 = r.ctx.launch_count()
+        step()
+        torch.cuda.synchronize()
+        assert r.ctx.launch_count() - n0 == 1 + 2 * (1 + 5 + 1)   # bucket; per delta: classify, five classes, SGMV
+        eager = y.cpu().numpy().copy()
+        ref = _oracle(p)
+        want = p["y_in"].astype(np.float64) + 2 * ref
+        assert np.max(np.abs(eager - want)) <= TOL_FP32_PATH * np.max(np.abs(ref)) + 2e-6 * np.max(np.abs(want))
+        s = torch.cuda.Stream()
+        s.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(s):
+            step()
+        torch.cuda.current_stream().wait_stream(s)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            step()
+        for _ in range(20):
+            y.copy_(y_in)
+            g.replay()
+            torch.cuda.synchronize()
+            assert y.cpu().numpy().tobytes() == eager.tobytes()
+        assert r.ctx.device_status() == 0
+    finally:
+        r.close()
+
+
 def test_empty_and_all_minus_one():
     p = random_problem(1, T=0, d_in=64, d_out=64, ranks=[8])
     r = Runner(p, max_tokens=8)
