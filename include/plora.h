@@ -192,6 +192,21 @@ PLORA_API plora_status plora_shrink(plora_ctx *ctx, const void *x_dev, const int
 PLORA_API plora_status plora_expand(plora_ctx *ctx, const float *m_dev, int32_t ldm, const int32_t *adapter_ids_dev,
                           int32_t n_tok, int32_t layer, int32_t proj, float *y_dev, void *stream);
 
+/* The same split with a 2-byte m, as the paper's strategy E4 ships it between the two halves
+ * (Section VI-B: its transfer term counts S = 2 bytes per value of m).
+ * plora_shrink_m16: m_bf16[t, 0..ldm) = bf16(x_t A[a_t]), rounded to nearest even from the fp32 sum;
+ * zeros beyond the adapter's rank and for tokens without an adapter.  plora_expand_m16:
+ * y_t += s * m_bf16[t] * B[a_t], values beyond the adapter's rank ignored.  m_bf16: device, bf16
+ * [n_tok, ldm] row-major, 16-byte aligned, ldm >= the pool's largest padded rank and a multiple of 8.
+ * One rounding of m to bf16 costs about 2e-3 of max|delta| (inside the 5e-3 contract, far above the
+ * fp32 path's 2e-7).  Same errors and stream semantics as plora_shrink / plora_expand. */
+PLORA_API plora_status plora_shrink_m16(plora_ctx *ctx, const void *x_bf16_dev, const int32_t *adapter_ids_dev,
+                                        int32_t n_tok, int32_t layer, int32_t proj, void *m_bf16_dev, int32_t ldm,
+                                        void *stream);
+PLORA_API plora_status plora_expand_m16(plora_ctx *ctx, const void *m_bf16_dev, int32_t ldm,
+                                        const int32_t *adapter_ids_dev, int32_t n_tok, int32_t layer, int32_t proj,
+                                        float *y_dev, void *stream);
+
 /*
  * Same operation as plora_lora_delta with HOST buffers: copies x, ids and y to
  * context-owned device staging buffers, buckets, runs the delta and copies y

@@ -30,6 +30,7 @@ PATH_AUTO, PATH_UNFUSED, PATH_FUSED, PATH_SGMV = 0, 1, 2, 3
 EXPORTS = (
     "plora_create", "plora_destroy", "plora_pool_slab_bytes", "plora_register_pool", "plora_pool_max_rank",
     "plora_bucket", "plora_bucket_view", "plora_lora_delta", "plora_lora_delta_group", "plora_shrink", "plora_expand",
+    "plora_shrink_m16", "plora_expand_m16",
     "plora_lora_delta_host", "plora_lora_delta_noalloc", "plora_set_path", "plora_device_status", "plora_launch_count", "plora_status_string",
     "plora_cost_model",
 )
@@ -91,6 +92,8 @@ def load(build_if_missing: bool = True):
         "plora_lora_delta_group": (i32, [vp, i32, vp, vp, i32, vp, vp, vp, vp]),
         "plora_shrink": (i32, [vp, vp, vp, i32, i32, i32, vp, i32, vp]),
         "plora_expand": (i32, [vp, vp, i32, vp, i32, i32, i32, vp, vp]),
+        "plora_shrink_m16": (i32, [vp, vp, vp, i32, i32, i32, vp, i32, vp]),
+        "plora_expand_m16": (i32, [vp, vp, i32, vp, i32, i32, i32, vp, vp]),
         "plora_lora_delta_host": (i32, [vp, vp, vp, i32, i32, i32, vp, vp]),
         "plora_lora_delta_noalloc": (i32, [vp, vp, vp, i32, i32, i32, vp, vp]),
         "plora_set_path": (i32, [vp, i32, i32]),
@@ -181,6 +184,14 @@ def plora_shrink(ctx, x_ptr, ids_ptr, n_tok, layer, proj, m_ptr, ldm, stream=0):
 
 def plora_expand(ctx, m_ptr, ldm, ids_ptr, n_tok, layer, proj, y_ptr, stream=0):
     return load().plora_expand(ctx, m_ptr, ldm, ids_ptr, n_tok, layer, proj, y_ptr, stream)
+
+
+def plora_shrink_m16(ctx, x_ptr, ids_ptr, n_tok, layer, proj, m_ptr, ldm, stream=0):
+    return load().plora_shrink_m16(ctx, x_ptr, ids_ptr, n_tok, layer, proj, m_ptr, ldm, stream)
+
+
+def plora_expand_m16(ctx, m_ptr, ldm, ids_ptr, n_tok, layer, proj, y_ptr, stream=0):
+    return load().plora_expand_m16(ctx, m_ptr, ldm, ids_ptr, n_tok, layer, proj, y_ptr, stream)
 
 
 def plora_lora_delta_host(ctx, x_host_ptr, ids_host_ptr, n_tok, layer, proj, y_host_ptr, stream=0):
@@ -343,6 +354,14 @@ class Context:
     def expand(self, m, ids, layer, proj, y, stream=None):
         _check(plora_expand(self._h, m.data_ptr(), int(m.shape[1]), ids.data_ptr(), int(ids.numel()), layer, proj,
                             y.data_ptr(), _stream_handle(stream)), "plora_expand")
+
+    def shrink_m16(self, x, ids, layer, proj, m_bf16, stream=None):
+        _check(plora_shrink_m16(self._h, x.data_ptr(), ids.data_ptr(), int(ids.numel()), layer, proj, m_bf16.data_ptr(),
+                                int(m_bf16.shape[1]), _stream_handle(stream)), "plora_shrink_m16")
+
+    def expand_m16(self, m_bf16, ids, layer, proj, y, stream=None):
+        _check(plora_expand_m16(self._h, m_bf16.data_ptr(), int(m_bf16.shape[1]), ids.data_ptr(), int(ids.numel()), layer,
+                                proj, y.data_ptr(), _stream_handle(stream)), "plora_expand_m16")
 
     def lora_delta_host(self, x_host, ids_host, layer, proj, y_host, stream=None):
         """x_host / ids_host / y_host: CPU torch tensors (pinned or not) or numpy arrays; y_host is updated in place."""

@@ -146,11 +146,11 @@ plora_status ensure_bucket(plora_ctx* ctx, const int32_t* ids, int32_t n_tok, in
 }
 
 cudaError_t launch_bgmv_one(BgmvMode mode, const PoolDev& pool, const BucketDev& bk, int n_tok, const void* x, float* y,
-                            float* m, int ldm, int32_t* status, int sm_count, bool early_tables, cudaStream_t stream,
-                            int* n_launches) {
+                            void* m, int ldm, int32_t* status, int sm_count, bool early_tables, cudaStream_t stream,
+                            int* n_launches, bool m16 = false) {
     const void* xs[1] = {x};
     float* ys[1] = {y};
-    return launch_bgmv(mode, &pool, 1, bk, n_tok, xs, ys, m, ldm, status, sm_count, early_tables, stream, n_launches);
+    return launch_bgmv(mode, &pool, 1, bk, n_tok, xs, ys, m, ldm, m16, status, sm_count, early_tables, stream, n_launches);
 }
 
 plora_status check_call(plora_ctx* ctx, const void* a, const void* ids, int32_t n_tok, const void* b) {
@@ -454,7 +454,7 @@ PLORA_API plora_status plora_lora_delta_group(plora_ctx* ctx, int32_t n, const v
     PoolDev pools[kMaxGroupPools];
     for (int g = 0; g < n; ++g) pools[g] = recs[g]->dev;
     int nl = 0;
-    cudaError_t e = launch_bgmv(kFused, pools, n, ctx->bk, n_tok, x, y, nullptr, 0, ctx->status_dev, ctx->sm_count,
+    cudaError_t e = launch_bgmv(kFused, pools, n, ctx->bk, n_tok, x, y, nullptr, 0, false, ctx->status_dev, ctx->sm_count,
                                 ctx->launches_since_bucket++ > 0, st, &nl);
     if (e == cudaSuccess && ctx->bucket_sgmv_min != INT_MAX)
         for (int g = 0; g < n && e == cudaSuccess; ++g)
@@ -463,51 +463,51 @@ PLORA_API plora_status plora_lora_delta_group(plora_ctx* ctx, int32_t n, const v
     return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
 }
 
-PLORA_API plora_status plora_shrink(plora_ctx* ctx, const void* x, const int32_t* ids, int32_t n_tok, int32_t layer, int32_t proj,
-                          float* m, int32_t ldm, void* stream) {
-    plora_status rc = check_call(ctx, x, ids, n_tok, m);
+namespace {
+// The split entry points always take the BGMV kernels: bucket with no tensor-core segments.
+plora_status split_call(plora_ctx* ctx, BgmvMode mode, const void* x, void* m, int32_t ldm, bool m16, const int32_t* ids,
+                        int32_t n_tok, int32_t layer, int32_t proj, float* y, void* stream) {
+    plora_status rc = check_call(ctx, mode == kShrinkOnly ? x : m, ids, n_tok, mode == kShrinkOnly ? m : (void*)y);
     if (rc != PLORA_OK) return rc;
     PoolRec* pool = find_pool(ctx, layer, proj);
     if (!pool) return PLORA_ERR_NOT_REGISTERED;
-    if (ldm < pool->dev.max_rp || (ldm & 3)) return PLORA_ERR_INVALID_ARG;
+    // rows of m start on 16-byte boundaries (the expand copies them in bulk)
+    if (ldm < pool->dev.max_rp || (ldm & (m16 ? 7 : 3))) return PLORA_ERR_INVALID_ARG;
     if (n_tok == 0) return PLORA_OK;
     DeviceGuard g(ctx->device);
     if (!g.ok) return PLORA_ERR_CUDA;
     cudaStream_t st = as_stream(stream);
-    // the split entry points always take the BGMV kernels: bucket with no tensor-core segments
     const int32_t saved = ctx->path;
     ctx->path = PLORA_PATH_UNFUSED;
     rc = ensure_bucket(ctx, ids, n_tok, pool->dev.n_adapters, st);
     ctx->path = saved;
     if (rc != PLORA_OK) return rc;
     int nl = 0;
-    cudaError_t e = launch_bgmv_one(kShrinkOnly, pool->dev, ctx->bk, n_tok, x, nullptr, m, ldm, ctx->status_dev,
-                                ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl);
+    cudaError_t e = launch_bgmv_one(mode, pool->dev, ctx->bk, n_tok, x, y, m, ldm, ctx->status_dev, ctx->sm_count,
+                                    ctx->launches_since_bucket++ > 0, st, &nl, m16);
     ctx->launches += nl;
     return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
+}
+}  // namespace
+
+PLORA_API plora_status plora_shrink(plora_ctx* ctx, const void* x, const int32_t* ids, int32_t n_tok, int32_t layer, int32_t proj,
+                          float* m, int32_t ldm, void* stream) {
+    return split_call(ctx, kShrinkOnly, x, m, ldm, false, ids, n_tok, layer, proj, nullptr, stream);
 }
 
 PLORA_API plora_status plora_expand(plora_ctx* ctx, const float* m, int32_t ldm, const int32_t* ids, int32_t n_tok,
                           int32_t layer, int32_t proj, float* y, void* stream) {
-    plora_status rc = check_call(ctx, m, ids, n_tok, y);
-    if (rc != PLORA_OK) return rc;
-    PoolRec* pool = find_pool(ctx, layer, proj);
-    if (!pool) return PLORA_ERR_NOT_REGISTERED;
-    if (ldm < pool->dev.max_rp || (ldm & 3)) return PLORA_ERR_INVALID_ARG;
-    if (n_tok == 0) return PLORA_OK;
-    DeviceGuard g(ctx->device);
-    if (!g.ok) return PLORA_ERR_CUDA;
-    cudaStream_t st = as_stream(stream);
-    const int32_t saved = ctx->path;
-    ctx->path = PLORA_PATH_UNFUSED;
-    rc = ensure_bucket(ctx, ids, n_tok, pool->dev.n_adapters, st);
-    ctx->path = saved;
-    if (rc != PLORA_OK) return rc;
-    int nl = 0;
-    cudaError_t e = launch_bgmv_one(kExpandOnly, pool->dev, ctx->bk, n_tok, nullptr, y, const_cast<float*>(m), ldm,
-                                ctx->status_dev, ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl);
-    ctx->launches += nl;
-    return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
+    return split_call(ctx, kExpandOnly, nullptr, const_cast<float*>(m), ldm, false, ids, n_tok, layer, proj, y, stream);
+}
+
+PLORA_API plora_status plora_shrink_m16(plora_ctx* ctx, const void* x, const int32_t* ids, int32_t n_tok, int32_t layer,
+                                        int32_t proj, void* m_bf16, int32_t ldm, void* stream) {
+    return split_call(ctx, kShrinkOnly, x, m_bf16, ldm, true, ids, n_tok, layer, proj, nullptr, stream);
+}
+
+PLORA_API plora_status plora_expand_m16(plora_ctx* ctx, const void* m_bf16, int32_t ldm, const int32_t* ids, int32_t n_tok,
+                                        int32_t layer, int32_t proj, float* y, void* stream) {
+    return split_call(ctx, kExpandOnly, nullptr, const_cast<void*>(m_bf16), ldm, true, ids, n_tok, layer, proj, y, stream);
 }
 
 PLORA_API plora_status plora_lora_delta_host(plora_ctx* ctx, const void* x_host, const int32_t* ids_host, int32_t n_tok,

@@ -73,8 +73,9 @@ struct Params {
     const AdapterEntry* table_g[kMaxGroup];
     const uint16_t* x_g[kMaxGroup];
     float* y_g[kMaxGroup];
-    float* m;
+    float* m;                 // shrink-only / expand-only: the caller's m, fp32 or (m16) bf16, ldm values per token
     int32_t ldm;
+    int32_t m16;              // m holds 2-byte values (the paper's strategy E4 ships m at S = 2 bytes)
     int32_t n_tok;
     int32_t runs_a, runs_b;   // tasks per unit in the shrink / expand phase
     int32_t early_tables;     // the bucket tables were complete before the previous kernel of the stream began
@@ -210,6 +211,15 @@ __device__ __forceinline__ int tok_at(const StageHdr& h, int t) {
 // the sorted order (row0 = projection * n_tok + position of the unit's first token).  The layout does
 // not depend on a launch's own number of runs or on its rank class: the class launches of one call
 // share an epoch, so their units must not meet in the workspace.
+// One value of the caller's m (shrink-only mode): fp32, or bf16 rounded to nearest even.
+__device__ __forceinline__ void store_m(const Params& p, size_t idx, float v) {
+    if (p.m16) {
+        const uint32_t u = __float_as_uint(v);
+        reinterpret_cast<uint16_t*>(p.m)[idx] = (uint16_t)((u + 0x7fffu + ((u >> 16) & 1u)) >> 16);
+    } else {
+        p.m[idx] = v;
+    }
+}
 __device__ __forceinline__ size_t part_index(const Params& p, int row0, int run, int t) {
     return (((size_t)row0 + t) * kMaxRunsA + run) * p.pool.max_rp;
 }
@@ -369,7 +379,7 @@ __device__ __forceinline__ void shrink_finish_cnt(const Params& p, const Smem& s
                     p.bk.m_part[part_index(p, h.unit, h.run, t) + k] =
                         ((unsigned long long)sm.epoch << 32) | (unsigned long long)__float_as_uint(val[j]);
                 } else {
-                    p.m[(size_t)tok_at(h, t) * p.ldm + k] = val[j];
+                    store_m(p, (size_t)tok_at(h, t) * p.ldm + k, val[j]);
                 }
             }
         }
@@ -390,7 +400,7 @@ __device__ __forceinline__ void shrink_finish(const Params& p, const Smem& sm, c
         const int extra = p.ldm - RP;
         for (int idx = warp * 32 + lane; idx < h.cnt * extra; idx += kConsumerThreads) {
             const int t = idx / extra, k = RP + idx % extra;
-            p.m[(size_t)tok_at(h, t) * p.ldm + k] = 0.f;
+            store_m(p, (size_t)tok_at(h, t) * p.ldm + k, 0.f);
         }
     }
 }
@@ -441,7 +451,14 @@ __device__ __forceinline__ void expand_tile_cnt(const Params& p, const Smem& sm,
         for (int q = 0; q < 4; ++q) braw[q] = lds32((b0 ^ (((kk + q) & 7) << 4)) + (kk + q) * 128);
 #pragma unroll
         for (int t = 0; t < CNT; ++t) {
-            mv[t] = lds128(mb + t * (RP * 4) + kk * 4);
+            if (MODE == kExpandOnly && p.m16) {
+                // 2-byte m: four bf16 values of this token, widened (exactly) to fp32
+                const uint32_t a16 = tile + kTileBytesMax + t * (RP * 2) + (mp.rg * M::RPG + kk) * 2;
+                const uint32_t w0 = lds32(a16), w1 = lds32(a16 + 4);
+                mv[t] = make_uint4(w0 << 16, w0 & 0xffff0000u, w1 << 16, w1 & 0xffff0000u);
+            } else {
+                mv[t] = lds128(mb + t * (RP * 4) + kk * 4);
+            }
             if (MODE == kExpandOnly && h.r < RP) {
                 // the caller's m may hold anything beyond the adapter's rank
                 const int k0 = mp.rg * M::RPG + kk;
@@ -755,7 +772,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
         for (long long i = (long long)blockIdx.x * (kThreads - 32) + wtid; i < total;
              i += (long long)gridDim.x * (kThreads - 32)) {
             const int pos = n_active + (int)(i / p.ldm);
-            p.m[(size_t)p.bk.perm[pos] * p.ldm + (int)(i % p.ldm)] = 0.f;
+            store_m(p, (size_t)p.bk.perm[pos] * p.ldm + (int)(i % p.ldm), 0.f);
         }
     }
 
@@ -822,7 +839,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
                 if (lane == b) {
                     const int cnt = mu.cnt;
                     // bytes a token adds to a stage besides the tile: its x piece (shrink) or its m row (expand-only)
-                    const uint32_t mbytes = (MODE == kExpandOnly) ? (uint32_t)me.rp * 4u : 0u;
+                    const uint32_t mbytes = (MODE == kExpandOnly) ? (uint32_t)me.rp * (p.m16 ? 2u : 4u) : 0u;
                     uint32_t it = my_it0;
                     for (int i = lo; i < hi; ++i, ++it) {
                         const uint32_t slot = it % kStages;
@@ -847,7 +864,8 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
 #pragma unroll
                             for (int t = 0; t < kTokChunk; ++t)   // the caller's m row, rp floats, lands as m[t][0..rp)
                                 if (t < cnt)
-                                    bulk_g2s(dst + kTileBytesMax + t * mbytes, p.m + (size_t)mu.tok[t] * p.ldm, mbytes, bar);
+                                    bulk_g2s(dst + kTileBytesMax + t * mbytes,
+                                             reinterpret_cast<const uint8_t*>(p.m) + (size_t)mu.tok[t] * p.ldm * (p.m16 ? 2 : 4), mbytes, bar);
                         }
                     }
                 }
@@ -979,7 +997,7 @@ cudaError_t bgmv_configure() {
 }
 
 cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const BucketDev& bk, int n_tok,
-                        const void* const* x, float* const* y, float* m, int ldm, int32_t* status, int sm_count,
+                        const void* const* x, float* const* y, void* m, int ldm, bool m16, int32_t* status, int sm_count,
                         bool early_tables, cudaStream_t stream, int* n_launches) {
     if (n_groups < 1 || n_groups > kMaxGroup || (mode != kFused && n_groups != 1)) return cudaErrorInvalidValue;
     const PoolDev& pool = pools[0];
@@ -996,8 +1014,9 @@ cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const
         p.y_g[g] = y ? y[gg] : nullptr;
         if (g < n_groups) rp_mask |= pools[g].rp_mask;
     }
-    p.m = m;
+    p.m = static_cast<float*>(m);
     p.ldm = ldm;
+    p.m16 = m16 ? 1 : 0;
     p.n_tok = n_tok;
     p.status = status;
     p.early_tables = early_tables ? 1 : 0;

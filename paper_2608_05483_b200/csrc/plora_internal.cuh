@@ -110,8 +110,9 @@ enum BgmvMode { kFused = 0, kShrinkOnly = 1, kExpandOnly = 2 };
 // pools[0 .. n_groups): projections of one launch (same shape; more than one only in fused mode);
 // x / y: per-projection pointers (x unused by the expand-only mode, y by the shrink-only mode)
 constexpr int kMaxGroupPools = 4;
+// m / ldm / m16: the caller's m of the shrink-only and expand-only modes, fp32 or (m16) bf16 values
 cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const BucketDev& bk, int n_tok,
-                        const void* const* x, float* const* y, float* m, int ldm, int32_t* status, int sm_count,
+                        const void* const* x, float* const* y, void* m, int ldm, bool m16, int32_t* status, int sm_count,
                         bool early_tables, cudaStream_t stream, int* n_launches);
 // after_bgmv_of_same_call: the launch follows fused BGMV launches of the same call (other tokens of the
 // same batch) and may overlap them

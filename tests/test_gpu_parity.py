@@ -282,6 +282,48 @@ def test_out_of_range_id_is_skipped_and_flagged():
     r.close()
 
 
+def test_two_byte_m_between_shrink_and_expand():
+    # the paper's strategy E4 ships m at 2 bytes per value: shrink rounds the fp32 sum to bf16, expand widens it again
+    from workloads import bf16_bits_to_f64, f32_to_bf16_bits
+    p = random_problem(78, T=53, d_in=776, d_out=520, ranks=[8, 24, 64, 5, 128], with_minus_one=True)
+    r = Runner(p)
+    try:
+        ldm = r.ctx.pool_max_rank(0, 0)
+        assert ldm == 128
+        m16 = torch.full((p["T"], ldm), 7.0, dtype=torch.bfloat16, device=DEV)
+        r.ctx.shrink_m16(r.x, r.ids, 0, 0, m16)
+        torch.cuda.synchronize()
+        got_bits = m16.view(torch.int16).cpu().numpy().view(np.uint16)
+        m_ref = oracle.shrink(p["x"], p["ids"], p["ranks"], p["A"], ldm=ldm)
+        want_bits = f32_to_bf16_bits(m_ref.astype(np.float32))
+        # the same value rounded from an fp32 sum (device) or from the float64 sum (oracle) may fall on either side
+        # of a rounding boundary: at most one bf16 step apart, and only rarely
+        step = np.abs(got_bits.astype(np.int32) - want_bits.astype(np.int32))
+        assert step.max() <= 1 and (step > 0).mean() < 0.01
+        assert np.all(got_bits[m_ref == 0] == 0)       # padding columns and id -1 rows are exact zeros
+        # expand from a given 2-byte m: no rounding decision left, the fp32-path bound applies
+        m_in = torch.from_numpy(want_bits.view(np.int16)).to(DEV).view(torch.bfloat16)
+        y = torch.from_numpy(p["y_in"]).to(DEV)
+        r.ctx.expand_m16(m_in, r.ids, 0, 0, y)
+        torch.cuda.synchronize()
+        ref = oracle.expand(bf16_bits_to_f64(want_bits), p["ids"], p["ranks"], p["scales"], p["B"], p["d_out"], p["y_in"])
+        delta = oracle.lora_delta(p["x"], p["ids"], p["ranks"], p["scales"], p["A"], p["B"], p["d_out"], None)
+        assert np.max(np.abs(y.cpu().numpy() - ref)) <= TOL_FP32_PATH * np.max(np.abs(delta)) + 1e-6 * np.max(np.abs(ref))
+        # the pair against the unrounded definition: inside the contract, with the cost of one bf16 rounding
+        y2 = torch.zeros((p["T"], p["d_out"]), dtype=torch.float32, device=DEV)
+        r.ctx.expand_m16(m16, r.ids, 0, 0, y2)
+        torch.cuda.synchronize()
+        err = rel_err(y2.cpu().numpy(), delta)
+        assert 1e-5 < err <= TOL_CONTRACT
+        # ldm must keep the rows of m 16-byte aligned
+        bad = torch.zeros((p["T"], ldm + 4), dtype=torch.bfloat16, device=DEV)
+        with pytest.raises(P.PloraError):
+            r.ctx.shrink_m16(r.x, r.ids, 0, 0, bad)
+        assert r.ctx.device_status() == 0
+    finally:
+        r.close()
+
+
 def test_host_buffer_entry_point():
     p = random_problem(6, T=33, d_in=512, d_out=384, ranks=[16, 8, 32])
     r = Runner(p, max_tokens=64)
