@@ -135,13 +135,16 @@ class ClockSampler:
 class DeviceWorkload:
     """Pools registered in a library context plus per-call activations, all resident in HBM."""
 
-    def __init__(self, wl, device_index: int, max_tokens=None):
+    def __init__(self, wl, device_index: int, max_tokens=None, fp16: bool = False):
         import torch
         import paper_2608_05483_b200 as P
         self.P, self.torch, self.wl = P, torch, wl
         self.dev = f"cuda:{device_index}"
         torch.cuda.set_device(device_index)
+        self.fp16 = fp16
         self.ctx = P.Context(max_tokens or wl.n_tok, wl.n_adapters, device=device_index)
+        if fp16:
+            self.ctx.set_input_type(True)
         self.ids = torch.from_numpy(wl.ids).to(self.dev)
         g = torch.Generator(device=self.dev)
         g.manual_seed(wl.seed)
@@ -150,13 +153,13 @@ class DeviceWorkload:
         self.grouped = True
         self._groups = None
         for pool in wl.pools:
-            A, B = gen_pool_device(wl, pool, self.dev)
+            A, B = gen_pool_device(wl, pool, self.dev, fp16)
             self.ctx.register_pool(pool.layer, pool.proj, pool.d_in, pool.d_out, wl.ranks, wl.scales, A, B)
             del A, B
             key = (pool.layer, pool.x_group)
             if key not in self.x:
                 self.x[key] = torch.randn((wl.n_tok, pool.d_in), generator=g, device=self.dev,
-                                          dtype=torch.float32).to(torch.bfloat16)
+                                          dtype=torch.float32).to(torch.float16 if fp16 else torch.bfloat16)
             self.y[(pool.layer, pool.proj)] = torch.randn((wl.n_tok, pool.d_out), generator=g, device=self.dev,
                                                           dtype=torch.float32)
         torch.cuda.synchronize()
@@ -189,7 +192,7 @@ class DeviceWorkload:
 
     def host_adapters(self, pool, adapters):
         """Logical A/B bit patterns of `adapters` of `pool`, regenerated on the device and copied to the host."""
-        A, B = gen_pool_device(self.wl, pool, self.dev)
+        A, B = gen_pool_device(self.wl, pool, self.dev, self.fp16)
         outA = [None] * self.wl.n_adapters
         outB = [None] * self.wl.n_adapters
         for a in adapters:
@@ -210,6 +213,15 @@ def bits_of(t):
 # the CPU oracle on a bounded sample (also a full-size parity check of sampled pools)
 # ----------------------------------------------------------------------------------
 def oracle_sample(dw: DeviceWorkload, n_pools: int, check_gpu: bool, target_s: float = 0.0):
+    import oracle
+    oracle.set_input_type(dw.fp16)
+    try:
+        return _oracle_sample(dw, n_pools, check_gpu, target_s)
+    finally:
+        oracle.set_input_type(False)
+
+
+def _oracle_sample(dw: DeviceWorkload, n_pools: int, check_gpu: bool, target_s: float = 0.0):
     """Times the oracle on `n_pools` (layer, proj) calls of the step at full size.  When one pass
     over them takes less than `target_s`, every call is repeated (same inputs) so that the whole
     sample is about `target_s` of CPU work; returns the time of ONE pass (the mean)."""
@@ -275,7 +287,7 @@ def run_ours(args):
     torch.cuda.set_device(local)
 
     wl = make_workload(args.config, n_layers=args.layers)
-    dw = DeviceWorkload(wl, local)
+    dw = DeviceWorkload(wl, local, fp16=args.dtype == "fp16")
     dw.grouped = not args.no_group
     ctx = dw.ctx
     ctx.set_path({"auto": P.PATH_AUTO, "fused": P.PATH_FUSED, "unfused": P.PATH_UNFUSED, "sgmv": P.PATH_SGMV}[args.path])
@@ -422,7 +434,7 @@ def run_ours(args):
         out = dict(metric="LoRA-delta tokens/sec at 1000 adapters (whole step: bucket + every layer x projection delta)",
                    value=whole_job_tokens_per_s(wl.n_tok, world, ms_per_step), unit="tokens/s", n_gpus=world, steps=args.steps,
                    warmup=max(3, args.warmup), ms_per_step=ms_per_step, higher_is_better=True, scaling="weak",
-                   vs_baseline=None, dtype="bf16", data="synthetic",
+                   vs_baseline=None, dtype=args.dtype, data="synthetic",
                    config=dict(workload=f"config {args.config} ({wl.name})", n_tok=wl.n_tok, n_adapters=wl.n_adapters,
                                layers=len({p.layer for p in wl.pools}), calls_per_step=n_calls,
                                ranks=sorted({int(r) for r in wl.ranks}), ids=wl.meta.get("ids"),
@@ -494,6 +506,7 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=20.0, dest="cpu_seconds",
                     help="target CPU time of the oracle sample (cpu_baseline leg)")
     ap.add_argument("--path", default="auto", choices=["auto", "fused", "unfused", "sgmv"])
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp16"], help="16-bit type of x, A and B (fp16 = the paper's own)")
     ap.add_argument("--no-group", action="store_true", dest="no_group",
                     help="one call per projection instead of grouping q/k/v and up/gate")
     ap.add_argument("--no-cpu", action="store_true", dest="no_cpu")

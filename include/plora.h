@@ -256,6 +256,15 @@ PLORA_API plora_status plora_lora_delta_noalloc(plora_ctx *ctx, const void *x_de
  * segment to the tensor-core path; pass 0 to keep the default. */
 PLORA_API plora_status plora_set_path(plora_ctx *ctx, int32_t path, int32_t sgmv_min_rows);
 
+/* The 16-bit type of x, A and B: bf16 (the default) or IEEE half, the paper's own FP16 (its cost model
+ * counts S = 2 bytes per value either way).  Pools are stored as 16-bit patterns, so the setting only
+ * tells the kernels how to read them: it applies to every later call on this context and must match
+ * what the caller registered and passes.  Accumulation and y stay fp32; the tensor-core path then
+ * carries m as half hi + lo.  plora_shrink_m16 / plora_expand_m16 keep a bf16 m. */
+#define PLORA_INPUT_BF16 0
+#define PLORA_INPUT_FP16 1
+PLORA_API plora_status plora_set_input_type(plora_ctx *ctx, int32_t type);
+
 /* Synchronise `stream`, copy the sticky device status word to *host_out (0 or a
  * PLORA_ERR_* value) and clear it. */
 PLORA_API plora_status plora_device_status(plora_ctx *ctx, void *stream, int32_t *host_out);

@@ -35,7 +35,7 @@ def build(force: bool = False) -> Path:
     _LIB.parent.mkdir(exist_ok=True)
     tmp = _LIB.with_suffix(f".tmp{os.getpid()}.so")
     cmd = ["gcc", "-O2", "-fopenmp", "-std=c11", "-fPIC", "-shared", "-ffp-contract=off",
-           "-Wall", "-o", str(tmp), str(_SRC)]
+           "-Wall", "-o", str(tmp), str(_SRC), "-lm"]
     subprocess.run(cmd, check=True)
     os.replace(tmp, _LIB)
     return _LIB
@@ -55,6 +55,20 @@ def _load():
             f.restype = ctypes.c_int
         _lib = lib
     return _lib
+
+
+def set_input_type(fp16: bool) -> None:
+    """x, A and B are read as IEEE half (True) or bf16 (False, the default) from now on."""
+    _load().plora_oracle_set_input_type(1 if fp16 else 0)
+
+
+def input_to_double(bits) -> np.ndarray:
+    """The float64 value of every 16-bit pattern under the current input type (exact)."""
+    lib = _load()
+    lib.plora_oracle_input_to_double.restype = ctypes.c_double
+    lib.plora_oracle_input_to_double.argtypes = [ctypes.c_uint16]
+    flat = np.ascontiguousarray(bits, np.uint16).ravel()
+    return np.array([lib.plora_oracle_input_to_double(int(b)) for b in flat], np.float64).reshape(np.shape(bits))
 
 
 def threads() -> int:

@@ -23,19 +23,45 @@
  */
 #include <stdint.h>
 #include <stdlib.h>
+#include <math.h>
 #include <string.h>
 
 #define ORACLE_OK 0
 #define ORACLE_ERR_INVALID_ARG (-1)
 #define ORACLE_ERR_BAD_ADAPTER_ID (-3)
 
-static double bf16_to_double(uint16_t bits)
+static double bf16_bits_to_double(uint16_t bits)
 {
     uint32_t u = (uint32_t)bits << 16;
     float f;
     memcpy(&f, &u, sizeof f);
     return (double)f;
 }
+
+/* IEEE half (the paper's FP16, Section VI-B: S = 2 bytes per value): 1 sign, 5 exponent, 10 fraction bits. */
+static double fp16_bits_to_double(uint16_t bits)
+{
+    const int sign = bits >> 15, e = (bits >> 10) & 31, f = bits & 1023;
+    double v;
+    if (e == 0)
+        v = ldexp((double)f, -24);                 /* zero and subnormals: f * 2^-24 */
+    else if (e == 31)
+        v = f ? NAN : INFINITY;
+    else
+        v = ldexp(1.0 + (double)f / 1024.0, e - 15);
+    return sign ? -v : v;
+}
+
+/* Which 16-bit type x, A and B hold: 0 = bf16 (default), 1 = IEEE half.  Set by the caller
+ * before a call; the conversion to double is exact for both. */
+static int g_input_is_fp16 = 0;
+void plora_oracle_set_input_type(int is_fp16) { g_input_is_fp16 = is_fp16 != 0; }
+double plora_oracle_input_to_double(uint16_t bits)
+{
+    return g_input_is_fp16 ? fp16_bits_to_double(bits) : bf16_bits_to_double(bits);
+}
+
+static double bf16_to_double(uint16_t bits) { return plora_oracle_input_to_double(bits); }
 
 /* ---------------------------------------------------------------------- */
 /* Bucketing: tokens stably sorted by adapter id, plus the segment list.   */

@@ -30,7 +30,7 @@ PATH_AUTO, PATH_UNFUSED, PATH_FUSED, PATH_SGMV = 0, 1, 2, 3
 EXPORTS = (
     "plora_create", "plora_destroy", "plora_pool_slab_bytes", "plora_register_pool", "plora_pool_max_rank",
     "plora_bucket", "plora_bucket_view", "plora_lora_delta", "plora_lora_delta_group", "plora_shrink", "plora_expand",
-    "plora_shrink_m16", "plora_expand_m16",
+    "plora_shrink_m16", "plora_expand_m16", "plora_set_input_type",
     "plora_lora_delta_host", "plora_lora_delta_noalloc", "plora_set_path", "plora_device_status", "plora_launch_count", "plora_status_string",
     "plora_cost_model",
 )
@@ -97,6 +97,7 @@ def load(build_if_missing: bool = True):
         "plora_lora_delta_host": (i32, [vp, vp, vp, i32, i32, i32, vp, vp]),
         "plora_lora_delta_noalloc": (i32, [vp, vp, vp, i32, i32, i32, vp, vp]),
         "plora_set_path": (i32, [vp, i32, i32]),
+        "plora_set_input_type": (i32, [vp, i32]),
         "plora_device_status": (i32, [vp, vp, ctypes.POINTER(i32)]),
         "plora_launch_count": (i64, [vp]),
         "plora_status_string": (ctypes.c_char_p, [i32]),
@@ -292,7 +293,7 @@ class Context:
                 ma = np.ascontiguousarray(ma, dtype=np.uint16)
                 mb = np.ascontiguousarray(mb, dtype=np.uint16)
             else:
-                assert ma.is_cuda == on_dev and mb.is_cuda == on_dev and ma.dtype == torch.bfloat16
+                assert ma.is_cuda == on_dev and mb.is_cuda == on_dev and ma.dtype in (torch.bfloat16, torch.float16)
                 ma, mb = ma.contiguous(), mb.contiguous()
             assert tuple(ma.shape) == (d_in, int(ranks[a])), (a, tuple(ma.shape))
             assert tuple(mb.shape) == (int(ranks[a]), d_out), (a, tuple(mb.shape))
@@ -377,6 +378,9 @@ class Context:
 
     def set_path(self, path: int, sgmv_min_rows: int = 0):
         _check(plora_set_path(self._h, path, sgmv_min_rows), "plora_set_path")
+
+    def set_input_type(self, fp16: bool):
+        _check(load().plora_set_input_type(self._h, 1 if fp16 else 0), "plora_set_input_type")
 
     def device_status(self, stream=None) -> int:
         rc, v = plora_device_status(self._h, _stream_handle(stream))

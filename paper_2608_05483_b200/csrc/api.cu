@@ -64,6 +64,7 @@ struct plora_ctx {
     // kernels launched through this context since the bucket kernel: from the second one on, the
     // bucket tables were complete before the kernel preceding it in the stream started
     int32_t launches_since_bucket = 0;
+    bool fp16 = false;   // x, A and B are IEEE half instead of bf16
 };
 
 namespace {
@@ -147,10 +148,11 @@ plora_status ensure_bucket(plora_ctx* ctx, const int32_t* ids, int32_t n_tok, in
 
 cudaError_t launch_bgmv_one(BgmvMode mode, const PoolDev& pool, const BucketDev& bk, int n_tok, const void* x, float* y,
                             void* m, int ldm, int32_t* status, int sm_count, bool early_tables, cudaStream_t stream,
-                            int* n_launches, bool m16 = false) {
+                            int* n_launches, bool m16, bool fp16) {
     const void* xs[1] = {x};
     float* ys[1] = {y};
-    return launch_bgmv(mode, &pool, 1, bk, n_tok, xs, ys, m, ldm, m16, status, sm_count, early_tables, stream, n_launches);
+    return launch_bgmv(mode, &pool, 1, bk, n_tok, xs, ys, m, ldm, m16, fp16, status, sm_count, early_tables, stream,
+                       n_launches);
 }
 
 plora_status check_call(plora_ctx* ctx, const void* a, const void* ids, int32_t n_tok, const void* b) {
@@ -389,6 +391,12 @@ PLORA_API plora_status plora_set_path(plora_ctx* ctx, int32_t path, int32_t sgmv
     return PLORA_OK;
 }
 
+PLORA_API plora_status plora_set_input_type(plora_ctx* ctx, int32_t type) {
+    if (!ctx || (type != PLORA_INPUT_BF16 && type != PLORA_INPUT_FP16)) return PLORA_ERR_INVALID_ARG;
+    ctx->fp16 = type == PLORA_INPUT_FP16;
+    return PLORA_OK;
+}
+
 PLORA_API plora_status plora_lora_delta(plora_ctx* ctx, const void* x, const int32_t* ids, int32_t n_tok, int32_t layer,
                               int32_t proj, float* y, void* stream) {
     plora_status rc = check_call(ctx, x, ids, n_tok, y);
@@ -405,18 +413,18 @@ PLORA_API plora_status plora_lora_delta(plora_ctx* ctx, const void* x, const int
     cudaError_t e = cudaSuccess;
     if (ctx->path == PLORA_PATH_UNFUSED) {
         e = launch_bgmv_one(kShrinkOnly, pool->dev, ctx->bk, n_tok, x, nullptr, ctx->m_ws, pool->dev.max_rp, ctx->status_dev,
-                        ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl);
+                        ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl, false, ctx->fp16);
         if (e == cudaSuccess)
             e = launch_bgmv_one(kExpandOnly, pool->dev, ctx->bk, n_tok, nullptr, y, ctx->m_ws, pool->dev.max_rp,
-                            ctx->status_dev, ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl);
+                            ctx->status_dev, ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl, false, ctx->fp16);
     } else {
         // a batch shorter than the threshold cannot hold a segment for the tensor-core path
         const bool may_bgmv = ctx->path != PLORA_PATH_SGMV;
         const bool may_sgmv = ctx->bucket_sgmv_min != INT_MAX;
         if (may_bgmv)
-            e = launch_bgmv_one(kFused, pool->dev, ctx->bk, n_tok, x, y, nullptr, 0, ctx->status_dev, ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl);
+            e = launch_bgmv_one(kFused, pool->dev, ctx->bk, n_tok, x, y, nullptr, 0, ctx->status_dev, ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl, false, ctx->fp16);
         if (e == cudaSuccess && may_sgmv)
-            e = launch_sgmv(pool->dev, ctx->bk, n_tok, ctx->bucket_sgmv_min, x, y, ctx->status_dev, ctx->sm_count, may_bgmv, st, &nl);
+            e = launch_sgmv(pool->dev, ctx->bk, n_tok, ctx->bucket_sgmv_min, x, y, ctx->fp16, ctx->status_dev, ctx->sm_count, may_bgmv, st, &nl);
     }
     ctx->launches += nl;
     return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
@@ -454,11 +462,11 @@ PLORA_API plora_status plora_lora_delta_group(plora_ctx* ctx, int32_t n, const v
     PoolDev pools[kMaxGroupPools];
     for (int g = 0; g < n; ++g) pools[g] = recs[g]->dev;
     int nl = 0;
-    cudaError_t e = launch_bgmv(kFused, pools, n, ctx->bk, n_tok, x, y, nullptr, 0, false, ctx->status_dev, ctx->sm_count,
+    cudaError_t e = launch_bgmv(kFused, pools, n, ctx->bk, n_tok, x, y, nullptr, 0, false, ctx->fp16, ctx->status_dev, ctx->sm_count,
                                 ctx->launches_since_bucket++ > 0, st, &nl);
     if (e == cudaSuccess && ctx->bucket_sgmv_min != INT_MAX)
         for (int g = 0; g < n && e == cudaSuccess; ++g)
-            e = launch_sgmv(pools[g], ctx->bk, n_tok, ctx->bucket_sgmv_min, x[g], y[g], ctx->status_dev, ctx->sm_count, true, st, &nl);
+            e = launch_sgmv(pools[g], ctx->bk, n_tok, ctx->bucket_sgmv_min, x[g], y[g], ctx->fp16, ctx->status_dev, ctx->sm_count, true, st, &nl);
     ctx->launches += nl;
     return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
 }
@@ -484,7 +492,7 @@ plora_status split_call(plora_ctx* ctx, BgmvMode mode, const void* x, void* m, i
     if (rc != PLORA_OK) return rc;
     int nl = 0;
     cudaError_t e = launch_bgmv_one(mode, pool->dev, ctx->bk, n_tok, x, y, m, ldm, ctx->status_dev, ctx->sm_count,
-                                    ctx->launches_since_bucket++ > 0, st, &nl, m16);
+                                    ctx->launches_since_bucket++ > 0, st, &nl, m16, ctx->fp16);
     ctx->launches += nl;
     return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
 }
@@ -625,10 +633,10 @@ PLORA_API plora_status plora_lora_delta_noalloc(plora_ctx* ctx, const void* x, c
     if (rc != PLORA_OK) return rc;
     int nl = 0;
     cudaError_t e = launch_bgmv_one(kShrinkOnly, pool->dev, ctx->bk, n_tok, x, nullptr, m, ldm, ctx->status_dev,
-                                ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl);
+                                ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl, false, ctx->fp16);
     if (e == cudaSuccess)
         e = launch_bgmv_one(kExpandOnly, pool->dev, ctx->bk, n_tok, nullptr, y, m, ldm, ctx->status_dev, ctx->sm_count,
-                        ctx->launches_since_bucket++ > 0, st, &nl);
+                        ctx->launches_since_bucket++ > 0, st, &nl, false, ctx->fp16);
     ctx->launches += nl;
     return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
 }

@@ -35,6 +35,8 @@
 // the caller's buffer, unscaled, one task per unit) and the expand-only path.
 // Every wait (mbarrier or arrival of a partial) is bounded: when it runs out the kernel records
 // PLORA_ERR_TIMEOUT in the status word and runs to completion without waiting again.
+#include <cuda_fp16.h>
+
 #include "plora_internal.cuh"
 
 namespace plora {
@@ -159,9 +161,19 @@ __device__ __forceinline__ void red_add_v2(float* p, float a, float b) {
 }
 __device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+// The two 16-bit values of a word as fp32: bf16 (H = false) or IEEE half (H = true) inputs.
+template <bool H>
+__device__ __forceinline__ float in_lo(uint32_t w) {
+    return H ? __half2float(__ushort_as_half((unsigned short)(w & 0xffffu))) : bf_lo(w);
+}
+template <bool H>
+__device__ __forceinline__ float in_hi(uint32_t w) {
+    return H ? __half2float(__ushort_as_half((unsigned short)(w >> 16))) : bf_hi(w);
+}
+template <bool H>
 __device__ __forceinline__ void unpack8(const uint4& v, float* f) {
-    f[0] = bf_lo(v.x); f[1] = bf_hi(v.x); f[2] = bf_lo(v.y); f[3] = bf_hi(v.y);
-    f[4] = bf_lo(v.z); f[5] = bf_hi(v.z); f[6] = bf_lo(v.w); f[7] = bf_hi(v.w);
+    f[0] = in_lo<H>(v.x); f[1] = in_hi<H>(v.x); f[2] = in_lo<H>(v.y); f[3] = in_hi<H>(v.y);
+    f[4] = in_lo<H>(v.z); f[5] = in_hi<H>(v.z); f[6] = in_lo<H>(v.w); f[7] = in_hi<H>(v.w);
 }
 
 struct Smem {
@@ -265,7 +277,7 @@ struct ShrinkMap {
 // CNT (tokens of the unit) is a template parameter: the loops unroll without branches, every
 // load of the tile is issued before the first use, and each (row, token, chunk) product
 // runs as two short chains (even / odd columns) instead of one long one.
-template <int RP, int CNT, bool CHECKED>
+template <int RP, int CNT, bool CHECKED, bool H>
 __device__ __forceinline__ void shrink_chunks(const ShrinkMap<RP>& mp, int cols_left, uint32_t tile,
                                               float (&acc)[kMaxRowsPerLane][kTokChunk]) {
     using M = ShrinkMap<RP>;
@@ -283,11 +295,11 @@ __device__ __forceinline__ void shrink_chunks(const ShrinkMap<RP>& mp, int cols_
         if (!CHECKED || mp.col0 + q * M::CHL * 8 < cols_left) {
             float xf[CNT][8];
 #pragma unroll
-            for (int t = 0; t < CNT; ++t) unpack8(xraw[q][t], xf[t]);
+            for (int t = 0; t < CNT; ++t) unpack8<H>(xraw[q][t], xf[t]);
 #pragma unroll
             for (int rr = 0; rr < M::RPL; ++rr) {
                 float af[8];
-                unpack8(araw[q][rr], af);
+                unpack8<H>(araw[q][rr], af);
 #pragma unroll
                 for (int t = 0; t < CNT; ++t) {
                     float e = xf[t][0] * af[0], o = xf[t][1] * af[1];
@@ -301,24 +313,24 @@ __device__ __forceinline__ void shrink_chunks(const ShrinkMap<RP>& mp, int cols_
     }
 }
 
-template <int RP, int CNT>
+template <int RP, int CNT, bool H>
 __device__ __forceinline__ void shrink_tile_cnt(const Params& p, const StageHdr& h, const ShrinkMap<RP>& mp,
                                                 uint32_t tile, float (&acc)[kMaxRowsPerLane][kTokChunk]) {
     const int cols_left = p.pool.d_in - h.tile * ShrinkMap<RP>::C;   // only the last tile can be ragged
     if (cols_left >= ShrinkMap<RP>::C)
-        shrink_chunks<RP, CNT, false>(mp, cols_left, tile, acc);
+        shrink_chunks<RP, CNT, false, H>(mp, cols_left, tile, acc);
     else
-        shrink_chunks<RP, CNT, true>(mp, cols_left, tile, acc);
+        shrink_chunks<RP, CNT, true, H>(mp, cols_left, tile, acc);
 }
 
-template <int RP>
+template <int RP, bool H>
 __device__ __forceinline__ void shrink_tile(const Params& p, const StageHdr& h, const ShrinkMap<RP>& mp, uint32_t tile,
                                             float (&acc)[kMaxRowsPerLane][kTokChunk]) {
     switch (h.cnt) {
-        case 1: shrink_tile_cnt<RP, 1>(p, h, mp, tile, acc); break;
-        case 2: shrink_tile_cnt<RP, 2>(p, h, mp, tile, acc); break;
-        case 3: shrink_tile_cnt<RP, 3>(p, h, mp, tile, acc); break;
-        default: shrink_tile_cnt<RP, 4>(p, h, mp, tile, acc); break;
+        case 1: shrink_tile_cnt<RP, 1, H>(p, h, mp, tile, acc); break;
+        case 2: shrink_tile_cnt<RP, 2, H>(p, h, mp, tile, acc); break;
+        case 3: shrink_tile_cnt<RP, 3, H>(p, h, mp, tile, acc); break;
+        default: shrink_tile_cnt<RP, 4, H>(p, h, mp, tile, acc); break;
     }
 }
 
@@ -430,7 +442,7 @@ struct ExpandMap {
     }
 };
 
-template <int MODE, int RP, int CNT>
+template <int MODE, int RP, int CNT, bool H>
 __device__ __forceinline__ void expand_tile_cnt(const Params& p, const Smem& sm, const StageHdr& h,
                                                 const ExpandMap<RP>& mp, uint32_t tile, uint32_t empty_bar, int lane) {
     using M = ExpandMap<RP>;
@@ -470,7 +482,7 @@ __device__ __forceinline__ void expand_tile_cnt(const Params& p, const Smem& sm,
         }
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-            const float blo = bf_lo(braw[q]), bhi = bf_hi(braw[q]);
+            const float blo = in_lo<H>(braw[q]), bhi = in_hi<H>(braw[q]);
 #pragma unroll
             for (int t = 0; t < CNT; ++t) {
                 const float mk = __uint_as_float(q == 0 ? mv[t].x : q == 1 ? mv[t].y : q == 2 ? mv[t].z : mv[t].w);
@@ -505,14 +517,14 @@ __device__ __forceinline__ void expand_tile_cnt(const Params& p, const Smem& sm,
     }
 }
 
-template <int MODE, int RP>
+template <int MODE, int RP, bool H>
 __device__ __forceinline__ void expand_tile(const Params& p, const Smem& sm, const StageHdr& h, const ExpandMap<RP>& mp,
                                             uint32_t tile, uint32_t empty_bar, int lane) {
     switch (h.cnt) {
-        case 1: expand_tile_cnt<MODE, RP, 1>(p, sm, h, mp, tile, empty_bar, lane); break;
-        case 2: expand_tile_cnt<MODE, RP, 2>(p, sm, h, mp, tile, empty_bar, lane); break;
-        case 3: expand_tile_cnt<MODE, RP, 3>(p, sm, h, mp, tile, empty_bar, lane); break;
-        default: expand_tile_cnt<MODE, RP, 4>(p, sm, h, mp, tile, empty_bar, lane); break;
+        case 1: expand_tile_cnt<MODE, RP, 1, H>(p, sm, h, mp, tile, empty_bar, lane); break;
+        case 2: expand_tile_cnt<MODE, RP, 2, H>(p, sm, h, mp, tile, empty_bar, lane); break;
+        case 3: expand_tile_cnt<MODE, RP, 3, H>(p, sm, h, mp, tile, empty_bar, lane); break;
+        default: expand_tile_cnt<MODE, RP, 4, H>(p, sm, h, mp, tile, empty_bar, lane); break;
     }
 }
 
@@ -528,7 +540,7 @@ struct LaneMaps {
 };
 
 // One stage, consumer side.
-template <int MODE, int RP>
+template <int MODE, int RP, bool H>
 __device__ __forceinline__ void consume_stage(const Params& p, const Smem& sm, const StageHdr& h,
                                               const LaneMaps<RP>& maps, uint32_t tile, uint32_t empty_bar,
                                               float (&acc)[kMaxRowsPerLane][kTokChunk], int warp, int lane) {
@@ -540,14 +552,14 @@ __device__ __forceinline__ void consume_stage(const Params& p, const Smem& sm, c
 #pragma unroll
                     for (int t = 0; t < kTokChunk; ++t) acc[rr][t] = 0.f;
             }
-            shrink_tile<RP>(p, h, maps.s, tile, acc);
+            shrink_tile<RP, H>(p, h, maps.s, tile, acc);
             __syncwarp();
             if (lane == 0) mbar_arrive(empty_bar);
             if (h.flags & kFlagLast) shrink_finish<MODE, RP>(p, sm, h, maps.s, acc, warp, lane);
         }
     } else {
         if (MODE != kShrinkOnly) {
-            expand_tile<MODE, RP>(p, sm, h, maps.e, tile, empty_bar, lane);
+            expand_tile<MODE, RP, H>(p, sm, h, maps.e, tile, empty_bar, lane);
         }
     }
 }
@@ -718,7 +730,7 @@ __global__ void __launch_bounds__(kClassifyThreads) classify_kernel(const Params
 // One instantiation per padded rank RPK.  The kernel handles the units whose adapter has that
 // padded rank and skips the others: a pool of mixed ranks is served by one launch per rank
 // class present in it, each with loops specialised (and registers allocated) for its rank.
-template <int MODE, int RPK>
+template <int MODE, int RPK, bool H>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params p) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     Smem sm;
@@ -946,7 +958,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
         const StageHdr h = read_hdr(tile + kHdrOffset);
         if ((h.flags & kFlagEnd) || lds32(smem_u32(const_cast<int*>(sm.abort_flag)))) break;
         const uint32_t empty_bar = sm.empty + slot * 8;
-        consume_stage<MODE, RPK>(p, sm, h, maps, tile, empty_bar, acc, warp, lane);
+        consume_stage<MODE, RPK, H>(p, sm, h, maps, tile, empty_bar, acc, warp, lane);
     }
     if (tid == 0 && p.defer_wait) grid_dependency_wait();
     if (MODE == kFused && tid == 0 && p.bump_epoch) {
@@ -961,23 +973,28 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
 
 using KernelFn = void (*)(const Params);
 
-template <int MODE>
+template <int MODE, bool H>
 KernelFn pick_rank(int rp) {
     switch (rp) {
-        case 8: return bgmv_kernel<MODE, 8>;
-        case 16: return bgmv_kernel<MODE, 16>;
-        case 32: return bgmv_kernel<MODE, 32>;
-        case 64: return bgmv_kernel<MODE, 64>;
-        default: return bgmv_kernel<MODE, 128>;
+        case 8: return bgmv_kernel<MODE, 8, H>;
+        case 16: return bgmv_kernel<MODE, 16, H>;
+        case 32: return bgmv_kernel<MODE, 32, H>;
+        case 64: return bgmv_kernel<MODE, 64, H>;
+        default: return bgmv_kernel<MODE, 128, H>;
     }
 }
 
-KernelFn pick_kernel(BgmvMode mode, int rp) {
+template <bool H>
+KernelFn pick_mode(BgmvMode mode, int rp) {
     switch (mode) {
-        case kFused: return pick_rank<kFused>(rp);
-        case kShrinkOnly: return pick_rank<kShrinkOnly>(rp);
-        default: return pick_rank<kExpandOnly>(rp);
+        case kFused: return pick_rank<kFused, H>(rp);
+        case kShrinkOnly: return pick_rank<kShrinkOnly, H>(rp);
+        default: return pick_rank<kExpandOnly, H>(rp);
     }
+}
+
+KernelFn pick_kernel(BgmvMode mode, int rp, bool fp16) {
+    return fp16 ? pick_mode<true>(mode, rp) : pick_mode<false>(mode, rp);
 }
 
 int clamp_runs(int tiles) { return tiles < 1 ? 1 : (tiles > kMaxRuns ? kMaxRuns : tiles); }
@@ -989,16 +1006,18 @@ cudaError_t bgmv_configure() {
     const int rps[5] = {8, 16, 32, 64, 128};
     for (int m : modes)
         for (int rp : rps) {
-            cudaError_t e = cudaFuncSetAttribute(pick_kernel((BgmvMode)m, rp),
-                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-            if (e != cudaSuccess) return e;
+            for (int h = 0; h < 2; ++h) {
+                cudaError_t e = cudaFuncSetAttribute(pick_kernel((BgmvMode)m, rp, h != 0),
+                                                     cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+                if (e != cudaSuccess) return e;
+            }
         }
     return cudaSuccess;
 }
 
 cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const BucketDev& bk, int n_tok,
-                        const void* const* x, float* const* y, void* m, int ldm, bool m16, int32_t* status, int sm_count,
-                        bool early_tables, cudaStream_t stream, int* n_launches) {
+                        const void* const* x, float* const* y, void* m, int ldm, bool m16, bool fp16, int32_t* status,
+                        int sm_count, bool early_tables, cudaStream_t stream, int* n_launches) {
     if (n_groups < 1 || n_groups > kMaxGroup || (mode != kFused && n_groups != 1)) return cudaErrorInvalidValue;
     const PoolDev& pool = pools[0];
     Params p;
@@ -1071,7 +1090,7 @@ cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const
         cfg.stream = stream;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        const cudaError_t e = cudaLaunchKernelEx(&cfg, pick_kernel(mode, rp), p);
+        const cudaError_t e = cudaLaunchKernelEx(&cfg, pick_kernel(mode, rp, fp16), p);
         ++*n_launches;
         if (e != cudaSuccess) return e;
         p.early_tables = 1;   // the next class's launch follows a kernel that is not the bucket kernel

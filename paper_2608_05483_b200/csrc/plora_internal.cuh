@@ -111,13 +111,14 @@ enum BgmvMode { kFused = 0, kShrinkOnly = 1, kExpandOnly = 2 };
 // x / y: per-projection pointers (x unused by the expand-only mode, y by the shrink-only mode)
 constexpr int kMaxGroupPools = 4;
 // m / ldm / m16: the caller's m of the shrink-only and expand-only modes, fp32 or (m16) bf16 values
+// fp16: x, A and B hold IEEE half values instead of bf16
 cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const BucketDev& bk, int n_tok,
-                        const void* const* x, float* const* y, void* m, int ldm, bool m16, int32_t* status, int sm_count,
-                        bool early_tables, cudaStream_t stream, int* n_launches);
+                        const void* const* x, float* const* y, void* m, int ldm, bool m16, bool fp16, int32_t* status,
+                        int sm_count, bool early_tables, cudaStream_t stream, int* n_launches);
 // after_bgmv_of_same_call: the launch follows fused BGMV launches of the same call (other tokens of the
 // same batch) and may overlap them
 cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, int sgmv_min_rows, const void* x, float* y,
-                        int32_t* status, int sm_count, bool after_bgmv_of_same_call, cudaStream_t stream,
+                        bool fp16, int32_t* status, int sm_count, bool after_bgmv_of_same_call, cudaStream_t stream,
                         int* n_launches);
 // per-device function attributes (dynamic shared memory); called by plora_create
 cudaError_t bucket_configure();

@@ -28,6 +28,7 @@
 // pipe.  Every wait is bounded: when one runs out the kernel records PLORA_ERR_TIMEOUT, every
 // role leaves its loop, and the tensor memory is freed before the CTA exits.
 #include <cuda.h>
+#include <cuda_fp16.h>
 
 #include "plora_internal.cuh"
 
@@ -90,6 +91,7 @@ struct Params {
     // wait for them.  It joins the stream order only when its CTAs are done, so that its completion
     // still implies the completion of everything before it.
     int32_t defer_wait;
+    int32_t fp16;       // x, A and B hold IEEE half values instead of bf16 (m is then split into half hi + lo)
 };
 
 // ---- PTX wrappers -----------------------------------------------------------------
@@ -162,9 +164,11 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes
     return (uint64_t)((saddr >> 4) & 0x3fffu) | ((uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16) |
            ((uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32) | ((uint64_t)1 << 46) | ((uint64_t)layout << 61);
 }
-// Instruction descriptor: fp32 accumulate, bf16 operands, A K-major, B K- or MN-major, M = 128.
-__device__ __forceinline__ uint32_t instr_desc(int n, bool b_mn_major) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) | ((uint32_t)(n >> 3) << 17) |
+// Instruction descriptor: fp32 accumulate, bf16 (format 1) or half (format 0) operands, A K-major,
+// B K- or MN-major, M = kRows.
+__device__ __forceinline__ uint32_t instr_desc(int n, bool b_mn_major, bool fp16) {
+    const uint32_t fmt = fp16 ? 0u : 1u;
+    return (1u << 4) | (fmt << 7) | (fmt << 10) | (b_mn_major ? (1u << 16) : 0u) | ((uint32_t)(n >> 3) << 17) |
            ((uint32_t)(kRows >> 4) << 24);
 }
 __device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, bool accumulate) {
@@ -297,7 +301,7 @@ __device__ __forceinline__ void mma_thread(const Params& p, const Smem& sm, uint
         const int rp = p.pool.table[wu.adapter].rp;
         const int KP = rp < 16 ? 16 : rp;      // N of the shrink, K of the expand
         // shrink: D[128, KP] (tensor-memory columns [0, KP)) = sum over stages of X[128, 64] * W[KP, 64]^T
-        const uint32_t idesc_s = instr_desc(KP, false);
+        const uint32_t idesc_s = instr_desc(KP, false, p.fp16 != 0);
         for (int kc = 0; kc < nK; ++kc, ++it) {
             const uint32_t slot = it % p.n_stages;
             if (!mbar_wait(sm.full + slot * 8, (it / p.n_stages) & 1, sm.abort_flag, p.status)) return;
@@ -312,7 +316,7 @@ __device__ __forceinline__ void mma_thread(const Params& p, const Smem& sm, uint
         // expand: for every 64-column block, D2[128, 64] = (m_hi + m_lo)[128, KP] * B[KP, 64]
         if (!mbar_wait(sm.m_ready, tile_idx & 1, sm.abort_flag, p.status)) return;
         tc_fence_after();
-        const uint32_t idesc_e = instr_desc(kKC, true);
+        const uint32_t idesc_e = instr_desc(kKC, true, p.fp16 != 0);
         for (int nc = 0; nc < nN; ++nc, ++it, ++d2) {
             const uint32_t slot = it % p.n_stages, b = d2 % kD2Bufs;
             if (!mbar_wait(sm.full + slot * 8, (it / p.n_stages) & 1, sm.abort_flag, p.status)) return;
@@ -374,8 +378,14 @@ __device__ __forceinline__ void epilogue_warp(const Params& p, const Smem& sm, u
                         for (int u = 0; u < 2; ++u) {
                             const int k = c0 + kc * 8 + 2 * j + u;
                             const float v = k < e.rp ? __uint_as_float(r[kc * 8 + 2 * j + u]) * e.scale : 0.f;
-                            h2[u] = f32_to_bf16_bits(v);
-                            l2[u] = f32_to_bf16_bits(v - __uint_as_float(h2[u] << 16));
+                            if (p.fp16) {
+                                const __half hv = __float2half_rn(v);
+                                h2[u] = __half_as_ushort(hv);
+                                l2[u] = __half_as_ushort(__float2half_rn(v - __half2float(hv)));
+                            } else {
+                                h2[u] = f32_to_bf16_bits(v);
+                                l2[u] = f32_to_bf16_bits(v - __uint_as_float(h2[u] << 16));
+                            }
                         }
                         hi[j] = h2[0] | (h2[1] << 16);
                         lo[j] = l2[0] | (l2[1] << 16);
@@ -509,7 +519,7 @@ cudaError_t sgmv_configure() {
 }
 
 cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, int sgmv_min_rows, const void* x, float* y,
-                        int32_t* status, int sm_count, bool after_bgmv_of_same_call, cudaStream_t stream,
+                        bool fp16, int32_t* status, int sm_count, bool after_bgmv_of_same_call, cudaStream_t stream,
                         int* n_launches) {
     Params p;
     p.pool = pool;
@@ -519,6 +529,7 @@ cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, int
     p.R = pool.max_rp < 16 ? 16 : pool.max_rp;
     p.n_stages = stages_for(p.R);
     p.defer_wait = after_bgmv_of_same_call ? 1 : 0;
+    p.fp16 = fp16 ? 1 : 0;
     // x as a 2-D tensor [n_tok][d_in] of bf16; a gather instruction copies 64 columns of four rows,
     // 128-byte swizzled (columns beyond d_in read as zeros)
     CUtensorMap tm, tm_box;
@@ -526,12 +537,12 @@ cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, int
     const cuuint64_t strides[1] = {(cuuint64_t)pool.d_in * 2};
     const cuuint32_t box[2] = {(cuuint32_t)kKC, 1};
     const cuuint32_t elem_strides[2] = {1, 1};
-    if (encode_tiled()(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(x), dims, strides, box, elem_strides,
+    if (encode_tiled()(&tm, (fp16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16), 2, const_cast<void*>(x), dims, strides, box, elem_strides,
                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return cudaErrorInvalidValue;
     const cuuint32_t box_rows[2] = {(cuuint32_t)kKC, (cuuint32_t)kBoxRows};
-    if (encode_tiled()(&tm_box, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(x), dims, strides, box_rows,
+    if (encode_tiled()(&tm_box, (fp16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16), 2, const_cast<void*>(x), dims, strides, box_rows,
                        elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                        CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return cudaErrorInvalidValue;

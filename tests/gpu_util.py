@@ -22,6 +22,8 @@ class Runner:
         self.prob = prob
         self.layer, self.proj = layer, proj
         self.ctx = P.Context(max_tokens or max(1, prob["T"]), prob["N"])
+        if prob.get("fp16"):
+            self.ctx.set_input_type(True)     # the 16-bit patterns are IEEE half; device tensors keep a bf16 label
         if on_device:
             A = [bits_to_dev(a) for a in prob["A"]]
             B = [bits_to_dev(b) for b in prob["B"]]

@@ -22,8 +22,12 @@ ALL_PATHS = [P.PATH_FUSED, P.PATH_UNFUSED, P.PATH_SGMV, P.PATH_AUTO]
 
 
 def _oracle(p, y_in=None, ids=None):
-    return oracle.lora_delta(p["x"], p["ids"] if ids is None else ids, p["ranks"], p["scales"], p["A"], p["B"],
-                             p["d_out"], y_in)
+    oracle.set_input_type(bool(p.get("fp16")))
+    try:
+        return oracle.lora_delta(p["x"], p["ids"] if ids is None else ids, p["ranks"], p["scales"], p["A"], p["B"],
+                                 p["d_out"], y_in)
+    finally:
+        oracle.set_input_type(False)
 
 
 def _problem_from_workload(wl, pool):
@@ -280,6 +284,19 @@ def test_out_of_range_id_is_skipped_and_flagged():
     assert np.array_equal(got[4], p["y_in"][4])
     assert np.max(np.abs(got - ref)) <= 1e-4 * np.max(np.abs(ref))
     r.close()
+
+
+@pytest.mark.parametrize("case", ["decode", "ragged", "segments"])
+def test_half_precision_inputs(case):
+    # the paper's own FP16: x, A and B as IEEE half; every path, the same bounds as for bf16
+    if case == "decode":
+        p = random_problem(501, T=61, d_in=1024, d_out=768, ranks=[16, 16, 8, 64, 128, 3], with_minus_one=True, fp16=True)
+    elif case == "ragged":
+        p = random_problem(502, T=19, d_in=520, d_out=1032, ranks=[8, 16, 32, 64, 128, 4], with_minus_one=True, fp16=True)
+    else:
+        p = random_problem(503, T=700, d_in=328, d_out=264, ranks=[8, 16, 32, 64, 128, 24], fp16=True)
+        p["ids"] = _ids_from_runs([(0, 129), (1, 64), (2, 255), (3, 33), (4, 130), (5, 89)])
+    _check_paths(p)
 
 
 def test_two_byte_m_between_shrink_and_expand():

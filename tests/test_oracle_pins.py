@@ -202,3 +202,39 @@ def test_tiny_config_against_numpy():
         a = int(wl.ids[t])
         ref = y_in[t].astype(np.float64) + 2.0 * ((xf[t] @ bf16_bits_to_f64(A[a])) @ bf16_bits_to_f64(B[a]))
         _close(y[t], ref)
+
+
+def test_input_conversions_match_numpy_for_every_bit_pattern():
+    # both 16-bit input types widen exactly; numpy's float16 and the bf16-as-upper-half-of-fp32 view are the references
+    bits = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    try:
+        oracle.set_input_type(True)
+        got = oracle.input_to_double(bits)
+        with np.errstate(invalid="ignore"):
+            want = bits.view(np.float16).astype(np.float64)
+        assert np.array_equal(np.isnan(got), np.isnan(want)) and np.array_equal(got[~np.isnan(got)], want[~np.isnan(want)])
+        assert np.array_equal(np.signbit(got), np.signbit(want))
+    finally:
+        oracle.set_input_type(False)
+    got = oracle.input_to_double(bits)
+    with np.errstate(invalid="ignore"):
+        want = (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    assert np.array_equal(np.isnan(got), np.isnan(want)) and np.array_equal(got[~np.isnan(got)], want[~np.isnan(want)])
+
+
+def test_half_inputs_reduce_to_a_matmul():
+    # same-adapter batch with IEEE-half inputs == two numpy float64 products of the widened matrices
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal((7, 40)).astype(np.float16)
+    A = (rng.standard_normal((40, 5)) / 6).astype(np.float16)
+    B = (rng.standard_normal((5, 24)) / 2).astype(np.float16)
+    try:
+        oracle.set_input_type(True)
+        got = oracle.lora_delta(x.view(np.uint16), np.zeros(7, np.int32), [5], [0.5], [A.view(np.uint16)], [B.view(np.uint16)], 24)
+    finally:
+        oracle.set_input_type(False)
+    want = 0.5 * (x.astype(np.float64) @ A.astype(np.float64)) @ B.astype(np.float64)
+    assert np.max(np.abs(got - want)) <= 1e-12 * np.max(np.abs(want))
+    # read as bf16 the same bits mean something else entirely
+    other = oracle.lora_delta(x.view(np.uint16), np.zeros(7, np.int32), [5], [0.5], [A.view(np.uint16)], [B.view(np.uint16)], 24)
+    assert np.max(np.abs(other - want)) > 1e-3 * np.max(np.abs(want))

@@ -12,6 +12,7 @@ from .gen import (  # noqa: F401
     bf16_bits_to_f64,
     bounded_zipf_pmf,
     f32_to_bf16_bits,
+    f32_to_fp16_bits,
     gen_adapter,
     gen_pool_device,
     gen_x,

@@ -58,6 +58,11 @@ def f32_to_bf16_bits(a: np.ndarray) -> np.ndarray:
     return ((u + bias) >> np.uint32(16)).astype(np.uint16)
 
 
+def f32_to_fp16_bits(a: np.ndarray) -> np.ndarray:
+    """Round fp32 to IEEE half (nearest even) and return the uint16 bit patterns."""
+    return np.ascontiguousarray(a, dtype=np.float32).astype(np.float16).view(np.uint16)
+
+
 def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
     return (np.ascontiguousarray(b, dtype=np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32)
 
@@ -256,7 +261,7 @@ def gen_adapter(wl: Workload, pool: PoolSpec, a: int):
 # --------------------------------------------------------------------------
 # device payload generator for full-size pools (tens of GB: too slow on host)
 # --------------------------------------------------------------------------
-def gen_pool_device(wl: Workload, pool: PoolSpec, device):
+def gen_pool_device(wl: Workload, pool: PoolSpec, device, fp16: bool = False):
     """Draw a whole pool on `device` with torch's seeded generator.
 
     Returns (A_list, B_list): per-adapter bf16 tensors, A_a [d_in, r_a] and
@@ -267,6 +272,7 @@ def gen_pool_device(wl: Workload, pool: PoolSpec, device):
     """
     import torch
 
+    dt = torch.float16 if fp16 else torch.bfloat16     # fp16: the same draws rounded to IEEE half instead
     g = torch.Generator(device=device)
     g.manual_seed((wl.seed * 1000003 + pool.layer * 101 + pool.proj) & 0x7FFFFFFFFFFF)
     n = wl.n_adapters
@@ -275,16 +281,16 @@ def gen_pool_device(wl: Workload, pool: PoolSpec, device):
     for r in sorted({int(v) for v in wl.ranks}):
         idx = np.nonzero(wl.ranks == r)[0]
         cnt = len(idx)
-        A_blk = torch.empty((cnt, pool.d_in, r), dtype=torch.bfloat16, device=device)
-        B_blk = torch.empty((cnt, r, pool.d_out), dtype=torch.bfloat16, device=device)
+        A_blk = torch.empty((cnt, pool.d_in, r), dtype=dt, device=device)
+        B_blk = torch.empty((cnt, r, pool.d_out), dtype=dt, device=device)
         # draw in slices so the fp32 temporaries stay small
         step = max(1, (64 << 20) // max(1, pool.d_in * r, r * pool.d_out))
         for s in range(0, cnt, step):
             e = min(cnt, s + step)
             t = torch.randn((e - s, pool.d_in, r), generator=g, device=device, dtype=torch.float32)
-            A_blk[s:e] = (t * (1.0 / float(np.sqrt(pool.d_in)))).to(torch.bfloat16)
+            A_blk[s:e] = (t * (1.0 / float(np.sqrt(pool.d_in)))).to(dt)
             t = torch.randn((e - s, r, pool.d_out), generator=g, device=device, dtype=torch.float32)
-            B_blk[s:e] = (t * (1.0 / float(np.sqrt(r)))).to(torch.bfloat16)
+            B_blk[s:e] = (t * (1.0 / float(np.sqrt(r)))).to(dt)
         for j, a in enumerate(idx):
             A_list[int(a)] = A_blk[j]
             B_list[int(a)] = B_blk[j]
