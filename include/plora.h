@@ -304,6 +304,30 @@ PLORA_API plora_status plora_cost_model(const plora_cost_hw *hw, int32_t n_adapt
                                         const double *batch, double d, double value_bytes, double t_base,
                                         plora_cost_terms *out);
 
+/* ---- Decode attention (paper Section V-B): for every request, one query token against the request's
+ * KV cache, O = softmax(scale * q K^T) V per head.  The cache is streamed once (the path is bound by
+ * HBM bandwidth on the KV bytes); chunks of 256 tokens of one (request, KV head) are the partitions of
+ * the paper's integral execution strategy: each runs all three steps with a partial softmax that keeps
+ * its anchor (maximum), a second kernel rescales the partial outputs into the exact result.
+ *
+ * q        device bf16 [n_req][n_kv_heads * q_per_kv][head_dim]; query head h reads KV head h / q_per_kv
+ * k_cache  device bf16 [n_req][n_kv_heads][max_kv_len][head_dim] (v_cache alike); 16-byte aligned
+ * kv_len   device int32 [n_req]: tokens of the request's cache that are valid (clamped to [0, max_kv_len]);
+ *          0 leaves a zero row of out.  What lies beyond kv_len is never used.
+ * out      device fp32 [n_req][n_kv_heads * q_per_kv][head_dim], overwritten
+ * workspace  device, 256-byte aligned, at least plora_attn_workspace_bytes(...) bytes; its first 256
+ *          bytes must be zero before the first call (they hold the sticky status word); contents are
+ *          scratch between calls.  One workspace serves one stream at a time.
+ * head_dim must be 128 and q_per_kv one of 1, 2, 4, 8 (else PLORA_ERR_UNSUPPORTED).  Work is only
+ * enqueued on `stream`.  A bounded device wait that runs out sets PLORA_ERR_TIMEOUT in the status word
+ * (plora_attn_status synchronises the stream, returns the word and clears it). */
+PLORA_API size_t plora_attn_workspace_bytes(int32_t n_req, int32_t max_kv_len, int32_t n_kv_heads, int32_t q_per_kv);
+PLORA_API plora_status plora_attn_decode(const void *q_bf16_dev, const void *k_cache_dev, const void *v_cache_dev,
+                                         const int32_t *kv_len_dev, int32_t n_req, int32_t max_kv_len,
+                                         int32_t n_kv_heads, int32_t q_per_kv, int32_t head_dim, float scale,
+                                         float *out_dev, void *workspace_dev, size_t workspace_bytes, void *stream);
+PLORA_API plora_status plora_attn_status(void *workspace_dev, void *stream, int32_t *host_out);
+
 #ifdef __cplusplus
 }
 #endif

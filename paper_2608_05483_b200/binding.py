@@ -32,7 +32,7 @@ EXPORTS = (
     "plora_bucket", "plora_bucket_view", "plora_lora_delta", "plora_lora_delta_group", "plora_shrink", "plora_expand",
     "plora_shrink_m16", "plora_expand_m16", "plora_set_input_type",
     "plora_lora_delta_host", "plora_lora_delta_noalloc", "plora_set_path", "plora_device_status", "plora_launch_count", "plora_status_string",
-    "plora_cost_model",
+    "plora_cost_model", "plora_attn_workspace_bytes", "plora_attn_decode", "plora_attn_status",
 )
 
 
@@ -101,6 +101,9 @@ def load(build_if_missing: bool = True):
         "plora_device_status": (i32, [vp, vp, ctypes.POINTER(i32)]),
         "plora_launch_count": (i64, [vp]),
         "plora_status_string": (ctypes.c_char_p, [i32]),
+        "plora_attn_workspace_bytes": (ctypes.c_size_t, [i32, i32, i32, i32]),
+        "plora_attn_decode": (i32, [vp, vp, vp, vp, i32, i32, i32, i32, i32, ctypes.c_float, vp, vp, ctypes.c_size_t, vp]),
+        "plora_attn_status": (i32, [vp, vp, ctypes.POINTER(i32)]),
         "plora_cost_model": (i32, [ctypes.POINTER(CostHw), i32, vp, vp, ctypes.c_double, ctypes.c_double, ctypes.c_double,
                                    ctypes.POINTER(CostTerms)]),
     }
@@ -139,6 +142,39 @@ def plora_cost_model(hw: dict, ranks, batch, d: float, value_bytes: float, t_bas
     terms = dict(t_gpu=list(out.t_gpu), t_dev_cpt=list(out.t_dev_cpt), t_dev_trs=list(out.t_dev_trs),
                  t_lora_gpu=out.t_lora_gpu, t_lora_dev=out.t_lora_dev, t_lora=out.t_lora)
     return rc, terms
+
+
+def plora_attn_workspace_bytes(n_req: int, max_kv_len: int, n_kv_heads: int, q_per_kv: int) -> int:
+    return int(load().plora_attn_workspace_bytes(n_req, max_kv_len, n_kv_heads, q_per_kv))
+
+
+def plora_attn_decode(q_ptr, k_ptr, v_ptr, kv_len_ptr, n_req, max_kv_len, n_kv_heads, q_per_kv, head_dim, scale, out_ptr,
+                      ws_ptr, ws_bytes, stream=0):
+    return load().plora_attn_decode(q_ptr, k_ptr, v_ptr, kv_len_ptr, n_req, max_kv_len, n_kv_heads, q_per_kv, head_dim,
+                                    float(scale), out_ptr, ws_ptr, ws_bytes, stream)
+
+
+def plora_attn_status(ws_ptr, stream=0):
+    v = ctypes.c_int32(0)
+    rc = load().plora_attn_status(ws_ptr, stream, ctypes.byref(v))
+    return rc, int(v.value)
+
+
+def attn_decode(q, k_cache, v_cache, kv_len, scale, out=None, workspace=None, stream=None):
+    """Torch convenience: q bf16 [B, Hq, 128], k_cache / v_cache bf16 [B, Hkv, Lmax, 128], kv_len int32 [B] (all CUDA);
+    returns (out fp32 [B, Hq, 128], workspace).  Pass the returned workspace back in to reuse it."""
+    import torch
+    B, Hq, d = q.shape
+    Hkv, Lmax = int(k_cache.shape[1]), int(k_cache.shape[2])
+    need = plora_attn_workspace_bytes(B, Lmax, Hkv, Hq // Hkv)
+    if workspace is None:
+        workspace = torch.zeros(need, dtype=torch.uint8, device=q.device)
+    if out is None:
+        out = torch.empty((B, Hq, d), dtype=torch.float32, device=q.device)
+    _check(plora_attn_decode(q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), kv_len.data_ptr(), B, Lmax, Hkv, Hq // Hkv,
+                             d, scale, out.data_ptr(), workspace.data_ptr(), int(workspace.numel()), _stream_handle(stream)),
+           "plora_attn_decode")
+    return out, workspace
 
 
 def plora_pool_slab_bytes(desc: PoolDesc) -> int:
