@@ -493,8 +493,86 @@ def run_reference(args):
     print(json.dumps(out))
 
 
+def run_attention(args):
+    """Decode attention (the paper's other memory-bound operator) on a synthetic batch: one query token per
+    request against a KV cache of the paper's request lengths, Llama-2-7B head shapes (32 heads of 128),
+    one layer's cache.  Prints its own JSON line; `bench.py` without --op stays the LoRA-delta benchmark."""
+    import torch
+    import paper_2608_05483_b200 as P
+    torch.cuda.set_device(0)
+    dev = "cuda:0"
+    long_ctx = args.attn_long
+    n_req, lo, hi = (64, 2048, 4096) if long_ctx else (256, 100, 1024)
+    n_req = args.attn_requests or n_req
+    H, d = 32, 128
+    rng = np.random.default_rng(20260805 * 10 + (8 if long_ctx else 7))
+    kv_len = rng.integers(lo, hi + 1, size=n_req).astype(np.int32)
+    g = torch.Generator(device=dev)
+    g.manual_seed(int(rng.integers(1 << 30)))
+    layers = args.attn_layers      # several layers' caches in turn, so that a step streams far more than L2 holds
+    q = torch.randn((layers, n_req, H, d), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    K = torch.randn((layers, n_req, H, hi, d), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    V = torch.randn((layers, n_req, H, hi, d), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    lens = torch.from_numpy(kv_len).to(dev)
+    scale = 1.0 / float(np.sqrt(d))
+    out = torch.empty((layers, n_req, H, d), dtype=torch.float32, device=dev)
+    ws = torch.zeros(P.plora_attn_workspace_bytes(n_req, hi, H, 1), dtype=torch.uint8, device=dev)
+
+    def step():
+        for l in range(layers):
+            P.attn_decode(q[l], K[l], V[l], lens, scale, out=out[l], workspace=ws)
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / args.steps
+    rc, status = P.plora_attn_status(ws.data_ptr())
+    kv_bytes = float(kv_len.sum()) * H * d * 2 * 2 * layers            # K and V, 2 bytes per value
+    other = layers * n_req * H * d * (2 + 4)                           # q read, out written
+    peaks = measured_peaks()
+    achieved = (kv_bytes + other) / (ms * 1e-3) / 1e9
+    # parity on sampled requests and the oracle's time on them
+    from oracle.attention import decode_attention
+    sample = np.unique(np.concatenate([[0, n_req - 1, int(np.argmax(kv_len)), int(np.argmin(kv_len))], rng.integers(0, n_req, size=4)]))
+    Ks = K[0][sample].float().cpu().numpy().astype(np.float64)
+    Vs = V[0][sample].float().cpu().numpy().astype(np.float64)
+    qs = q[0][sample].float().cpu().numpy().astype(np.float64)
+    t0 = time.perf_counter()
+    ref = decode_attention(qs, Ks, Vs, kv_len[sample], scale)
+    cpu_s = time.perf_counter() - t0
+    err = float(np.max(np.abs(out[0][sample].cpu().numpy() - ref)) / max(1.0, np.max(np.abs(ref))))
+    print(json.dumps(dict(
+        metric="decode-attention requests/sec (one query token per request, one layer's KV cache per call)",
+        value=n_req * layers / (ms * 1e-3), unit="requests/s", n_gpus=1, steps=args.steps, warmup=max(3, args.warmup),
+        ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16", data="synthetic",
+        config=dict(workload="decode attention, Llama-2-7B heads (32 x 128), %d requests, cache lengths U[%d, %d]" % (n_req, lo, hi),
+                    calls_per_step=layers, kv_tokens=int(kv_len.sum()), accumulate="fp32",
+                    l2="inputs larger than L2: a step streams %.2f GB of KV cache" % (kv_bytes / 1e9)),
+        clocks=clocks, gpu_launches=3 * layers * (args.steps + max(3, args.warmup)),
+        roofline=dict(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s", frac=achieved / peaks["hbm_gbs"],
+                      traffic=None, kernel="attn partial_kernel (chunked partial softmax)", peak_source=peaks["source"],
+                      algorithmic_bytes_per_step=kv_bytes + other),
+        cpu_baseline=dict(value=len(sample) / cpu_s, unit="requests/s", cores=1, kind="oracle",
+                          sample="%d requests of one layer, numpy float64" % len(sample)),
+        parity_max_rel_err=err, device_status=status)))
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--op", default="lora", choices=["lora", "attention"],
+                    help="lora: the LoRA-delta benchmark (the default, the headline); attention: decode attention")
+    ap.add_argument("--attn-long", action="store_true", dest="attn_long", help="attention: 64 requests of 2048..4096 tokens")
+    ap.add_argument("--attn-layers", type=int, default=4, dest="attn_layers")
+    ap.add_argument("--attn-requests", type=int, default=0, dest="attn_requests")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
@@ -512,7 +590,9 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", dest="no_cpu")
     ap.add_argument("--no-e2e", action="store_true", dest="no_e2e")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.op == "attention":
+        run_attention(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
