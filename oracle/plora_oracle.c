@@ -14,11 +14,13 @@
  *     strategy E4 names the two halves, shrink m = x A and expand y = m B.
  *   - Section VI-B: a step serves requests tagged by adapter id; B_i is the
  *     number of requests of adapter i; values are 2 bytes wide.
- * Readings the paper leaves open (scale factor s, token with no adapter, the
- * output being accumulated into the base projection) are listed in the design doc.
+ * Readings the paper leaves open: a per-adapter fp32 scale s_a multiplies the
+ * delta; a token with id -1 has no adapter and keeps its row of y; the delta is
+ * added to the caller's y (the base projection output); an id outside
+ * [-1, N) is an error.
  *
- * All arithmetic is float64.  Inputs are the raw bf16 bit patterns the GPU
- * gets (bf16 -> double is exact).  Nothing is blocked, fused or reordered: the
+ * All arithmetic is float64.  Inputs are the raw 16-bit patterns the GPU gets,
+ * bf16 or IEEE half (widening either to double is exact).  Nothing is blocked, fused or reordered: the
  * loops are the definition written out.  Pins: tests/test_oracle_*.py.
  */
 #include <stdint.h>
