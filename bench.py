@@ -504,19 +504,21 @@ def run_attention(args):
     long_ctx = args.attn_long
     n_req, lo, hi = (64, 2048, 4096) if long_ctx else (256, 100, 1024)
     n_req = args.attn_requests or n_req
-    H, d = 32, 128
+    G = args.attn_q_per_kv
+    H, d = 32 // G, 128      # KV heads: 32 query heads in all, G of them per KV head
+    Hq = H * G
     rng = np.random.default_rng(20260805 * 10 + (8 if long_ctx else 7))
     kv_len = rng.integers(lo, hi + 1, size=n_req).astype(np.int32)
     g = torch.Generator(device=dev)
     g.manual_seed(int(rng.integers(1 << 30)))
     layers = args.attn_layers      # several layers' caches in turn, so that a step streams far more than L2 holds
-    q = torch.randn((layers, n_req, H, d), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    q = torch.randn((layers, n_req, Hq, d), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
     K = torch.randn((layers, n_req, H, hi, d), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
     V = torch.randn((layers, n_req, H, hi, d), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
     lens = torch.from_numpy(kv_len).to(dev)
     scale = 1.0 / float(np.sqrt(d))
-    out = torch.empty((layers, n_req, H, d), dtype=torch.float32, device=dev)
-    ws = torch.zeros(P.plora_attn_workspace_bytes(n_req, hi, H, 1), dtype=torch.uint8, device=dev)
+    out = torch.empty((layers, n_req, Hq, d), dtype=torch.float32, device=dev)
+    ws = torch.zeros(P.plora_attn_workspace_bytes(n_req, hi, H, G), dtype=torch.uint8, device=dev)
 
     def step():
         for l in range(layers):
@@ -537,7 +539,7 @@ def run_attention(args):
     ms = e0.elapsed_time(e1) / args.steps
     rc, status = P.plora_attn_status(ws.data_ptr())
     kv_bytes = float(kv_len.sum()) * H * d * 2 * 2 * layers            # K and V, 2 bytes per value
-    other = layers * n_req * H * d * (2 + 4)                           # q read, out written
+    other = layers * n_req * Hq * d * (2 + 4)                          # q read, out written
     peaks = measured_peaks()
     achieved = (kv_bytes + other) / (ms * 1e-3) / 1e9
     # parity on sampled requests and the oracle's time on them
@@ -554,7 +556,7 @@ def run_attention(args):
         metric="decode-attention requests/sec (one query token per request, one layer's KV cache per call)",
         value=n_req * layers / (ms * 1e-3), unit="requests/s", n_gpus=1, steps=args.steps, warmup=max(3, args.warmup),
         ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16", data="synthetic",
-        config=dict(workload="decode attention, Llama-2-7B heads (32 x 128), %d requests, cache lengths U[%d, %d]" % (n_req, lo, hi),
+        config=dict(workload="decode attention, %d KV heads x %d query heads each x 128, %d requests, cache lengths U[%d, %d]" % (H, G, n_req, lo, hi),
                     calls_per_step=layers, kv_tokens=int(kv_len.sum()), accumulate="fp32",
                     l2="inputs larger than L2: a step streams %.2f GB of KV cache" % (kv_bytes / 1e9)),
         clocks=clocks, gpu_launches=3 * layers * (args.steps + max(3, args.warmup)),
@@ -573,6 +575,8 @@ def main():
     ap.add_argument("--attn-long", action="store_true", dest="attn_long", help="attention: 64 requests of 2048..4096 tokens")
     ap.add_argument("--attn-layers", type=int, default=4, dest="attn_layers")
     ap.add_argument("--attn-requests", type=int, default=0, dest="attn_requests")
+    ap.add_argument("--attn-q-per-kv", type=int, default=1, choices=[1, 2, 4, 8], dest="attn_q_per_kv",
+                    help="attention: query heads per KV head (1 = the Llama-2 7B / 13B shapes)")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
