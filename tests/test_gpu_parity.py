@@ -235,6 +235,31 @@ def test_cuda_graph_replay_of_a_mixed_call_sequence():
         r.close()
 
 
+@pytest.mark.parametrize("seed", range(24))
+def test_random_shapes_ranks_and_id_mixes(seed):
+    # a sweep over what the kernels branch on: ragged dimensions, every rank class alone and mixed, ids that are
+    # uniform, skewed, run-structured or mostly absent, batch sizes on both sides of the tensor-core threshold
+    rng = np.random.default_rng(9000 + seed)
+    d_in = int(rng.integers(1, 260)) * 8
+    d_out = int(rng.integers(1, 260)) * 8
+    N = int(rng.integers(1, 48))
+    rank_sets = [[8], [16], [64], [128], [1, 2, 3], [8, 16, 32, 64, 128], [5, 33, 100], [16, 64]]
+    ranks = rng.choice(rank_sets[seed % len(rank_sets)], size=N)
+    T = int(rng.choice([1, 3, 17, 64, 200, 513, 700, 1500]))
+    kind = seed % 4
+    if kind == 0:
+        ids = rng.integers(0, N, size=T)
+    elif kind == 1:
+        ids = np.minimum((rng.pareto(1.0, size=T)).astype(np.int64), N - 1)
+    elif kind == 2:
+        ids = np.repeat(rng.integers(0, N, size=T // 37 + 1), 37)[:T]
+    else:
+        ids = np.where(rng.random(T) < 0.7, -1, rng.integers(0, N, size=T))
+    p = random_problem(9100 + seed, T=T, d_in=d_in, d_out=d_out, ranks=ranks, fp16=bool(seed & 8))
+    p["ids"] = ids.astype(np.int32)
+    _check_paths(p)
+
+
 def test_empty_and_all_minus_one():
     p = random_problem(1, T=0, d_in=64, d_out=64, ranks=[8])
     r = Runner(p, max_tokens=8)
