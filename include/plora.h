@@ -210,11 +210,33 @@ PLORA_API plora_status plora_expand_m16(plora_ctx *ctx, const void *m_bf16_dev, 
 /*
  * Same operation as plora_lora_delta with HOST buffers: copies x, ids and y to
  * context-owned device staging buffers, buckets, runs the delta and copies y
- * back, all on `stream`, then synchronises `stream`.  Pinned host memory makes
+ * back, then waits until y_host holds the result.  Pinned host memory makes
  * the copies asynchronous to each other but is not required.
  */
 PLORA_API plora_status plora_lora_delta_host(plora_ctx *ctx, const void *x_host, const int32_t *adapter_ids_host,
                                    int32_t n_tok, int32_t layer, int32_t proj, float *y_host, void *stream);
+
+/*
+ * The pipelined form of the above, for a step that makes many such calls (one per layer and
+ * projection, Section II-A).  It queues the work and returns; y_host[g] holds its result only
+ * after plora_host_sync.  n projections (1..4) that share one input are served together:
+ * x_host is copied once, y_host[g] += delta of pool (layers[g], projs[g]); all n pools must have
+ * the same d_in.  The copies to the device run on a stream of the context's own, the kernels on
+ * `stream`, the copies back on a second stream of the context's own, over a ring of four staging
+ * sets, so one call's copy back, the next call's kernels and the following call's copy in overlap
+ * (both directions of the host link in use at once).  x_host, adapter_ids_host and y_host[g]
+ * must stay untouched until plora_host_sync returns, and should be pinned: from pageable memory
+ * the copies are correct but each blocks the calling thread.  The same ids may be passed to
+ * every call of a step; they are bucketed again per call.
+ * Errors as plora_lora_delta_group; PLORA_ERR_INVALID_ARG also if the pools' d_in differ.
+ * The first call at a new largest shape allocates staging memory and synchronises.
+ *
+ * plora_host_sync: blocks the calling thread until every queued call's result is in host memory.
+ */
+PLORA_API plora_status plora_lora_delta_host_async(plora_ctx *ctx, int32_t n, const void *x_host,
+                                                   const int32_t *adapter_ids_host, int32_t n_tok, const int32_t *layers,
+                                                   const int32_t *projs, float *const *y_host, void *stream);
+PLORA_API plora_status plora_host_sync(plora_ctx *ctx);
 
 /*
  * The LoRA delta for callers that must not allocate device memory.  (The paper has no

@@ -31,7 +31,7 @@ EXPORTS = (
     "plora_create", "plora_destroy", "plora_pool_slab_bytes", "plora_register_pool", "plora_pool_max_rank",
     "plora_bucket", "plora_bucket_view", "plora_lora_delta", "plora_lora_delta_group", "plora_shrink", "plora_expand",
     "plora_shrink_m16", "plora_expand_m16", "plora_set_input_type",
-    "plora_lora_delta_host", "plora_lora_delta_noalloc", "plora_set_path", "plora_device_status", "plora_launch_count", "plora_status_string",
+    "plora_lora_delta_host", "plora_lora_delta_host_async", "plora_host_sync", "plora_lora_delta_noalloc", "plora_set_path", "plora_device_status", "plora_launch_count", "plora_status_string",
     "plora_cost_model", "plora_attn_workspace_bytes", "plora_attn_decode", "plora_attn_status",
 )
 
@@ -96,6 +96,8 @@ def load(build_if_missing: bool = True):
         "plora_expand_m16": (i32, [vp, vp, i32, vp, i32, i32, i32, vp, vp]),
         "plora_lora_delta_host": (i32, [vp, vp, vp, i32, i32, i32, vp, vp]),
         "plora_lora_delta_noalloc": (i32, [vp, vp, vp, i32, i32, i32, vp, vp]),
+        "plora_lora_delta_host_async": (i32, [vp, i32, vp, vp, i32, vp, vp, vp, vp]),
+        "plora_host_sync": (i32, [vp]),
         "plora_set_path": (i32, [vp, i32, i32]),
         "plora_set_input_type": (i32, [vp, i32]),
         "plora_device_status": (i32, [vp, vp, ctypes.POINTER(i32)]),
@@ -233,6 +235,18 @@ def plora_expand_m16(ctx, m_ptr, ldm, ids_ptr, n_tok, layer, proj, y_ptr, stream
 
 def plora_lora_delta_host(ctx, x_host_ptr, ids_host_ptr, n_tok, layer, proj, y_host_ptr, stream=0):
     return load().plora_lora_delta_host(ctx, x_host_ptr, ids_host_ptr, n_tok, layer, proj, y_host_ptr, stream)
+
+
+def plora_lora_delta_host_async(ctx, x_host_ptr, ids_host_ptr, n_tok, layers, projs, y_host_ptrs, stream=0):
+    n = len(layers)
+    la = (ctypes.c_int32 * n)(*layers)
+    pa = (ctypes.c_int32 * n)(*projs)
+    ya = (ctypes.c_void_p * n)(*y_host_ptrs)
+    return load().plora_lora_delta_host_async(ctx, n, x_host_ptr, ids_host_ptr, n_tok, la, pa, ya, stream)
+
+
+def plora_host_sync(ctx):
+    return load().plora_host_sync(ctx)
 
 
 def plora_lora_delta_noalloc(ctx, x_ptr, ids_ptr, n_tok, layer, proj, y_ptr, stream=0):
@@ -405,6 +419,18 @@ class Context:
         n_tok = int(ids_host.shape[0])
         _check(plora_lora_delta_host(self._h, _data_ptr(x_host), _data_ptr(ids_host), n_tok, layer, proj,
                                      _data_ptr(y_host), _stream_handle(stream)), "plora_lora_delta_host")
+
+    def lora_delta_host_async(self, x_host, ids_host, layers, projs, ys_host, stream=None):
+        """Queues y_host[g] += delta of pool (layers[g], projs[g]) for projections that share x_host;
+        the results are in host memory after host_sync().  The host tensors must stay alive and
+        untouched until then."""
+        n_tok = int(ids_host.shape[0])
+        _check(plora_lora_delta_host_async(self._h, _data_ptr(x_host), _data_ptr(ids_host), n_tok, list(layers), list(projs),
+                                           [_data_ptr(y) for y in ys_host], _stream_handle(stream)),
+               "plora_lora_delta_host_async")
+
+    def host_sync(self):
+        _check(plora_host_sync(self._h), "plora_host_sync")
 
     def lora_delta_noalloc(self, x, ids, layer, proj, y, stream=None):
         """The delta for callers that must not allocate: same result as lora_delta, with the

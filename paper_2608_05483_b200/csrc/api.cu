@@ -54,11 +54,20 @@ struct plora_ctx {
     int32_t bucket_sgmv_min = INT_MAX;   // threshold the current bucket was built with
     // workspace for the unfused path's m
     float* m_ws = nullptr;
-    // staging for the host-buffer entry point
-    void* x_stage = nullptr;
-    float* y_stage = nullptr;
-    int32_t* ids_stage = nullptr;
-    size_t x_stage_bytes = 0, y_stage_bytes = 0;
+    // staging for the host-buffer entry points: a ring of sets, so that one call's copy back to the
+    // host, the next call's kernels and the call after that's copy to the device run at the same time
+    struct HostStage {
+        void* x = nullptr;
+        int32_t* ids = nullptr;
+        float* y[kMaxGroupPools] = {};
+        size_t x_bytes = 0, y_bytes[kMaxGroupPools] = {};
+        cudaEvent_t up = nullptr, done = nullptr, freed = nullptr;
+        bool in_flight = false;
+    };
+    static constexpr int kHostStages = 4;
+    HostStage stage[kHostStages];
+    cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
+    int next_stage = 0;
     std::vector<PoolRec> pools;
     int64_t launches = 0;
     // kernels launched through this context since the bucket kernel: from the second one on, the
@@ -261,9 +270,16 @@ PLORA_API plora_status plora_destroy(plora_ctx* ctx) {
     cudaDeviceSynchronize();
     for (auto& p : ctx->pools) cudaFree(p.table_dev);
     cudaFree(ctx->bucket_block);
-    cudaFree(ctx->x_stage);
-    cudaFree(ctx->y_stage);
-    cudaFree(ctx->ids_stage);
+    for (auto& hs : ctx->stage) {
+        cudaFree(hs.x);
+        cudaFree(hs.ids);
+        for (float* y : hs.y) cudaFree(y);
+        if (hs.up) cudaEventDestroy(hs.up);
+        if (hs.done) cudaEventDestroy(hs.done);
+        if (hs.freed) cudaEventDestroy(hs.freed);
+    }
+    if (ctx->h2d_stream) cudaStreamDestroy(ctx->h2d_stream);
+    if (ctx->d2h_stream) cudaStreamDestroy(ctx->d2h_stream);
     delete ctx;
     return PLORA_OK;
 }
@@ -518,48 +534,116 @@ PLORA_API plora_status plora_expand_m16(plora_ctx* ctx, const void* m_bf16, int3
     return split_call(ctx, kExpandOnly, nullptr, const_cast<void*>(m_bf16), ldm, true, ids, n_tok, layer, proj, y, stream);
 }
 
-PLORA_API plora_status plora_lora_delta_host(plora_ctx* ctx, const void* x_host, const int32_t* ids_host, int32_t n_tok,
-                                   int32_t layer, int32_t proj, float* y_host, void* stream) {
-    if (!ctx || n_tok < 0 || n_tok > ctx->max_tokens) return PLORA_ERR_INVALID_ARG;
-    if (n_tok > 0 && (!x_host || !ids_host || !y_host)) return PLORA_ERR_INVALID_ARG;
-    PoolRec* pool = find_pool(ctx, layer, proj);
-    if (!pool) return PLORA_ERR_NOT_REGISTERED;
-    if (n_tok == 0) return PLORA_OK;
+namespace {
+
+bool grow(void** p, size_t* have, size_t want) {
+    if (*have >= want) return true;
+    cudaFree(*p);
+    *p = nullptr;
+    *have = 0;
+    if (cudaMalloc(p, want) != cudaSuccess) return false;
+    *have = want;
+    return true;
+}
+
+}  // namespace
+
+PLORA_API plora_status plora_host_sync(plora_ctx* ctx) {
+    if (!ctx) return PLORA_ERR_INVALID_ARG;
+    if (!ctx->d2h_stream) return PLORA_OK;   // nothing was ever queued
     DeviceGuard g(ctx->device);
     if (!g.ok) return PLORA_ERR_CUDA;
+    // the copy-back stream is last in every call's chain, and in order across calls
+    if (cudaStreamSynchronize(ctx->d2h_stream) != cudaSuccess) return PLORA_ERR_CUDA;
+    for (auto& hs : ctx->stage) hs.in_flight = false;
+    return PLORA_OK;
+}
+
+PLORA_API plora_status plora_lora_delta_host_async(plora_ctx* ctx, int32_t n, const void* x_host, const int32_t* ids_host,
+                                                   int32_t n_tok, const int32_t* layers, const int32_t* projs,
+                                                   float* const* y_host, void* stream) {
+    if (!ctx || n < 1 || n > kMaxGroupPools || !layers || !projs || !y_host) return PLORA_ERR_INVALID_ARG;
+    if (n_tok < 0 || n_tok > ctx->max_tokens) return PLORA_ERR_INVALID_ARG;
+    if (n_tok > 0 && (!x_host || !ids_host)) return PLORA_ERR_INVALID_ARG;
+    PoolRec* recs[kMaxGroupPools];
+    for (int g = 0; g < n; ++g) {
+        if (n_tok > 0 && !y_host[g]) return PLORA_ERR_INVALID_ARG;
+        recs[g] = find_pool(ctx, layers[g], projs[g]);
+        if (!recs[g]) return PLORA_ERR_NOT_REGISTERED;
+        if (recs[g]->dev.d_in != recs[0]->dev.d_in) return PLORA_ERR_INVALID_ARG;   // one x serves the whole group
+    }
+    if (n_tok == 0) return PLORA_OK;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return PLORA_ERR_CUDA;
     cudaStream_t st = as_stream(stream);
-    const size_t xb = (size_t)ctx->max_tokens * pool->dev.d_in * 2, yb = (size_t)ctx->max_tokens * pool->dev.d_out * 4;
-    if (xb > ctx->x_stage_bytes) {
-        cudaStreamSynchronize(st);
-        cudaFree(ctx->x_stage);
-        ctx->x_stage = nullptr;
-        ctx->x_stage_bytes = 0;
-        if (cudaMalloc(&ctx->x_stage, xb) != cudaSuccess) return PLORA_ERR_WORKSPACE;
-        ctx->x_stage_bytes = xb;
+    if (!ctx->h2d_stream) {
+        if (cudaStreamCreateWithFlags(&ctx->h2d_stream, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaStreamCreateWithFlags(&ctx->d2h_stream, cudaStreamNonBlocking) != cudaSuccess)
+            return PLORA_ERR_CUDA;
     }
-    if (yb > ctx->y_stage_bytes) {
-        cudaStreamSynchronize(st);
-        cudaFree(ctx->y_stage);
-        ctx->y_stage = nullptr;
-        ctx->y_stage_bytes = 0;
-        if (cudaMalloc(&ctx->y_stage, yb) != cudaSuccess) return PLORA_ERR_WORKSPACE;
-        ctx->y_stage_bytes = yb;
+    plora_ctx::HostStage& hs = ctx->stage[ctx->next_stage];
+    ctx->next_stage = (ctx->next_stage + 1) % plora_ctx::kHostStages;
+    if (!hs.up) {
+        if (cudaEventCreateWithFlags(&hs.up, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&hs.done, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&hs.freed, cudaEventDisableTiming) != cudaSuccess)
+            return PLORA_ERR_CUDA;
     }
-    if (!ctx->ids_stage && cudaMalloc(&ctx->ids_stage, (size_t)ctx->max_tokens * 4) != cudaSuccess)
-        return PLORA_ERR_WORKSPACE;
-    const size_t nx = (size_t)n_tok * pool->dev.d_in * 2, ny = (size_t)n_tok * pool->dev.d_out * 4;
-    if (cudaMemcpyAsync(ctx->ids_stage, ids_host, (size_t)n_tok * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(ctx->x_stage, x_host, nx, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(ctx->y_stage, y_host, ny, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    // buffers sized for the context's largest batch, so they are allocated once per shape
+    const size_t want_x = (size_t)ctx->max_tokens * recs[0]->dev.d_in * 2;
+    bool fits = hs.x_bytes >= want_x && hs.ids != nullptr;
+    for (int g = 0; g < n; ++g) fits = fits && hs.y_bytes[g] >= (size_t)ctx->max_tokens * recs[g]->dev.d_out * 4;
+    if (!fits) {
+        plora_status rc = plora_host_sync(ctx);   // nothing may still be using what is freed here
+        if (rc != PLORA_OK) return rc;
+        if (cudaStreamSynchronize(st) != cudaSuccess) return PLORA_ERR_CUDA;
+        if (!grow(&hs.x, &hs.x_bytes, want_x)) return PLORA_ERR_WORKSPACE;
+        if (!hs.ids && cudaMalloc(&hs.ids, (size_t)ctx->max_tokens * 4) != cudaSuccess) return PLORA_ERR_WORKSPACE;
+        for (int g = 0; g < n; ++g)
+            if (!grow((void**)&hs.y[g], &hs.y_bytes[g], (size_t)ctx->max_tokens * recs[g]->dev.d_out * 4))
+                return PLORA_ERR_WORKSPACE;
+    }
+    // to the device, once the set's previous user has copied its result out
+    if (hs.in_flight && cudaStreamWaitEvent(ctx->h2d_stream, hs.freed, 0) != cudaSuccess) return PLORA_ERR_CUDA;
+    hs.in_flight = true;
+    const size_t nx = (size_t)n_tok * recs[0]->dev.d_in * 2;
+    if (cudaMemcpyAsync(hs.ids, ids_host, (size_t)n_tok * 4, cudaMemcpyHostToDevice, ctx->h2d_stream) != cudaSuccess ||
+        cudaMemcpyAsync(hs.x, x_host, nx, cudaMemcpyHostToDevice, ctx->h2d_stream) != cudaSuccess)
         return PLORA_ERR_CUDA;
-    ctx->bucket_valid = false;   // the staged ids changed under the same pointer
-    plora_status rc = plora_lora_delta(ctx, ctx->x_stage, ctx->ids_stage, n_tok, layer, proj, ctx->y_stage, stream);
+    for (int g = 0; g < n; ++g)
+        if (cudaMemcpyAsync(hs.y[g], y_host[g], (size_t)n_tok * recs[g]->dev.d_out * 4, cudaMemcpyHostToDevice,
+                            ctx->h2d_stream) != cudaSuccess)
+            return PLORA_ERR_CUDA;
+    if (cudaEventRecord(hs.up, ctx->h2d_stream) != cudaSuccess || cudaStreamWaitEvent(st, hs.up, 0) != cudaSuccess)
+        return PLORA_ERR_CUDA;
+    // the delta, on the caller's stream
+    ctx->bucket_valid = false;   // another set's ids, or new ids under the same pointer
+    const void* xs[kMaxGroupPools];
+    float* ys[kMaxGroupPools];
+    for (int g = 0; g < n; ++g) {
+        xs[g] = hs.x;
+        ys[g] = hs.y[g];
+    }
+    plora_status rc = n == 1 ? plora_lora_delta(ctx, hs.x, hs.ids, n_tok, layers[0], projs[0], hs.y[0], stream)
+                             : plora_lora_delta_group(ctx, n, xs, hs.ids, n_tok, layers, projs, ys, stream);
     ctx->bucket_valid = false;
     if (rc != PLORA_OK) return rc;
-    if (cudaMemcpyAsync(y_host, ctx->y_stage, ny, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
-        cudaStreamSynchronize(st) != cudaSuccess)
+    if (cudaEventRecord(hs.done, st) != cudaSuccess || cudaStreamWaitEvent(ctx->d2h_stream, hs.done, 0) != cudaSuccess)
         return PLORA_ERR_CUDA;
+    // back to the host
+    for (int g = 0; g < n; ++g)
+        if (cudaMemcpyAsync(y_host[g], hs.y[g], (size_t)n_tok * recs[g]->dev.d_out * 4, cudaMemcpyDeviceToHost,
+                            ctx->d2h_stream) != cudaSuccess)
+            return PLORA_ERR_CUDA;
+    if (cudaEventRecord(hs.freed, ctx->d2h_stream) != cudaSuccess) return PLORA_ERR_CUDA;
     return PLORA_OK;
+}
+
+PLORA_API plora_status plora_lora_delta_host(plora_ctx* ctx, const void* x_host, const int32_t* ids_host, int32_t n_tok,
+                                   int32_t layer, int32_t proj, float* y_host, void* stream) {
+    plora_status rc = plora_lora_delta_host_async(ctx, 1, x_host, ids_host, n_tok, &layer, &proj, &y_host, stream);
+    if (rc != PLORA_OK) return rc;
+    return plora_host_sync(ctx);
 }
 
 PLORA_API plora_status plora_device_status(plora_ctx* ctx, void* stream, int32_t* host_out) {

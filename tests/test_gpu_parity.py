@@ -383,6 +383,53 @@ def test_host_buffer_entry_point():
     r.close()
 
 
+def test_pipelined_host_calls_overlap_and_keep_every_result():
+    # more queued calls than staging sets, each with its own ids, x and y; q/k/v share one x and go
+    # as one call, o goes alone; every result equals the device-buffer path bit for bit
+    wl = make_workload(2, n_adapters=48, d_model=512, n_layers=1, n_tok=120)
+    ctx = P.Context(wl.n_tok, wl.n_adapters)
+    probs = {}
+    for pool in wl.pools:
+        pr = _problem_from_workload(wl, pool)
+        probs[pool.proj] = pr
+        ctx.register_pool(pool.layer, pool.proj, pool.d_in, pool.d_out, wl.ranks, wl.scales, pr["A"], pr["B"])
+    ctx.set_path(P.PATH_AUTO)
+    rng = np.random.default_rng(5)
+    calls = []
+    for i in range(9):
+        n_tok = int(rng.integers(1, wl.n_tok + 1))
+        ids = rng.integers(-1, wl.n_adapters, n_tok).astype(np.int32)
+        projs = [0, 1, 2] if i % 2 == 0 else [3]
+        x = probs[projs[0]]["x"][:n_tok].copy()
+        x[:, :8] = x[::-1, :8]                      # a different x per call
+        ys = [rng.standard_normal((n_tok, probs[pj]["d_out"])).astype(np.float32) for pj in projs]
+        calls.append(dict(ids=ids, projs=projs, x=x, y_in=[y.copy() for y in ys],
+                          x_h=torch.from_numpy(x.view(np.int16)).pin_memory(), ids_h=torch.from_numpy(ids).pin_memory(),
+                          y_h=[torch.from_numpy(y).pin_memory() for y in ys]))
+    for c in calls:
+        ctx.lora_delta_host_async(c["x_h"], c["ids_h"], [0] * len(c["projs"]), c["projs"], c["y_h"])
+    ctx.host_sync()
+    for c in calls:
+        ids_d = torch.from_numpy(c["ids"]).to(DEV)
+        x_d = bits_to_dev(c["x"])
+        for g, pj in enumerate(c["projs"]):
+            y_d = torch.from_numpy(c["y_in"][g]).to(DEV)
+            ctx.lora_delta(x_d, ids_d, 0, pj, y_d)
+            torch.cuda.synchronize()
+            assert c["y_h"][g].numpy().tobytes() == y_d.cpu().numpy().tobytes(), (c["projs"], g)
+            pr = dict(probs[pj], T=len(c["ids"]), ids=c["ids"], x=c["x"])
+            ref = _oracle(pr, y_in=c["y_in"][g])
+            delta = np.max(np.abs(ref - c["y_in"][g]))
+            assert np.max(np.abs(c["y_h"][g].numpy() - ref)) <= TOL_FP32_PATH * delta + 1e-6 * np.max(np.abs(ref))
+    assert ctx.device_status() == 0
+    # one x cannot serve pools of different input width; unknown pools are refused
+    assert P.plora_lora_delta_host_async(ctx.handle, 0, 0, 0, [0], [9], [0]) == P.ERR_NOT_REGISTERED
+    c = calls[0]
+    assert P.plora_lora_delta_host_async(ctx.handle, c["x_h"].data_ptr(), c["ids_h"].data_ptr(), len(c["ids"]), [0] * 5,
+                                         [0] * 5, [c["y_h"][0].data_ptr()] * 5) == P.ERR_INVALID_ARG
+    ctx.close()
+
+
 def test_grouped_projections_share_a_launch():
     # q, k, v of one layer read the same x; o has its own.  Grouped q/k/v = one launch, bit-identical
     # to three separate calls (every y element still receives exactly one addition).
