@@ -80,6 +80,7 @@ struct Params {
     int32_t m16;              // m holds 2-byte values (the paper's strategy E4 ships m at S = 2 bytes)
     int32_t n_tok;
     int32_t runs_a, runs_b;   // tasks per unit in the shrink / expand phase
+    int32_t runs_a_sliced;    // column runs per unit when the launch cuts its units into row slices
     int32_t early_tables;     // the bucket tables were complete before the previous kernel of the stream began
     int32_t by_class;         // the launch walks its class's part of bk.cls_list (pools of mixed ranks)
     // The class launches of one call work on different units: a later one need not wait for the
@@ -189,7 +190,7 @@ struct Smem {
 };
 
 // What a stage holds (written by the producer into the stage, read by every consumer warp).
-constexpr int kFlagExpand = 1, kFlagFirst = 2, kFlagLast = 4, kFlagEnd = 8;
+constexpr int kFlagExpand = 1, kFlagFirst = 2, kFlagLast = 4, kFlagEnd = 8, kFlagSlice = 16;
 struct StageHdr {
     int32_t flags;
     int32_t unit, run, tile;
@@ -199,17 +200,19 @@ struct StageHdr {
     float scale;
     int32_t m_seq;    // fused expand stages: running number of the expand task in this CTA (m-ring entry = m_seq % kMRing)
     int32_t group;    // which projection of the launch's group (unit = group * n_units + bucket unit)
+    int32_t k0;       // shrink stages of a row slice: first rank row of the slice (otherwise 0)
 };
 
 __device__ __forceinline__ StageHdr read_hdr(uint32_t a) {
     const uint4 q0 = lds128(a), q1 = lds128(a + 16), q2 = lds128(a + 32);
-    const uint32_t q3 = lds32(a + 48), q4 = lds32(a + 52);
+    const uint32_t q3 = lds32(a + 48), q4 = lds32(a + 52), q5 = lds32(a + 56);
     StageHdr h;
     h.flags = (int)q0.x; h.unit = (int)q0.y; h.run = (int)q0.z; h.tile = (int)q0.w;
     h.cnt = (int)q1.x; h.tok[0] = (int)q1.y; h.tok[1] = (int)q1.z; h.tok[2] = (int)q1.w;
     h.tok[3] = (int)q2.x; h.rp = (int)q2.y; h.r = (int)q2.z; h.scale = __uint_as_float(q2.w);
     h.m_seq = (int)q3;
     h.group = (int)q4;
+    h.k0 = (int)q5;
     return h;
 }
 __device__ __forceinline__ void sts128(uint32_t a, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
@@ -385,7 +388,7 @@ __device__ __forceinline__ void shrink_finish_cnt(const Params& p, const Smem& s
         for (int j = 0; j < kLeft; ++j) {
             const int rr = (idx + j) / CNT, t = (idx + j) % CNT;
             if (t < h.cnt) {
-                const int k = mp.row0 + rr;
+                const int k = h.k0 + mp.row0 + rr;
                 if (MODE == kFused) {
                     // value and epoch leave in one 64-bit store: no fence, nobody waits for it here
                     p.bk.m_part[part_index(p, h.unit, h.run, t) + k] =
@@ -419,7 +422,16 @@ __device__ __forceinline__ void shrink_finish(const Params& p, const Smem& sm, c
 
 // ---- expand: one tile of B; the result goes straight to y ------------------------------------------
 // Lane mapping: a lane owns two adjacent output columns; when the warp's slice has fewer
-// than 32 column pairs, lane groups split the rank rows and meet by shuffles.
+// than 32 column pairs, RG lane groups split the rank rows and meet by shuffles.
+//
+// Which rows a group takes decides the bank conflicts of the B loads.  All rows of a sub-tile
+// start at the same bank (a row is 128 bytes) and only the swizzle, by the row's number mod 8,
+// moves a column's chunk.  Groups that took blocks of consecutive rows would read rows of the same
+// swizzle class at the same time, the same 16 bytes' banks RG times over (8-way at rank 128).  In
+// the fused kernel group g therefore takes the rows g, g + RG, g + 2 RG, ...: at every step the RG
+// groups read RG different classes, that is RG different chunks of the 128-byte bank window, and the
+// gather warp stores m so that a group's rows are consecutive (m_slot_of).  The expand-only kernel
+// gets m from the caller in natural order and keeps the blocks.
 template <int RP>
 struct ExpandMap {
     static constexpr int NSUB = (kMaxRank / RP > kMaxSubPerTile) ? kMaxSubPerTile : kMaxRank / RP;
@@ -427,8 +439,7 @@ struct ExpandMap {
     static constexpr int P = 4 * NSUB;      // column pairs per warp per tile
     static constexpr int RG = 32 / P;       // lane groups that split the rank rows
     static constexpr int RPG = RP / RG;     // rows per group (8 or 16)
-    uint32_t b_off;    // byte offset inside the tile of (first row of the group, this lane's pair), swizzle class 0
-    uint32_t m_off;    // byte offset inside the stage of m[0][first row of the group]
+    uint32_t b_col;    // byte offset inside the tile of (row 0, this lane's pair), swizzle class 0
     int colw;          // this lane's first column inside the tile
     int rg;
     __device__ __forceinline__ void init(int warp, int lane) {
@@ -437,20 +448,25 @@ struct ExpandMap {
         colw = warp * (NSUB * 8) + 2 * pair;
         // the chunk index sits in address bits 4..6 and everything else leaves them clear, so
         // the swizzle of row class j is one XOR with (j << 4)
-        b_off = (colw >> 6) * (RP * 128) + rg * RPG * 128 + (((colw & 63) >> 3) << 4) + (colw & 7) * 2;
-        m_off = kTileBytesMax + rg * RPG * 4;
+        b_col = (colw >> 6) * (RP * 128) + (((colw & 63) >> 3) << 4) + (colw & 7) * 2;
     }
+    // where the gather warp puts m[k] of a token (fused kernel): group-major
+    __device__ static __forceinline__ int m_slot_of(int k) { return (k % RG) * RPG + k / RG; }
 };
 
 template <int MODE, int RP, int CNT, bool H>
 __device__ __forceinline__ void expand_tile_cnt(const Params& p, const Smem& sm, const StageHdr& h,
                                                 const ExpandMap<RP>& mp, uint32_t tile, uint32_t empty_bar, int lane) {
     using M = ExpandMap<RP>;
-    const uint32_t b0 = tile + mp.b_off;
+    constexpr bool kInterleaved = MODE == kFused;   // group g takes rows g + RG * j (else rows g * RPG + j)
+    // address of this lane's pair in the group's row j: base ^ (class(j) << 4) + row(j) * 128
+    const uint32_t b0 = kInterleaved ? ((tile + mp.b_col) ^ ((uint32_t)mp.rg << 4)) + mp.rg * 128
+                                     : tile + mp.b_col + mp.rg * M::RPG * 128;
     const int m_slot = h.m_seq % kMRing;
     if (MODE == kFused && (h.flags & kFlagFirst))   // the gather warp has assembled this task's m
         mbar_wait(sm.m_full + m_slot * 8, (h.m_seq / kMRing) & 1, sm.abort_flag, sm.status);
-    // m[t][k], RP floats per token: in the m ring (fused) or in the stage next to the tile (expand-only)
+    // m of the group's rows, RPG consecutive floats per token: in the m ring (fused, group-major) or
+    // in the stage next to the tile (expand-only, natural order)
     const uint32_t mb = (MODE == kFused ? sm.m_ring + m_slot * kMRingBytes : tile + kTileBytesMax) + mp.rg * M::RPG * 4;
     float acc[2][CNT][2];   // [even / odd rank row][token][column]
 #pragma unroll
@@ -460,7 +476,11 @@ __device__ __forceinline__ void expand_tile_cnt(const Params& p, const Smem& sm,
         uint4 mv[CNT];
         uint32_t braw[4];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) braw[q] = lds32((b0 ^ (((kk + q) & 7) << 4)) + (kk + q) * 128);
+        for (int q = 0; q < 4; ++q) {
+            const int j = kk + q;
+            braw[q] = kInterleaved ? lds32((b0 ^ (((j * M::RG) & 7) << 4)) + j * (M::RG * 128))
+                                   : lds32((b0 ^ ((j & 7) << 4)) + j * 128);
+        }
 #pragma unroll
         for (int t = 0; t < CNT; ++t) {
             if (MODE == kExpandOnly && p.m16) {
@@ -528,13 +548,52 @@ __device__ __forceinline__ void expand_tile(const Params& p, const Smem& sm, con
     }
 }
 
-// Per-lane constants of both phases for one padded rank.
-template <int RP>
+// Row slices.  A unit of padded rank 64 or 128 has few, large tiles (16 KiB for 64 columns at rank
+// 128): cut into at most kMaxRunsA column runs, its shrink keeps only a few CTAs busy when the
+// launch has few units (a rank class of a mixed pool, a small batch).  A fused launch that finds
+// fewer shrink tasks than CTAs therefore also cuts along the rank: a task takes kSliceRows rank
+// rows of a column run.  The rows [k0, k0 + 32) of a sub-tile are contiguous (32 rows of 128 bytes)
+// and keep their swizzle (k0 is a multiple of 8), so four of them, from four consecutive sub-tiles,
+// put side by side in a stage are exactly a tile of a rank-32 adapter over 256 columns: the
+// consumers run the rank-32 code on it and add k0 to the row number when they hand the sums over.
+// The partial words of the slices of one column run fill disjoint rows of the same run, so the
+// workspace and the gather are as without slices; x pieces are fetched once per slice (from L2
+// after the first).  With many units the slices only add copies and hand-overs (measured: 0.86 of
+// the roofline instead of 0.98 on the 13B decode shapes at rank 64), hence the choice per launch.
+constexpr int kSliceRows = 32;
+template <int MODE, int RPK>
+struct SliceCfg {
+    static constexpr bool kCan = MODE == kFused && RPK > kSliceRows;
+    static constexpr int kSlices = kCan ? RPK / kSliceRows : 1;   // when the launch slices
+    static constexpr int kSliceRp = kCan ? kSliceRows : RPK;      // geometry of a slice stage
+};
+// How a launch cuts the shrink of its units.  Every CTA computes the same plan from the same counts.
+struct ShrinkPlan {
+    int runs;     // column runs per unit
+    int slices;   // row slices per column run
+};
+template <int MODE, int RPK>
+__device__ __forceinline__ ShrinkPlan shrink_plan(const Params& p, int n_vunits) {
+    ShrinkPlan pl;
+    pl.runs = p.runs_a;
+    pl.slices = 1;
+    if (SliceCfg<MODE, RPK>::kCan && n_vunits * p.runs_a < (int)gridDim.x) {
+        pl.runs = p.runs_a_sliced;
+        pl.slices = SliceCfg<MODE, RPK>::kSlices;
+    }
+    return pl;
+}
+
+// Per-lane constants of both phases: shrink stages have the geometry of padded rank RP or, for
+// slice stages, RPS; expand stages that of RP.
+template <int RP, int RPS>
 struct LaneMaps {
     ShrinkMap<RP> s;
+    ShrinkMap<RPS> s2;
     ExpandMap<RP> e;
     __device__ __forceinline__ void init(int warp, int lane) {
         s.init(warp, lane);
+        if (RPS != RP) s2.init(warp, lane);
         e.init(warp, lane);
     }
 };
@@ -542,7 +601,7 @@ struct LaneMaps {
 // One stage, consumer side.
 template <int MODE, int RP, bool H>
 __device__ __forceinline__ void consume_stage(const Params& p, const Smem& sm, const StageHdr& h,
-                                              const LaneMaps<RP>& maps, uint32_t tile, uint32_t empty_bar,
+                                              const LaneMaps<RP, SliceCfg<MODE, RP>::kSliceRp>& maps, uint32_t tile, uint32_t empty_bar,
                                               float (&acc)[kMaxRowsPerLane][kTokChunk], int warp, int lane) {
     if (!(h.flags & kFlagExpand)) {
         if (MODE != kExpandOnly) {
@@ -552,10 +611,18 @@ __device__ __forceinline__ void consume_stage(const Params& p, const Smem& sm, c
 #pragma unroll
                     for (int t = 0; t < kTokChunk; ++t) acc[rr][t] = 0.f;
             }
-            shrink_tile<RP, H>(p, h, maps.s, tile, acc);
-            __syncwarp();
-            if (lane == 0) mbar_arrive(empty_bar);
-            if (h.flags & kFlagLast) shrink_finish<MODE, RP>(p, sm, h, maps.s, acc, warp, lane);
+            constexpr int RPS = SliceCfg<MODE, RP>::kSliceRp;
+            if (RPS != RP && (h.flags & kFlagSlice)) {
+                shrink_tile<RPS, H>(p, h, maps.s2, tile, acc);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty_bar);
+                if (h.flags & kFlagLast) shrink_finish<MODE, RPS>(p, sm, h, maps.s2, acc, warp, lane);
+            } else {
+                shrink_tile<RP, H>(p, h, maps.s, tile, acc);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty_bar);
+                if (h.flags & kFlagLast) shrink_finish<MODE, RP>(p, sm, h, maps.s, acc, warp, lane);
+            }
         }
     } else {
         if (MODE != kShrinkOnly) {
@@ -575,12 +642,12 @@ __device__ __forceinline__ const unsigned long long* partial_src(const Params& p
     const int t = idx >> sh, k = idx & (rp - 1);
     return p.bk.m_part + part_index(p, unit, 0, t) + k;
 }
-__device__ __forceinline__ void partial_load(const Params& p, uint32_t epoch, const unsigned long long* src,
+__device__ __forceinline__ void partial_load(const Params& p, int runs_a, uint32_t epoch, const unsigned long long* src,
                                              unsigned long long (&w)[kMaxRunsA]) {
     const size_t run_stride = (size_t)p.pool.max_rp;
 #pragma unroll
     for (int j = 0; j < kMaxRunsA; ++j)
-        w[j] = j < p.runs_a ? ldg_cg_u64(src + j * run_stride) : ((unsigned long long)epoch << 32);
+        w[j] = j < runs_a ? ldg_cg_u64(src + j * run_stride) : ((unsigned long long)epoch << 32);
 }
 __device__ __forceinline__ bool partial_sum(uint32_t epoch, const unsigned long long (&w)[kMaxRunsA], uint32_t dst) {
     bool ok = true;
@@ -596,18 +663,21 @@ __device__ __forceinline__ bool partial_sum(uint32_t epoch, const unsigned long 
 // The words of up to kGatherDepth values per lane are requested before the first of them is
 // used: a unit's m costs one round trip to L2 per 32 * kGatherDepth values, not one per 32.
 constexpr int kGatherDepth = 2;
-__device__ __forceinline__ bool gather_m(const Params& p, uint32_t epoch, int unit, int cnt, int rp, int lane,
-                                         uint32_t mdst) {
+template <int RP>
+__device__ __forceinline__ bool gather_m(const Params& p, int runs_a, uint32_t epoch, int unit, int cnt, int lane, uint32_t mdst) {
     bool ok = true;
-    const int n = cnt * rp;
+    const int n = cnt * RP;
     for (int i0 = lane; i0 < n; i0 += 32 * kGatherDepth) {
         unsigned long long w[kGatherDepth][kMaxRunsA];
 #pragma unroll
         for (int q = 0; q < kGatherDepth; ++q)
-            if (i0 + q * 32 < n) partial_load(p, epoch, partial_src(p, unit, i0 + q * 32, rp), w[q]);
+            if (i0 + q * 32 < n) partial_load(p, runs_a, epoch, partial_src(p, unit, i0 + q * 32, RP), w[q]);
 #pragma unroll
-        for (int q = 0; q < kGatherDepth; ++q)
-            if (i0 + q * 32 < n) ok = partial_sum(epoch, w[q], mdst + (i0 + q * 32) * 4) && ok;
+        for (int q = 0; q < kGatherDepth; ++q) {
+            const int i = i0 + q * 32;
+            // value k of token t goes where the expand lanes of its row group look for it
+            if (i < n) ok = partial_sum(epoch, w[q], mdst + ((i / RP) * RP + ExpandMap<RP>::m_slot_of(i % RP)) * 4) && ok;
+        }
     }
     return ok;
 }
@@ -620,14 +690,20 @@ struct Task {
     int unit;
     int phase;   // 0 = shrink, 1 = expand
     int run;
+    int slice;   // shrink: which row slice of the column run (0 when the unit is not sliced)
 };
 
-__device__ __forceinline__ Task decode_task(int t, int n_shrink_tasks, int runs_a, int runs_b) {
+// Shrink tasks of a unit: run-major, the slices of one column run next to one another (their x
+// pieces are the same bytes).
+__device__ __forceinline__ Task decode_task(int t, int n_shrink_tasks, int runs_a, int slices, int runs_b) {
     Task k;
+    k.slice = 0;
     if (t < n_shrink_tasks) {
         k.phase = 0;
-        k.unit = t / runs_a;
-        k.run = t - k.unit * runs_a;
+        k.unit = t / (runs_a * slices);
+        const int rem = t - k.unit * (runs_a * slices);
+        k.run = rem / slices;
+        k.slice = rem - k.run * slices;
     } else {
         t -= n_shrink_tasks;
         k.phase = 1;
@@ -635,6 +711,20 @@ __device__ __forceinline__ Task decode_task(int t, int n_shrink_tasks, int runs_
         k.run = t - k.unit * runs_b;
     }
     return k;
+}
+
+// Expand tasks per unit.  The host proposes a number from the shapes alone; a launch that turns out
+// to have few units (the CTAs see the count, the host does not) cuts its units finer, down to two
+// tiles per task, until there are about two tasks per CTA.  Every CTA computes the same number.
+template <int MODE, int RPK>
+__device__ __forceinline__ int expand_runs(const Params& p, int n_vunits) {
+    int runs = p.runs_b;
+    if (MODE == kFused) {
+        const int cap = max(runs, tiles_for(p.pool.d_out, RPK) / 2);
+        const int want = (2 * (int)gridDim.x + n_vunits - 1) / max(n_vunits, 1);
+        runs = min(cap, max(runs, want));
+    }
+    return runs;
 }
 
 // The (group, unit) pairs a launch walks: all of them (pools of one rank), or its class's part
@@ -804,8 +894,12 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
         const int n_units = *p.bk.n_bgmv_units;
         const ClassList cl = class_list<RPK>(p, n_units);   // the (group, unit) pairs of this launch
         const int n_vunits = cl.n;
-        const int n_shrink = MODE == kExpandOnly ? 0 : n_vunits * p.runs_a;
-        const int n_tasks = n_shrink + (MODE == kShrinkOnly ? 0 : n_vunits * p.runs_b);
+        using SC = SliceCfg<MODE, RPK>;
+        const ShrinkPlan plan = shrink_plan<MODE, RPK>(p, n_vunits);
+        const bool sliced = SC::kCan && plan.slices > 1;
+        const int runs_b = expand_runs<MODE, RPK>(p, n_vunits);
+        const int n_shrink = MODE == kExpandOnly ? 0 : n_vunits * plan.runs * plan.slices;
+        const int n_tasks = n_shrink + (MODE == kShrinkOnly ? 0 : n_vunits * runs_b);
         const int stride = gridDim.x;
         const unsigned full = 0xffffffffu;
         uint32_t it_base = 0;
@@ -813,19 +907,21 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
         for (int base = blockIdx.x; base < n_tasks; base += 32 * stride) {
             const int my_task = base + lane * stride;
             const bool in_range = my_task < n_tasks;
-            Task mine = decode_task(in_range ? my_task : base, n_shrink, p.runs_a, p.runs_b);
+            Task mine = decode_task(in_range ? my_task : base, n_shrink, plan.runs, plan.slices, runs_b);
             mine.unit = cl.at(mine.unit);   // group * n_units + unit
             const int my_group = mine.unit / max(n_units, 1);
             const WorkUnit mu = p.bk.bgmv_units[mine.unit - my_group * n_units];
             const AdapterEntry me = p.table_g[my_group][mu.adapter];
             const bool has = in_range && me.rp == RPK;   // units of other rank classes belong to other launches
             const int in_batch = min(32, (n_tasks - base + stride - 1) / stride);
-            const int C = tile_cols(me.rp);
-            const uint32_t tb = (uint32_t)tile_bytes(me.rp);
+            // a shrink stage of a sliced unit has the geometry of a rank-kSliceRows tile
+            const int C = tile_cols(!mine.phase && sliced ? SC::kSliceRp : RPK);
+            const uint32_t tb = (uint32_t)tile_bytes(RPK);   // bytes of a slab tile
             const int d = mine.phase ? p.pool.d_out : p.pool.d_in;
-            const int runs = mine.phase ? p.runs_b : p.runs_a;
-            const int nT = tiles_for(d, me.rp);
+            const int runs = mine.phase ? runs_b : plan.runs;
+            const int nT = (d + C - 1) / C;
             const int lo = has ? mine.run * nT / runs : 0, hi = has ? (mine.run + 1) * nT / runs : 0;
+            const int k0 = mine.slice * kSliceRows;
             const uint8_t* src = p.slab_g[my_group] + (mine.phase ? me.offB : me.offA);
             const uint16_t* my_x = p.x_g[my_group];
             if (!waited) {
@@ -859,13 +955,29 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
                         const uint32_t bar = sm.full + slot * 8;
                         const uint32_t tbytes = mine.phase ? mbytes : (uint32_t)min(C, d - i * C) * 2u;
                         mbar_wait(sm.empty + slot * 8, ((it / kStages) & 1) ^ 1, sm.abort_flag, p.status);
-                        const int flags = (mine.phase ? kFlagExpand : 0) | (i == lo ? kFlagFirst : 0) | (i == hi - 1 ? kFlagLast : 0);
+                        const int flags = (mine.phase ? kFlagExpand : 0) | (i == lo ? kFlagFirst : 0) | (i == hi - 1 ? kFlagLast : 0) |
+                                          (!mine.phase && sliced ? kFlagSlice : 0);
                         sts128(dst + kHdrOffset, (uint32_t)flags, (uint32_t)(my_group * p.n_tok + mu.pos0), (uint32_t)mine.run, (uint32_t)i);
                         sts128(dst + kHdrOffset + 16, (uint32_t)cnt, (uint32_t)mu.tok[0], (uint32_t)mu.tok[1], (uint32_t)mu.tok[2]);
                         sts128(dst + kHdrOffset + 32, (uint32_t)mu.tok[3], (uint32_t)me.rp, (uint32_t)me.r, __float_as_uint(me.scale));
-                        sts128(dst + kHdrOffset + 48, m_seq, (uint32_t)my_group, 0u, 0u);
-                        mbar_arrive_expect_tx(bar, tb + (uint32_t)cnt * tbytes);
-                        bulk_g2s(dst, src + (size_t)i * tb, tb, bar);
+                        sts128(dst + kHdrOffset + 48, m_seq, (uint32_t)my_group, (uint32_t)k0, 0u);
+                        if (SC::kCan && sliced && !mine.phase) {
+                            // rows [k0, k0 + kSliceRows) of up to four consecutive sub-tiles of A^T, side by side
+                            constexpr int kNsub = RPK > kMaxRank / kMaxSubPerTile ? kMaxRank / RPK : kMaxSubPerTile;   // sub-tiles per slab tile
+                            constexpr uint32_t kPiece = kSliceRows * kSubCols * 2;
+                            const int n_sub = (d + kSubCols - 1) / kSubCols;
+                            const int n_here = min(C / kSubCols, n_sub - i * (C / kSubCols));
+                            mbar_arrive_expect_tx(bar, (uint32_t)n_here * kPiece + (uint32_t)cnt * tbytes);
+                            for (int j = 0; j < n_here; ++j) {
+                                const int g = i * (C / kSubCols) + j;
+                                bulk_g2s(dst + j * kPiece,
+                                         src + (size_t)(g / kNsub) * tb + (size_t)(g % kNsub) * (RPK * kSubCols * 2) + (size_t)k0 * (kSubCols * 2),
+                                         kPiece, bar);
+                            }
+                        } else {
+                            mbar_arrive_expect_tx(bar, tb + (uint32_t)cnt * tbytes);
+                            bulk_g2s(dst, src + (size_t)i * tb, tb, bar);
+                        }
                         if (!mine.phase) {
 #pragma unroll
                             for (int t = 0; t < kTokChunk; ++t)
@@ -904,8 +1016,10 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
         const int n_units = *p.bk.n_bgmv_units;
         const ClassList cl = class_list<RPK>(p, n_units);
         const int n_vunits = cl.n;
-        const int n_shrink = n_vunits * p.runs_a;
-        const int n_tasks = n_shrink + n_vunits * p.runs_b;
+        const ShrinkPlan plan = shrink_plan<MODE, RPK>(p, n_vunits);
+        const int runs_b = expand_runs<MODE, RPK>(p, n_vunits);
+        const int n_shrink = n_vunits * plan.runs * plan.slices;
+        const int n_tasks = n_shrink + n_vunits * runs_b;
         const int stride = gridDim.x;
         const unsigned full = 0xffffffffu;
         // this CTA's first expand task
@@ -915,7 +1029,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
         for (int base = t; base < n_tasks; base += 32 * stride) {
             const int my_task = base + lane * stride;
             const bool in_range = my_task < n_tasks;
-            const int my_unit = cl.at((in_range ? my_task - n_shrink : base - n_shrink) / p.runs_b);
+            const int my_unit = cl.at((in_range ? my_task - n_shrink : base - n_shrink) / runs_b);
             const int my_group = my_unit / max(n_units, 1);
             const WorkUnit mu = p.bk.bgmv_units[my_unit - my_group * n_units];
             const int my_rp = p.table_g[my_group][mu.adapter].rp;
@@ -928,11 +1042,11 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
                 if (lane == 0) mbar_wait(sm.m_empty + e * 8, ((seq / kMRing) & 1) ^ 1, sm.abort_flag, p.status);
                 __syncwarp();
                 const uint32_t mdst = sm.m_ring + e * kMRingBytes;
-                if (!__all_sync(full, gather_m(p, sm.epoch, unit_b, cnt_b, rp_b, lane, mdst))) {
+                if (!__all_sync(full, gather_m<RPK>(p, plan.runs, sm.epoch, unit_b, cnt_b, lane, mdst))) {
                     const long long t0 = clock64();
                     for (;;) {
                         __nanosleep(100);
-                        if (__all_sync(full, gather_m(p, sm.epoch, unit_b, cnt_b, rp_b, lane, mdst)) || *sm.abort_flag) break;
+                        if (__all_sync(full, gather_m<RPK>(p, plan.runs, sm.epoch, unit_b, cnt_b, lane, mdst)) || *sm.abort_flag) break;
                         if (clock64() - t0 > kWaitCycles) {
                             if (lane == 0) give_up(sm.abort_flag, p.status);
                             break;
@@ -949,7 +1063,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
 
     // ------------------------------- consumer warps -------------------------------
     float acc[kMaxRowsPerLane][kTokChunk];
-    LaneMaps<RPK> maps;   // per-lane constants of both phases
+    LaneMaps<RPK, SliceCfg<MODE, RPK>::kSliceRp> maps;   // per-lane constants of both phases
     maps.init(warp, lane);
     for (uint32_t it = 0;; ++it) {
         const uint32_t slot = it % kStages;
@@ -1067,6 +1181,11 @@ cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const
         p.bump_epoch = rp == last_rp;
         // a unit of this class has tiles_for(d, rp) tiles per phase: cut each phase into runs
         p.runs_a = mode == kShrinkOnly ? 1 : clamp_runs(tiles_for(pool.d_in, rp));
+        // (a fused launch with few units of padded rank above kSliceRows cuts them into row slices,
+        // whose stages have the rank-kSliceRows geometry)
+        const int slices = mode == kFused && rp > kSliceRows ? rp / kSliceRows : 1;
+        p.runs_a_sliced = clamp_runs(tiles_for(pool.d_in, kSliceRows));
+        if (p.runs_a_sliced > kMaxRunsA) p.runs_a_sliced = kMaxRunsA;
         // an expand task pays one round trip for its m before its first tile: give it at least two tiles
         p.runs_b = clamp_runs(tiles_for(pool.d_out, rp) / (mode == kFused ? 2 : 1));
         // every shrink task ends with a hand-over of its partial m (and every expand task reads all of
@@ -1079,7 +1198,7 @@ cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const
             if (need > bk.m_part_bytes) return cudaErrorMemoryAllocation;
         }
         // persistent grid: two CTAs per SM, never more CTAs than there can be tasks
-        const long long max_tasks = (long long)n_tok * n_groups * (p.runs_a + p.runs_b);
+        const long long max_tasks = (long long)n_tok * n_groups * (p.runs_a * slices + p.runs_b);
         int grid = kCtasPerSm * sm_count;
         if (grid > max_tasks) grid = (int)max_tasks;
         if (grid < 1) grid = 1;

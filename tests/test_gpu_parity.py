@@ -12,6 +12,7 @@ import oracle
 import paper_2608_05483_b200 as P
 from gpu_util import DEV, Runner, bits_to_dev
 from helpers import TOL_CONTRACT, TOL_FP32_PATH, random_problem, rel_err
+from workloads.gen import f32_to_bf16_bits
 from workloads import gen_adapter, gen_x, gen_y_in, make_workload
 
 pytestmark = pytest.mark.gpu
@@ -364,6 +365,24 @@ def test_two_byte_m_between_shrink_and_expand():
         assert r.ctx.device_status() == 0
     finally:
         r.close()
+
+
+@pytest.mark.parametrize("rank", [40, 64, 100, 128])
+@pytest.mark.parametrize("n_distinct", [3, 30, 140])
+def test_high_rank_units_few_and_many(rank, n_distinct):
+    # a launch with few units of padded rank 64 or 128 cuts their shrink into row slices, one with
+    # many units does not (the launch decides from its unit count); the widths are ragged against
+    # both geometries (64 and 256 columns per stage) and units have 1..4 tokens
+    rng = np.random.default_rng(rank * 1000 + n_distinct)
+    N = n_distinct + 5
+    p = random_problem(rank + n_distinct, T=1, d_in=584, d_out=328, ranks=[rank] * N)
+    ids = np.concatenate([np.repeat(np.arange(n_distinct), 1), rng.integers(0, n_distinct, n_distinct // 2 + 2)]).astype(np.int32)
+    rng.shuffle(ids)
+    T = len(ids)
+    p["T"], p["ids"] = T, ids
+    p["x"] = f32_to_bf16_bits(rng.standard_normal((T, p["d_in"]), dtype=np.float32))
+    p["y_in"] = rng.standard_normal((T, p["d_out"]), dtype=np.float32)
+    _check_paths(p, paths=(P.PATH_FUSED, P.PATH_AUTO))
 
 
 def test_host_buffer_entry_point():
