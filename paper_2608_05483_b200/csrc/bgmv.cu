@@ -427,11 +427,11 @@ __device__ __forceinline__ void shrink_finish(const Params& p, const Smem& sm, c
 // Which rows a group takes decides the bank conflicts of the B loads.  All rows of a sub-tile
 // start at the same bank (a row is 128 bytes) and only the swizzle, by the row's number mod 8,
 // moves a column's chunk.  Groups that took blocks of consecutive rows would read rows of the same
-// swizzle class at the same time, the same 16 bytes' banks RG times over (8-way at rank 128).  In
-// the fused kernel group g therefore takes the rows g, g + RG, g + 2 RG, ...: at every step the RG
-// groups read RG different classes, that is RG different chunks of the 128-byte bank window, and the
-// gather warp stores m so that a group's rows are consecutive (m_slot_of).  The expand-only kernel
-// gets m from the caller in natural order and keeps the blocks.
+// swizzle class at the same time, the same 16 bytes' banks RG times over (8-way at rank 128).
+// Group g therefore takes the rows g, g + RG, g + 2 RG, ...: at every step the RG groups read RG
+// different classes, that is RG different chunks of the 128-byte bank window.  In the fused kernel
+// the gather warp stores m so that a group's rows are consecutive (m_slot_of); the expand-only
+// kernel gets m from the caller in natural order and reads it value by value.
 template <int RP>
 struct ExpandMap {
     static constexpr int NSUB = (kMaxRank / RP > kMaxSubPerTile) ? kMaxSubPerTile : kMaxRank / RP;
@@ -458,22 +458,24 @@ template <int MODE, int RP, int CNT, bool H>
 __device__ __forceinline__ void expand_tile_cnt(const Params& p, const Smem& sm, const StageHdr& h,
                                                 const ExpandMap<RP>& mp, uint32_t tile, uint32_t empty_bar, int lane) {
     using M = ExpandMap<RP>;
-    constexpr bool kInterleaved = MODE == kFused;   // group g takes rows g + RG * j (else rows g * RPG + j)
-    // address of this lane's pair in the group's row j: base ^ (class(j) << 4) + row(j) * 128
+    // Interleaved: group g takes the rows g + RG * j, and the address of this lane's pair in row j is
+    // base ^ (class(j) << 4) + row(j) * 128.  The expand-only kernel with RG <= 2 keeps blocks of rows
+    // (g * RPG + j): it would pay more for fetching its m value by value than the two-way conflict costs.
+    constexpr bool kInterleaved = MODE == kFused || M::RG >= 4;
     const uint32_t b0 = kInterleaved ? ((tile + mp.b_col) ^ ((uint32_t)mp.rg << 4)) + mp.rg * 128
                                      : tile + mp.b_col + mp.rg * M::RPG * 128;
     const int m_slot = h.m_seq % kMRing;
     if (MODE == kFused && (h.flags & kFlagFirst))   // the gather warp has assembled this task's m
         mbar_wait(sm.m_full + m_slot * 8, (h.m_seq / kMRing) & 1, sm.abort_flag, sm.status);
-    // m of the group's rows, RPG consecutive floats per token: in the m ring (fused, group-major) or
-    // in the stage next to the tile (expand-only, natural order)
-    const uint32_t mb = (MODE == kFused ? sm.m_ring + m_slot * kMRingBytes : tile + kTileBytesMax) + mp.rg * M::RPG * 4;
+    // fused: m in the m ring, group-major, so the group's rows are RPG consecutive floats per token;
+    // expand-only: the caller's m next to the tile, in natural order
+    const uint32_t mb = MODE == kFused ? sm.m_ring + m_slot * kMRingBytes + mp.rg * M::RPG * 4 : tile + kTileBytesMax;
     float acc[2][CNT][2];   // [even / odd rank row][token][column]
 #pragma unroll
     for (int t = 0; t < CNT; ++t) acc[0][t][0] = acc[0][t][1] = acc[1][t][0] = acc[1][t][1] = 0.f;
 #pragma unroll
     for (int kk = 0; kk < M::RPG; kk += 4) {
-        uint4 mv[CNT];
+        uint32_t mv[CNT][4];
         uint32_t braw[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
@@ -483,21 +485,29 @@ __device__ __forceinline__ void expand_tile_cnt(const Params& p, const Smem& sm,
         }
 #pragma unroll
         for (int t = 0; t < CNT; ++t) {
-            if (MODE == kExpandOnly && p.m16) {
-                // 2-byte m: four bf16 values of this token, widened (exactly) to fp32
-                const uint32_t a16 = tile + kTileBytesMax + t * (RP * 2) + (mp.rg * M::RPG + kk) * 2;
-                const uint32_t w0 = lds32(a16), w1 = lds32(a16 + 4);
-                mv[t] = make_uint4(w0 << 16, w0 & 0xffff0000u, w1 << 16, w1 & 0xffff0000u);
+            if (MODE == kFused) {
+                const uint4 v = lds128(mb + t * (RP * 4) + kk * 4);
+                mv[t][0] = v.x; mv[t][1] = v.y; mv[t][2] = v.z; mv[t][3] = v.w;
+            } else if (!kInterleaved && !p.m16) {
+                const int row = mp.rg * M::RPG + kk;   // four consecutive fp32 values
+                const uint4 v = lds128(mb + t * (RP * 4) + row * 4);
+                mv[t][0] = row + 0 < h.r ? v.x : 0u;
+                mv[t][1] = row + 1 < h.r ? v.y : 0u;
+                mv[t][2] = row + 2 < h.r ? v.z : 0u;
+                mv[t][3] = row + 3 < h.r ? v.w : 0u;
             } else {
-                mv[t] = lds128(mb + t * (RP * 4) + kk * 4);
-            }
-            if (MODE == kExpandOnly && h.r < RP) {
-                // the caller's m may hold anything beyond the adapter's rank
-                const int k0 = mp.rg * M::RPG + kk;
-                if (k0 + 0 >= h.r) mv[t].x = 0u;
-                if (k0 + 1 >= h.r) mv[t].y = 0u;
-                if (k0 + 2 >= h.r) mv[t].z = 0u;
-                if (k0 + 3 >= h.r) mv[t].w = 0u;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int row = kInterleaved ? mp.rg + (kk + q) * M::RG : mp.rg * M::RPG + kk + q;
+                    uint32_t v;
+                    if (p.m16) {   // 2-byte m: a bf16 value, widened (exactly) to fp32
+                        const uint32_t w = lds32(mb + t * (RP * 2) + (row & ~1) * 2);
+                        v = (row & 1) ? (w & 0xffff0000u) : (w << 16);
+                    } else {
+                        v = lds32(mb + t * (RP * 4) + row * 4);
+                    }
+                    mv[t][q] = row < h.r ? v : 0u;   // the caller's m may hold anything beyond the adapter's rank
+                }
             }
         }
 #pragma unroll
@@ -505,7 +515,7 @@ __device__ __forceinline__ void expand_tile_cnt(const Params& p, const Smem& sm,
             const float blo = in_lo<H>(braw[q]), bhi = in_hi<H>(braw[q]);
 #pragma unroll
             for (int t = 0; t < CNT; ++t) {
-                const float mk = __uint_as_float(q == 0 ? mv[t].x : q == 1 ? mv[t].y : q == 2 ? mv[t].z : mv[t].w);
+                const float mk = __uint_as_float(mv[t][q]);
                 acc[q & 1][t][0] = fmaf(mk, blo, acc[q & 1][t][0]);
                 acc[q & 1][t][1] = fmaf(mk, bhi, acc[q & 1][t][1]);
             }
