@@ -1183,10 +1183,12 @@ cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const
         p.early_tables = 0;   // the first class launch reads what the classify pass has just written
     }
     // one launch per padded-rank class present in the pool
-    int last_rp = 8;
-    for (int rp = 8; rp <= kMaxRank; rp <<= 1)
+    // The class launches of a call overlap (see defer_wait).  The class with the largest units goes
+    // first: the others' CTAs move in as its CTAs retire and fill its tail.
+    int last_rp = kMaxRank;
+    for (int rp = kMaxRank; rp >= 8; rp >>= 1)
         if (rp_mask & rp) last_rp = rp;
-    for (int rp = 8; rp <= kMaxRank; rp <<= 1) {
+    for (int rp = kMaxRank; rp >= 8; rp >>= 1) {
         if (!(rp_mask & rp)) continue;
         p.bump_epoch = rp == last_rp;
         // a unit of this class has tiles_for(d, rp) tiles per phase: cut each phase into runs
