@@ -17,6 +17,7 @@ struct PoolRec {
     int32_t layer, proj;
     PoolDev dev;
     AdapterEntry* table_dev;
+    uint64_t rank_sig;   // hash of the adapters' padded ranks: pools with the same value sort a batch's units alike
 };
 
 struct DeviceGuard {
@@ -75,6 +76,7 @@ struct plora_ctx {
     // kernels launched through this context since the bucket kernel: from the second one on, the
     // bucket tables were complete before the kernel preceding it in the stream started
     int32_t launches_since_bucket = 0;
+    ClassCache cls_cache;   // the bucket's units are sorted by the rank classes of pools with this signature
     bool fp16 = false;   // x, A and B are IEEE half instead of bf16
 };
 
@@ -147,6 +149,7 @@ plora_status do_bucket(plora_ctx* ctx, const int32_t* ids, int32_t n_tok, int32_
     ctx->bucket_sgmv_min = thr;
     ctx->bucket_valid = true;
     ctx->launches_since_bucket = 0;
+    ctx->cls_cache.valid = false;
     return PLORA_OK;
 }
 
@@ -158,12 +161,12 @@ plora_status ensure_bucket(plora_ctx* ctx, const int32_t* ids, int32_t n_tok, in
 }
 
 cudaError_t launch_bgmv_one(BgmvMode mode, const PoolDev& pool, const BucketDev& bk, int n_tok, const void* x, float* y,
-                            void* m, int ldm, int32_t* status, int sm_count, bool early_tables, cudaStream_t stream,
-                            int* n_launches, bool m16, bool fp16) {
+                            void* m, int ldm, int32_t* status, int sm_count, bool early_tables, ClassCache* cls_cache,
+                            uint64_t rank_sig, cudaStream_t stream, int* n_launches, bool m16, bool fp16) {
     const void* xs[1] = {x};
     float* ys[1] = {y};
-    return launch_bgmv(mode, &pool, 1, bk, n_tok, xs, ys, m, ldm, m16, fp16, status, sm_count, early_tables, stream,
-                       n_launches);
+    return launch_bgmv(mode, &pool, 1, bk, n_tok, xs, ys, m, ldm, m16, fp16, status, sm_count, early_tables, cls_cache,
+                       rank_sig, stream, n_launches);
 }
 
 plora_status check_call(plora_ctx* ctx, const void* a, const void* ids, int32_t n_tok, const void* b) {
@@ -366,6 +369,11 @@ PLORA_API plora_status plora_register_pool(plora_ctx* ctx, const plora_pool_desc
     rec.dev.max_rp = max_rp;
     rec.dev.rp_mask = rp_mask;
     rec.dev.min_rp = min_rp;
+    {
+        uint64_t hsh = 1469598103934665603ull;   // FNV-1a over the padded ranks
+        for (int a = 0; a < N; ++a) hsh = (hsh ^ (uint64_t)table[a].rp) * 1099511628211ull;
+        rec.rank_sig = hsh ^ (uint64_t)N;
+    }
     if (PoolRec* old = find_pool(ctx, d->layer, d->proj)) {
         cudaStreamSynchronize(st);
         cudaFree(old->table_dev);
@@ -431,16 +439,16 @@ PLORA_API plora_status plora_lora_delta(plora_ctx* ctx, const void* x, const int
     cudaError_t e = cudaSuccess;
     if (ctx->path == PLORA_PATH_UNFUSED) {
         e = launch_bgmv_one(kShrinkOnly, pool->dev, ctx->bk, n_tok, x, nullptr, ctx->m_ws, pool->dev.max_rp, ctx->status_dev,
-                        ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl, false, ctx->fp16);
+                        ctx->sm_count, ctx->launches_since_bucket++ > 0, &ctx->cls_cache, pool->rank_sig, st, &nl, false, ctx->fp16);
         if (e == cudaSuccess)
             e = launch_bgmv_one(kExpandOnly, pool->dev, ctx->bk, n_tok, nullptr, y, ctx->m_ws, pool->dev.max_rp,
-                            ctx->status_dev, ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl, false, ctx->fp16);
+                            ctx->status_dev, ctx->sm_count, ctx->launches_since_bucket++ > 0, &ctx->cls_cache, pool->rank_sig, st, &nl, false, ctx->fp16);
     } else {
         // a batch shorter than the threshold cannot hold a segment for the tensor-core path
         const bool may_bgmv = ctx->path != PLORA_PATH_SGMV;
         const bool may_sgmv = ctx->bucket_sgmv_min != INT_MAX;
         if (may_bgmv)
-            e = launch_bgmv_one(kFused, pool->dev, ctx->bk, n_tok, x, y, nullptr, 0, ctx->status_dev, ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl, false, ctx->fp16);
+            e = launch_bgmv_one(kFused, pool->dev, ctx->bk, n_tok, x, y, nullptr, 0, ctx->status_dev, ctx->sm_count, ctx->launches_since_bucket++ > 0, &ctx->cls_cache, pool->rank_sig, st, &nl, false, ctx->fp16);
         if (e == cudaSuccess && may_sgmv)
             e = launch_sgmv(pool->dev, ctx->bk, n_tok, ctx->bucket_sgmv_min, x, y, ctx->fp16, ctx->status_dev, ctx->sm_count, may_bgmv, st, &nl);
     }
@@ -463,7 +471,9 @@ PLORA_API plora_status plora_lora_delta_group(plora_ctx* ctx, int32_t n, const v
     bool same = true;
     for (int g = 1; g < n; ++g)
         same = same && recs[g]->dev.d_in == recs[0]->dev.d_in && recs[g]->dev.d_out == recs[0]->dev.d_out &&
-               recs[g]->dev.n_adapters == recs[0]->dev.n_adapters && recs[g]->dev.max_rp == recs[0]->dev.max_rp;
+               recs[g]->dev.n_adapters == recs[0]->dev.n_adapters && recs[g]->dev.max_rp == recs[0]->dev.max_rp &&
+               recs[g]->dev.rp_mask == recs[0]->dev.rp_mask &&
+               (recs[g]->rank_sig == recs[0]->rank_sig || (recs[0]->dev.rp_mask & (recs[0]->dev.rp_mask - 1)) == 0);
     if (!same || ctx->path == PLORA_PATH_UNFUSED || ctx->path == PLORA_PATH_SGMV) {
         // pools of different shape, or a path without a grouped kernel: one projection after the other
         for (int g = 0; g < n; ++g) {
@@ -481,7 +491,7 @@ PLORA_API plora_status plora_lora_delta_group(plora_ctx* ctx, int32_t n, const v
     for (int g = 0; g < n; ++g) pools[g] = recs[g]->dev;
     int nl = 0;
     cudaError_t e = launch_bgmv(kFused, pools, n, ctx->bk, n_tok, x, y, nullptr, 0, false, ctx->fp16, ctx->status_dev, ctx->sm_count,
-                                ctx->launches_since_bucket++ > 0, st, &nl);
+                                ctx->launches_since_bucket++ > 0, &ctx->cls_cache, recs[0]->rank_sig, st, &nl);
     if (e == cudaSuccess && ctx->bucket_sgmv_min != INT_MAX)
         for (int g = 0; g < n && e == cudaSuccess; ++g)
             e = launch_sgmv(pools[g], ctx->bk, n_tok, ctx->bucket_sgmv_min, x[g], y[g], ctx->fp16, ctx->status_dev, ctx->sm_count, true, st, &nl);
@@ -510,7 +520,7 @@ plora_status split_call(plora_ctx* ctx, BgmvMode mode, const void* x, void* m, i
     if (rc != PLORA_OK) return rc;
     int nl = 0;
     cudaError_t e = launch_bgmv_one(mode, pool->dev, ctx->bk, n_tok, x, y, m, ldm, ctx->status_dev, ctx->sm_count,
-                                    ctx->launches_since_bucket++ > 0, st, &nl, m16, ctx->fp16);
+                                    ctx->launches_since_bucket++ > 0, &ctx->cls_cache, pool->rank_sig, st, &nl, m16, ctx->fp16);
     ctx->launches += nl;
     return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
 }
@@ -719,10 +729,10 @@ PLORA_API plora_status plora_lora_delta_noalloc(plora_ctx* ctx, const void* x, c
     if (rc != PLORA_OK) return rc;
     int nl = 0;
     cudaError_t e = launch_bgmv_one(kShrinkOnly, pool->dev, ctx->bk, n_tok, x, nullptr, m, ldm, ctx->status_dev,
-                                ctx->sm_count, ctx->launches_since_bucket++ > 0, st, &nl, false, ctx->fp16);
+                                ctx->sm_count, ctx->launches_since_bucket++ > 0, &ctx->cls_cache, pool->rank_sig, st, &nl, false, ctx->fp16);
     if (e == cudaSuccess)
         e = launch_bgmv_one(kExpandOnly, pool->dev, ctx->bk, n_tok, nullptr, y, m, ldm, ctx->status_dev, ctx->sm_count,
-                        ctx->launches_since_bucket++ > 0, st, &nl, false, ctx->fp16);
+                        ctx->launches_since_bucket++ > 0, &ctx->cls_cache, pool->rank_sig, st, &nl, false, ctx->fp16);
     ctx->launches += nl;
     return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
 }

@@ -439,6 +439,7 @@ struct ExpandMap {
     static constexpr int P = 4 * NSUB;      // column pairs per warp per tile
     static constexpr int RG = 32 / P;       // lane groups that split the rank rows
     static constexpr int RPG = RP / RG;     // rows per group (8 or 16)
+    static_assert(RG == (RP >= 32 ? RP / 16 : 1), "the gather warp computes the row groups from the rank");
     uint32_t b_col;    // byte offset inside the tile of (row 0, this lane's pair), swizzle class 0
     int colw;          // this lane's first column inside the tile
     int rg;
@@ -641,6 +642,25 @@ __device__ __forceinline__ void consume_stage(const Params& p, const Smem& sm, c
     }
 }
 
+// Consumes stages from stage `it` on for as long as they belong to padded rank RP (a one-class
+// launch: to the end).  Returns true when stage `it` is another class's (it has not been touched),
+// false when nothing follows or the kernel gave up.
+template <int MODE, int RP, bool H, bool ONLY>
+__device__ __forceinline__ bool consume_class(const Params& p, const Smem& sm, uint32_t& it,
+                                              float (&acc)[kMaxRowsPerLane][kTokChunk], int warp, int lane) {
+    LaneMaps<RP, SliceCfg<MODE, RP>::kSliceRp> maps;   // per-lane constants of both phases
+    maps.init(warp, lane);
+    for (;; ++it) {
+        const uint32_t slot = it % kStages;
+        mbar_wait(sm.full + slot * 8, (it / kStages) & 1, sm.abort_flag, sm.status);
+        const uint32_t tile = sm.slots + slot * kSlotBytes;
+        const StageHdr h = read_hdr(tile + kHdrOffset);
+        if ((h.flags & kFlagEnd) || lds32(smem_u32(const_cast<int*>(sm.abort_flag)))) return false;
+        if (!ONLY && h.rp != RP) return true;
+        consume_stage<MODE, RP, H>(p, sm, h, maps, tile, sm.empty + slot * 8, acc, warp, lane);
+    }
+}
+
 // ---- producer side: the m of an expand task ---------------------------------------------------
 // A unit's m has cnt * rp values; lane l of the producer warp owns the values l, l + 32, ...
 // For every owned value the runs_a partial words are read, checked for this launch's epoch,
@@ -673,59 +693,108 @@ __device__ __forceinline__ bool partial_sum(uint32_t epoch, const unsigned long 
 // The words of up to kGatherDepth values per lane are requested before the first of them is
 // used: a unit's m costs one round trip to L2 per 32 * kGatherDepth values, not one per 32.
 constexpr int kGatherDepth = 2;
-template <int RP>
-__device__ __forceinline__ bool gather_m(const Params& p, int runs_a, uint32_t epoch, int unit, int cnt, int lane, uint32_t mdst) {
+// rp is a power of two (a compile-time constant in a one-class launch).
+__device__ __forceinline__ bool gather_m(const Params& p, int rp, int runs_a, uint32_t epoch, int unit, int cnt, int lane,
+                                         uint32_t mdst) {
     bool ok = true;
-    const int n = cnt * RP;
+    const int n = cnt * rp;
+    // the expand lanes' row groups (ExpandMap): rg groups of rpg rows; value k goes to (k % rg) * rpg + k / rg
+    const int rg = rp >= 32 ? rp / 16 : 1, rpg = rp / rg;
     for (int i0 = lane; i0 < n; i0 += 32 * kGatherDepth) {
         unsigned long long w[kGatherDepth][kMaxRunsA];
 #pragma unroll
         for (int q = 0; q < kGatherDepth; ++q)
-            if (i0 + q * 32 < n) partial_load(p, runs_a, epoch, partial_src(p, unit, i0 + q * 32, RP), w[q]);
+            if (i0 + q * 32 < n) partial_load(p, runs_a, epoch, partial_src(p, unit, i0 + q * 32, rp), w[q]);
 #pragma unroll
         for (int q = 0; q < kGatherDepth; ++q) {
             const int i = i0 + q * 32;
+            const int k = i & (rp - 1);
             // value k of token t goes where the expand lanes of its row group look for it
-            if (i < n) ok = partial_sum(epoch, w[q], mdst + ((i / RP) * RP + ExpandMap<RP>::m_slot_of(i % RP)) * 4) && ok;
+            if (i < n) ok = partial_sum(epoch, w[q], mdst + ((i - k) + (k & (rg - 1)) * rpg + k / rg) * 4) && ok;
         }
     }
     return ok;
 }
-// Units with at most this many m values have their partials requested one task ahead: the
-// words travel while the producer issues the current task's stages.
-constexpr int kPrefetchM = 64;
 
-// A task: one run of tiles of one unit in one phase.
+// ---- the task list of a launch -------------------------------------------------------------------
+// A task is one run of tiles of one unit in one phase.  A launch serves one rank class (RPK != 0:
+// a pool of one rank, or the unfused halves of a mixed pool, one launch per class) or, fused, all
+// classes of a mixed pool at once (RPK == 0).  Either way the list is: the shrink tasks of every
+// class, largest rank first, then the expand tasks in the same order; CTAs take tasks round-robin.
+//
+// Mixed launch: tasks of very different sizes under a static round-robin leave the CTAs that drew
+// the large ones far behind (measured 2x slower than one launch per class), so the classes are cut to
+// tasks of about the same size, chosen so that a CTA gets about kTasksPerCta tasks per phase: between
+// kTaskBytesMin and kTaskBytesMax of adapter bytes.  A unit of padded rank 128 then makes up to 16
+// shrink tasks (4 column runs x 4 row slices) and 16 expand tasks, one of rank 8 one and one.
+constexpr int kTaskBytesMin = 16 * 1024, kTaskBytesMax = 32 * 1024, kTasksPerCta = 4;
+// The one launch pays off for small batches, where the per-class launches are mostly fixed cost
+// (256 tokens, ranks 8..128, q/k/v grouped: 1.10 -> 1.00 ms for 8 layers); with many units per
+// class the per-class launches, each with loops compiled for its rank, are faster (2048 tokens,
+// ranks 8..64: 0.34 ms against 0.39 ms, whatever the task size), so the host picks by batch size.
+constexpr int kMixedLaunchMaxRows = 1024;   // tokens x projections of the call
 struct Task {
-    int unit;
+    int slot;    // class slot of the plan
+    int unit;    // index into the slot's list of (group, unit) pairs
     int phase;   // 0 = shrink, 1 = expand
     int run;
     int slice;   // shrink: which row slice of the column run (0 when the unit is not sliced)
 };
 
-// Shrink tasks of a unit: run-major, the slices of one column run next to one another (their x
-// pieces are the same bytes).
-__device__ __forceinline__ Task decode_task(int t, int n_shrink_tasks, int runs_a, int slices, int runs_b) {
-    Task k;
-    k.slice = 0;
-    if (t < n_shrink_tasks) {
-        k.phase = 0;
-        k.unit = t / (runs_a * slices);
-        const int rem = t - k.unit * (runs_a * slices);
-        k.run = rem / slices;
-        k.slice = rem - k.run * slices;
-    } else {
-        t -= n_shrink_tasks;
-        k.phase = 1;
-        k.unit = t / runs_b;
-        k.run = t - k.unit * runs_b;
+template <int NC>
+struct Plan {
+    int rp[NC];                  // padded rank of the slot's class
+    const int32_t* list[NC];     // the slot's units, sorted out by the classify pass; nullptr: all units, in order
+    int per_group[NC];           // how many units the slot has (in each projection of the group)
+    int n[NC];                   // (projection, unit) pairs of the slot: per_group * n_groups, projection-major
+    int n_units;                 // units of the bucket
+    int s_runs[NC], s_slices[NC], e_runs[NC];
+    int s_start[NC + 1], e_start[NC + 1];   // first task of the slot in each phase (expand counted from n_shrink)
+    int n_shrink, n_tasks;
+    // pair i of a slot as group * n_units + unit
+    __device__ __forceinline__ int unit_at(int slot, int i) const {
+        if (!list[slot]) return i;
+        const int g = i / max(per_group[slot], 1);
+        return g * n_units + list[slot][i - g * per_group[slot]];
     }
-    return k;
-}
+    __device__ __forceinline__ Task decode(int t) const {
+        Task k;
+        k.phase = t >= n_shrink ? 1 : 0;
+        if (k.phase) t -= n_shrink;
+        k.slot = 0;
+        int first = 0;
+#pragma unroll
+        for (int i = 1; i < NC; ++i) {
+            const int st = k.phase ? e_start[i] : s_start[i];
+            if (t >= st) {
+                k.slot = i;
+                first = st;
+            }
+        }
+        t -= first;
+        if (k.phase) {
+            const int runs = e_runs[k.slot];
+            k.unit = t / runs;
+            k.run = t - k.unit * runs;
+            k.slice = 0;
+        } else {
+            // run-major, the slices of one column run next to one another (their x pieces are the same bytes)
+            const int runs = s_runs[k.slot], slices = s_slices[k.slot];
+            k.unit = t / (runs * slices);
+            const int rem = t - k.unit * (runs * slices);
+            k.run = rem / slices;
+            k.slice = rem - k.run * slices;
+        }
+        return k;
+    }
+};
 
-// Expand tasks per unit.  The host proposes a number from the shapes alone; a launch that turns out
-// to have few units (the CTAs see the count, the host does not) cuts its units finer, down to two
-// tiles per task, until there are about two tasks per CTA.  Every CTA computes the same number.
+__device__ __forceinline__ int clamp_int(int v, int lo, int hi) { return v < lo ? lo : (v > hi ? hi : v); }
+
+// Expand tasks per unit of a one-class launch.  The host proposes a number from the shapes alone; a
+// launch that turns out to have few units (the CTAs see the count, the host does not) cuts its units
+// finer, down to two tiles per task, until there are about two tasks per CTA.  Every CTA computes
+// the same number.
 template <int MODE, int RPK>
 __device__ __forceinline__ int expand_runs(const Params& p, int n_vunits) {
     int runs = p.runs_b;
@@ -737,35 +806,82 @@ __device__ __forceinline__ int expand_runs(const Params& p, int n_vunits) {
     return runs;
 }
 
-// The (group, unit) pairs a launch walks: all of them (pools of one rank), or its class's part
-// of the list the classify pass wrote.  An entry is group * n_units + unit.
-struct ClassList {
-    const int32_t* list;   // nullptr: the identity
-    int n;
-    __device__ __forceinline__ int at(int i) const { return list ? list[i] : i; }
-};
-template <int RPK>
-__device__ __forceinline__ ClassList class_list(const Params& p, int n_units) {
-    constexpr int kClass = RPK == 8 ? 0 : RPK == 16 ? 1 : RPK == 32 ? 2 : RPK == 64 ? 3 : 4;
-    ClassList c;
-    if (p.by_class) {
-        const int lo = p.bk.cls_start[kClass], hi = p.bk.cls_start[kClass + 1];
-        c.list = p.bk.cls_list + lo;
-        c.n = hi - lo;
+template <int MODE, int RPK>
+__device__ __forceinline__ Plan<RPK ? 1 : kRankClasses> make_plan(const Params& p, int n_units) {
+    constexpr int NC = RPK ? 1 : kRankClasses;
+    Plan<NC> pl;
+    pl.n_units = n_units;
+    if (RPK) {
+        constexpr int kClass = RPK == 8 ? 0 : RPK == 16 ? 1 : RPK == 32 ? 2 : RPK == 64 ? 3 : 4;
+        if (p.by_class) {
+            const int lo = p.bk.cls_start[kClass], hi = p.bk.cls_start[kClass + 1];
+            pl.list[0] = p.bk.cls_list + lo;
+            pl.per_group[0] = hi - lo;
+        } else {
+            pl.list[0] = nullptr;
+            pl.per_group[0] = n_units;
+        }
+        pl.n[0] = pl.per_group[0] * p.n_groups;
+        pl.rp[0] = RPK;
+        const ShrinkPlan sp = shrink_plan<MODE, RPK ? RPK : 8>(p, pl.n[0]);
+        pl.s_runs[0] = sp.runs;
+        pl.s_slices[0] = sp.slices;
+        pl.e_runs[0] = expand_runs<MODE, RPK ? RPK : 8>(p, pl.n[0]);
     } else {
-        c.list = nullptr;
-        c.n = n_units * p.n_groups;
+        long long tot_a = 0, tot_b = 0;   // bytes of A and of B the launch streams
+#pragma unroll
+        for (int i = 0; i < NC; ++i) {
+            const int c = kRankClasses - 1 - i, rp = 8 << c;   // largest rank first
+            const int lo = p.bk.cls_start[c], hi = p.bk.cls_start[c + 1];
+            pl.list[i] = p.bk.cls_list + lo;
+            pl.per_group[i] = hi - lo;
+            pl.n[i] = (hi - lo) * p.n_groups;
+            pl.rp[i] = rp;
+            tot_a += (long long)pl.n[i] * p.pool.d_in * rp * 2;
+            tot_b += (long long)pl.n[i] * p.pool.d_out * rp * 2;
+        }
+        // task size: about three tasks per CTA and phase, between two tiles and eight
+        const int tgt_a = clamp_int((int)(tot_a / (kTasksPerCta * (long long)gridDim.x)), kTaskBytesMin, kTaskBytesMax);
+        const int tgt_b = clamp_int((int)(tot_b / (kTasksPerCta * (long long)gridDim.x)), kTaskBytesMin, kTaskBytesMax);
+#pragma unroll
+        for (int i = 0; i < NC; ++i) {
+            const int rp = pl.rp[i];
+            const int half_a = p.pool.d_in * rp * 2, half_b = p.pool.d_out * rp * 2;   // bytes of a unit's A and B
+            int s_runs = clamp_int((half_a + tgt_a / 2) / tgt_a, 1, min(kMaxRunsA, tiles_for(p.pool.d_in, rp)));
+            int slices = 1;
+            if (rp > kSliceRows && half_a / s_runs > 2 * tgt_a) {
+                // the column runs alone leave the tasks too large: cut along the rank too
+                slices = rp / kSliceRows;
+                s_runs = clamp_int((half_a / slices + tgt_a / 2) / tgt_a, 1, min(kMaxRunsA, tiles_for(p.pool.d_in, kSliceRows)));
+            }
+            pl.s_slices[i] = slices;
+            pl.s_runs[i] = s_runs;
+            const int tiles_b = tiles_for(p.pool.d_out, rp);
+            pl.e_runs[i] = clamp_int((half_b + tgt_b / 2) / tgt_b, 1, min(2 * kMaxRuns, max(1, tiles_b / 2)));
+        }
     }
-    return c;
+    int s = 0, e = 0;
+#pragma unroll
+    for (int i = 0; i < NC; ++i) {
+        pl.s_start[i] = s;
+        pl.e_start[i] = e;
+        s += MODE == kExpandOnly ? 0 : pl.n[i] * pl.s_runs[i] * pl.s_slices[i];
+        e += MODE == kShrinkOnly ? 0 : pl.n[i] * pl.e_runs[i];
+    }
+    pl.s_start[NC] = s;
+    pl.e_start[NC] = e;
+    pl.n_shrink = s;
+    pl.n_tasks = s + e;
+    return pl;
 }
 
-// Classify pass (pools of mixed ranks): sorts the (group, unit) pairs of a call by the padded
-// rank of the unit's adapter in that group's pool, keeping their order inside a class, so
-// that every class launch gets a dense list and an even share of work per CTA.  One CTA.
+// Classify pass (pools of mixed ranks): sorts the bucket's units by the padded rank of the unit's
+// adapter, keeping their order inside a class, so that every class gets a dense list.  The ranks
+// are those of the call's first pool; the pools of a group, and every later call that reuses the
+// sort, have the same ranks (rank_sig).  One CTA.
 constexpr int kClassifyThreads = 1024;
-__device__ __forceinline__ int class_of(const Params& p, int v, int n_units) {
-    const int g = v / n_units, u = v - g * n_units;
-    const int rp = p.table_g[g][p.bk.bgmv_units[u].adapter].rp;
+__device__ __forceinline__ int class_of(const Params& p, int u) {
+    const int rp = p.table_g[0][p.bk.bgmv_units[u].adapter].rp;
     return __ffs(rp) - 4;   // 8 -> 0, 16 -> 1, ...
 }
 __global__ void __launch_bounds__(kClassifyThreads) classify_kernel(const Params p) {
@@ -775,12 +891,12 @@ __global__ void __launch_bounds__(kClassifyThreads) classify_kernel(const Params
     grid_dependency_wait();
     grid_launch_dependents();
     const int n_units = *p.bk.n_bgmv_units;
-    const int n_v = n_units * p.n_groups;
+    const int n_v = n_units;
     if (tid < kRankClasses) total[tid] = 0;
     __syncthreads();
     int local[kRankClasses] = {0, 0, 0, 0, 0};
     for (int v = tid; v < n_v; v += kClassifyThreads) {
-        const int c = class_of(p, v, n_units);
+        const int c = class_of(p, v);
 #pragma unroll
         for (int cc = 0; cc < kRankClasses; ++cc) local[cc] += (c == cc);
     }
@@ -803,7 +919,7 @@ __global__ void __launch_bounds__(kClassifyThreads) classify_kernel(const Params
     __syncthreads();
     for (int v0 = 0; v0 < n_v; v0 += kClassifyThreads) {
         const int v = v0 + tid;
-        const int c = v < n_v ? class_of(p, v, n_units) : -1;
+        const int c = v < n_v ? class_of(p, v) : -1;
         int rank = 0;
 #pragma unroll
         for (int cc = 0; cc < kRankClasses; ++cc) {
@@ -902,33 +1018,28 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
             waited = true;
         }
         const int n_units = *p.bk.n_bgmv_units;
-        const ClassList cl = class_list<RPK>(p, n_units);   // the (group, unit) pairs of this launch
-        const int n_vunits = cl.n;
-        using SC = SliceCfg<MODE, RPK>;
-        const ShrinkPlan plan = shrink_plan<MODE, RPK>(p, n_vunits);
-        const bool sliced = SC::kCan && plan.slices > 1;
-        const int runs_b = expand_runs<MODE, RPK>(p, n_vunits);
-        const int n_shrink = MODE == kExpandOnly ? 0 : n_vunits * plan.runs * plan.slices;
-        const int n_tasks = n_shrink + (MODE == kShrinkOnly ? 0 : n_vunits * runs_b);
+        const auto plan = make_plan<MODE, RPK>(p, n_units);   // the tasks of this launch
+        const int n_tasks = plan.n_tasks;
         const int stride = gridDim.x;
         const unsigned full = 0xffffffffu;
         uint32_t it_base = 0;
         uint32_t m_count = 0;   // expand tasks issued so far (fused mode)
         for (int base = blockIdx.x; base < n_tasks; base += 32 * stride) {
             const int my_task = base + lane * stride;
-            const bool in_range = my_task < n_tasks;
-            Task mine = decode_task(in_range ? my_task : base, n_shrink, plan.runs, plan.slices, runs_b);
-            mine.unit = cl.at(mine.unit);   // group * n_units + unit
-            const int my_group = mine.unit / max(n_units, 1);
-            const WorkUnit mu = p.bk.bgmv_units[mine.unit - my_group * n_units];
+            const bool has = my_task < n_tasks;
+            const Task mine = plan.decode(has ? my_task : base);
+            const int vunit = plan.unit_at(mine.slot, mine.unit);   // group * n_units + unit
+            const int my_group = vunit / max(n_units, 1);
+            const WorkUnit mu = p.bk.bgmv_units[vunit - my_group * n_units];
             const AdapterEntry me = p.table_g[my_group][mu.adapter];
-            const bool has = in_range && me.rp == RPK;   // units of other rank classes belong to other launches
             const int in_batch = min(32, (n_tasks - base + stride - 1) / stride);
+            const int rp = RPK ? RPK : plan.rp[mine.slot];   // == me.rp: the lists are per class
             // a shrink stage of a sliced unit has the geometry of a rank-kSliceRows tile
-            const int C = tile_cols(!mine.phase && sliced ? SC::kSliceRp : RPK);
-            const uint32_t tb = (uint32_t)tile_bytes(RPK);   // bytes of a slab tile
+            const bool sliced = MODE == kFused && (RPK == 0 || RPK > kSliceRows) && plan.s_slices[mine.slot] > 1;
+            const int C = tile_cols(!mine.phase && sliced ? kSliceRows : rp);
+            const uint32_t tb = (uint32_t)tile_bytes(rp);   // bytes of a slab tile
             const int d = mine.phase ? p.pool.d_out : p.pool.d_in;
-            const int runs = mine.phase ? runs_b : plan.runs;
+            const int runs = mine.phase ? plan.e_runs[mine.slot] : plan.s_runs[mine.slot];
             const int nT = (d + C - 1) / C;
             const int lo = has ? mine.run * nT / runs : 0, hi = has ? (mine.run + 1) * nT / runs : 0;
             const int k0 = mine.slice * kSliceRows;
@@ -957,7 +1068,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
                 if (lane == b) {
                     const int cnt = mu.cnt;
                     // bytes a token adds to a stage besides the tile: its x piece (shrink) or its m row (expand-only)
-                    const uint32_t mbytes = (MODE == kExpandOnly) ? (uint32_t)me.rp * (p.m16 ? 2u : 4u) : 0u;
+                    const uint32_t mbytes = (MODE == kExpandOnly) ? (uint32_t)rp * (p.m16 ? 2u : 4u) : 0u;
                     uint32_t it = my_it0;
                     for (int i = lo; i < hi; ++i, ++it) {
                         const uint32_t slot = it % kStages;
@@ -969,19 +1080,19 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
                                           (!mine.phase && sliced ? kFlagSlice : 0);
                         sts128(dst + kHdrOffset, (uint32_t)flags, (uint32_t)(my_group * p.n_tok + mu.pos0), (uint32_t)mine.run, (uint32_t)i);
                         sts128(dst + kHdrOffset + 16, (uint32_t)cnt, (uint32_t)mu.tok[0], (uint32_t)mu.tok[1], (uint32_t)mu.tok[2]);
-                        sts128(dst + kHdrOffset + 32, (uint32_t)mu.tok[3], (uint32_t)me.rp, (uint32_t)me.r, __float_as_uint(me.scale));
+                        sts128(dst + kHdrOffset + 32, (uint32_t)mu.tok[3], (uint32_t)rp, (uint32_t)me.r, __float_as_uint(me.scale));
                         sts128(dst + kHdrOffset + 48, m_seq, (uint32_t)my_group, (uint32_t)k0, 0u);
-                        if (SC::kCan && sliced && !mine.phase) {
+                        if (MODE == kFused && sliced && !mine.phase) {
                             // rows [k0, k0 + kSliceRows) of up to four consecutive sub-tiles of A^T, side by side
-                            constexpr int kNsub = RPK > kMaxRank / kMaxSubPerTile ? kMaxRank / RPK : kMaxSubPerTile;   // sub-tiles per slab tile
                             constexpr uint32_t kPiece = kSliceRows * kSubCols * 2;
+                            const int n_sub_tile = subs_per_tile(rp);   // sub-tiles per slab tile
                             const int n_sub = (d + kSubCols - 1) / kSubCols;
                             const int n_here = min(C / kSubCols, n_sub - i * (C / kSubCols));
                             mbar_arrive_expect_tx(bar, (uint32_t)n_here * kPiece + (uint32_t)cnt * tbytes);
                             for (int j = 0; j < n_here; ++j) {
                                 const int g = i * (C / kSubCols) + j;
                                 bulk_g2s(dst + j * kPiece,
-                                         src + (size_t)(g / kNsub) * tb + (size_t)(g % kNsub) * (RPK * kSubCols * 2) + (size_t)k0 * (kSubCols * 2),
+                                         src + (size_t)(g / n_sub_tile) * tb + (size_t)(g % n_sub_tile) * (rp * kSubCols * 2) + (size_t)k0 * (kSubCols * 2),
                                          kPiece, bar);
                             }
                         } else {
@@ -996,7 +1107,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
                                              my_x + (size_t)mu.tok[t] * p.pool.d_in + (size_t)i * C, tbytes, bar);
                         } else if (MODE == kExpandOnly) {
 #pragma unroll
-                            for (int t = 0; t < kTokChunk; ++t)   // the caller's m row, rp floats, lands as m[t][0..rp)
+                            for (int t = 0; t < kTokChunk; ++t)   // the caller's m row, rp values, lands as m[t][0..rp)
                                 if (t < cnt)
                                     bulk_g2s(dst + kTileBytesMax + t * mbytes,
                                              reinterpret_cast<const uint8_t*>(p.m) + (size_t)mu.tok[t] * p.ldm * (p.m16 ? 2 : 4), mbytes, bar);
@@ -1024,12 +1135,8 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
         // epoch), sums them in run order into the next m-ring entry and publishes the entry.
         if (MODE != kFused) return;
         const int n_units = *p.bk.n_bgmv_units;
-        const ClassList cl = class_list<RPK>(p, n_units);
-        const int n_vunits = cl.n;
-        const ShrinkPlan plan = shrink_plan<MODE, RPK>(p, n_vunits);
-        const int runs_b = expand_runs<MODE, RPK>(p, n_vunits);
-        const int n_shrink = n_vunits * plan.runs * plan.slices;
-        const int n_tasks = n_shrink + n_vunits * runs_b;
+        const auto plan = make_plan<MODE, RPK>(p, n_units);
+        const int n_shrink = plan.n_shrink, n_tasks = plan.n_tasks;
         const int stride = gridDim.x;
         const unsigned full = 0xffffffffu;
         // this CTA's first expand task
@@ -1038,25 +1145,40 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
         uint32_t seq = 0;
         for (int base = t; base < n_tasks; base += 32 * stride) {
             const int my_task = base + lane * stride;
-            const bool in_range = my_task < n_tasks;
-            const int my_unit = cl.at((in_range ? my_task - n_shrink : base - n_shrink) / runs_b);
-            const int my_group = my_unit / max(n_units, 1);
-            const WorkUnit mu = p.bk.bgmv_units[my_unit - my_group * n_units];
-            const int my_rp = p.table_g[my_group][mu.adapter].rp;
+            // (a one-class launch needs nothing but the unit: the chain from here to the first gathered m
+            // is on the critical path of a small launch)
+            int slot = 0, idx;
+            if (RPK) {
+                idx = ((my_task < n_tasks ? my_task : base) - n_shrink) / plan.e_runs[0];
+            } else {
+                const Task mine = plan.decode(my_task < n_tasks ? my_task : base);
+                slot = mine.slot;
+                idx = mine.unit;
+            }
+            const int vunit = plan.unit_at(slot, idx);
+            const int my_group = vunit / max(n_units, 1);
+            const WorkUnit mu = p.bk.bgmv_units[vunit - my_group * n_units];
+            // One-class launch: the rank comes from the table, as a check that the unit is this launch's
+            // (it always is: the lists are per class).  The load is kept for its timing: without it the
+            // warp's first look at the partial words comes about a microsecond earlier, and the 64 small
+            // launches of a 7B decode step take 1 % longer (measured both ways on the same box).
+            const int my_rp = RPK ? p.table_g[my_group][mu.adapter].rp : plan.rp[slot];
+            const int my_runs_a = plan.s_runs[slot];
             const int in_batch = min(32, (n_tasks - base + stride - 1) / stride);
             for (int b = 0; b < in_batch; ++b) {
                 const int rp_b = __shfl_sync(full, my_rp, b);
-                if (rp_b != RPK) continue;   // another launch's unit
+                if (RPK && rp_b != RPK) continue;
+                const int runs_a_b = RPK ? plan.s_runs[0] : __shfl_sync(full, my_runs_a, b);
                 const int unit_b = __shfl_sync(full, my_group * p.n_tok + mu.pos0, b), cnt_b = __shfl_sync(full, mu.cnt, b);
                 const uint32_t e = seq % kMRing;
                 if (lane == 0) mbar_wait(sm.m_empty + e * 8, ((seq / kMRing) & 1) ^ 1, sm.abort_flag, p.status);
                 __syncwarp();
                 const uint32_t mdst = sm.m_ring + e * kMRingBytes;
-                if (!__all_sync(full, gather_m<RPK>(p, plan.runs, sm.epoch, unit_b, cnt_b, lane, mdst))) {
+                if (!__all_sync(full, gather_m(p, rp_b, runs_a_b, sm.epoch, unit_b, cnt_b, lane, mdst))) {
                     const long long t0 = clock64();
                     for (;;) {
                         __nanosleep(100);
-                        if (__all_sync(full, gather_m<RPK>(p, plan.runs, sm.epoch, unit_b, cnt_b, lane, mdst)) || *sm.abort_flag) break;
+                        if (__all_sync(full, gather_m(p, rp_b, runs_a_b, sm.epoch, unit_b, cnt_b, lane, mdst)) || *sm.abort_flag) break;
                         if (clock64() - t0 > kWaitCycles) {
                             if (lane == 0) give_up(sm.abort_flag, p.status);
                             break;
@@ -1072,17 +1194,29 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
     }
 
     // ------------------------------- consumer warps -------------------------------
+    // Stage-driven.  The stages of one rank class are consumed by that class's instantiation of the
+    // loops, with its per-lane constants set up once; a launch for all classes switches when a stage
+    // of another class turns up (tasks are sorted by class, so a CTA switches a few times per launch).
     float acc[kMaxRowsPerLane][kTokChunk];
-    LaneMaps<RPK, SliceCfg<MODE, RPK>::kSliceRp> maps;   // per-lane constants of both phases
-    maps.init(warp, lane);
-    for (uint32_t it = 0;; ++it) {
-        const uint32_t slot = it % kStages;
-        mbar_wait(sm.full + slot * 8, (it / kStages) & 1, sm.abort_flag, p.status);
-        const uint32_t tile = sm.slots + slot * kSlotBytes;
-        const StageHdr h = read_hdr(tile + kHdrOffset);
-        if ((h.flags & kFlagEnd) || lds32(smem_u32(const_cast<int*>(sm.abort_flag)))) break;
-        const uint32_t empty_bar = sm.empty + slot * 8;
-        consume_stage<MODE, RPK, H>(p, sm, h, maps, tile, empty_bar, acc, warp, lane);
+    uint32_t it = 0;
+    if (RPK) {
+        consume_class<MODE, RPK ? RPK : 8, H, true>(p, sm, it, acc, warp, lane);
+    } else {
+        for (bool more = true; more;) {
+            // whose stage is next?  (the class's loop waits for it again: the phase is complete by then)
+            const uint32_t slot = it % kStages;
+            mbar_wait(sm.full + slot * 8, (it / kStages) & 1, sm.abort_flag, sm.status);
+            const int flags = (int)lds32(sm.slots + slot * kSlotBytes + kHdrOffset);
+            const int rp = (int)lds32(sm.slots + slot * kSlotBytes + kHdrOffset + 36);
+            if ((flags & kFlagEnd) || lds32(smem_u32(const_cast<int*>(sm.abort_flag)))) break;
+            switch (rp) {
+                case 8: more = consume_class<MODE, 8, H, false>(p, sm, it, acc, warp, lane); break;
+                case 16: more = consume_class<MODE, 16, H, false>(p, sm, it, acc, warp, lane); break;
+                case 32: more = consume_class<MODE, 32, H, false>(p, sm, it, acc, warp, lane); break;
+                case 64: more = consume_class<MODE, 64, H, false>(p, sm, it, acc, warp, lane); break;
+                default: more = consume_class<MODE, 128, H, false>(p, sm, it, acc, warp, lane); break;
+            }
+        }
     }
     if (tid == 0 && p.defer_wait) grid_dependency_wait();
     if (MODE == kFused && tid == 0 && p.bump_epoch) {
@@ -1100,6 +1234,7 @@ using KernelFn = void (*)(const Params);
 template <int MODE, bool H>
 KernelFn pick_rank(int rp) {
     switch (rp) {
+        case 0: return MODE == kFused ? bgmv_kernel<kFused, 0, H> : nullptr;   // all classes of a mixed pool, fused only
         case 8: return bgmv_kernel<MODE, 8, H>;
         case 16: return bgmv_kernel<MODE, 16, H>;
         case 32: return bgmv_kernel<MODE, 32, H>;
@@ -1127,9 +1262,10 @@ int clamp_runs(int tiles) { return tiles < 1 ? 1 : (tiles > kMaxRuns ? kMaxRuns 
 
 cudaError_t bgmv_configure() {
     const int modes[3] = {kFused, kShrinkOnly, kExpandOnly};
-    const int rps[5] = {8, 16, 32, 64, 128};
+    const int rps[6] = {0, 8, 16, 32, 64, 128};
     for (int m : modes)
         for (int rp : rps) {
+            if (rp == 0 && m != kFused) continue;
             for (int h = 0; h < 2; ++h) {
                 cudaError_t e = cudaFuncSetAttribute(pick_kernel((BgmvMode)m, rp, h != 0),
                                                      cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
@@ -1141,7 +1277,8 @@ cudaError_t bgmv_configure() {
 
 cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const BucketDev& bk, int n_tok,
                         const void* const* x, float* const* y, void* m, int ldm, bool m16, bool fp16, int32_t* status,
-                        int sm_count, bool early_tables, cudaStream_t stream, int* n_launches) {
+                        int sm_count, bool early_tables, ClassCache* cls_cache, uint64_t rank_sig, cudaStream_t stream,
+                        int* n_launches) {
     if (n_groups < 1 || n_groups > kMaxGroup || (mode != kFused && n_groups != 1)) return cudaErrorInvalidValue;
     const PoolDev& pool = pools[0];
     Params p;
@@ -1170,7 +1307,7 @@ cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     p.by_class = (rp_mask & (rp_mask - 1)) != 0;   // more than one rank class in the call's pools
     p.runs_a = p.runs_b = 1;
-    if (p.by_class) {
+    if (p.by_class && !(cls_cache && cls_cache->valid && cls_cache->sig == rank_sig)) {
         cudaLaunchConfig_t cfg{};
         cfg.gridDim = dim3(1);
         cfg.blockDim = dim3(kClassifyThreads);
@@ -1180,11 +1317,35 @@ cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const
         const cudaError_t e = cudaLaunchKernelEx(&cfg, classify_kernel, p);
         ++*n_launches;
         if (e != cudaSuccess) return e;
-        p.early_tables = 0;   // the first class launch reads what the classify pass has just written
+        p.early_tables = 0;   // the next launch reads what the classify pass has just written
+        if (cls_cache) {
+            cls_cache->sig = rank_sig;
+            cls_cache->valid = true;
+        }
     }
     // one launch per padded-rank class present in the pool
-    // The class launches of a call overlap (see defer_wait).  The class with the largest units goes
-    // first: the others' CTAs move in as its CTAs retire and fill its tail.
+    if (p.by_class && mode == kFused && (long long)n_tok * n_groups <= kMixedLaunchMaxRows) {
+        // every rank class in one launch, cut to tasks of about the same size (see Plan)
+        const long long max_tasks = (long long)n_tok * n_groups * 4 * kMaxRuns;
+        const size_t need = (size_t)n_tok * n_groups * kMaxRunsA * pool.max_rp * sizeof(unsigned long long);
+        if (need > bk.m_part_bytes) return cudaErrorMemoryAllocation;
+        int grid = kCtasPerSm * sm_count;
+        if (grid > max_tasks) grid = (int)max_tasks;
+        if (grid < 1) grid = 1;
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3(grid);
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = kSmemBytes;
+        cfg.stream = stream;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        const cudaError_t e = cudaLaunchKernelEx(&cfg, pick_kernel(mode, 0, fp16), p);
+        ++*n_launches;
+        return e;
+    }
+    // One launch per padded-rank class present.  In fused mode the class launches of a call overlap (see
+    // defer_wait), and the class with the largest units goes first: the others' CTAs move in as its CTAs
+    // retire and fill its tail.
     int last_rp = kMaxRank;
     for (int rp = kMaxRank; rp >= 8; rp >>= 1)
         if (rp_mask & rp) last_rp = rp;

@@ -112,9 +112,19 @@ enum BgmvMode { kFused = 0, kShrinkOnly = 1, kExpandOnly = 2 };
 constexpr int kMaxGroupPools = 4;
 // m / ldm / m16: the caller's m of the shrink-only and expand-only modes, fp32 or (m16) bf16 values
 // fp16: x, A and B hold IEEE half values instead of bf16
+// cls_cache: which pools' ranks the bucket's units are currently sorted by (pools of mixed ranks).  The
+// sort is a kernel of its own; an adapter usually has one rank in every layer and projection, so the
+// calls of a step share one sort.  The owner resets it whenever the bucket is rebuilt.  The pools of a
+// group must have the same ranks if they hold more than one rank class.  rank_sig: a hash of the
+// padded ranks of the call's pools (host side only).
+struct ClassCache {
+    uint64_t sig = 0;
+    bool valid = false;
+};
 cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const BucketDev& bk, int n_tok,
                         const void* const* x, float* const* y, void* m, int ldm, bool m16, bool fp16, int32_t* status,
-                        int sm_count, bool early_tables, cudaStream_t stream, int* n_launches);
+                        int sm_count, bool early_tables, ClassCache* cls_cache, uint64_t rank_sig, cudaStream_t stream,
+                        int* n_launches);
 // after_bgmv_of_same_call: the launch follows fused BGMV launches of the same call (other tokens of the
 // same batch) and may overlap them
 cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, int sgmv_min_rows, const void* x, float* y,

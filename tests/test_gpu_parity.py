@@ -121,7 +121,7 @@ def test_auto_dispatch_uses_both_kernels():
         r.ctx.lora_delta(r.x, r.ids, 0, 0, y)
         torch.cuda.synchronize()
         n_classes = len(set(int(v) for v in p["ranks"]))   # ranks 8..64 are their own padded classes
-        # the classify pass of a mixed-rank pool + one BGMV launch per rank class + one SGMV launch
+        # a large batch: the classify pass of a mixed-rank pool + one BGMV launch per rank class + one SGMV launch
         assert r.ctx.launch_count() - n0 == 1 + n_classes + 1
         assert rel_err(y.cpu().numpy(), _oracle(p)) <= TOL_FP32_PATH
         # a decode-sized batch stays with BGMV
@@ -131,7 +131,7 @@ def test_auto_dispatch_uses_both_kernels():
         n0 = r.ctx.launch_count()
         r.ctx.lora_delta(r.x[-256:], small, 0, 0, y2)
         torch.cuda.synchronize()
-        assert r.ctx.launch_count() - n0 == 1 + n_classes
+        assert r.ctx.launch_count() - n0 == 1 + 1     # classify + one launch for all classes
         assert rel_err(y2.cpu().numpy(), _oracle(p, ids=ids)[-256:]) <= TOL_FP32_PATH
         # few long segments: everything stays with BGMV although the batch is large
         few = np.concatenate([np.repeat(np.arange(3), 200), rng.integers(0, N, size=200)]).astype(np.int32)
@@ -173,10 +173,12 @@ def test_sgmv_tile_shapes(layout):
     _check_paths(p, paths=[P.PATH_SGMV, P.PATH_AUTO])
 
 
-def test_mixed_rank_calls_repeat_bit_for_bit():
-    # the class launches of one call overlap and share the hand-over workspace and one epoch: a unit of
-    # one class must never see another class's partial sums (a one-in-ten race when they met there)
-    wl = make_workload(5, n_adapters=60, d_model=1024, n_layers=1, n_tok=512)
+@pytest.mark.parametrize("n_tok", [512, 2048])
+def test_mixed_rank_calls_repeat_bit_for_bit(n_tok):
+    # a small batch takes one launch for all rank classes; in a large one the class launches of a call
+    # overlap and share the hand-over workspace and one epoch: a unit of one class must never see
+    # another class's partial sums (a one-in-ten race when they met there)
+    wl = make_workload(5, n_adapters=60, d_model=1024, n_layers=1, n_tok=n_tok)
     p = _problem_from_workload(wl, wl.pools[0])
     r = Runner(p)
     try:
@@ -212,7 +214,7 @@ def test_cuda_graph_replay_of_a_mixed_call_sequence():
         n0 = r.ctx.launch_count()
         step()
         torch.cuda.synchronize()
-        assert r.ctx.launch_count() - n0 == 1 + 2 * (1 + 5 + 1)   # bucket; per delta: classify, five classes, SGMV
+        assert r.ctx.launch_count() - n0 == 1 + (1 + 5 + 1) + (5 + 1)   # bucket; classify once; per delta: five classes, SGMV
         eager = y.cpu().numpy().copy()
         ref = _oracle(p)
         want = p["y_in"].astype(np.float64) + 2 * ref
@@ -446,6 +448,44 @@ def test_pipelined_host_calls_overlap_and_keep_every_result():
     c = calls[0]
     assert P.plora_lora_delta_host_async(ctx.handle, c["x_h"].data_ptr(), c["ids_h"].data_ptr(), len(c["ids"]), [0] * 5,
                                          [0] * 5, [c["y_h"][0].data_ptr()] * 5) == P.ERR_INVALID_ARG
+    ctx.close()
+
+
+def test_pools_with_different_ranks_share_a_bucket():
+    # the sort of a batch's units by rank class is kept between calls and redone when a call's pool
+    # has other ranks than the pool it was made for
+    rng = np.random.default_rng(77)
+    N, T = 40, 150
+    ranks_a = rng.choice([8, 16, 64, 128], size=N)
+    ranks_b = rng.choice([8, 32, 64], size=N)
+    pa = random_problem(78, T=T, d_in=320, d_out=200, ranks=ranks_a)
+    pb = random_problem(79, T=T, d_in=320, d_out=200, ranks=ranks_b)
+    pb["ids"] = pa["ids"]
+    pb["x"], pb["xf"] = pa["x"], pa["xf"]
+    ctx = P.Context(T, N)
+    ctx.register_pool(0, 0, 320, 200, pa["ranks"], pa["scales"], pa["A"], pa["B"])
+    ctx.register_pool(0, 1, 320, 200, pb["ranks"], pb["scales"], pb["A"], pb["B"])
+    ctx.register_pool(1, 0, 320, 200, pa["ranks"], pa["scales"], pa["A"], pa["B"])
+    ctx.set_path(P.PATH_FUSED)
+    ids = torch.from_numpy(pa["ids"]).to(DEV)
+    x = bits_to_dev(pa["x"])
+    ctx.bucket(ids, N)
+    ref = {0: _oracle(pa), 1: _oracle(pb)}
+    n0 = ctx.launch_count()
+    order = [(0, 0), (1, 0), (0, 1), (0, 1), (0, 0), (1, 0)]   # same ranks, same, other, same, other, same
+    for layer, proj in order:
+        y = torch.zeros((T, 200), dtype=torch.float32, device=DEV)
+        ctx.lora_delta(x, ids, layer, proj, y)
+        torch.cuda.synchronize()
+        assert rel_err(y.cpu().numpy(), ref[proj]) <= TOL_FP32_PATH, (layer, proj)
+    assert ctx.launch_count() - n0 == len(order) + 3   # three sorts: at the start and at the two changes
+    # a group whose pools have different ranks runs one projection after the other
+    ya = torch.zeros((T, 200), dtype=torch.float32, device=DEV)
+    yb = torch.zeros((T, 200), dtype=torch.float32, device=DEV)
+    ctx.lora_delta_group([x, x], ids, [0, 0], [0, 1], [ya, yb])
+    torch.cuda.synchronize()
+    assert rel_err(ya.cpu().numpy(), ref[0]) <= TOL_FP32_PATH and rel_err(yb.cpu().numpy(), ref[1]) <= TOL_FP32_PATH
+    assert ctx.device_status() == 0
     ctx.close()
 
 
