@@ -177,6 +177,15 @@ __device__ __forceinline__ void unpack8(const uint4& v, float* f) {
     f[4] = in_lo<H>(v.z); f[5] = in_hi<H>(v.z); f[6] = in_lo<H>(v.w); f[7] = in_hi<H>(v.w);
 }
 
+// The four words of a 16-byte chunk as four (even column, odd column) pairs.
+template <bool H>
+__device__ __forceinline__ void unpack4x2(const uint4& v, float2* f) {
+    f[0] = make_float2(in_lo<H>(v.x), in_hi<H>(v.x));
+    f[1] = make_float2(in_lo<H>(v.y), in_hi<H>(v.y));
+    f[2] = make_float2(in_lo<H>(v.z), in_hi<H>(v.z));
+    f[3] = make_float2(in_lo<H>(v.w), in_hi<H>(v.w));
+}
+
 struct Smem {
     uint32_t slots;      // shared address of stage 0
     uint32_t full;       // full[kStages] barriers
@@ -296,20 +305,23 @@ __device__ __forceinline__ void shrink_chunks(const ShrinkMap<RP>& mp, int cols_
 #pragma unroll
     for (int q = 0; q < M::CPL; ++q) {
         if (!CHECKED || mp.col0 + q * M::CHL * 8 < cols_left) {
-            float xf[CNT][8];
+            // The two values of a 32-bit word (even / odd column) stay together as a pair and every
+            // multiply-add is the packed one (two fp32 FMAs per instruction on sm_100): the even and the
+            // odd chain of a product advance in one issue slot.
+            float2 xp[CNT][4];
 #pragma unroll
-            for (int t = 0; t < CNT; ++t) unpack8<H>(xraw[q][t], xf[t]);
+            for (int t = 0; t < CNT; ++t) unpack4x2<H>(xraw[q][t], xp[t]);
 #pragma unroll
             for (int rr = 0; rr < M::RPL; ++rr) {
-                float af[8];
-                unpack8<H>(araw[q][rr], af);
+                float2 ap[4];
+                unpack4x2<H>(araw[q][rr], ap);
 #pragma unroll
                 for (int t = 0; t < CNT; ++t) {
-                    float e = xf[t][0] * af[0], o = xf[t][1] * af[1];
-                    e = fmaf(xf[t][2], af[2], e); o = fmaf(xf[t][3], af[3], o);
-                    e = fmaf(xf[t][4], af[4], e); o = fmaf(xf[t][5], af[5], o);
-                    e = fmaf(xf[t][6], af[6], e); o = fmaf(xf[t][7], af[7], o);
-                    acc[rr][t] += e + o;
+                    float2 eo = __fmul2_rn(xp[t][0], ap[0]);
+                    eo = __ffma2_rn(xp[t][1], ap[1], eo);
+                    eo = __ffma2_rn(xp[t][2], ap[2], eo);
+                    eo = __ffma2_rn(xp[t][3], ap[3], eo);
+                    acc[rr][t] += eo.x + eo.y;
                 }
             }
         }
@@ -471,9 +483,11 @@ __device__ __forceinline__ void expand_tile_cnt(const Params& p, const Smem& sm,
     // fused: m in the m ring, group-major, so the group's rows are RPG consecutive floats per token;
     // expand-only: the caller's m next to the tile, in natural order
     const uint32_t mb = MODE == kFused ? sm.m_ring + m_slot * kMRingBytes + mp.rg * M::RPG * 4 : tile + kTileBytesMax;
-    float acc[2][CNT][2];   // [even / odd rank row][token][column]
+    // accumulators: per token and column a pair (sum over the even rows, sum over the odd rows), so
+    // that two rows advance per packed multiply-add
+    float2 acc[CNT][2];
 #pragma unroll
-    for (int t = 0; t < CNT; ++t) acc[0][t][0] = acc[0][t][1] = acc[1][t][0] = acc[1][t][1] = 0.f;
+    for (int t = 0; t < CNT; ++t) acc[t][0] = acc[t][1] = make_float2(0.f, 0.f);
 #pragma unroll
     for (int kk = 0; kk < M::RPG; kk += 4) {
         uint32_t mv[CNT][4];
@@ -512,13 +526,15 @@ __device__ __forceinline__ void expand_tile_cnt(const Params& p, const Smem& sm,
             }
         }
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const float blo = in_lo<H>(braw[q]), bhi = in_hi<H>(braw[q]);
+        for (int q = 0; q < 4; q += 2) {
+            // rows q and q + 1 of this step: (row q, row q + 1) pairs of the first and of the second column
+            const float2 b0 = make_float2(in_lo<H>(braw[q]), in_lo<H>(braw[q + 1]));
+            const float2 b1 = make_float2(in_hi<H>(braw[q]), in_hi<H>(braw[q + 1]));
 #pragma unroll
             for (int t = 0; t < CNT; ++t) {
-                const float mk = __uint_as_float(mv[t][q]);
-                acc[q & 1][t][0] = fmaf(mk, blo, acc[q & 1][t][0]);
-                acc[q & 1][t][1] = fmaf(mk, bhi, acc[q & 1][t][1]);
+                const float2 mk = make_float2(__uint_as_float(mv[t][q]), __uint_as_float(mv[t][q + 1]));
+                acc[t][0] = __ffma2_rn(mk, b0, acc[t][0]);
+                acc[t][1] = __ffma2_rn(mk, b1, acc[t][1]);
             }
         }
     }
@@ -530,8 +546,8 @@ __device__ __forceinline__ void expand_tile_cnt(const Params& p, const Smem& sm,
     float out[CNT][2];
 #pragma unroll
     for (int t = 0; t < CNT; ++t) {
-        out[t][0] = acc[0][t][0] + acc[1][t][0];
-        out[t][1] = acc[0][t][1] + acc[1][t][1];
+        out[t][0] = acc[t][0].x + acc[t][0].y;
+        out[t][1] = acc[t][1].x + acc[t][1].y;
     }
 #pragma unroll
     for (int d = M::P; d < 32; d <<= 1)
