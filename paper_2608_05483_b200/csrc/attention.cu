@@ -289,15 +289,18 @@ partial_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 #pragma unroll
         for (int g = 0; g < G; ++g) {
             // q piece: dims [32 qr, +32) of query head g, bf16 in the stage
-            float s = 0.f;
+            // packed multiply-adds (two fp32 FMAs per instruction on sm_100): the even and the odd dims
+            // of a 32-bit word advance together, two chains of 16 instead of one of 32
+            float2 s2 = make_float2(0.f, 0.f);
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const uint4 qw = lds128(st + kQOffset + g * (kHeadDim * 2) + qr * 64 + i * 16);
-                s = fmaf(bf_lo(qw.x), bf_lo(kraw[i].x), s); s = fmaf(bf_hi(qw.x), bf_hi(kraw[i].x), s);
-                s = fmaf(bf_lo(qw.y), bf_lo(kraw[i].y), s); s = fmaf(bf_hi(qw.y), bf_hi(kraw[i].y), s);
-                s = fmaf(bf_lo(qw.z), bf_lo(kraw[i].z), s); s = fmaf(bf_hi(qw.z), bf_hi(kraw[i].z), s);
-                s = fmaf(bf_lo(qw.w), bf_lo(kraw[i].w), s); s = fmaf(bf_hi(qw.w), bf_hi(kraw[i].w), s);
+                s2 = __ffma2_rn(make_float2(bf_lo(qw.x), bf_hi(qw.x)), make_float2(bf_lo(kraw[i].x), bf_hi(kraw[i].x)), s2);
+                s2 = __ffma2_rn(make_float2(bf_lo(qw.y), bf_hi(qw.y)), make_float2(bf_lo(kraw[i].y), bf_hi(kraw[i].y)), s2);
+                s2 = __ffma2_rn(make_float2(bf_lo(qw.z), bf_hi(qw.z)), make_float2(bf_lo(kraw[i].z), bf_hi(kraw[i].z)), s2);
+                s2 = __ffma2_rn(make_float2(bf_lo(qw.w), bf_hi(qw.w)), make_float2(bf_lo(kraw[i].w), bf_hi(kraw[i].w)), s2);
             }
+            float s = s2.x + s2.y;
             s += __shfl_xor_sync(0xffffffffu, s, 8);
             s += __shfl_xor_sync(0xffffffffu, s, 16);
             s = valid ? s * p.scale_log2e : -INFINITY;      // every lane of a token now holds its score
@@ -314,14 +317,15 @@ partial_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             psum += __shfl_xor_sync(0xffffffffu, psum, 2);
             psum += __shfl_xor_sync(0xffffffffu, psum, 4);
             l_run[g] = l_run[g] * alpha + psum;
-            float o0 = o_run[g][0] * alpha, o1 = o_run[g][1] * alpha, o2 = o_run[g][2] * alpha, o3 = o_run[g][3] * alpha;
+            float2 o01 = make_float2(o_run[g][0] * alpha, o_run[g][1] * alpha), o23 = make_float2(o_run[g][2] * alpha, o_run[g][3] * alpha);
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 const float pj = __shfl_sync(0xffffffffu, pt, j);     // lane j (quarter 0) holds token j's weight
-                o0 = fmaf(pj, bf_lo(vraw[j].x), o0); o1 = fmaf(pj, bf_hi(vraw[j].x), o1);
-                o2 = fmaf(pj, bf_lo(vraw[j].y), o2); o3 = fmaf(pj, bf_hi(vraw[j].y), o3);
+                const float2 pp = make_float2(pj, pj);
+                o01 = __ffma2_rn(pp, make_float2(bf_lo(vraw[j].x), bf_hi(vraw[j].x)), o01);
+                o23 = __ffma2_rn(pp, make_float2(bf_lo(vraw[j].y), bf_hi(vraw[j].y)), o23);
             }
-            o_run[g][0] = o0; o_run[g][1] = o1; o_run[g][2] = o2; o_run[g][3] = o3;
+            o_run[g][0] = o01.x; o_run[g][1] = o01.y; o_run[g][2] = o23.x; o_run[g][3] = o23.y;
             m_run[g] = m_new;
         }
         __syncwarp();
