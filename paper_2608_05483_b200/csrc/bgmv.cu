@@ -6,11 +6,13 @@
 // the adapters present, once per adapter whatever its batch), so the kernel is a
 // streaming pipeline:
 //
-//   - a unit's shrink is cut into up to kMaxRunsA tasks (runs of consecutive A tiles)
-//     and its expand into up to kMaxRuns tasks (runs of B tiles); all shrink tasks
-//     come first in the task list and persistent CTAs take tasks round-robin, so
-//     the tiles of one adapter stream through many SMs at once and the load is
-//     balanced at tile granularity whatever the adapter popularity;
+//   - a unit's shrink is cut into up to kMaxRunsA tasks (runs of consecutive A tiles; a launch with
+//     few units of padded rank 64 or 128 also cuts along the rank, see "Row slices") and its expand
+//     into runs of B tiles; all shrink tasks come first in the task list and persistent CTAs take
+//     tasks round-robin, so the tiles of one adapter stream through many SMs at once and the load
+//     is balanced at tile granularity whatever the adapter popularity.  A launch serves one padded
+//     rank (its loops are compiled for that rank) or, for a small batch on a pool of mixed ranks,
+//     all ranks at once, with the classes cut to tasks of equal size (see "the task list of a launch");
 //   - one producer warp per CTA fetches the descriptors of its next 32 tasks at once,
 //     then issues bulk asynchronous copies (cp.async.bulk, completion counted on an
 //     mbarrier) of whole slab tiles, plus the matching pieces of the unit's x rows,
@@ -22,14 +24,15 @@
 //     matching chunks of x, fp32 accumulation) and meet by shuffles at the end of the
 //     task, so a warp owns complete sums of its rows and no warp waits for another;
 //     the task's partial m goes to an L2-resident workspace as 64-bit words
-//     {value, launch epoch} with plain stores and no fence.  Expand: the producer
-//     warp of the CTA that owns the expand task loads the unit's partials (a word
-//     whose epoch matches has arrived, otherwise it is read again), sums them in a
-//     fixed order, scales them and puts m into the stage next to the B tile; a
-//     consumer lane owns two output columns, walks the rank rows, and adds its
-//     result to y with one vector reduction per element (no read of y on the SM;
-//     one addition per element, so the result is bit-reproducible).  Consumer
-//     warps therefore never wait on global memory.
+//     {value, launch epoch} with plain stores and no fence.  Expand: a gather warp of the CTA
+//     that owns the expand task loads the unit's partials (a word whose epoch matches has
+//     arrived, otherwise it is read again), sums them in a fixed order and puts m into a small
+//     ring next to the stages; a consumer lane owns two output columns, walks the rank rows, and
+//     adds its result to y with one vector reduction per element (no read of y on the SM;
+//     one addition per element, so the result is bit-reproducible).  Consumer warps therefore
+//     never wait on global memory.  Both inner loops use the packed fp32 multiply-add of sm_100
+//     (two FMAs per instruction): the kernel is bound by instruction issue where HBM does not
+//     bound it.
 //
 // The same template provides the fused path, the shrink-only path (m written to
 // the caller's buffer, unscaled, one task per unit) and the expand-only path.
