@@ -41,8 +41,13 @@ FALLBACK_HBM_GBS = 6650.0   # used only when MEASURED_PEAKS.json is absent
 # (profiles/*.md say which capture each number comes from); None = not captured.
 # Per (layer, proj) delta; the roofline entry scales it to the average launch (a launch may carry a group).
 NCU_TRAFFIC_BYTES = {
-    "decode7b": 40.17e6,   # profiles/bgmv_fused_config2_decode7b.md: (116.41 + 3.89 + 40.29 + 0.09) MB over q/k/v + o
+    "decode7b": 40.17e6,   # profiles/bgmv_fused_config2_decode7b.md: (116.44 + 3.84 + 40.31 + 0.09) MB over q/k/v + o
+    # profiles/bgmv_fused_config3_decode13b.md: captured on the four 5120 -> 5120 projections, 567.3 MB each against
+    # 565.0 MB of algorithmic bytes; the step's other projections (5120 <-> 13824) are scaled by their algorithmic bytes
+    "decode13b": ("of_algorithmic", 567.3 / 565.0),
     "prefill": 622.7e6,    # profiles/sgmv_config4_prefill.md
+    "mixed": 518.8e6,      # profiles/launch_list_config5_mixed.md: the four class launches of a projection
+    "skew7b": 91.5e6,      # profiles/launch_list_config6_skew7b.md: (272.8 + 93.3) MB over q/k/v + o
 }
 
 
@@ -397,7 +402,8 @@ def run_ours(args):
     achieved = bytes_per_launch / (launch_us * 1e-6) / 1e9
     traffic = NCU_TRAFFIC_BYTES.get(wl.name)
     roofline = dict(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s", frac=achieved / peaks["hbm_gbs"],
-                    traffic=None if traffic is None else traffic * n_calls / delta_launches,
+                    traffic=None if traffic is None else (traffic[1] * bytes_per_launch if isinstance(traffic, tuple)
+                                                           else traffic * n_calls / delta_launches),
                     kernel="sgmv_kernel (tensor-core segmented GEMM)" if wl.name == "prefill" else "bgmv_kernel (fused shrink+expand)",
                     peak_source=peaks["source"], avg_launch_us=launch_us, launches_per_step=delta_launches,
                     per_projection_us=kernel_ms * 1e3, algorithmic_bytes_per_launch=bytes_per_launch,

@@ -131,7 +131,12 @@ size_t layout_pool(const plora_pool_desc* d, std::vector<AdapterEntry>* table, i
 int32_t effective_sgmv_min(const plora_ctx* ctx, int32_t n_tok) {
     switch (ctx->path) {
         case PLORA_PATH_SGMV: return 1;
-        case PLORA_PATH_AUTO: return n_tok >= kSgmvMinBatch ? ctx->sgmv_min_rows : INT_MAX;
+        case PLORA_PATH_AUTO:
+            // kSgmvMinTiles tiles hold at least kSgmvMinTiles * sgmv_min_rows tokens: a smaller batch
+            // cannot have a tensor-core segment, and is spared the launch that would find none
+            return n_tok >= kSgmvMinBatch && (long long)n_tok >= (long long)kSgmvMinTiles * ctx->sgmv_min_rows
+                       ? ctx->sgmv_min_rows
+                       : INT_MAX;
         default: return INT_MAX;
     }
 }
