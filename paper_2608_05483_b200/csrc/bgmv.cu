@@ -1064,12 +1064,6 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
             const int k0 = mine.slice * kSliceRows;
             const uint8_t* src = p.slab_g[my_group] + (mine.phase ? me.offB : me.offA);
             const uint16_t* my_x = p.x_g[my_group];
-            if (!waited) {
-                // this CTA's first descriptors are in registers: join the stream order
-                grid_dependency_wait();
-                waited = true;
-            }
-            if (base == (int)blockIdx.x) sm.epoch = MODE == kFused ? *p.bk.epoch : 0u;
             // first stage number of every lane's task: exclusive prefix sum of the stage counts
             int incl = hi - lo;
 #pragma unroll
@@ -1080,60 +1074,83 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
             const uint32_t my_it0 = it_base + (uint32_t)(incl - (hi - lo));
             it_base += (uint32_t)__shfl_sync(full, incl, 31);
 
-            for (int b = 0; b < in_batch; ++b) {
-                // fused mode: the running number of this expand task tells the consumers where its m is
-                const uint32_t m_seq = m_count;
-                if (MODE == kFused && __shfl_sync(full, (int)(has && mine.phase), b)) ++m_count;
-                if (lane == b) {
-                    const int cnt = mu.cnt;
-                    // bytes a token adds to a stage besides the tile: its x piece (shrink) or its m row (expand-only)
-                    const uint32_t mbytes = (MODE == kExpandOnly) ? (uint32_t)rp * (p.m16 ? 2u : 4u) : 0u;
-                    uint32_t it = my_it0;
-                    for (int i = lo; i < hi; ++i, ++it) {
-                        const uint32_t slot = it % kStages;
-                        const uint32_t dst = sm.slots + slot * kSlotBytes;
-                        const uint32_t bar = sm.full + slot * 8;
-                        const uint32_t tbytes = mine.phase ? mbytes : (uint32_t)min(C, d - i * C) * 2u;
-                        mbar_wait(sm.empty + slot * 8, ((it / kStages) & 1) ^ 1, sm.abort_flag, p.status);
-                        const int flags = (mine.phase ? kFlagExpand : 0) | (i == lo ? kFlagFirst : 0) | (i == hi - 1 ? kFlagLast : 0) |
-                                          (!mine.phase && sliced ? kFlagSlice : 0);
-                        sts128(dst + kHdrOffset, (uint32_t)flags, (uint32_t)(my_group * p.n_tok + mu.pos0), (uint32_t)mine.run, (uint32_t)i);
-                        sts128(dst + kHdrOffset + 16, (uint32_t)cnt, (uint32_t)mu.tok[0], (uint32_t)mu.tok[1], (uint32_t)mu.tok[2]);
-                        sts128(dst + kHdrOffset + 32, (uint32_t)mu.tok[3], (uint32_t)rp, (uint32_t)me.r, __float_as_uint(me.scale));
-                        sts128(dst + kHdrOffset + 48, m_seq, (uint32_t)my_group, (uint32_t)k0, 0u);
-                        if (MODE == kFused && sliced && !mine.phase) {
-                            // rows [k0, k0 + kSliceRows) of up to four consecutive sub-tiles of A^T, side by side
-                            constexpr uint32_t kPiece = kSliceRows * kSubCols * 2;
-                            const int n_sub_tile = subs_per_tile(rp);   // sub-tiles per slab tile
-                            const int n_sub = (d + kSubCols - 1) / kSubCols;
-                            const int n_here = min(C / kSubCols, n_sub - i * (C / kSubCols));
-                            mbar_arrive_expect_tx(bar, (uint32_t)n_here * kPiece + (uint32_t)cnt * tbytes);
-                            for (int j = 0; j < n_here; ++j) {
-                                const int g = i * (C / kSubCols) + j;
-                                bulk_g2s(dst + j * kPiece,
-                                         src + (size_t)(g / n_sub_tile) * tb + (size_t)(g % n_sub_tile) * (rp * kSubCols * 2) + (size_t)k0 * (kSubCols * 2),
-                                         kPiece, bar);
+            // This CTA's first descriptors are in registers.  If it has not joined the stream order yet, the
+            // slab tiles of the ring's first turn go out before it does (pass 1): no kernel ever writes the
+            // slab, and the previous kernel's last CTAs leave most of the memory system idle.  What the
+            // previous kernel may have written (x, the caller's m) follows after the wait (pass 2, which
+            // also issues everything beyond the first turn).  Otherwise one pass issues everything (pass 0).
+            const bool early = !waited;
+            for (int pass = early ? 1 : 0; pass <= (early ? 2 : 0); ++pass) {
+                if (pass == 2) {
+                    grid_dependency_wait();
+                    waited = true;
+                }
+                if (pass != 1 && base == (int)blockIdx.x) sm.epoch = MODE == kFused ? *p.bk.epoch : 0u;
+                uint32_t mc = m_count;
+                for (int b = 0; b < in_batch; ++b) {
+                    // fused mode: the running number of this expand task tells the consumers where its m is
+                    const uint32_t m_seq = mc;
+                    if (MODE == kFused && __shfl_sync(full, (int)(has && mine.phase), b)) ++mc;
+                    if (lane == b) {
+                        const int cnt = mu.cnt;
+                        // bytes a token adds to a stage besides the tile: its x piece (shrink) or its m row (expand-only)
+                        const uint32_t mbytes = (MODE == kExpandOnly) ? (uint32_t)rp * (p.m16 ? 2u : 4u) : 0u;
+                        uint32_t it = my_it0;
+                        for (int i = lo; i < hi; ++i, ++it) {
+                            const bool first_turn = it < (uint32_t)kStages;
+                            if (pass == 1 && !first_turn) break;
+                            const bool head = pass != 2 || !first_turn;   // header, byte count and slab tile
+                            const bool tail = pass != 1;                  // what may depend on the previous kernel
+                            const uint32_t slot = it % kStages;
+                            const uint32_t dst = sm.slots + slot * kSlotBytes;
+                            const uint32_t bar = sm.full + slot * 8;
+                            const uint32_t tbytes = mine.phase ? mbytes : (uint32_t)min(C, d - i * C) * 2u;
+                            if (head) {
+                                mbar_wait(sm.empty + slot * 8, ((it / kStages) & 1) ^ 1, sm.abort_flag, p.status);
+                                const int flags = (mine.phase ? kFlagExpand : 0) | (i == lo ? kFlagFirst : 0) | (i == hi - 1 ? kFlagLast : 0) |
+                                                  (!mine.phase && sliced ? kFlagSlice : 0);
+                                sts128(dst + kHdrOffset, (uint32_t)flags, (uint32_t)(my_group * p.n_tok + mu.pos0), (uint32_t)mine.run, (uint32_t)i);
+                                sts128(dst + kHdrOffset + 16, (uint32_t)cnt, (uint32_t)mu.tok[0], (uint32_t)mu.tok[1], (uint32_t)mu.tok[2]);
+                                sts128(dst + kHdrOffset + 32, (uint32_t)mu.tok[3], (uint32_t)rp, (uint32_t)me.r, __float_as_uint(me.scale));
+                                sts128(dst + kHdrOffset + 48, m_seq, (uint32_t)my_group, (uint32_t)k0, 0u);
+                                if (MODE == kFused && sliced && !mine.phase) {
+                                    // rows [k0, k0 + kSliceRows) of up to four consecutive sub-tiles of A^T, side by side
+                                    constexpr uint32_t kPiece = kSliceRows * kSubCols * 2;
+                                    const int n_sub_tile = subs_per_tile(rp);   // sub-tiles per slab tile
+                                    const int n_sub = (d + kSubCols - 1) / kSubCols;
+                                    const int n_here = min(C / kSubCols, n_sub - i * (C / kSubCols));
+                                    mbar_arrive_expect_tx(bar, (uint32_t)n_here * kPiece + (uint32_t)cnt * tbytes);
+                                    for (int j = 0; j < n_here; ++j) {
+                                        const int g = i * (C / kSubCols) + j;
+                                        bulk_g2s(dst + j * kPiece,
+                                                 src + (size_t)(g / n_sub_tile) * tb + (size_t)(g % n_sub_tile) * (rp * kSubCols * 2) + (size_t)k0 * (kSubCols * 2),
+                                                 kPiece, bar);
+                                    }
+                                } else {
+                                    mbar_arrive_expect_tx(bar, tb + (uint32_t)cnt * tbytes);
+                                    bulk_g2s(dst, src + (size_t)i * tb, tb, bar);
+                                }
                             }
-                        } else {
-                            mbar_arrive_expect_tx(bar, tb + (uint32_t)cnt * tbytes);
-                            bulk_g2s(dst, src + (size_t)i * tb, tb, bar);
-                        }
-                        if (!mine.phase) {
+                            if (tail) {
+                                if (!mine.phase) {
 #pragma unroll
-                            for (int t = 0; t < kTokChunk; ++t)
-                                if (t < cnt)
-                                    bulk_g2s(dst + kTileBytesMax + t * kXBytesPerTok,
-                                             my_x + (size_t)mu.tok[t] * p.pool.d_in + (size_t)i * C, tbytes, bar);
-                        } else if (MODE == kExpandOnly) {
+                                    for (int t = 0; t < kTokChunk; ++t)
+                                        if (t < cnt)
+                                            bulk_g2s(dst + kTileBytesMax + t * kXBytesPerTok,
+                                                     my_x + (size_t)mu.tok[t] * p.pool.d_in + (size_t)i * C, tbytes, bar);
+                                } else if (MODE == kExpandOnly) {
 #pragma unroll
-                            for (int t = 0; t < kTokChunk; ++t)   // the caller's m row, rp values, lands as m[t][0..rp)
-                                if (t < cnt)
-                                    bulk_g2s(dst + kTileBytesMax + t * mbytes,
-                                             reinterpret_cast<const uint8_t*>(p.m) + (size_t)mu.tok[t] * p.ldm * (p.m16 ? 2 : 4), mbytes, bar);
+                                    for (int t = 0; t < kTokChunk; ++t)   // the caller's m row, rp values, lands as m[t][0..rp)
+                                        if (t < cnt)
+                                            bulk_g2s(dst + kTileBytesMax + t * mbytes,
+                                                     reinterpret_cast<const uint8_t*>(p.m) + (size_t)mu.tok[t] * p.ldm * (p.m16 ? 2 : 4), mbytes, bar);
+                                }
+                            }
                         }
                     }
+                    __syncwarp();
                 }
-                __syncwarp();
+                if (pass != 1) m_count = mc;
             }
         }
         if (!waited) grid_dependency_wait();
