@@ -117,6 +117,9 @@ PLORA_API size_t plora_pool_slab_bytes(const plora_pool_desc *desc);
  * with zeros) and record its offset table under (layer, proj), replacing any
  * earlier registration of that pair.  The source matrices are not needed after
  * the call returns: it synchronises `stream` (registration is a set-up step).
+ * From then on the slab is read-only for the library and must not be written by
+ * the caller while the pool is registered: the delta kernels fetch adapter tiles
+ * before they have joined the stream's order behind the preceding kernel.
  * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE (slab_bytes too small or more
  * adapters than the context allows), CUDA.
  */
@@ -141,6 +144,15 @@ PLORA_API int32_t plora_pool_max_rank(plora_ctx *ctx, int32_t layer, int32_t pro
  * with cap = min(n_tok, n_adapters).  The result is unique (stable order) and
  * deterministic.  Errors: INVALID_ARG (null, n_tok < 0 or > max_tokens,
  * n_adapters < 1 or > max_adapters).
+ *
+ * The bucket, and for pools of mixed ranks the ordering of its work units by rank
+ * that the first delta call on such a pool adds to it, are device state of the
+ * context, produced in stream order.  The library tracks on the host which ids
+ * and which pool ranks that state belongs to and rebuilds it when a call needs
+ * another; a captured CUDA graph replays only the launches that were needed at
+ * capture time, so a graph should contain its own plora_bucket call (then it is
+ * self-contained), or nothing that changes the bucket or uses a pool with other
+ * ranks may run on the context between its replays.
  */
 PLORA_API plora_status plora_bucket(plora_ctx *ctx, const int32_t *adapter_ids_dev, int32_t n_tok, int32_t n_adapters,
                           void *stream);
