@@ -387,6 +387,18 @@ def test_high_rank_units_few_and_many(rank, n_distinct):
     _check_paths(p, paths=(P.PATH_FUSED, P.PATH_AUTO))
 
 
+def test_widest_projection_highest_and_lowest_rank_largest_batch_per_adapter():
+    # the corners of the paper's parameter ranges (Section V-A: D up to 16384, R from 2 to 128, up to 256
+    # requests on one adapter) in one batch
+    ranks = [128, 2, 64, 3, 128, 17]
+    rng = np.random.default_rng(404)
+    ids = np.concatenate([np.full(256, 0), np.full(40, 1), rng.integers(2, 6, size=60), np.full(3, -1)]).astype(np.int32)
+    rng.shuffle(ids)
+    p = random_problem(405, T=len(ids), d_in=16384, d_out=16384, ranks=ranks)
+    p["ids"] = ids
+    _check_paths(p, paths=(P.PATH_FUSED, P.PATH_UNFUSED, P.PATH_SGMV, P.PATH_AUTO))
+
+
 def test_host_buffer_entry_point():
     p = random_problem(6, T=33, d_in=512, d_out=384, ranks=[16, 8, 32])
     r = Runner(p, max_tokens=64)
