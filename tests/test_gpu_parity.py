@@ -501,6 +501,44 @@ def test_pools_with_different_ranks_share_a_bucket():
     ctx.close()
 
 
+def test_grouped_projections_of_a_mixed_rank_pool():
+    # q, k, v with ranks from every class in one all-classes launch (small batch): bit-identical to three
+    # separate calls, repeatable, and equal to the oracle
+    rng = np.random.default_rng(611)
+    N, T, d = 30, 90, 264
+    ranks = rng.choice([4, 8, 16, 32, 64, 128], size=N)
+    probs = [random_problem(612 + j, T=T, d_in=d, d_out=d, ranks=ranks) for j in range(3)]
+    for pr in probs[1:]:
+        pr["ids"], pr["x"], pr["xf"] = probs[0]["ids"], probs[0]["x"], probs[0]["xf"]
+    ctx = P.Context(T, N)
+    for j, pr in enumerate(probs):
+        ctx.register_pool(0, j, d, d, pr["ranks"], pr["scales"], pr["A"], pr["B"])
+    ctx.set_path(P.PATH_AUTO)
+    ids = torch.from_numpy(probs[0]["ids"]).to(DEV)
+    x = bits_to_dev(probs[0]["x"])
+    ctx.bucket(ids, N)
+    sep = []
+    for j in range(3):
+        y = torch.from_numpy(probs[j]["y_in"]).to(DEV)
+        ctx.lora_delta(x, ids, 0, j, y)
+        sep.append(y)
+    torch.cuda.synchronize()
+    for rep in range(20):
+        ys = [torch.from_numpy(probs[j]["y_in"]).to(DEV) for j in range(3)]
+        n0 = ctx.launch_count()
+        ctx.lora_delta_group([x, x, x], ids, [0, 0, 0], [0, 1, 2], ys)
+        torch.cuda.synchronize()
+        assert ctx.launch_count() - n0 == 1      # the sort by rank class is kept from the first call
+        for j in range(3):
+            assert ys[j].cpu().numpy().tobytes() == sep[j].cpu().numpy().tobytes(), (rep, j)
+    for j in range(3):
+        ref = _oracle(probs[j], y_in=probs[j]["y_in"])
+        delta = np.max(np.abs(ref - probs[j]["y_in"]))
+        assert np.max(np.abs(sep[j].cpu().numpy() - ref)) <= TOL_FP32_PATH * delta + 1e-6 * np.max(np.abs(ref))
+    assert ctx.device_status() == 0
+    ctx.close()
+
+
 def test_grouped_projections_share_a_launch():
     # q, k, v of one layer read the same x; o has its own.  Grouped q/k/v = one launch, bit-identical
     # to three separate calls (every y element still receives exactly one addition).
