@@ -13,10 +13,11 @@
 //                   (tensor-map box copies into 128-byte-swizzled shared memory; the query rows of the
 //                   item ride along with a bulk copy) through a ring of stages; eight consumer warps
 //                   take 8 tokens of every tile each: scores with 4 lanes per token, an online softmax
-//                   per warp (anchor m, sum l, output o, in the base-2 domain with the scale folded
-//                   into q), the weighted sum of V with a lane per 4 dimensions; at the end of an item
-//                   the warps' triples meet in shared memory and the item's (m, l, o) goes to the
-//                   workspace;
+//                   per warp (anchor m, sum l, output o, in the base-2 domain), the weighted sum of V
+//                   with a lane per 4 dimensions; with several query heads per KV head both products
+//                   run on the tensor cores instead (mma.sync, the query heads as rows of the 16-row
+//                   operand); at the end of an item the warps' triples meet in shared memory and the
+//                   item's (m, l, o) goes to the workspace;
 //   merge kernel    one warp per (request, query head) rescales the chunks' partial outputs by their
 //                   anchors: O = sum 2^(m_c - m) o_c / sum 2^(m_c - m) l_c.
 //
@@ -136,6 +137,32 @@ __device__ __forceinline__ void sts128(uint32_t a, uint32_t x, uint32_t y, uint3
 __device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
+// ---- tensor-core pieces of the grouped-query path -----------------------------------------------------
+__device__ __forceinline__ void ldmatrix_x4(uint32_t a, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t a, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
+// D[16 x 8] += A[16 x 16] B[16 x 8], bf16 in, fp32 out; rows 8..15 of A are zero (registers a1, a3)
+__device__ __forceinline__ void mma_16816(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+    const uint32_t z = 0u;
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3]) : "r"(a0), "r"(z), "r"(a2), "r"(z), "r"(b0), "r"(b1));
+}
+// D[16 x 8] += A[16 x 8] B[8 x 8]; rows 8..15 of A are zero, so d2 and d3 stay what they were
+__device__ __forceinline__ void mma_1688(float& d0, float& d1, float& d2, float& d3, uint32_t a0, uint32_t b0) {
+    const uint32_t z = 0u;
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
+                 : "+f"(d0), "+f"(d1), "+f"(d2), "+f"(d3) : "r"(a0), "r"(z), "r"(b0));
+}
+__device__ __forceinline__ uint32_t bf16_rn_bits(float v) {
+    const uint32_t u = __float_as_uint(v);
+    return (u + 0x7fffu + ((u >> 16) & 1u)) >> 16;   // finite, non-negative inputs only
+}
+
 // ---- prep: the list of (request, chunk) units -------------------------------------------------------
 __global__ void __launch_bounds__(1024) prep_kernel(const Params p) {
     __shared__ int warp_sum[32];
@@ -249,6 +276,12 @@ partial_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     const uint32_t v_sub = (uint32_t)(lane >> 4) * (kKBytes / 2);
     const int v_chunk = (lane >> 1) & 7, v_byte = (lane & 1) * 8;
     float m_run[G], l_run[G], o_run[G][4];
+    // grouped queries (G > 1), tensor-core path: lane (g, c) = (lane / 4, lane % 4) holds, for query head g, the
+    // anchor and the sum of its warp's tokens, the output dims 8 n + 2 c, 8 n + 2 c + 1 (n = 0..15), and the
+    // query fragments of the eight 16-dim steps
+    const int mg = lane >> 2, mc = lane & 3;
+    float mm = -INFINITY, ml = 0.f, mo[16][2];
+    uint32_t qf[8][2];
     uint32_t meetings = 0;
     bool alive = true;
     auto consumer_meet = [&]() {
@@ -273,71 +306,189 @@ partial_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
                 o_run[g][0] = o_run[g][1] = o_run[g][2] = o_run[g][3] = 0.f;
             }
         }
-        // K piece of this lane: 32 dims = 4 chunks of 16 bytes, chunk c of row r stored at c ^ (r & 7)
-        uint4 kraw[4];
+        if constexpr (G == 1) {
+            // K piece of this lane: 32 dims = 4 chunks of 16 bytes, chunk c of row r stored at c ^ (r & 7)
+            uint4 kraw[4];
+    #pragma unroll
+            for (int i = 0; i < 4; ++i) kraw[i] = lds128(st + k_off + ((((qr & 1) * 4 + i) ^ (trow & 7)) << 4));
+            // V pieces of the warp's 8 tokens for this lane's 4 dims
+            uint2 vraw[8];
+    #pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int r = warp * 8 + j;
+                vraw[j] = lds64(st + kKBytes + v_sub + r * 128 + ((v_chunk ^ (r & 7)) << 4) + v_byte);
+                if (r >= h.n_tok) vraw[j] = make_uint2(0u, 0u);   // beyond the cache's end: whatever lies there must not reach the sum
+            }
+            const bool valid = trow < h.n_tok;
+    #pragma unroll
+            for (int g = 0; g < G; ++g) {
+                // q piece: dims [32 qr, +32) of query head g, bf16 in the stage
+                // packed multiply-adds (two fp32 FMAs per instruction on sm_100): the even and the odd dims
+                // of a 32-bit word advance together, two chains of 16 instead of one of 32
+                float2 s2 = make_float2(0.f, 0.f);
+    #pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint4 qw = lds128(st + kQOffset + g * (kHeadDim * 2) + qr * 64 + i * 16);
+                    s2 = __ffma2_rn(make_float2(bf_lo(qw.x), bf_hi(qw.x)), make_float2(bf_lo(kraw[i].x), bf_hi(kraw[i].x)), s2);
+                    s2 = __ffma2_rn(make_float2(bf_lo(qw.y), bf_hi(qw.y)), make_float2(bf_lo(kraw[i].y), bf_hi(kraw[i].y)), s2);
+                    s2 = __ffma2_rn(make_float2(bf_lo(qw.z), bf_hi(qw.z)), make_float2(bf_lo(kraw[i].z), bf_hi(kraw[i].z)), s2);
+                    s2 = __ffma2_rn(make_float2(bf_lo(qw.w), bf_hi(qw.w)), make_float2(bf_lo(kraw[i].w), bf_hi(kraw[i].w)), s2);
+                }
+                float s = s2.x + s2.y;
+                s += __shfl_xor_sync(0xffffffffu, s, 8);
+                s += __shfl_xor_sync(0xffffffffu, s, 16);
+                s = valid ? s * p.scale_log2e : -INFINITY;      // every lane of a token now holds its score
+                float mx = s;
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+                const float m_new = fmaxf(m_run[g], mx);
+                // a warp whose tokens are all beyond the tile's end keeps its state (m_new may still be -inf)
+                const float alpha = m_new == -INFINITY ? 1.f : exp2f(m_run[g] - m_new);
+                const float pt = valid ? exp2f(s - m_new) : 0.f;
+                float psum = pt;
+                psum += __shfl_xor_sync(0xffffffffu, psum, 1);
+                psum += __shfl_xor_sync(0xffffffffu, psum, 2);
+                psum += __shfl_xor_sync(0xffffffffu, psum, 4);
+                l_run[g] = l_run[g] * alpha + psum;
+                float2 o01 = make_float2(o_run[g][0] * alpha, o_run[g][1] * alpha), o23 = make_float2(o_run[g][2] * alpha, o_run[g][3] * alpha);
+    #pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float pj = __shfl_sync(0xffffffffu, pt, j);     // lane j (quarter 0) holds token j's weight
+                    const float2 pp = make_float2(pj, pj);
+                    o01 = __ffma2_rn(pp, make_float2(bf_lo(vraw[j].x), bf_hi(vraw[j].x)), o01);
+                    o23 = __ffma2_rn(pp, make_float2(bf_lo(vraw[j].y), bf_hi(vraw[j].y)), o23);
+                }
+                o_run[g][0] = o01.x; o_run[g][1] = o01.y; o_run[g][2] = o23.x; o_run[g][3] = o23.y;
+                m_run[g] = m_new;
+            }
+        } else {
+            // ---- grouped queries: S = Q K^T and O += P V on the tensor cores (mma.sync), this warp's 8 tokens ----
+            // The G query heads are the first rows of the 16-row operand (the others are zero registers).
+            // Scores: 16-dim steps over K, B fragments by ldmatrix from the swizzled rows of the warp's
+            // tokens.  Values: the probabilities, as bf16 hi + lo halves (two MMAs, fp32-grade accuracy),
+            // against 8-dim blocks of V by ldmatrix.trans.  The instruction count no longer grows with G.
+            if (h.flags & kFlagFirst) {
+                mm = -INFINITY;
+                ml = 0.f;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) kraw[i] = lds128(st + k_off + ((((qr & 1) * 4 + i) ^ (trow & 7)) << 4));
-        // V pieces of the warp's 8 tokens for this lane's 4 dims
-        uint2 vraw[8];
+                for (int n = 0; n < 16; ++n) mo[n][0] = mo[n][1] = 0.f;
+                const uint32_t qa = st + kQOffset + mg * (kHeadDim * 2) + mc * 4;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int r = warp * 8 + j;
-            vraw[j] = lds64(st + kKBytes + v_sub + r * 128 + ((v_chunk ^ (r & 7)) << 4) + v_byte);
-            if (r >= h.n_tok) vraw[j] = make_uint2(0u, 0u);   // beyond the cache's end: whatever lies there must not reach the sum
-        }
-        const bool valid = trow < h.n_tok;
-#pragma unroll
-        for (int g = 0; g < G; ++g) {
-            // q piece: dims [32 qr, +32) of query head g, bf16 in the stage
-            // packed multiply-adds (two fp32 FMAs per instruction on sm_100): the even and the odd dims
-            // of a 32-bit word advance together, two chains of 16 instead of one of 32
-            float2 s2 = make_float2(0.f, 0.f);
+                for (int ks = 0; ks < 8; ++ks) {
+                    qf[ks][0] = mg < G ? lds32(qa + ks * 32) : 0u;
+                    qf[ks][1] = mg < G ? lds32(qa + ks * 32 + 16) : 0u;
+                }
+            }
+            const int row0 = warp * 8;
+            if (row0 + 8 > h.n_tok) {
+                // beyond the cache's end: whatever lies there must not reach the sum (0 * NaN); this warp alone reads these rows
+                for (int i = lane; i < 8 * 16; i += 32) {
+                    const int r = row0 + (i >> 4), c = i & 15;
+                    if (r >= h.n_tok) sts128(st + kKBytes + (c >> 3) * (kKBytes / 2) + r * 128 + ((c & 7) << 4), 0u, 0u, 0u, 0u);
+                }
+                __syncwarp();
+            }
+            // the lane's row of the 8 x 8 blocks it addresses: token row0 + (lane & 7), 16-byte chunk 4 i + (lane >> 3)
+            const int lrow = row0 + (lane & 7), lch = lane >> 3;
+            float sc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const uint4 qw = lds128(st + kQOffset + g * (kHeadDim * 2) + qr * 64 + i * 16);
-                s2 = __ffma2_rn(make_float2(bf_lo(qw.x), bf_hi(qw.x)), make_float2(bf_lo(kraw[i].x), bf_hi(kraw[i].x)), s2);
-                s2 = __ffma2_rn(make_float2(bf_lo(qw.y), bf_hi(qw.y)), make_float2(bf_lo(kraw[i].y), bf_hi(kraw[i].y)), s2);
-                s2 = __ffma2_rn(make_float2(bf_lo(qw.z), bf_hi(qw.z)), make_float2(bf_lo(kraw[i].z), bf_hi(kraw[i].z)), s2);
-                s2 = __ffma2_rn(make_float2(bf_lo(qw.w), bf_hi(qw.w)), make_float2(bf_lo(kraw[i].w), bf_hi(kraw[i].w)), s2);
+                const int ch = 4 * i + lch;
+                uint32_t b[4];
+                ldmatrix_x4(st + (ch >> 3) * (kKBytes / 2) + lrow * 128 + (((ch & 7) ^ (lrow & 7)) << 4), b);
+                mma_16816(sc, qf[2 * i][0], qf[2 * i][1], b[0], b[1]);
+                mma_16816(sc, qf[2 * i + 1][0], qf[2 * i + 1][1], b[2], b[3]);
             }
-            float s = s2.x + s2.y;
-            s += __shfl_xor_sync(0xffffffffu, s, 8);
-            s += __shfl_xor_sync(0xffffffffu, s, 16);
-            s = valid ? s * p.scale_log2e : -INFINITY;      // every lane of a token now holds its score
-            float mx = s;
+            const int t0 = row0 + 2 * mc;
+            const float s0 = t0 < h.n_tok ? sc[0] * p.scale_log2e : -INFINITY;
+            const float s1 = t0 + 1 < h.n_tok ? sc[1] * p.scale_log2e : -INFINITY;
+            float mx = fmaxf(s0, s1);
             mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
             mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
-            const float m_new = fmaxf(m_run[g], mx);
-            // a warp whose tokens are all beyond the tile's end keeps its state (m_new may still be -inf)
-            const float alpha = m_new == -INFINITY ? 1.f : exp2f(m_run[g] - m_new);
-            const float pt = valid ? exp2f(s - m_new) : 0.f;
-            float psum = pt;
+            const float m_new = fmaxf(mm, mx);
+            const float alpha = m_new == -INFINITY ? 1.f : exp2f(mm - m_new);
+            const float p0 = t0 < h.n_tok ? exp2f(s0 - m_new) : 0.f;
+            const float p1 = t0 + 1 < h.n_tok ? exp2f(s1 - m_new) : 0.f;
+            float psum = p0 + p1;
             psum += __shfl_xor_sync(0xffffffffu, psum, 1);
             psum += __shfl_xor_sync(0xffffffffu, psum, 2);
-            psum += __shfl_xor_sync(0xffffffffu, psum, 4);
-            l_run[g] = l_run[g] * alpha + psum;
-            float2 o01 = make_float2(o_run[g][0] * alpha, o_run[g][1] * alpha), o23 = make_float2(o_run[g][2] * alpha, o_run[g][3] * alpha);
+            ml = ml * alpha + psum;
+            mm = m_new;
+            const uint32_t h0 = bf16_rn_bits(p0), h1 = bf16_rn_bits(p1);
+            const uint32_t p_hi = h0 | (h1 << 16);
+            const uint32_t p_lo = bf16_rn_bits(p0 - __uint_as_float(h0 << 16)) | (bf16_rn_bits(p1 - __uint_as_float(h1 << 16)) << 16);
+            float z2 = 0.f, z3 = 0.f;   // rows 8..15 of the output block: zero in, zero out
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const float pj = __shfl_sync(0xffffffffu, pt, j);     // lane j (quarter 0) holds token j's weight
-                const float2 pp = make_float2(pj, pj);
-                o01 = __ffma2_rn(pp, make_float2(bf_lo(vraw[j].x), bf_hi(vraw[j].x)), o01);
-                o23 = __ffma2_rn(pp, make_float2(bf_lo(vraw[j].y), bf_hi(vraw[j].y)), o23);
+            for (int i = 0; i < 4; ++i) {
+                const int ch = 4 * i + lch;
+                uint32_t b[4];
+                ldmatrix_x4_trans(st + kKBytes + (ch >> 3) * (kKBytes / 2) + lrow * 128 + (((ch & 7) ^ (lrow & 7)) << 4), b);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int n = 4 * i + j;
+                    mo[n][0] *= alpha;
+                    mo[n][1] *= alpha;
+                    mma_1688(mo[n][0], mo[n][1], z2, z3, p_hi, b[j]);
+                    mma_1688(mo[n][0], mo[n][1], z2, z3, p_lo, b[j]);
+                }
             }
-            o_run[g][0] = o01.x; o_run[g][1] = o01.y; o_run[g][2] = o23.x; o_run[g][3] = o23.y;
-            m_run[g] = m_new;
         }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(empty + slot * 8);
-        if (h.flags & kFlagLast) {
-            // anchor merge of the eight warps' shares of this item, one query head at a time
-            for (int g = 0; g < G; ++g) {
+        if constexpr (G > 1) {
+            if (h.flags & kFlagLast) {
+                // Anchor merge of the eight warps' shares, all query heads at once.  The item's last tile is
+                // consumed, so its stage (34 KB of K, V and q) serves as the meeting place: every warp
+                // puts its G triples there, then warp g combines query head g.  Two meetings per item.
+                consumer_meet();   // nobody reads the tile any more
+                float* scr = reinterpret_cast<float*>(base + slot * kSlotBytes);
+                static_assert(kConsumerWarps * kMaxQPerKv * kMergeStride * 4 <= kHdrOffset, "the meeting place fits in a stage");
+                if (mg < G) {
+                    float* mine = scr + (warp * G + mg) * kMergeStride;
+#pragma unroll
+                    for (int n = 0; n < 16; ++n) *reinterpret_cast<float2*>(mine + 8 * n + 2 * mc) = make_float2(mo[n][0], mo[n][1]);
+                    if (mc == 0) {
+                        mine[kHeadDim] = mm;
+                        mine[kHeadDim + 1] = ml;
+                    }
+                }
+                consumer_meet();
+                if (warp < G && alive) {
+                    const int g = warp;
+                    float M = -INFINITY;
+#pragma unroll
+                    for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, scr[(w * G + g) * kMergeStride + kHeadDim]);
+                    float L = 0.f;
+                    float4 O = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                    for (int w = 0; w < kConsumerWarps; ++w) {
+                        const float* src = scr + (w * G + g) * kMergeStride;
+                        const float mw = src[kHeadDim];
+                        const float f = mw == -INFINITY ? 0.f : exp2f(mw - M);
+                        L = fmaf(f, src[kHeadDim + 1], L);
+                        const float4 ow = *reinterpret_cast<const float4*>(src + 4 * lane);
+                        O.x = fmaf(f, ow.x, O.x); O.y = fmaf(f, ow.y, O.y); O.z = fmaf(f, ow.z, O.z); O.w = fmaf(f, ow.w, O.w);
+                    }
+                    float* dst = p.w.partials + ((size_t)h.unit * (p.n_kv_heads * G) + h.head * G + g) * kPartFloats;
+                    *reinterpret_cast<float4*>(dst + 4 * lane) = O;
+                    if (lane == 0) {
+                        dst[kHeadDim] = M;
+                        dst[kHeadDim + 1] = L;
+                    }
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the stage goes back to the copy engine
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty + slot * 8);
+        } else {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty + slot * 8);
+            if (h.flags & kFlagLast) {
+                // anchor merge of the eight warps' shares of this item
                 float* mine = merge + warp * kMergeStride;
-                *reinterpret_cast<float4*>(mine + 4 * lane) = make_float4(o_run[g][0], o_run[g][1], o_run[g][2], o_run[g][3]);
+                *reinterpret_cast<float4*>(mine + 4 * lane) = make_float4(o_run[0][0], o_run[0][1], o_run[0][2], o_run[0][3]);
                 if (lane == 0) {
-                    mine[kHeadDim] = m_run[g];
-                    mine[kHeadDim + 1] = l_run[g];
+                    mine[kHeadDim] = m_run[0];
+                    mine[kHeadDim + 1] = l_run[0];
                 }
                 consumer_meet();
                 if (warp == 0) {
@@ -354,7 +505,7 @@ partial_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
                         const float4 ow = *reinterpret_cast<const float4*>(merge + w * kMergeStride + 4 * lane);
                         O.x = fmaf(f, ow.x, O.x); O.y = fmaf(f, ow.y, O.y); O.z = fmaf(f, ow.z, O.z); O.w = fmaf(f, ow.w, O.w);
                     }
-                    float* dst = p.w.partials + ((size_t)h.unit * (p.n_kv_heads * G) + h.head * G + g) * kPartFloats;
+                    float* dst = p.w.partials + ((size_t)h.unit * p.n_kv_heads + h.head) * kPartFloats;
                     *reinterpret_cast<float4*>(dst + 4 * lane) = O;
                     if (lane == 0) {
                         dst[kHeadDim] = M;
