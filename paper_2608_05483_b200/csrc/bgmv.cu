@@ -53,7 +53,9 @@ constexpr int kGatherWarp = kConsumerWarps + 1;     // fused mode: assembles the
 constexpr int kThreads = kConsumerThreads + 64;
 constexpr int kCtasPerSm = 2;   // persistent CTAs per SM
 constexpr int kStages = 5;
-constexpr int kXBytesPerTok = kMaxSubPerTile * kSubCols * 2;             // x piece of one token for one tile
+// x piece of one token for one tile, plus 32 bytes: the pieces of a unit's (up to four) tokens then start in
+// different banks, and the tensor-core shrink reads one word of each at a time
+constexpr int kXBytesPerTok = kMaxSubPerTile * kSubCols * 2 + 32;
 constexpr int kHdrOffset = kTileBytesMax + kTokChunk * kXBytesPerTok;
 constexpr int kSlotBytes = kHdrOffset + 128;                             // tile + x pieces + stage header
 // m of the expand tasks in flight (fused mode): a ring filled by the gather warp and drained by
@@ -435,6 +437,78 @@ __device__ __forceinline__ void shrink_finish(const Params& p, const Smem& sm, c
     }
 }
 
+// ---- shrink on the tensor cores: units of several tokens (padded rank >= 16) ----------------------------
+// A unit of 2..4 tokens costs the CUDA-core loop 2..2.6 times the instructions of a one-token unit.  Here
+// m^T[16 rank rows x 8] += A^T[16 x 16 columns] x^T[16 x 8] by mma.sync.m16n8k16: warp w takes the rank
+// rows [16 w, 16 w + 16) of every sub-tile of the stage (warps beyond RP / 16 have nothing to do and only
+// release the stage), A fragments by ldmatrix from the swizzled sub-tile (conflict-free), x fragments as
+// one word per lane from the unit's x pieces (tokens beyond the unit's count read some other token's
+// piece: their columns of the result are never stored).  The accumulator fragment holds complete sums of
+// the warp's rows for the task's columns, so the end of a task is one store per value: no shuffles.
+__device__ __forceinline__ void ldmatrix_x4(uint32_t a, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
+template <bool H>
+__device__ __forceinline__ void mma_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    if (H)
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                     : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3]) : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+    else
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                     : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3]) : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+template <int RP, bool H>
+__device__ __forceinline__ void shrink_tile_mma(const Params& p, const StageHdr& h, uint32_t tile, float (&d)[4], int warp, int lane) {
+    constexpr int NSUB = (kMaxRank / RP > kMaxSubPerTile) ? kMaxSubPerTile : kMaxRank / RP;
+    if (warp >= RP / 16) return;
+    const int g = lane >> 2, q = lane & 3;
+    const int cols_left = p.pool.d_in - h.tile * (NSUB * kSubCols);   // only the last tile can be ragged
+    const int arow = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;  // the lane's row of the 8 x 8 blocks it addresses
+    const uint32_t xrow = tile + kTileBytesMax + (g & (kTokChunk - 1)) * kXBytesPerTok;
+#pragma unroll
+    for (int sb = 0; sb < NSUB; ++sb) {
+        if (sb * kSubCols >= cols_left) break;   // nothing was copied for these columns
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks) {
+            uint32_t a[4];
+            const int ch = 2 * ks + (lane >> 4);
+            ldmatrix_x4(tile + sb * (RP * 128) + arow * 128 + ((ch ^ (arow & 7)) << 4), a);
+            const int col = sb * kSubCols + ks * 16 + 2 * q;
+            // columns beyond d_in: the slab holds zeros there, the x piece holds whatever was in the stage
+            const uint32_t b0 = col < cols_left ? lds32(xrow + col * 2) : 0u;
+            const uint32_t b1 = col + 8 < cols_left ? lds32(xrow + col * 2 + 16) : 0u;
+            mma_16816<H>(d, a, b0, b1);
+        }
+    }
+}
+template <int MODE, int RP>
+__device__ __forceinline__ void shrink_finish_mma(const Params& p, const Smem& sm, const StageHdr& h, const float (&d)[4],
+                                                  int warp, int lane) {
+    if (warp < RP / 16) {
+        const int g = lane >> 2, q = lane & 3;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int t = 2 * q + (j & 1), k = h.k0 + warp * 16 + g + (j >> 1) * 8;
+            if (t < h.cnt) {
+                if (MODE == kFused)
+                    p.bk.m_part[part_index(p, h.unit, h.run, t) + k] =
+                        ((unsigned long long)sm.epoch << 32) | (unsigned long long)__float_as_uint(d[j]);
+                else
+                    store_m(p, (size_t)tok_at(h, t) * p.ldm + k, d[j]);
+            }
+        }
+    }
+    if (MODE != kFused) {
+        // columns beyond this adapter's padded rank are zeros
+        const int extra = p.ldm - RP;
+        for (int idx = warp * 32 + lane; idx < h.cnt * extra; idx += kConsumerThreads) {
+            const int t = idx / extra, k = RP + idx % extra;
+            store_m(p, (size_t)tok_at(h, t) * p.ldm + k, 0.f);
+        }
+    }
+}
+
 // ---- expand: one tile of B; the result goes straight to y ------------------------------------------
 // Lane mapping: a lane owns two adjacent output columns; when the warp's slice has fewer
 // than 32 column pairs, RG lane groups split the rank rows and meet by shuffles.
@@ -629,7 +703,7 @@ struct LaneMaps {
 };
 
 // One stage, consumer side.
-template <int MODE, int RP, bool H>
+template <int MODE, int RP, bool H, bool TC>
 __device__ __forceinline__ void consume_stage(const Params& p, const Smem& sm, const StageHdr& h,
                                               const LaneMaps<RP, SliceCfg<MODE, RP>::kSliceRp>& maps, uint32_t tile, uint32_t empty_bar,
                                               float (&acc)[kMaxRowsPerLane][kTokChunk], int warp, int lane) {
@@ -642,11 +716,25 @@ __device__ __forceinline__ void consume_stage(const Params& p, const Smem& sm, c
                     for (int t = 0; t < kTokChunk; ++t) acc[rr][t] = 0.f;
             }
             constexpr int RPS = SliceCfg<MODE, RP>::kSliceRp;
+            // several tokens: the tensor-core loop (its accumulator fragment lives in acc[0]) where it has at least
+            // four warps to run on (padded rank 64 and 128); with two warps (rank 32, row slices) or one (rank 16)
+            // it loses against the CUDA-core loop on all eight (measured)
+            const bool tc4 = TC && h.cnt >= 2;   // (not in the launch for all classes, which cuts these ranks into slices)
             if (RPS != RP && (h.flags & kFlagSlice)) {
-                shrink_tile<RPS, H>(p, h, maps.s2, tile, acc);
+                const bool tc = RPS >= 64 && tc4;
+                if (tc) shrink_tile_mma<RPS < 16 ? 16 : RPS, H>(p, h, tile, acc[0], warp, lane);
+                else shrink_tile<RPS, H>(p, h, maps.s2, tile, acc);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(empty_bar);
-                if (h.flags & kFlagLast) shrink_finish<MODE, RPS>(p, sm, h, maps.s2, acc, warp, lane);
+                if (h.flags & kFlagLast) {
+                    if (tc) shrink_finish_mma<MODE, RPS < 16 ? 16 : RPS>(p, sm, h, acc[0], warp, lane);
+                    else shrink_finish<MODE, RPS>(p, sm, h, maps.s2, acc, warp, lane);
+                }
+            } else if (RP >= 64 && tc4) {
+                shrink_tile_mma<RP < 16 ? 16 : RP, H>(p, h, tile, acc[0], warp, lane);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty_bar);
+                if (h.flags & kFlagLast) shrink_finish_mma<MODE, RP < 16 ? 16 : RP>(p, sm, h, acc[0], warp, lane);
             } else {
                 shrink_tile<RP, H>(p, h, maps.s, tile, acc);
                 __syncwarp();
@@ -676,7 +764,7 @@ __device__ __forceinline__ bool consume_class(const Params& p, const Smem& sm, u
         const StageHdr h = read_hdr(tile + kHdrOffset);
         if ((h.flags & kFlagEnd) || lds32(smem_u32(const_cast<int*>(sm.abort_flag)))) return false;
         if (!ONLY && h.rp != RP) return true;
-        consume_stage<MODE, RP, H>(p, sm, h, maps, tile, sm.empty + slot * 8, acc, warp, lane);
+        consume_stage<MODE, RP, H, ONLY>(p, sm, h, maps, tile, sm.empty + slot * 8, acc, warp, lane);
     }
 }
 
