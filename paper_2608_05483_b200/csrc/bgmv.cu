@@ -32,7 +32,8 @@
 //     one addition per element, so the result is bit-reproducible).  Consumer warps therefore
 //     never wait on global memory.  Both inner loops use the packed fp32 multiply-add of sm_100
 //     (two FMAs per instruction): the kernel is bound by instruction issue where HBM does not
-//     bound it.
+//     bound it.  The shrink of a unit with several tokens at padded rank 64 or 128 runs on the
+//     tensor cores (mma.sync) in one-rank launches.
 //
 // The same template provides the fused path, the shrink-only path (m written to
 // the caller's buffer, unscaled, one task per unit) and the expand-only path.
