@@ -152,11 +152,10 @@ __device__ __forceinline__ void mma_16816(float (&d)[4], uint32_t a0, uint32_t a
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3]) : "r"(a0), "r"(z), "r"(a2), "r"(z), "r"(b0), "r"(b1));
 }
-// D[16 x 8] += A[16 x 8] B[8 x 8]; rows 8..15 of A are zero, so d2 and d3 stay what they were
-__device__ __forceinline__ void mma_1688(float& d0, float& d1, float& d2, float& d3, uint32_t a0, uint32_t b0) {
-    const uint32_t z = 0u;
+// D[16 x 8] += A[16 x 8] B[8 x 8]; a0 holds rows 0..7 of A, a1 rows 8..15
+__device__ __forceinline__ void mma_1688(float& d0, float& d1, float& d2, float& d3, uint32_t a0, uint32_t a1, uint32_t b0) {
     asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
-                 : "+f"(d0), "+f"(d1), "+f"(d2), "+f"(d3) : "r"(a0), "r"(z), "r"(b0));
+                 : "+f"(d0), "+f"(d1), "+f"(d2), "+f"(d3) : "r"(a0), "r"(a1), "r"(b0));
 }
 __device__ __forceinline__ uint32_t bf16_rn_bits(float v) {
     const uint32_t u = __float_as_uint(v);
@@ -418,7 +417,8 @@ partial_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             const uint32_t h0 = bf16_rn_bits(p0), h1 = bf16_rn_bits(p1);
             const uint32_t p_hi = h0 | (h1 << 16);
             const uint32_t p_lo = bf16_rn_bits(p0 - __uint_as_float(h0 << 16)) | (bf16_rn_bits(p1 - __uint_as_float(h1 << 16)) << 16);
-            float z2 = 0.f, z3 = 0.f;   // rows 8..15 of the output block: zero in, zero out
+            // the hi halves ride in rows 0..7 of the operand and the lo halves in rows 8..15 (there are at most
+            // eight query heads): one MMA per block gives both products, in rows g and g + 8 of the result
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const int ch = 4 * i + lch;
@@ -427,10 +427,10 @@ partial_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const int n = 4 * i + j;
-                    mo[n][0] *= alpha;
-                    mo[n][1] *= alpha;
-                    mma_1688(mo[n][0], mo[n][1], z2, z3, p_hi, b[j]);
-                    mma_1688(mo[n][0], mo[n][1], z2, z3, p_lo, b[j]);
+                    float d0 = mo[n][0] * alpha, d1 = mo[n][1] * alpha, d2 = 0.f, d3 = 0.f;
+                    mma_1688(d0, d1, d2, d3, p_hi, p_lo, b[j]);
+                    mo[n][0] = d0 + d2;
+                    mo[n][1] = d1 + d3;
                 }
             }
         }
