@@ -145,6 +145,15 @@ PLORA_API int32_t plora_pool_max_rank(plora_ctx *ctx, int32_t layer, int32_t pro
  * deterministic.  Errors: INVALID_ARG (null, n_tok < 0 or > max_tokens,
  * n_adapters < 1 or > max_adapters).
  *
+ * Reuse rule.  A bucket made by plora_bucket is the caller's statement that the ids
+ * buffer keeps its contents: every later delta call that passes the same
+ * (adapter_ids_dev, n_tok) and a pool of the same n_adapters uses it as it is, until
+ * the next plora_bucket.  Call plora_bucket again after writing new ids into the
+ * buffer, also when the pointer is unchanged.  A delta call that finds no such bucket
+ * buckets for itself, and that bucket serves this one call only (all projections of a
+ * grouped call share it): the library cannot see whether the buffer was rewritten, or
+ * its address given to another tensor, before the next call.
+ *
  * The bucket, and for pools of mixed ranks the ordering of its work units by rank
  * that the first delta call on such a pool adds to it, are device state of the
  * context, produced in stream order.  The library tracks on the host which ids
@@ -169,9 +178,18 @@ PLORA_API plora_status plora_bucket_view(plora_ctx *ctx, const int32_t **perm, c
  * output on entry), both on the device; d_in/d_out are the registered pool's.
  * Uses the context's current bucket when plora_bucket was last called with this
  * same (adapter_ids_dev, n_tok) and the pool's n_adapters; otherwise buckets
- * first.  Every adapter present in the batch is read from HBM once per call,
- * whatever its number of tokens (Section VI-B).  Each element of y receives
- * exactly one addition, so results are bit-reproducible run to run.
+ * first, for this call only (see the reuse rule at plora_bucket).  Every adapter
+ * present in the batch is read from HBM once per call, whatever its number of tokens
+ * (Section VI-B).  Each element of y receives exactly one addition, so results are
+ * bit-reproducible run to run.
+ * Tensor memory.  Segments that take the tensor-core path (PLORA_PATH_AUTO on batches
+ * of 512+ tokens, PLORA_PATH_SGMV always) run in a kernel whose CTAs each allocate 256
+ * of an SM's 512 tensor-memory columns, two CTAs per SM (one per SM for pools with
+ * ranks above 64).  The allocation instruction has no time limit: it blocks while
+ * another kernel resident on the same SM (a base-model GEMM on a second stream, say)
+ * holds the columns it needs, and goes on when they are freed.  Do not run this call
+ * concurrently with a kernel that keeps more than half of the tensor memory for its
+ * whole lifetime and itself waits for this call.
  * Errors: INVALID_ARG, NOT_REGISTERED, CUDA.
  */
 PLORA_API plora_status plora_lora_delta(plora_ctx *ctx, const void *x_dev, const int32_t *adapter_ids_dev, int32_t n_tok,
@@ -257,8 +275,9 @@ PLORA_API plora_status plora_host_sync(plora_ctx *ctx);
  * Some hosts of this library cannot call cudaMalloc at the point where they need the
  * delta: a serving loop that may not stall (cudaMalloc and cudaFree synchronise the whole
  * device), a process whose device memory was handed out in full at start-up, or code
- * running under an allocator it does not control.  This call computes exactly what
- * plora_lora_delta computes, by the shrink kernel followed by the expand kernel, and keeps
+ * running under an allocator it does not control.  This call computes what
+ * plora_lora_delta computes (the same result within the tolerance of the fp32 paths: the
+ * order of the additions differs), by the shrink kernel followed by the expand kernel, and keeps
  * the intermediate m = x A in a fixed array that is part of the library image instead of
  * in allocated workspace.  It calls no cudaMalloc, no cudaFree and no allocating library
  * routine; it only enqueues kernels on `stream` (bucketing first if the context's current
@@ -271,7 +290,11 @@ PLORA_API plora_status plora_host_sync(plora_ctx *ctx);
  * PLORA_ERR_WORKSPACE before anything is launched.
  *
  * The first call on a device looks up the array's device address (once per device) before
- * it launches; make that first call outside any stream capture.  All calls, on all
+ * it launches; that lookup may make the CUDA runtime load the library's device code onto the
+ * device, which allocates and synchronises inside the driver, so only the calls after the first
+ * are free of allocation.  Make the first call during set-up, outside any stream capture, and not
+ * at the same time as another thread's first call on that device (the address is cached without
+ * a lock; later calls only read it).  All calls, on all
  * contexts of a device, share the one array, and it keeps what the previous call left in
  * it: the shrink kernel rewrites every row the expand kernel will read (rows of tokens
  * without an adapter are written as zeros), so nothing has to be cleared between calls,
@@ -298,6 +321,37 @@ PLORA_API plora_status plora_set_path(plora_ctx *ctx, int32_t path, int32_t sgmv
 #define PLORA_INPUT_BF16 0
 #define PLORA_INPUT_FP16 1
 PLORA_API plora_status plora_set_input_type(plora_ctx *ctx, int32_t type);
+
+/*
+ * Diagnostics of the bounded device-side waits (no counterpart in the paper).  Every wait inside the
+ * kernels (on a shared-memory barrier, or on partial sums from another CTA) gives up after a number of
+ * SM clock cycles, records PLORA_ERR_TIMEOUT in the status word, and the kernel winds down: no role
+ * issues further copies, the copies already issued are waited for, tensor memory is freed, y may hold
+ * partial results for that call.  The context stays usable.
+ * plora_set_wait_limit: cycles > 0 sets the limit for this context's later launches; 0 restores the
+ * default (4e9, about two seconds).
+ * plora_set_test_hook: for tests only.  PLORA_HOOK_WITHHOLD_RELEASE makes one consumer of every CTA
+ * never hand its stages back to the copy warp, so that the copy warp's wait for a free stage runs out
+ * (at that point every copy it issued has landed).  Accepted only while a wait limit of at most
+ * PLORA_HOOK_MAX_CYCLES is set; PLORA_HOOK_NONE switches it off.
+ */
+#define PLORA_HOOK_NONE 0
+#define PLORA_HOOK_WITHHOLD_RELEASE 1
+#define PLORA_HOOK_MAX_CYCLES (1 << 24)
+PLORA_API plora_status plora_set_wait_limit(plora_ctx *ctx, int64_t cycles);
+PLORA_API plora_status plora_set_test_hook(plora_ctx *ctx, int32_t hook);
+
+/*
+ * Read-bandwidth probe (no counterpart in the paper; a measuring aid for the roofline).  Reads
+ * `bytes` bytes (a multiple of 16, 16-byte aligned) of device memory at buf_dev once, with 16-byte
+ * loads from every SM, and folds them into a checksum in sink_dev (device, at least 4 bytes per
+ * launched block: 64 KiB always suffices), so the loads cannot be optimised away.  The caller times
+ * it with events on `stream`; bytes / time is what a kernel that only reads can get from HBM on this
+ * part, which is the fair ceiling for the decode path (its traffic is almost all adapter reads),
+ * whereas a copy's figure counts reads and writes.  Runs on the current device.
+ */
+PLORA_API plora_status plora_stream_read(const void *buf_dev, size_t bytes, void *sink_dev, size_t sink_bytes,
+                                         void *stream);
 
 /* Synchronise `stream`, copy the sticky device status word to *host_out (0 or a
  * PLORA_ERR_* value) and clear it. */
@@ -361,6 +415,11 @@ PLORA_API plora_status plora_attn_decode(const void *q_bf16_dev, const void *k_c
                                          int32_t n_kv_heads, int32_t q_per_kv, int32_t head_dim, float scale,
                                          float *out_dev, void *workspace_dev, size_t workspace_bytes, void *stream);
 PLORA_API plora_status plora_attn_status(void *workspace_dev, void *stream, int32_t *host_out);
+/* The wait limit and test hook of plora_set_wait_limit / plora_set_test_hook for the attention kernels,
+ * which have no context: the settings live in the workspace's header (zero = defaults) and hold for later
+ * calls with this workspace.  cycles 0 restores the default limit; a hook other than PLORA_HOOK_NONE needs
+ * 0 < cycles <= PLORA_HOOK_MAX_CYCLES.  Synchronises `stream`. */
+PLORA_API plora_status plora_attn_set_debug(void *workspace_dev, int64_t cycles, int32_t hook, void *stream);
 
 #ifdef __cplusplus
 }

@@ -32,8 +32,11 @@ EXPORTS = (
     "plora_bucket", "plora_bucket_view", "plora_lora_delta", "plora_lora_delta_group", "plora_shrink", "plora_expand",
     "plora_shrink_m16", "plora_expand_m16", "plora_set_input_type",
     "plora_lora_delta_host", "plora_lora_delta_host_async", "plora_host_sync", "plora_lora_delta_noalloc", "plora_set_path", "plora_device_status", "plora_launch_count", "plora_status_string",
-    "plora_cost_model", "plora_attn_workspace_bytes", "plora_attn_decode", "plora_attn_status",
+    "plora_cost_model", "plora_attn_workspace_bytes", "plora_attn_decode", "plora_attn_status", "plora_attn_set_debug",
+    "plora_set_wait_limit", "plora_set_test_hook", "plora_stream_read",
 )
+
+HOOK_NONE, HOOK_WITHHOLD_RELEASE, HOOK_MAX_CYCLES = 0, 1, 1 << 24
 
 
 class PoolDesc(ctypes.Structure):
@@ -106,6 +109,10 @@ def load(build_if_missing: bool = True):
         "plora_attn_workspace_bytes": (ctypes.c_size_t, [i32, i32, i32, i32]),
         "plora_attn_decode": (i32, [vp, vp, vp, vp, i32, i32, i32, i32, i32, ctypes.c_float, vp, vp, ctypes.c_size_t, vp]),
         "plora_attn_status": (i32, [vp, vp, ctypes.POINTER(i32)]),
+        "plora_attn_set_debug": (i32, [vp, i64, i32, vp]),
+        "plora_set_wait_limit": (i32, [vp, i64]),
+        "plora_set_test_hook": (i32, [vp, i32]),
+        "plora_stream_read": (i32, [vp, ctypes.c_size_t, vp, ctypes.c_size_t, vp]),
         "plora_cost_model": (i32, [ctypes.POINTER(CostHw), i32, vp, vp, ctypes.c_double, ctypes.c_double, ctypes.c_double,
                                    ctypes.POINTER(CostTerms)]),
     }
@@ -160,6 +167,22 @@ def plora_attn_status(ws_ptr, stream=0):
     v = ctypes.c_int32(0)
     rc = load().plora_attn_status(ws_ptr, stream, ctypes.byref(v))
     return rc, int(v.value)
+
+
+def plora_attn_set_debug(ws_ptr, cycles: int, hook: int, stream=0):
+    return load().plora_attn_set_debug(ws_ptr, int(cycles), int(hook), stream)
+
+
+def plora_set_wait_limit(ctx, cycles: int):
+    return load().plora_set_wait_limit(ctx, int(cycles))
+
+
+def plora_set_test_hook(ctx, hook: int):
+    return load().plora_set_test_hook(ctx, int(hook))
+
+
+def plora_stream_read(buf_ptr, nbytes: int, sink_ptr, sink_bytes: int, stream=0):
+    return load().plora_stream_read(buf_ptr, int(nbytes), sink_ptr, int(sink_bytes), stream)
 
 
 def attn_decode(q, k_cache, v_cache, kv_len, scale, out=None, workspace=None, stream=None):
@@ -440,6 +463,12 @@ class Context:
 
     def set_path(self, path: int, sgmv_min_rows: int = 0):
         _check(plora_set_path(self._h, path, sgmv_min_rows), "plora_set_path")
+
+    def set_wait_limit(self, cycles: int):
+        _check(plora_set_wait_limit(self._h, cycles), "plora_set_wait_limit")
+
+    def set_test_hook(self, hook: int):
+        _check(plora_set_test_hook(self._h, hook), "plora_set_test_hook")
 
     def set_input_type(self, fp16: bool):
         _check(load().plora_set_input_type(self._h, 1 if fp16 else 0), "plora_set_input_type")

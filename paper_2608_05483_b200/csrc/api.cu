@@ -5,6 +5,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <unordered_map>
 #include <vector>
 
 #include "plora_internal.cuh"
@@ -52,6 +53,14 @@ struct plora_ctx {
     const int32_t* cur_ids = nullptr;
     int32_t cur_ntok = -1, cur_nadapters = -1;
     bool bucket_valid = false;
+    // Who made the current bucket.  plora_bucket makes an explicit one: the caller vouches that the ids
+    // buffer keeps its contents until the next plora_bucket, so every later call with that buffer reuses
+    // it.  A delta call that finds no such bucket makes an implicit one, good for that call alone: the
+    // library cannot know whether the caller rewrote the buffer (or the allocator handed the address to
+    // a new tensor) before the next call.
+    bool bucket_explicit = false;
+    uint64_t call_gen = 0;     // one per entry into the library through a delta entry point
+    uint64_t bucket_gen = 0;   // the call that made the implicit bucket
     int32_t path = PLORA_PATH_AUTO;
     int32_t sgmv_min_rows = kDefaultSgmvMinRows;
     int32_t bucket_sgmv_min = INT_MAX;   // threshold the current bucket was built with
@@ -72,22 +81,25 @@ struct plora_ctx {
     cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
     int next_stage = 0;
     std::vector<PoolRec> pools;
+    std::unordered_map<uint64_t, size_t> pool_index;   // (layer, proj) -> position in pools
     int64_t launches = 0;
     // kernels launched through this context since the bucket kernel: from the second one on, the
     // bucket tables were complete before the kernel preceding it in the stream started
     int32_t launches_since_bucket = 0;
     ClassCache cls_cache;   // the bucket's units are sorted by the rank classes of pools with this signature
     bool fp16 = false;   // x, A and B are IEEE half instead of bf16
+    DebugCfg dbg;        // wait limit and test hook of the kernels' bounded waits
 };
 
 namespace {
 
 inline cudaStream_t as_stream(void* s) { return static_cast<cudaStream_t>(s); }
 
+inline uint64_t pool_key(int32_t layer, int32_t proj) { return ((uint64_t)(uint32_t)layer << 32) | (uint32_t)proj; }
+
 PoolRec* find_pool(plora_ctx* ctx, int32_t layer, int32_t proj) {
-    for (auto& p : ctx->pools)
-        if (p.layer == layer && p.proj == proj) return &p;
-    return nullptr;
+    const auto it = ctx->pool_index.find(pool_key(layer, proj));
+    return it == ctx->pool_index.end() ? nullptr : &ctx->pools[it->second];
 }
 
 bool desc_shape_ok(const plora_pool_desc* d, plora_status* why) {
@@ -141,7 +153,8 @@ int32_t effective_sgmv_min(const plora_ctx* ctx, int32_t n_tok) {
     }
 }
 
-plora_status do_bucket(plora_ctx* ctx, const int32_t* ids, int32_t n_tok, int32_t n_adapters, cudaStream_t st) {
+plora_status do_bucket(plora_ctx* ctx, const int32_t* ids, int32_t n_tok, int32_t n_adapters, cudaStream_t st,
+                       bool is_explicit) {
     const int32_t thr = effective_sgmv_min(ctx, n_tok);
     int nl = 0;
     cudaError_t e = launch_bucket(ids, n_tok, n_adapters, thr, ctx->path == PLORA_PATH_AUTO ? kSgmvMinTiles : 0, ctx->bk,
@@ -153,25 +166,29 @@ plora_status do_bucket(plora_ctx* ctx, const int32_t* ids, int32_t n_tok, int32_
     ctx->cur_nadapters = n_adapters;
     ctx->bucket_sgmv_min = thr;
     ctx->bucket_valid = true;
+    ctx->bucket_explicit = is_explicit;
+    ctx->bucket_gen = ctx->call_gen;
     ctx->launches_since_bucket = 0;
     ctx->cls_cache.valid = false;
     return PLORA_OK;
 }
 
 plora_status ensure_bucket(plora_ctx* ctx, const int32_t* ids, int32_t n_tok, int32_t n_adapters, cudaStream_t st) {
-    if (ctx->bucket_valid && ctx->cur_ids == ids && ctx->cur_ntok == n_tok && ctx->cur_nadapters == n_adapters &&
-        ctx->bucket_sgmv_min == effective_sgmv_min(ctx, n_tok))
+    // an explicit bucket serves every call that names its ids; an implicit one only the call that made it
+    if (ctx->bucket_valid && (ctx->bucket_explicit || ctx->bucket_gen == ctx->call_gen) && ctx->cur_ids == ids &&
+        ctx->cur_ntok == n_tok && ctx->cur_nadapters == n_adapters && ctx->bucket_sgmv_min == effective_sgmv_min(ctx, n_tok))
         return PLORA_OK;
-    return do_bucket(ctx, ids, n_tok, n_adapters, st);
+    return do_bucket(ctx, ids, n_tok, n_adapters, st, false);
 }
 
 cudaError_t launch_bgmv_one(BgmvMode mode, const PoolDev& pool, const BucketDev& bk, int n_tok, const void* x, float* y,
                             void* m, int ldm, int32_t* status, int sm_count, bool early_tables, ClassCache* cls_cache,
-                            uint64_t rank_sig, cudaStream_t stream, int* n_launches, bool m16, bool fp16) {
+                            uint64_t rank_sig, cudaStream_t stream, int* n_launches, bool m16, bool fp16,
+                            const DebugCfg& dbg) {
     const void* xs[1] = {x};
     float* ys[1] = {y};
     return launch_bgmv(mode, &pool, 1, bk, n_tok, xs, ys, m, ldm, m16, fp16, status, sm_count, early_tables, cls_cache,
-                       rank_sig, stream, n_launches);
+                       rank_sig, dbg, stream, n_launches);
 }
 
 plora_status check_call(plora_ctx* ctx, const void* a, const void* ids, int32_t n_tok, const void* b) {
@@ -384,6 +401,7 @@ PLORA_API plora_status plora_register_pool(plora_ctx* ctx, const plora_pool_desc
         cudaFree(old->table_dev);
         *old = rec;
     } else {
+        ctx->pool_index[pool_key(d->layer, d->proj)] = ctx->pools.size();
         ctx->pools.push_back(rec);
     }
     return PLORA_OK;
@@ -401,7 +419,7 @@ PLORA_API plora_status plora_bucket(plora_ctx* ctx, const int32_t* ids, int32_t 
     if (n_tok > 0 && !ids) return PLORA_ERR_INVALID_ARG;
     DeviceGuard g(ctx->device);
     if (!g.ok) return PLORA_ERR_CUDA;
-    return do_bucket(ctx, ids, n_tok, n_adapters, as_stream(stream));
+    return do_bucket(ctx, ids, n_tok, n_adapters, as_stream(stream), true);
 }
 
 PLORA_API plora_status plora_bucket_view(plora_ctx* ctx, const int32_t** perm, const int32_t** seg_adapter,
@@ -422,14 +440,33 @@ PLORA_API plora_status plora_set_path(plora_ctx* ctx, int32_t path, int32_t sgmv
     return PLORA_OK;
 }
 
+PLORA_API plora_status plora_set_wait_limit(plora_ctx* ctx, int64_t cycles) {
+    if (!ctx || cycles < 0) return PLORA_ERR_INVALID_ARG;
+    ctx->dbg.wait_cycles = cycles;
+    if (cycles == 0 || cycles > PLORA_HOOK_MAX_CYCLES) ctx->dbg.test_hook = PLORA_HOOK_NONE;   // a hook needs a short limit
+    return PLORA_OK;
+}
+
+PLORA_API plora_status plora_set_test_hook(plora_ctx* ctx, int32_t hook) {
+    if (!ctx || (hook != PLORA_HOOK_NONE && hook != PLORA_HOOK_WITHHOLD_RELEASE)) return PLORA_ERR_INVALID_ARG;
+    if (hook != PLORA_HOOK_NONE && (ctx->dbg.wait_cycles < 1 || ctx->dbg.wait_cycles > PLORA_HOOK_MAX_CYCLES))
+        return PLORA_ERR_INVALID_ARG;
+    ctx->dbg.test_hook = hook;
+    return PLORA_OK;
+}
+
 PLORA_API plora_status plora_set_input_type(plora_ctx* ctx, int32_t type) {
     if (!ctx || (type != PLORA_INPUT_BF16 && type != PLORA_INPUT_FP16)) return PLORA_ERR_INVALID_ARG;
     ctx->fp16 = type == PLORA_INPUT_FP16;
     return PLORA_OK;
 }
 
-PLORA_API plora_status plora_lora_delta(plora_ctx* ctx, const void* x, const int32_t* ids, int32_t n_tok, int32_t layer,
-                              int32_t proj, float* y, void* stream) {
+}  // extern "C"
+
+namespace {
+// One projection's delta; the caller has opened the call (call_gen).
+plora_status delta_one(plora_ctx* ctx, const void* x, const int32_t* ids, int32_t n_tok, int32_t layer, int32_t proj,
+                       float* y, void* stream) {
     plora_status rc = check_call(ctx, x, ids, n_tok, y);
     if (rc != PLORA_OK) return rc;
     PoolRec* pool = find_pool(ctx, layer, proj);
@@ -444,27 +481,37 @@ PLORA_API plora_status plora_lora_delta(plora_ctx* ctx, const void* x, const int
     cudaError_t e = cudaSuccess;
     if (ctx->path == PLORA_PATH_UNFUSED) {
         e = launch_bgmv_one(kShrinkOnly, pool->dev, ctx->bk, n_tok, x, nullptr, ctx->m_ws, pool->dev.max_rp, ctx->status_dev,
-                        ctx->sm_count, ctx->launches_since_bucket++ > 0, &ctx->cls_cache, pool->rank_sig, st, &nl, false, ctx->fp16);
+                        ctx->sm_count, ctx->launches_since_bucket++ > 0, &ctx->cls_cache, pool->rank_sig, st, &nl, false, ctx->fp16, ctx->dbg);
         if (e == cudaSuccess)
             e = launch_bgmv_one(kExpandOnly, pool->dev, ctx->bk, n_tok, nullptr, y, ctx->m_ws, pool->dev.max_rp,
-                            ctx->status_dev, ctx->sm_count, ctx->launches_since_bucket++ > 0, &ctx->cls_cache, pool->rank_sig, st, &nl, false, ctx->fp16);
+                            ctx->status_dev, ctx->sm_count, ctx->launches_since_bucket++ > 0, &ctx->cls_cache, pool->rank_sig, st, &nl, false, ctx->fp16, ctx->dbg);
     } else {
         // a batch shorter than the threshold cannot hold a segment for the tensor-core path
         const bool may_bgmv = ctx->path != PLORA_PATH_SGMV;
         const bool may_sgmv = ctx->bucket_sgmv_min != INT_MAX;
         if (may_bgmv)
-            e = launch_bgmv_one(kFused, pool->dev, ctx->bk, n_tok, x, y, nullptr, 0, ctx->status_dev, ctx->sm_count, ctx->launches_since_bucket++ > 0, &ctx->cls_cache, pool->rank_sig, st, &nl, false, ctx->fp16);
+            e = launch_bgmv_one(kFused, pool->dev, ctx->bk, n_tok, x, y, nullptr, 0, ctx->status_dev, ctx->sm_count, ctx->launches_since_bucket++ > 0, &ctx->cls_cache, pool->rank_sig, st, &nl, false, ctx->fp16, ctx->dbg);
         if (e == cudaSuccess && may_sgmv)
-            e = launch_sgmv(pool->dev, ctx->bk, n_tok, ctx->bucket_sgmv_min, x, y, ctx->fp16, ctx->status_dev, ctx->sm_count, may_bgmv, st, &nl);
+            e = launch_sgmv(pool->dev, ctx->bk, n_tok, ctx->bucket_sgmv_min, x, y, ctx->fp16, ctx->status_dev, ctx->sm_count, may_bgmv, ctx->dbg, st, &nl);
     }
     ctx->launches += nl;
     return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
+}
+}  // namespace
+
+extern "C" {
+
+PLORA_API plora_status plora_lora_delta(plora_ctx* ctx, const void* x, const int32_t* ids, int32_t n_tok, int32_t layer,
+                                        int32_t proj, float* y, void* stream) {
+    if (ctx) ++ctx->call_gen;
+    return delta_one(ctx, x, ids, n_tok, layer, proj, y, stream);
 }
 
 PLORA_API plora_status plora_lora_delta_group(plora_ctx* ctx, int32_t n, const void* const* x, const int32_t* ids,
                                               int32_t n_tok, const int32_t* layers, const int32_t* projs, float* const* y,
                                               void* stream) {
     if (!ctx || n < 1 || n > kMaxGroupPools || !x || !y || !layers || !projs) return PLORA_ERR_INVALID_ARG;
+    ++ctx->call_gen;
     PoolRec* recs[kMaxGroupPools];
     for (int g = 0; g < n; ++g) {
         plora_status rc = check_call(ctx, x[g], ids, n_tok, y[g]);
@@ -482,7 +529,7 @@ PLORA_API plora_status plora_lora_delta_group(plora_ctx* ctx, int32_t n, const v
     if (!same || ctx->path == PLORA_PATH_UNFUSED || ctx->path == PLORA_PATH_SGMV) {
         // pools of different shape, or a path without a grouped kernel: one projection after the other
         for (int g = 0; g < n; ++g) {
-            plora_status rc = plora_lora_delta(ctx, x[g], ids, n_tok, layers[g], projs[g], y[g], stream);
+            plora_status rc = delta_one(ctx, x[g], ids, n_tok, layers[g], projs[g], y[g], stream);
             if (rc != PLORA_OK) return rc;
         }
         return PLORA_OK;
@@ -496,10 +543,10 @@ PLORA_API plora_status plora_lora_delta_group(plora_ctx* ctx, int32_t n, const v
     for (int g = 0; g < n; ++g) pools[g] = recs[g]->dev;
     int nl = 0;
     cudaError_t e = launch_bgmv(kFused, pools, n, ctx->bk, n_tok, x, y, nullptr, 0, false, ctx->fp16, ctx->status_dev, ctx->sm_count,
-                                ctx->launches_since_bucket++ > 0, &ctx->cls_cache, recs[0]->rank_sig, st, &nl);
+                                ctx->launches_since_bucket++ > 0, &ctx->cls_cache, recs[0]->rank_sig, ctx->dbg, st, &nl);
     if (e == cudaSuccess && ctx->bucket_sgmv_min != INT_MAX)
         for (int g = 0; g < n && e == cudaSuccess; ++g)
-            e = launch_sgmv(pools[g], ctx->bk, n_tok, ctx->bucket_sgmv_min, x[g], y[g], ctx->fp16, ctx->status_dev, ctx->sm_count, true, st, &nl);
+            e = launch_sgmv(pools[g], ctx->bk, n_tok, ctx->bucket_sgmv_min, x[g], y[g], ctx->fp16, ctx->status_dev, ctx->sm_count, true, ctx->dbg, st, &nl);
     ctx->launches += nl;
     return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
 }
@@ -510,6 +557,7 @@ plora_status split_call(plora_ctx* ctx, BgmvMode mode, const void* x, void* m, i
                         int32_t n_tok, int32_t layer, int32_t proj, float* y, void* stream) {
     plora_status rc = check_call(ctx, mode == kShrinkOnly ? x : m, ids, n_tok, mode == kShrinkOnly ? m : (void*)y);
     if (rc != PLORA_OK) return rc;
+    ++ctx->call_gen;
     PoolRec* pool = find_pool(ctx, layer, proj);
     if (!pool) return PLORA_ERR_NOT_REGISTERED;
     // rows of m start on 16-byte boundaries (the expand copies them in bulk)
@@ -525,7 +573,7 @@ plora_status split_call(plora_ctx* ctx, BgmvMode mode, const void* x, void* m, i
     if (rc != PLORA_OK) return rc;
     int nl = 0;
     cudaError_t e = launch_bgmv_one(mode, pool->dev, ctx->bk, n_tok, x, y, m, ldm, ctx->status_dev, ctx->sm_count,
-                                    ctx->launches_since_bucket++ > 0, &ctx->cls_cache, pool->rank_sig, st, &nl, m16, ctx->fp16);
+                                    ctx->launches_since_bucket++ > 0, &ctx->cls_cache, pool->rank_sig, st, &nl, m16, ctx->fp16, ctx->dbg);
     ctx->launches += nl;
     return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
 }
@@ -716,6 +764,7 @@ PLORA_API plora_status plora_lora_delta_noalloc(plora_ctx* ctx, const void* x, c
                                                 int32_t layer, int32_t proj, float* y, void* stream) {
     plora_status rc = check_call(ctx, x, ids, n_tok, y);
     if (rc != PLORA_OK) return rc;
+    ++ctx->call_gen;
     PoolRec* pool = find_pool(ctx, layer, proj);
     if (!pool) return PLORA_ERR_NOT_REGISTERED;
     if (n_tok == 0) return PLORA_OK;
@@ -734,10 +783,10 @@ PLORA_API plora_status plora_lora_delta_noalloc(plora_ctx* ctx, const void* x, c
     if (rc != PLORA_OK) return rc;
     int nl = 0;
     cudaError_t e = launch_bgmv_one(kShrinkOnly, pool->dev, ctx->bk, n_tok, x, nullptr, m, ldm, ctx->status_dev,
-                                ctx->sm_count, ctx->launches_since_bucket++ > 0, &ctx->cls_cache, pool->rank_sig, st, &nl, false, ctx->fp16);
+                                ctx->sm_count, ctx->launches_since_bucket++ > 0, &ctx->cls_cache, pool->rank_sig, st, &nl, false, ctx->fp16, ctx->dbg);
     if (e == cudaSuccess)
         e = launch_bgmv_one(kExpandOnly, pool->dev, ctx->bk, n_tok, nullptr, y, m, ldm, ctx->status_dev, ctx->sm_count,
-                        ctx->launches_since_bucket++ > 0, &ctx->cls_cache, pool->rank_sig, st, &nl, false, ctx->fp16);
+                        ctx->launches_since_bucket++ > 0, &ctx->cls_cache, pool->rank_sig, st, &nl, false, ctx->fp16, ctx->dbg);
     ctx->launches += nl;
     return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
 }

@@ -46,7 +46,10 @@ constexpr int kMergeStride = kHeadDim + 4;            // floats per warp in the 
 constexpr int kMergeFloats = kConsumerWarps * kMergeStride;
 constexpr int kSmemBytes = 1024 + kStages * kSlotBytes + kMergeFloats * 4 + (2 * kStages + 1) * 8 + 16;
 constexpr int kPartFloats = kHeadDim + 4;             // per (unit, query head): o[128], m, l, pad
-constexpr long long kWaitCycles = 4000000000ll;
+constexpr long long kWaitCycles = 4000000000ll;   // default limit of a wait: about two seconds of SM clock
+// Words of the workspace header (its first 256 bytes; word 0 is the status word, word 1 the unit count):
+constexpr int kHookWord = 8;     // PLORA_HOOK_*: tests make a wait run out with it
+constexpr int kLimitWord = 10;   // 64-bit: limit of a wait in SM clock cycles, 0 = the default
 constexpr int kFlagFirst = 1, kFlagLast = 2, kFlagEnd = 4;
 
 struct Work {
@@ -88,19 +91,35 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
+__device__ __forceinline__ long long wait_limit(const int32_t* status) {
+    const long long v = *reinterpret_cast<const volatile long long*>(status + kLimitWord);
+    return v > 0 ? v : kWaitCycles;
+}
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+    const long long t0 = clock64(), limit = wait_limit(status);
     for (;;) {
-        for (int i = 0; i < 64; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitCycles) break;
+        for (int i = 0; i < 16; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (clock64() - t0 > limit) break;
     }
     *abort_flag = 1;
     __threadfence_block();
     atomicCAS(status, 0, PLORA_ERR_TIMEOUT);
     return false;
+}
+// Bounded wait on an mbarrier phase; false when the CTA has given up (here or elsewhere).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag, status);
+}
+// The copy thread's last look at a stage before it leaves: waits whatever the abort flag says, for at
+// most the limit (a CTA must not retire with a copy still on its way into its shared memory).
+__device__ __noinline__ bool mbar_drain(uint32_t bar, uint32_t parity, long long limit) {
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity))
+        if (clock64() - t0 > limit) return false;
+    return true;
 }
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
@@ -236,7 +255,8 @@ partial_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         // ------------------------------- producer warp (one lane) -------------------------------
         if (lane != 0) return;
         uint32_t it = 0;
-        for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+        bool stopped = false;   // a wait ran out somewhere in this CTA: nothing more is issued
+        for (int item = blockIdx.x; item < n_items && !stopped; item += gridDim.x) {
             const int unit = item / p.n_kv_heads, head = item - unit * p.n_kv_heads;
             const int req = p.w.unit_req[unit], chunk = p.w.unit_chunk[unit];
             int len = p.kv_len[req];
@@ -247,7 +267,10 @@ partial_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             const uint16_t* qsrc = p.q + ((size_t)req * p.n_kv_heads + head) * G * kHeadDim;
             for (int t = 0; t < n_tiles; ++t, ++it) {
                 const uint32_t slot = it % kStages, dst = slots + slot * kSlotBytes, bar = full + slot * 8;
-                if (!mbar_wait(empty + slot * 8, ((it / kStages) & 1) ^ 1, abort_flag, p.w.status)) return;
+                if (!mbar_wait(empty + slot * 8, ((it / kStages) & 1) ^ 1, abort_flag, p.w.status)) {
+                    stopped = true;
+                    break;
+                }
                 const int flags = (t == 0 ? kFlagFirst : 0) | (t == n_tiles - 1 ? kFlagLast : 0);
                 sts128(dst + kHdrOffset, (uint32_t)flags, (uint32_t)unit, (uint32_t)head,
                        (uint32_t)min(kTileTokens, n_in_chunk - t * kTileTokens));
@@ -261,9 +284,19 @@ partial_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             }
         }
         const uint32_t slot = it % kStages;   // tell the consumers that nothing follows
-        if (!mbar_wait(empty + slot * 8, ((it / kStages) & 1) ^ 1, abort_flag, p.w.status)) return;
-        sts128(slots + slot * kSlotBytes + kHdrOffset, (uint32_t)kFlagEnd, 0u, 0u, 0u);
-        mbar_arrive(full + slot * 8);
+        if (!stopped && mbar_wait(empty + slot * 8, ((it / kStages) & 1) ^ 1, abort_flag, p.w.status)) {
+            sts128(slots + slot * kSlotBytes + kHdrOffset, (uint32_t)kFlagEnd, 0u, 0u, 0u);
+            mbar_arrive(full + slot * 8);
+            ++it;   // the closing stage counts as armed: its slot's barrier has moved on one phase
+        }
+        // Before the thread leaves, the copies of the stages it armed last (stages it - 1, it - 2, ...) must
+        // have landed: the CTA's shared memory goes to another CTA when its last warp is gone.  In an orderly
+        // run these waits return at once or overlap the consumers' last tiles.
+        const long long limit = wait_limit(p.w.status);
+        for (uint32_t k = 1; k <= (uint32_t)kStages && k <= it; ++k) {
+            const uint32_t j = it - k;
+            if (!mbar_drain(full + (j % kStages) * 8, (j / kStages) & 1, limit)) atomicCAS(p.w.status, 0, PLORA_ERR_TIMEOUT);
+        }
         return;
     }
 
@@ -283,15 +316,18 @@ partial_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     uint32_t qf[8][2];
     uint32_t meetings = 0;
     bool alive = true;
+    // test hook: warp 0 never hands a stage back, so the copy thread's wait for a free stage runs out
+    const bool withhold = warp == 0 && p.w.status[kHookWord] == PLORA_HOOK_WITHHOLD_RELEASE;
+    // (every decision to stop is a vote: the lanes of a warp meet in shuffles and must leave together)
     auto consumer_meet = [&]() {
         __syncwarp();
         if (lane == 0) mbar_arrive(meet);
-        alive = alive && mbar_wait(meet, meetings & 1, abort_flag, p.w.status);
+        alive = __all_sync(0xffffffffu, alive && mbar_wait(meet, meetings & 1, abort_flag, p.w.status));
         ++meetings;
     };
     for (uint32_t it = 0; alive; ++it) {
         const uint32_t slot = it % kStages;
-        if (!mbar_wait(full + slot * 8, (it / kStages) & 1, abort_flag, p.w.status)) break;
+        if (!__all_sync(0xffffffffu, mbar_wait(full + slot * 8, (it / kStages) & 1, abort_flag, p.w.status))) break;
         const uint32_t st = slots + slot * kSlotBytes;
         const uint4 hw = lds128(st + kHdrOffset);
         StageHdr h;
@@ -478,10 +514,10 @@ partial_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the stage goes back to the copy engine
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(empty + slot * 8);
+            if (lane == 0 && !withhold) mbar_arrive(empty + slot * 8);
         } else {
             __syncwarp();
-            if (lane == 0) mbar_arrive(empty + slot * 8);
+            if (lane == 0 && !withhold) mbar_arrive(empty + slot * 8);
             if (h.flags & kFlagLast) {
                 // anchor merge of the eight warps' shares of this item
                 float* mine = merge + warp * kMergeStride;
@@ -661,6 +697,18 @@ extern "C" PLORA_API plora_status plora_attn_decode(const void* q, const void* k
     mc.numAttrs = 1;
     if (cudaLaunchKernelEx(&mc, merge_kernel, p) != cudaSuccess) return PLORA_ERR_CUDA;
     return PLORA_OK;
+}
+
+extern "C" PLORA_API plora_status plora_attn_set_debug(void* workspace, int64_t cycles, int32_t hook, void* stream) {
+    if (!workspace || cycles < 0 || (hook != PLORA_HOOK_NONE && hook != PLORA_HOOK_WITHHOLD_RELEASE)) return PLORA_ERR_INVALID_ARG;
+    if (hook != PLORA_HOOK_NONE && (cycles < 1 || cycles > PLORA_HOOK_MAX_CYCLES)) return PLORA_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t* w = static_cast<int32_t*>(workspace);
+    const long long lim = cycles;
+    if (cudaMemcpyAsync(w + kHookWord, &hook, 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(w + kLimitWord, &lim, 8, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return PLORA_ERR_CUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
 }
 
 extern "C" PLORA_API plora_status plora_attn_status(void* workspace, void* stream, int32_t* host_out) {

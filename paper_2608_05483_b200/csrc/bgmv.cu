@@ -66,7 +66,7 @@ constexpr int kMRingBytes = kTokChunk * kMaxRank * 4;
 constexpr int kNumBarriers = 2 * kStages + 2 * kMRing;
 constexpr int kSmemBytes = kStages * kSlotBytes + kMRing * kMRingBytes + kNumBarriers * 8 + 16;
 constexpr uint32_t kSuspendHintNs = 20000;   // a waiting thread may sleep this long inside one try_wait
-constexpr long long kWaitCycles = 4000000000ll;   // about two seconds of SM clock
+constexpr long long kWaitCycles = 4000000000ll;   // default limit of a wait: about two seconds of SM clock
 
 // Projections that do not depend on one another (q, k and v of a layer; up and gate) can share a
 // launch: the task list simply runs over "virtual units" (group, unit).  The pools of a group have
@@ -95,6 +95,8 @@ struct Params {
     int32_t defer_wait;
     int32_t bump_epoch;
     int32_t* status;
+    long long wait_cycles;    // limit of every bounded wait, in SM clock cycles
+    int32_t test_hook;        // PLORA_HOOK_*: tests make a wait run out with it
 };
 
 // ---- PTX wrappers -----------------------------------------------------------------
@@ -128,17 +130,37 @@ __device__ __forceinline__ void give_up(volatile int* abort_flag, int32_t* statu
     __threadfence_block();
     atomicCAS(status, 0, PLORA_ERR_TIMEOUT);
 }
-// Bounded wait on an mbarrier phase.
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
-    if (mbar_try_wait(bar, parity)) return;
+// Bounded wait on an mbarrier phase.  True: the phase is complete.  False: the wait ran out, here
+// (then the status word says so) or in another role of this CTA (the abort flag); the caller stops
+// what it is doing: consumers leave their loop, the copy warp issues nothing more.
+struct WaitCtl {
+    volatile int* abort_flag;
+    int32_t* status;
+    long long limit;
+};
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, const WaitCtl& w) {
     const long long t0 = clock64();
     for (;;) {
-        for (int i = 0; i < 256; ++i)
-            if (mbar_try_wait(bar, parity)) return;
-        if (*abort_flag) return;
-        if (clock64() - t0 > kWaitCycles) break;
+        if (*w.abort_flag) return mbar_try_wait(bar, parity);
+        for (int i = 0; i < 16; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (clock64() - t0 > w.limit) break;
     }
-    give_up(abort_flag, status);
+    give_up(w.abort_flag, w.status);
+    return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtl& w) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, w);
+}
+// The copy warp's last look at a stage before it leaves: has everything it asked for arrived?  Waits
+// whatever the abort flag says, for at most the limit (a CTA must not retire with a bulk copy still on
+// its way into its shared memory).
+__device__ __noinline__ bool mbar_drain(uint32_t bar, uint32_t parity, long long limit) {
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity))
+        if (clock64() - t0 > limit) return false;
+    return true;
 }
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
@@ -196,13 +218,17 @@ struct Smem {
     uint32_t slots;      // shared address of stage 0
     uint32_t full;       // full[kStages] barriers
     uint32_t empty;      // empty[kStages]
-    volatile int* abort_flag;
+    WaitCtl wait;        // abort flag of the CTA, status word, limit of a wait
     uint32_t m_ring;     // shared address of the m ring (fused mode): kMRing entries of kMRingBytes
     uint32_t m_full;     // m_full[kMRing]: the gather warp has written the entry
     uint32_t m_empty;    // m_empty[kMRing]: every consumer warp is done with the entry
-    int32_t* status;
     uint32_t epoch;      // this launch's epoch (fused mode)
+    bool withhold;       // test hook: this warp never hands a stage back
 };
+// A consumer warp is done with a stage.
+__device__ __forceinline__ void release_stage(const Smem& sm, uint32_t empty_bar, int lane) {
+    if (lane == 0 && !sm.withhold) mbar_arrive(empty_bar);
+}
 
 // What a stage holds (written by the producer into the stage, read by every consumer warp).
 constexpr int kFlagExpand = 1, kFlagFirst = 2, kFlagLast = 4, kFlagEnd = 8, kFlagSlice = 16;
@@ -216,7 +242,10 @@ struct StageHdr {
     int32_t m_seq;    // fused expand stages: running number of the expand task in this CTA (m-ring entry = m_seq % kMRing)
     int32_t group;    // which projection of the launch's group (unit = group * n_units + bucket unit)
     int32_t k0;       // shrink stages of a row slice: first rank row of the slice (otherwise 0)
+    // (the word after k0 holds the stage's running number, for the copy warp's own use: kStampOffset)
 };
+constexpr int kStampOffset = 60;            // byte offset inside the header
+constexpr uint32_t kNoStamp = 0xffffffffu;  // the stage was never armed
 
 __device__ __forceinline__ StageHdr read_hdr(uint32_t a) {
     const uint4 q0 = lds128(a), q1 = lds128(a + 16), q2 = lds128(a + 32);
@@ -557,7 +586,8 @@ __device__ __forceinline__ void expand_tile_cnt(const Params& p, const Smem& sm,
                                      : tile + mp.b_col + mp.rg * M::RPG * 128;
     const int m_slot = h.m_seq % kMRing;
     if (MODE == kFused && (h.flags & kFlagFirst))   // the gather warp has assembled this task's m
-        mbar_wait(sm.m_full + m_slot * 8, (h.m_seq / kMRing) & 1, sm.abort_flag, sm.status);
+        if (!__all_sync(0xffffffffu, mbar_wait(sm.m_full + m_slot * 8, (h.m_seq / kMRing) & 1, sm.wait)))
+            return;   // gave up: nothing of this tile reaches y
     // fused: m in the m ring, group-major, so the group's rows are RPG consecutive floats per token;
     // expand-only: the caller's m next to the tile, in natural order
     const uint32_t mb = MODE == kFused ? sm.m_ring + m_slot * kMRingBytes + mp.rg * M::RPG * 4 : tile + kTileBytesMax;
@@ -617,10 +647,8 @@ __device__ __forceinline__ void expand_tile_cnt(const Params& p, const Smem& sm,
         }
     }
     __syncwarp();
-    if (lane == 0) {
-        mbar_arrive(empty_bar);
-        if (MODE == kFused && (h.flags & kFlagLast)) mbar_arrive(sm.m_empty + m_slot * 8);
-    }
+    release_stage(sm, empty_bar, lane);
+    if (lane == 0 && MODE == kFused && (h.flags & kFlagLast)) mbar_arrive(sm.m_empty + m_slot * 8);
     float out[CNT][2];
 #pragma unroll
     for (int t = 0; t < CNT; ++t) {
@@ -726,7 +754,7 @@ __device__ __forceinline__ void consume_stage(const Params& p, const Smem& sm, c
                 if (tc) shrink_tile_mma<RPS < 16 ? 16 : RPS, H>(p, h, tile, acc[0], warp, lane);
                 else shrink_tile<RPS, H>(p, h, maps.s2, tile, acc);
                 __syncwarp();
-                if (lane == 0) mbar_arrive(empty_bar);
+                release_stage(sm, empty_bar, lane);
                 if (h.flags & kFlagLast) {
                     if (tc) shrink_finish_mma<MODE, RPS < 16 ? 16 : RPS>(p, sm, h, acc[0], warp, lane);
                     else shrink_finish<MODE, RPS>(p, sm, h, maps.s2, acc, warp, lane);
@@ -734,12 +762,12 @@ __device__ __forceinline__ void consume_stage(const Params& p, const Smem& sm, c
             } else if (RP >= 64 && tc4) {
                 shrink_tile_mma<RP < 16 ? 16 : RP, H>(p, h, tile, acc[0], warp, lane);
                 __syncwarp();
-                if (lane == 0) mbar_arrive(empty_bar);
+                release_stage(sm, empty_bar, lane);
                 if (h.flags & kFlagLast) shrink_finish_mma<MODE, RP < 16 ? 16 : RP>(p, sm, h, acc[0], warp, lane);
             } else {
                 shrink_tile<RP, H>(p, h, maps.s, tile, acc);
                 __syncwarp();
-                if (lane == 0) mbar_arrive(empty_bar);
+                release_stage(sm, empty_bar, lane);
                 if (h.flags & kFlagLast) shrink_finish<MODE, RP>(p, sm, h, maps.s, acc, warp, lane);
             }
         }
@@ -760,10 +788,11 @@ __device__ __forceinline__ bool consume_class(const Params& p, const Smem& sm, u
     maps.init(warp, lane);
     for (;; ++it) {
         const uint32_t slot = it % kStages;
-        mbar_wait(sm.full + slot * 8, (it / kStages) & 1, sm.abort_flag, sm.status);
+        // (the vote makes the decision the same in every lane: the code below meets in shuffles)
+        if (!__all_sync(0xffffffffu, mbar_wait(sm.full + slot * 8, (it / kStages) & 1, sm.wait))) return false;
         const uint32_t tile = sm.slots + slot * kSlotBytes;
         const StageHdr h = read_hdr(tile + kHdrOffset);
-        if ((h.flags & kFlagEnd) || lds32(smem_u32(const_cast<int*>(sm.abort_flag)))) return false;
+        if (h.flags & kFlagEnd) return false;
         if (!ONLY && h.rp != RP) return true;
         consume_stage<MODE, RP, H, ONLY>(p, sm, h, maps, tile, sm.empty + slot * 8, acc, warp, lane);
     }
@@ -1065,22 +1094,42 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
     sm.empty = sm.full + kStages * 8;
     sm.m_full = sm.empty + kStages * 8;
     sm.m_empty = sm.m_full + kMRing * 8;
-    sm.abort_flag = reinterpret_cast<volatile int*>(bars + kNumBarriers * 8);
-    sm.status = p.status;
+    sm.wait.abort_flag = reinterpret_cast<volatile int*>(bars + kNumBarriers * 8);
+    sm.wait.status = p.status;
+    sm.wait.limit = p.wait_cycles;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    sm.withhold = p.test_hook == PLORA_HOOK_WITHHOLD_RELEASE && warp == 0;
+    if (MODE != kShrinkOnly && p.early_tables) {
+        // A launch that has nothing to do (every segment of the batch went to the tensor-core path, or
+        // the pool's rank class has no unit in this batch) leaves before it sets up its ring.  The
+        // tables it looks at are older than the previous kernel of the stream, hence complete.  It
+        // still joins the stream order, so that its completion implies that of everything before it.
+        // (The shrink-only kernel always has the rows of tokens without an adapter to clear.)
+        int n = *p.bk.n_bgmv_units;
+        // (the class launch that advances the epoch for its call stays: the other classes' words need it)
+        if (n != 0 && RPK && p.by_class && !(MODE == kFused && p.bump_epoch)) {
+            constexpr int kClass = RPK == 8 ? 0 : RPK == 16 ? 1 : RPK == 32 ? 2 : RPK == 64 ? 3 : 4;
+            n = p.bk.cls_start[kClass + 1] - p.bk.cls_start[kClass];
+        }
+        if (n == 0) {
+            if (tid == 0) grid_dependency_wait();
+            return;
+        }
+    }
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(sm.full + s * 8, 1);
             mbar_init(sm.empty + s * 8, kConsumerWarps);
             // a stage that was never filled reads as "nothing follows"
             sts128(sm.slots + s * kSlotBytes + kHdrOffset, (uint32_t)kFlagEnd, 0u, 0u, 0u);
+            sts128(sm.slots + s * kSlotBytes + kHdrOffset + 48, 0u, 0u, 0u, kNoStamp);
         }
         for (int e = 0; e < kMRing; ++e) {
             mbar_init(sm.m_full + e * 8, 1);
             mbar_init(sm.m_empty + e * 8, kConsumerWarps);
         }
-        *sm.abort_flag = 0;
+        *sm.wait.abort_flag = 0;
         fence_barrier_init();
     }
     __syncthreads();
@@ -1133,7 +1182,8 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
         const unsigned full = 0xffffffffu;
         uint32_t it_base = 0;
         uint32_t m_count = 0;   // expand tasks issued so far (fused mode)
-        for (int base = blockIdx.x; base < n_tasks; base += 32 * stride) {
+        bool stopped = false;   // a wait ran out somewhere in this CTA: nothing more is issued
+        for (int base = blockIdx.x; base < n_tasks && !stopped; base += 32 * stride) {
             const int my_task = base + lane * stride;
             const bool has = my_task < n_tasks;
             const Task mine = plan.decode(has ? my_task : base);
@@ -1170,14 +1220,15 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
             // previous kernel may have written (x, the caller's m) follows after the wait (pass 2, which
             // also issues everything beyond the first turn).  Otherwise one pass issues everything (pass 0).
             const bool early = !waited;
-            for (int pass = early ? 1 : 0; pass <= (early ? 2 : 0); ++pass) {
+            for (int pass = early ? 1 : 0; pass <= (early ? 2 : 0) && !stopped; ++pass) {
                 if (pass == 2) {
                     grid_dependency_wait();
                     waited = true;
                 }
                 if (pass != 1 && base == (int)blockIdx.x) sm.epoch = MODE == kFused ? *p.bk.epoch : 0u;
                 uint32_t mc = m_count;
-                for (int b = 0; b < in_batch; ++b) {
+                bool failed = false;
+                for (int b = 0; b < in_batch && !stopped; ++b) {
                     // fused mode: the running number of this expand task tells the consumers where its m is
                     const uint32_t m_seq = mc;
                     if (MODE == kFused && __shfl_sync(full, (int)(has && mine.phase), b)) ++mc;
@@ -1196,13 +1247,16 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
                             const uint32_t bar = sm.full + slot * 8;
                             const uint32_t tbytes = mine.phase ? mbytes : (uint32_t)min(C, d - i * C) * 2u;
                             if (head) {
-                                mbar_wait(sm.empty + slot * 8, ((it / kStages) & 1) ^ 1, sm.abort_flag, p.status);
+                                if (!mbar_wait(sm.empty + slot * 8, ((it / kStages) & 1) ^ 1, sm.wait)) {
+                                    failed = true;
+                                    break;
+                                }
                                 const int flags = (mine.phase ? kFlagExpand : 0) | (i == lo ? kFlagFirst : 0) | (i == hi - 1 ? kFlagLast : 0) |
                                                   (!mine.phase && sliced ? kFlagSlice : 0);
                                 sts128(dst + kHdrOffset, (uint32_t)flags, (uint32_t)(my_group * p.n_tok + mu.pos0), (uint32_t)mine.run, (uint32_t)i);
                                 sts128(dst + kHdrOffset + 16, (uint32_t)cnt, (uint32_t)mu.tok[0], (uint32_t)mu.tok[1], (uint32_t)mu.tok[2]);
                                 sts128(dst + kHdrOffset + 32, (uint32_t)mu.tok[3], (uint32_t)rp, (uint32_t)me.r, __float_as_uint(me.scale));
-                                sts128(dst + kHdrOffset + 48, m_seq, (uint32_t)my_group, (uint32_t)k0, 0u);
+                                sts128(dst + kHdrOffset + 48, m_seq, (uint32_t)my_group, (uint32_t)k0, it);   // it: kStampOffset
                                 if (MODE == kFused && sliced && !mine.phase) {
                                     // rows [k0, k0 + kSliceRows) of up to four consecutive sub-tiles of A^T, side by side
                                     constexpr uint32_t kPiece = kSliceRows * kSubCols * 2;
@@ -1238,18 +1292,32 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
                             }
                         }
                     }
-                    __syncwarp();
+                    stopped = __any_sync(full, failed);   // (also the warp's meeting point after the owner's turn)
                 }
                 if (pass != 1) m_count = mc;
             }
         }
         if (!waited) grid_dependency_wait();
-        if (lane == 0) {   // tell the consumers that nothing follows
-            const uint32_t it = it_base;
-            const uint32_t slot = it % kStages;
-            mbar_wait(sm.empty + slot * 8, ((it / kStages) & 1) ^ 1, sm.abort_flag, p.status);
-            sts128(sm.slots + slot * kSlotBytes + kHdrOffset, (uint32_t)kFlagEnd, 0u, 0u, 0u);
-            mbar_arrive(sm.full + slot * 8);
+        if (lane == 0) {
+            if (!stopped) {   // tell the consumers that nothing follows
+                const uint32_t it = it_base;
+                const uint32_t slot = it % kStages;
+                if (mbar_wait(sm.empty + slot * 8, ((it / kStages) & 1) ^ 1, sm.wait)) {
+                    sts128(sm.slots + slot * kSlotBytes + kHdrOffset, (uint32_t)kFlagEnd, 0u, 0u, 0u);
+                    sts128(sm.slots + slot * kSlotBytes + kHdrOffset + 48, 0u, 0u, 0u, it);
+                    mbar_arrive(sm.full + slot * 8);
+                }
+            }
+            // Before the warp leaves, every copy it asked for must have landed: the CTA's shared memory goes
+            // to another CTA when the last warp is gone.  Each stage's header names the phase it was last
+            // armed for.  In an orderly run these waits return at once or overlap the consumers' last stages.
+            // After a give-up between the two passes of the first turn a stage may be armed for bytes that
+            // were never asked for: its wait runs out, which is harmless (nothing is on its way there).
+            for (int s2 = 0; s2 < kStages; ++s2) {
+                const uint32_t stamp = lds32(sm.slots + s2 * kSlotBytes + kHdrOffset + kStampOffset);
+                if (stamp != kNoStamp && !mbar_drain(sm.full + s2 * 8, (stamp / kStages) & 1, p.wait_cycles))
+                    atomicCAS(p.status, 0, PLORA_ERR_TIMEOUT);
+            }
         }
         return;
     }
@@ -1297,18 +1365,25 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
                 const int runs_a_b = RPK ? plan.s_runs[0] : __shfl_sync(full, my_runs_a, b);
                 const int unit_b = __shfl_sync(full, my_group * p.n_tok + mu.pos0, b), cnt_b = __shfl_sync(full, mu.cnt, b);
                 const uint32_t e = seq % kMRing;
-                if (lane == 0) mbar_wait(sm.m_empty + e * 8, ((seq / kMRing) & 1) ^ 1, sm.abort_flag, p.status);
-                __syncwarp();
+                bool ok = true;
+                if (lane == 0) ok = mbar_wait(sm.m_empty + e * 8, ((seq / kMRing) & 1) ^ 1, sm.wait);
+                if (!__all_sync(full, ok)) return;   // gave up: the consumers see the flag at their own waits
                 const uint32_t mdst = sm.m_ring + e * kMRingBytes;
                 if (!__all_sync(full, gather_m(p, rp_b, runs_a_b, sm.epoch, unit_b, cnt_b, lane, mdst))) {
                     const long long t0 = clock64();
                     for (;;) {
                         __nanosleep(100);
-                        if (__all_sync(full, gather_m(p, rp_b, runs_a_b, sm.epoch, unit_b, cnt_b, lane, mdst)) || *sm.abort_flag) break;
-                        if (clock64() - t0 > kWaitCycles) {
-                            if (lane == 0) give_up(sm.abort_flag, p.status);
-                            break;
+                        if (__all_sync(full, gather_m(p, rp_b, runs_a_b, sm.epoch, unit_b, cnt_b, lane, mdst))) break;
+                        // one lane decides for the warp, so that all lanes leave together
+                        int quit = 0;
+                        if (lane == 0) {
+                            if (*sm.wait.abort_flag) quit = 1;
+                            else if (clock64() - t0 > sm.wait.limit) {
+                                give_up(sm.wait.abort_flag, p.status);
+                                quit = 1;
+                            }
                         }
+                        if (__shfl_sync(full, quit, 0)) return;   // the entry is never published: no expand task uses a partial m
                     }
                 }
                 __syncwarp();
@@ -1331,10 +1406,10 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
         for (bool more = true; more;) {
             // whose stage is next?  (the class's loop waits for it again: the phase is complete by then)
             const uint32_t slot = it % kStages;
-            mbar_wait(sm.full + slot * 8, (it / kStages) & 1, sm.abort_flag, sm.status);
+            if (!__all_sync(0xffffffffu, mbar_wait(sm.full + slot * 8, (it / kStages) & 1, sm.wait))) break;
             const int flags = (int)lds32(sm.slots + slot * kSlotBytes + kHdrOffset);
             const int rp = (int)lds32(sm.slots + slot * kSlotBytes + kHdrOffset + 36);
-            if ((flags & kFlagEnd) || lds32(smem_u32(const_cast<int*>(sm.abort_flag)))) break;
+            if (flags & kFlagEnd) break;
             switch (rp) {
                 case 8: more = consume_class<MODE, 8, H, false>(p, sm, it, acc, warp, lane); break;
                 case 16: more = consume_class<MODE, 16, H, false>(p, sm, it, acc, warp, lane); break;
@@ -1403,8 +1478,8 @@ cudaError_t bgmv_configure() {
 
 cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const BucketDev& bk, int n_tok,
                         const void* const* x, float* const* y, void* m, int ldm, bool m16, bool fp16, int32_t* status,
-                        int sm_count, bool early_tables, ClassCache* cls_cache, uint64_t rank_sig, cudaStream_t stream,
-                        int* n_launches) {
+                        int sm_count, bool early_tables, ClassCache* cls_cache, uint64_t rank_sig, const DebugCfg& dbg,
+                        cudaStream_t stream, int* n_launches) {
     if (n_groups < 1 || n_groups > kMaxGroup || (mode != kFused && n_groups != 1)) return cudaErrorInvalidValue;
     const PoolDev& pool = pools[0];
     Params p;
@@ -1425,6 +1500,8 @@ cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const
     p.m16 = m16 ? 1 : 0;
     p.n_tok = n_tok;
     p.status = status;
+    p.wait_cycles = dbg.wait_cycles > 0 ? dbg.wait_cycles : kWaitCycles;
+    p.test_hook = dbg.test_hook;
     p.early_tables = early_tables ? 1 : 0;
     p.defer_wait = 0;
     p.bump_epoch = 1;

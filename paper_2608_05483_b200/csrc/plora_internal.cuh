@@ -121,15 +121,20 @@ struct ClassCache {
     uint64_t sig = 0;
     bool valid = false;
 };
+// Diagnostics of the bounded waits (plora_set_wait_limit, plora_set_test_hook).
+struct DebugCfg {
+    long long wait_cycles = 0;   // 0: the kernels' default
+    int32_t test_hook = 0;       // PLORA_HOOK_*
+};
 cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const BucketDev& bk, int n_tok,
                         const void* const* x, float* const* y, void* m, int ldm, bool m16, bool fp16, int32_t* status,
-                        int sm_count, bool early_tables, ClassCache* cls_cache, uint64_t rank_sig, cudaStream_t stream,
-                        int* n_launches);
+                        int sm_count, bool early_tables, ClassCache* cls_cache, uint64_t rank_sig, const DebugCfg& dbg,
+                        cudaStream_t stream, int* n_launches);
 // after_bgmv_of_same_call: the launch follows fused BGMV launches of the same call (other tokens of the
 // same batch) and may overlap them
 cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, int sgmv_min_rows, const void* x, float* y,
-                        bool fp16, int32_t* status, int sm_count, bool after_bgmv_of_same_call, cudaStream_t stream,
-                        int* n_launches);
+                        bool fp16, int32_t* status, int sm_count, bool after_bgmv_of_same_call, const DebugCfg& dbg,
+                        cudaStream_t stream, int* n_launches);
 // per-device function attributes (dynamic shared memory); called by plora_create
 cudaError_t bucket_configure();
 cudaError_t bgmv_configure();

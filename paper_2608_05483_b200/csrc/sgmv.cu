@@ -61,7 +61,7 @@ constexpr int kStagePitch = kKC * 4 + 16;                  // row pitch of the e
 constexpr int kStagingBytes = kEpiWarps * kRowsPerWarp * kStagePitch;
 constexpr int kSmemBudget = 227 * 1024;                    // of an SM
 constexpr int kSmemPerCta = kSmemBudget / 2 - 1024;        // two CTAs per SM, so that one tile's shrink overlaps another's expand
-constexpr long long kWaitCycles = 4000000000ll;            // about two seconds of SM clock
+constexpr long long kWaitCycles = 4000000000ll;            // default limit of a wait: about two seconds of SM clock
 
 // Shared memory, sized for R = max(16, largest padded rank of the pool):
 //   ring of n_stages x (x block 8 KiB + weight sub-tile R x 128 B)       1024-byte aligned
@@ -92,6 +92,8 @@ struct Params {
     // still implies the completion of everything before it.
     int32_t defer_wait;
     int32_t fp16;       // x, A and B hold IEEE half values instead of bf16 (m is then split into half hi + lo)
+    long long wait_cycles;   // limit of every bounded wait, in SM clock cycles
+    int32_t test_hook;       // PLORA_HOOK_*: tests make a wait run out with it
 };
 
 // ---- PTX wrappers -----------------------------------------------------------------
@@ -117,19 +119,34 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait on an mbarrier phase; false when the CTA has given up (here or elsewhere).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
-    if (mbar_try_wait(bar, parity)) return true;
+struct WaitCtl {
+    volatile int* abort_flag;
+    int32_t* status;
+    long long limit;
+};
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, const WaitCtl& w) {
     const long long t0 = clock64();
     for (;;) {
-        for (int i = 0; i < 64; ++i)
+        if (*w.abort_flag) return false;
+        for (int i = 0; i < 16; ++i)
             if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitCycles) break;
+        if (clock64() - t0 > w.limit) break;
     }
-    *abort_flag = 1;
+    *w.abort_flag = 1;
     __threadfence_block();
-    atomicCAS(status, 0, PLORA_ERR_TIMEOUT);
+    atomicCAS(w.status, 0, PLORA_ERR_TIMEOUT);
     return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtl& w) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, w);
+}
+// Winding down after a give-up: wait for a phase whatever the abort flag says, for at most the limit.
+__device__ __noinline__ bool mbar_drain(uint32_t bar, uint32_t parity, long long limit) {
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity))
+        if (clock64() - t0 > limit) return false;
+    return true;
 }
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
@@ -212,8 +229,10 @@ struct Smem {
     uint32_t d_full;      // the shrink accumulator is complete
     uint32_t m_ready;     // the epilogue has stored m hi / lo (and is done with the shrink accumulator)
     uint32_t d2_full, d2_empty;   // [kD2Bufs] each
-    volatile int* abort_flag;
+    uint32_t wind_down;   // after a give-up: the MMAs issued so far have completed
+    WaitCtl wait;         // abort flag of the CTA, status word, limit of a wait
     uint32_t* tmem_slot;
+    uint32_t* armed;      // [kMaxStages]: 1 + the running number of the stage a slot was last armed for (0: never)
 };
 
 __device__ __forceinline__ Smem carve(uint8_t* raw, const Params& p) {
@@ -234,8 +253,13 @@ __device__ __forceinline__ Smem carve(uint8_t* raw, const Params& p) {
     s.m_ready = s.d_full + 8;
     s.d2_full = s.m_ready + 8;
     s.d2_empty = s.d2_full + kD2Bufs * 8;
-    s.abort_flag = reinterpret_cast<volatile int*>(bars + (2 * kMaxStages + 2 + 2 * kD2Bufs) * 8);
-    s.tmem_slot = reinterpret_cast<uint32_t*>(bars + (2 * kMaxStages + 2 + 2 * kD2Bufs) * 8 + 8);
+    s.wind_down = s.d2_empty + kD2Bufs * 8;
+    uint8_t* words = bars + (2 * kMaxStages + 3 + 2 * kD2Bufs) * 8;
+    s.wait.abort_flag = reinterpret_cast<volatile int*>(words);
+    s.wait.status = p.status;
+    s.wait.limit = p.wait_cycles;
+    s.tmem_slot = reinterpret_cast<uint32_t*>(words + 8);
+    s.armed = reinterpret_cast<uint32_t*>(words + 16);
     return s;
 }
 
@@ -273,8 +297,9 @@ __device__ __forceinline__ void producer_warp(const Params& p, const Smem& sm, c
             const bool shrink = c < nK;
             int ok = 1;
             if (lane == 0) {
-                ok = mbar_wait(sm.empty + slot * 8, ((it / p.n_stages) & 1) ^ 1, sm.abort_flag, p.status);
+                ok = mbar_wait(sm.empty + slot * 8, ((it / p.n_stages) & 1) ^ 1, sm.wait);
                 if (ok) {
+                    sm.armed[slot] = it + 1;
                     mbar_arrive_expect_tx(bar, wbytes + (shrink ? xbytes : 0u));
                     bulk_g2s(dst + kXStageBytes, shrink ? a_src + (size_t)c * wbytes : b_src + (size_t)(c - nK) * wbytes,
                              wbytes, bar);
@@ -296,6 +321,7 @@ __device__ __forceinline__ void mma_thread(const Params& p, const Smem& sm, uint
     const int nK = (p.pool.d_in + kKC - 1) / kKC, nN = (p.pool.d_out + kKC - 1) / kKC;
     const int stage = stage_bytes(p.R);
     uint32_t it = 0, d2 = 0, tile_idx = 0;
+    const bool withhold = p.test_hook == PLORA_HOOK_WITHHOLD_RELEASE;   // test hook: shrink stages are never handed back
     for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++tile_idx) {
         const WorkUnit wu = p.bk.sgmv_tiles[t];
         const int rp = p.pool.table[wu.adapter].rp;
@@ -304,23 +330,23 @@ __device__ __forceinline__ void mma_thread(const Params& p, const Smem& sm, uint
         const uint32_t idesc_s = instr_desc(KP, false, p.fp16 != 0);
         for (int kc = 0; kc < nK; ++kc, ++it) {
             const uint32_t slot = it % p.n_stages;
-            if (!mbar_wait(sm.full + slot * 8, (it / p.n_stages) & 1, sm.abort_flag, p.status)) return;
+            if (!mbar_wait(sm.full + slot * 8, (it / p.n_stages) & 1, sm.wait)) return;
             tc_fence_after();
             const uint32_t xa = sm.ring + slot * stage, wa = xa + kXStageBytes;
 #pragma unroll
             for (int k = 0; k < kKC / 16; ++k)   // 16 columns = 32 bytes further along the swizzled rows
                 umma(tmem, smem_desc(xa + k * 32, 16, 1024, 2), smem_desc(wa + k * 32, 16, 1024, 2), idesc_s, kc > 0 || k > 0);
-            umma_commit(sm.empty + slot * 8);
+            if (!withhold) umma_commit(sm.empty + slot * 8);
         }
         umma_commit(sm.d_full);
         // expand: for every 64-column block, D2[128, 64] = (m_hi + m_lo)[128, KP] * B[KP, 64]
-        if (!mbar_wait(sm.m_ready, tile_idx & 1, sm.abort_flag, p.status)) return;
+        if (!mbar_wait(sm.m_ready, tile_idx & 1, sm.wait)) return;
         tc_fence_after();
         const uint32_t idesc_e = instr_desc(kKC, true, p.fp16 != 0);
         for (int nc = 0; nc < nN; ++nc, ++it, ++d2) {
             const uint32_t slot = it % p.n_stages, b = d2 % kD2Bufs;
-            if (!mbar_wait(sm.full + slot * 8, (it / p.n_stages) & 1, sm.abort_flag, p.status)) return;
-            if (!mbar_wait(sm.d2_empty + b * 8, ((d2 / kD2Bufs) & 1) ^ 1, sm.abort_flag, p.status)) return;
+            if (!mbar_wait(sm.full + slot * 8, (it / p.n_stages) & 1, sm.wait)) return;
+            if (!mbar_wait(sm.d2_empty + b * 8, ((d2 / kD2Bufs) & 1) ^ 1, sm.wait)) return;
             tc_fence_after();
             const uint32_t wa = sm.ring + slot * stage + kXStageBytes;
             const uint32_t dst = tmem + kTmemD2 + b * kKC;
@@ -359,7 +385,7 @@ __device__ __forceinline__ void epilogue_warp(const Params& p, const Smem& sm, u
         epi_barrier();   // every epilogue thread is done with the previous tile's token indices
         if (owner) sm.tok[row] = p.bk.perm[wu.pos0 + min(row, cnt - 1)];
         epi_barrier();
-        if (alive) alive = __all_sync(full, mbar_wait(sm.d_full, tile_idx & 1, sm.abort_flag, p.status));
+        if (alive) alive = __all_sync(full, mbar_wait(sm.d_full, tile_idx & 1, sm.wait));
         if (!alive) continue;
         tc_fence_after();
         // m = s * (x A), split into bf16 hi + lo; columns beyond the padded rank (rank 8 only) are zeros
@@ -405,7 +431,7 @@ __device__ __forceinline__ void epilogue_warp(const Params& p, const Smem& sm, u
             if ((int)(d2 % kEpiGroups) != grp) continue;   // the other group's block
             // lane (h, c) handles the 16-byte piece c of rows 2i + h of its warp's 32 rows
             const int c = lane & 15, col = nc * kKC + c * 4;
-            alive = __all_sync(full, mbar_wait(sm.d2_full + b * 8, (d2 / kD2Bufs) & 1, sm.abort_flag, p.status));
+            alive = __all_sync(full, mbar_wait(sm.d2_full + b * 8, (d2 / kD2Bufs) & 1, sm.wait));
             if (!alive) break;
             tc_fence_after();
             uint32_t r0[32], r1[32];
@@ -466,7 +492,9 @@ sgmv_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CU
             mbar_init(sm.d2_full + b * 8, 1);
             mbar_init(sm.d2_empty + b * 8, 4);   // one arrival per warp of the group that drains the block
         }
-        *sm.abort_flag = 0;
+        mbar_init(sm.wind_down, 1);
+        for (int s = 0; s < kMaxStages; ++s) sm.armed[s] = 0;
+        *sm.wait.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     // The weight area of every stage starts as zeros: a rank-8 sub-tile fills 8 of the 16 rows
@@ -493,6 +521,22 @@ sgmv_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CU
     }
     tc_fence_before();
     __syncthreads();
+    if (*sm.wait.abort_flag) {
+        // A wait ran out and every role has left its loop.  Before the tensor memory is freed and the CTA's
+        // shared memory goes to another CTA, the MMAs issued so far must have completed and every copy asked
+        // for must have landed (bounded waits again; they return at once unless something is truly stuck).
+        if (warp == kMmaWarp && lane == 0) {
+            umma_commit(sm.wind_down);
+            if (!mbar_drain(sm.wind_down, 0, p.wait_cycles)) atomicCAS(p.status, 0, PLORA_ERR_TIMEOUT);
+        }
+        if (tid == 0)
+            for (int s = 0; s < p.n_stages; ++s) {
+                const uint32_t a = sm.armed[s];
+                if (a && !mbar_drain(sm.full + s * 8, ((a - 1) / p.n_stages) & 1, p.wait_cycles))
+                    atomicCAS(p.status, 0, PLORA_ERR_TIMEOUT);
+            }
+        __syncthreads();
+    }
     if (warp == kMmaWarp)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)kTmemCols) : "memory");
     if (p.defer_wait && tid == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -519,8 +563,8 @@ cudaError_t sgmv_configure() {
 }
 
 cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, int sgmv_min_rows, const void* x, float* y,
-                        bool fp16, int32_t* status, int sm_count, bool after_bgmv_of_same_call, cudaStream_t stream,
-                        int* n_launches) {
+                        bool fp16, int32_t* status, int sm_count, bool after_bgmv_of_same_call, const DebugCfg& dbg,
+                        cudaStream_t stream, int* n_launches) {
     Params p;
     p.pool = pool;
     p.bk = bk;
@@ -530,6 +574,8 @@ cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, int
     p.n_stages = stages_for(p.R);
     p.defer_wait = after_bgmv_of_same_call ? 1 : 0;
     p.fp16 = fp16 ? 1 : 0;
+    p.wait_cycles = dbg.wait_cycles > 0 ? dbg.wait_cycles : kWaitCycles;
+    p.test_hook = dbg.test_hook;
     // x as a 2-D tensor [n_tok][d_in] of bf16; a gather instruction copies 64 columns of four rows,
     // 128-byte swizzled (columns beyond d_in read as zeros)
     CUtensorMap tm, tm_box;

@@ -600,3 +600,40 @@ def test_two_pools_and_bucket_reuse():
     for key, pr in probs.items():
         assert rel_err(ys[key].cpu().numpy(), _oracle(pr)) <= TOL_FP32_PATH
     ctx.close()
+
+
+def test_ids_rewritten_in_place_between_calls_without_plora_bucket():
+    """A serving loop that refills one ids buffer every step and never calls plora_bucket: every call must
+    bucket the ids it is given (a bucket made inside a delta call serves that call only), while a bucket made
+    by plora_bucket is reused until the next plora_bucket."""
+    p = random_problem(77, T=96, d_in=256, d_out=264, ranks=[8, 16, 32, 64, 8, 16], with_minus_one=True)
+    r = Runner(p)
+    try:
+        ids_dev = r.ids.clone()
+        rng = np.random.default_rng(1)
+        for path in (P.PATH_FUSED, P.PATH_UNFUSED, P.PATH_AUTO):
+            r.ctx.set_path(path)
+            for step in range(3):
+                ids = rng.integers(-1, p["N"], size=p["T"]).astype(np.int32)
+                ids_dev.copy_(torch.from_numpy(ids))            # same address, new contents, no plora_bucket
+                y = torch.from_numpy(p["y_in"]).to(DEV)
+                n0 = r.ctx.launch_count()
+                r.ctx.lora_delta(r.x, ids_dev, 0, 0, y)
+                torch.cuda.synchronize()
+                assert r.ctx.launch_count() - n0 >= 2           # the bucket kernel ran again
+                want = oracle.lora_delta(p["x"], ids, p["ranks"], p["scales"], p["A"], p["B"], p["d_out"], p["y_in"])
+                scale = np.max(np.abs(want - p["y_in"]))
+                assert np.max(np.abs(y.cpu().numpy() - want)) <= TOL_FP32_PATH * scale + 1e-6 * np.max(np.abs(want)), (path, step)
+        # an explicit bucket is reused: the second call launches no bucket kernel
+        r.ctx.set_path(P.PATH_FUSED)
+        r.ctx.bucket(ids_dev, p["N"])
+        y = torch.zeros((p["T"], p["d_out"]), dtype=torch.float32, device=DEV)
+        r.ctx.lora_delta(r.x, ids_dev, 0, 0, y)
+        n0 = r.ctx.launch_count()
+        r.ctx.lora_delta(r.x, ids_dev, 0, 0, y)
+        per_call = r.ctx.launch_count() - n0
+        r.ctx.lora_delta(r.x, ids_dev.clone(), 0, 0, y)         # other buffer: buckets again
+        assert r.ctx.launch_count() - n0 - per_call >= per_call + 1   # + the bucket kernel (and the rank sort)
+        assert r.ctx.device_status() == 0
+    finally:
+        r.close()
