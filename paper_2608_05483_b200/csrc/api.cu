@@ -165,6 +165,7 @@ plora_status do_bucket(plora_ctx* ctx, const int32_t* ids, int32_t n_tok, int32_
     ctx->cur_ntok = n_tok;
     ctx->cur_nadapters = n_adapters;
     ctx->bucket_sgmv_min = thr;
+    ctx->dbg.maybe_empty = thr != INT_MAX;   // segments may have gone to the tensor-core path, perhaps all of them
     ctx->bucket_valid = true;
     ctx->bucket_explicit = is_explicit;
     ctx->bucket_gen = ctx->call_gen;

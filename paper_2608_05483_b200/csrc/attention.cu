@@ -95,27 +95,24 @@ __device__ __forceinline__ long long wait_limit(const int32_t* status) {
     const long long v = *reinterpret_cast<const volatile long long*>(status + kLimitWord);
     return v > 0 ? v : kWaitCycles;
 }
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
-    const long long t0 = clock64(), limit = wait_limit(status);
+// Bounded wait on an mbarrier phase; false when the CTA has given up (here or elsewhere).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
     for (;;) {
-        if (*abort_flag) return false;
-        for (int i = 0; i < 16; ++i)
+        for (int i = 0; i < 64; ++i)
             if (mbar_try_wait(bar, parity)) return true;
-        if (clock64() - t0 > limit) break;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > wait_limit(status)) break;
     }
     *abort_flag = 1;
     __threadfence_block();
     atomicCAS(status, 0, PLORA_ERR_TIMEOUT);
     return false;
 }
-// Bounded wait on an mbarrier phase; false when the CTA has given up (here or elsewhere).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
-    if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, abort_flag, status);
-}
 // The copy thread's last look at a stage before it leaves: waits whatever the abort flag says, for at
 // most the limit (a CTA must not retire with a copy still on its way into its shared memory).
-__device__ __noinline__ bool mbar_drain(uint32_t bar, uint32_t parity, long long limit) {
+__device__ __forceinline__ bool mbar_drain(uint32_t bar, uint32_t parity, long long limit) {
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity))
         if (clock64() - t0 > limit) return false;
@@ -318,7 +315,9 @@ partial_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     bool alive = true;
     // test hook: warp 0 never hands a stage back, so the copy thread's wait for a free stage runs out
     const bool withhold = warp == 0 && p.w.status[kHookWord] == PLORA_HOOK_WITHHOLD_RELEASE;
-    // (every decision to stop is a vote: the lanes of a warp meet in shuffles and must leave together)
+    // A lane whose wait for a stage fails leaves the loop and, with it, the kernel, without another
+    // warp-level operation (shuffles and warp barriers are defined over the lanes that have not exited);
+    // at the meetings, which are rare, the warp votes so that its lanes go on or stop together.
     auto consumer_meet = [&]() {
         __syncwarp();
         if (lane == 0) mbar_arrive(meet);
@@ -327,7 +326,7 @@ partial_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     };
     for (uint32_t it = 0; alive; ++it) {
         const uint32_t slot = it % kStages;
-        if (!__all_sync(0xffffffffu, mbar_wait(full + slot * 8, (it / kStages) & 1, abort_flag, p.w.status))) break;
+        if (!mbar_wait(full + slot * 8, (it / kStages) & 1, abort_flag, p.w.status)) break;
         const uint32_t st = slots + slot * kSlotBytes;
         const uint4 hw = lds128(st + kHdrOffset);
         StageHdr h;

@@ -88,6 +88,7 @@ struct Params {
     int32_t runs_a, runs_b;   // tasks per unit in the shrink / expand phase
     int32_t runs_a_sliced;    // column runs per unit when the launch cuts its units into row slices
     int32_t early_tables;     // the bucket tables were complete before the previous kernel of the stream began
+    int32_t maybe_empty;      // the batch may have sent every segment to the tensor-core path: look before setting up
     int32_t by_class;         // the launch walks its class's part of bk.cls_list (pools of mixed ranks)
     // The class launches of one call work on different units: a later one need not wait for the
     // one before it.  It joins the stream order only when its CTAs are done (so that its completion
@@ -131,32 +132,34 @@ __device__ __forceinline__ void give_up(volatile int* abort_flag, int32_t* statu
     atomicCAS(status, 0, PLORA_ERR_TIMEOUT);
 }
 // Bounded wait on an mbarrier phase.  True: the phase is complete.  False: the wait ran out, here
-// (then the status word says so) or in another role of this CTA (the abort flag); the caller stops
-// what it is doing: consumers leave their loop, the copy warp issues nothing more.
+// (then the status word says so) or in another role of this CTA (the abort flag).  What the caller
+// does with a false: a consumer lane leaves the kernel at once, executing no warp-level operation on
+// its way out (the lanes of a warp may get different answers in the instant a give-up happens, and
+// the shuffles and warp barriers further on are defined over the lanes that have not exited); the
+// copy warp and the gather warp let one lane decide and broadcast it, and stop issuing.
 struct WaitCtl {
     volatile int* abort_flag;
     int32_t* status;
     long long limit;
 };
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, const WaitCtl& w) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtl& w) {
+    if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
-        if (*w.abort_flag) return mbar_try_wait(bar, parity);
-        for (int i = 0; i < 16; ++i)
+        for (int i = 0; i < 256; ++i)
             if (mbar_try_wait(bar, parity)) return true;
+        if (*w.abort_flag) return false;
         if (clock64() - t0 > w.limit) break;
     }
     give_up(w.abort_flag, w.status);
     return false;
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtl& w) {
-    if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, w);
-}
 // The copy warp's last look at a stage before it leaves: has everything it asked for arrived?  Waits
 // whatever the abort flag says, for at most the limit (a CTA must not retire with a bulk copy still on
 // its way into its shared memory).
-__device__ __noinline__ bool mbar_drain(uint32_t bar, uint32_t parity, long long limit) {
+// (Inlined on purpose, like every wait here: a real call anywhere in the kernel made the whole kernel slower, 1.6 % on
+// the 7B decode step for this one, 4 % for a called slow path of mbar_wait.)
+__device__ __forceinline__ bool mbar_drain(uint32_t bar, uint32_t parity, long long limit) {
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity))
         if (clock64() - t0 > limit) return false;
@@ -575,7 +578,7 @@ struct ExpandMap {
 };
 
 template <int MODE, int RP, int CNT, bool H>
-__device__ __forceinline__ void expand_tile_cnt(const Params& p, const Smem& sm, const StageHdr& h,
+__device__ __forceinline__ bool expand_tile_cnt(const Params& p, const Smem& sm, const StageHdr& h,
                                                 const ExpandMap<RP>& mp, uint32_t tile, uint32_t empty_bar, int lane) {
     using M = ExpandMap<RP>;
     // Interleaved: group g takes the rows g + RG * j, and the address of this lane's pair in row j is
@@ -586,8 +589,7 @@ __device__ __forceinline__ void expand_tile_cnt(const Params& p, const Smem& sm,
                                      : tile + mp.b_col + mp.rg * M::RPG * 128;
     const int m_slot = h.m_seq % kMRing;
     if (MODE == kFused && (h.flags & kFlagFirst))   // the gather warp has assembled this task's m
-        if (!__all_sync(0xffffffffu, mbar_wait(sm.m_full + m_slot * 8, (h.m_seq / kMRing) & 1, sm.wait)))
-            return;   // gave up: nothing of this tile reaches y
+        if (!mbar_wait(sm.m_full + m_slot * 8, (h.m_seq / kMRing) & 1, sm.wait)) return false;   // gave up: nothing of this tile reaches y
     // fused: m in the m ring, group-major, so the group's rows are RPG consecutive floats per token;
     // expand-only: the caller's m next to the tile, in natural order
     const uint32_t mb = MODE == kFused ? sm.m_ring + m_slot * kMRingBytes + mp.rg * M::RPG * 4 : tile + kTileBytesMax;
@@ -668,16 +670,17 @@ __device__ __forceinline__ void expand_tile_cnt(const Params& p, const Smem& sm,
         for (int t = 0; t < CNT; ++t)
             red_add_v2(p.y_g[h.group] + (size_t)h.tok[t] * p.pool.d_out + col, out[t][0] * h.scale, out[t][1] * h.scale);
     }
+    return true;
 }
 
 template <int MODE, int RP, bool H>
-__device__ __forceinline__ void expand_tile(const Params& p, const Smem& sm, const StageHdr& h, const ExpandMap<RP>& mp,
+__device__ __forceinline__ bool expand_tile(const Params& p, const Smem& sm, const StageHdr& h, const ExpandMap<RP>& mp,
                                             uint32_t tile, uint32_t empty_bar, int lane) {
     switch (h.cnt) {
-        case 1: expand_tile_cnt<MODE, RP, 1, H>(p, sm, h, mp, tile, empty_bar, lane); break;
-        case 2: expand_tile_cnt<MODE, RP, 2, H>(p, sm, h, mp, tile, empty_bar, lane); break;
-        case 3: expand_tile_cnt<MODE, RP, 3, H>(p, sm, h, mp, tile, empty_bar, lane); break;
-        default: expand_tile_cnt<MODE, RP, 4, H>(p, sm, h, mp, tile, empty_bar, lane); break;
+        case 1: return expand_tile_cnt<MODE, RP, 1, H>(p, sm, h, mp, tile, empty_bar, lane);
+        case 2: return expand_tile_cnt<MODE, RP, 2, H>(p, sm, h, mp, tile, empty_bar, lane);
+        case 3: return expand_tile_cnt<MODE, RP, 3, H>(p, sm, h, mp, tile, empty_bar, lane);
+        default: return expand_tile_cnt<MODE, RP, 4, H>(p, sm, h, mp, tile, empty_bar, lane);
     }
 }
 
@@ -732,8 +735,9 @@ struct LaneMaps {
 };
 
 // One stage, consumer side.
+// (false: this lane gave up inside the stage)
 template <int MODE, int RP, bool H, bool TC>
-__device__ __forceinline__ void consume_stage(const Params& p, const Smem& sm, const StageHdr& h,
+__device__ __forceinline__ bool consume_stage(const Params& p, const Smem& sm, const StageHdr& h,
                                               const LaneMaps<RP, SliceCfg<MODE, RP>::kSliceRp>& maps, uint32_t tile, uint32_t empty_bar,
                                               float (&acc)[kMaxRowsPerLane][kTokChunk], int warp, int lane) {
     if (!(h.flags & kFlagExpand)) {
@@ -772,29 +776,33 @@ __device__ __forceinline__ void consume_stage(const Params& p, const Smem& sm, c
             }
         }
     } else {
-        if (MODE != kShrinkOnly) {
-            expand_tile<MODE, RP, H>(p, sm, h, maps.e, tile, empty_bar, lane);
-        }
+        if (MODE != kShrinkOnly) return expand_tile<MODE, RP, H>(p, sm, h, maps.e, tile, empty_bar, lane);
     }
+    return true;
 }
 
 // Consumes stages from stage `it` on for as long as they belong to padded rank RP (a one-class
 // launch: to the end).  Returns true when stage `it` is another class's (it has not been touched),
-// false when nothing follows or the kernel gave up.
+// false when nothing follows or this lane gave up (gave_up: it must leave the kernel now).
 template <int MODE, int RP, bool H, bool ONLY>
-__device__ __forceinline__ bool consume_class(const Params& p, const Smem& sm, uint32_t& it,
+__device__ __forceinline__ bool consume_class(const Params& p, const Smem& sm, uint32_t& it, bool& gave_up,
                                               float (&acc)[kMaxRowsPerLane][kTokChunk], int warp, int lane) {
     LaneMaps<RP, SliceCfg<MODE, RP>::kSliceRp> maps;   // per-lane constants of both phases
     maps.init(warp, lane);
     for (;; ++it) {
         const uint32_t slot = it % kStages;
-        // (the vote makes the decision the same in every lane: the code below meets in shuffles)
-        if (!__all_sync(0xffffffffu, mbar_wait(sm.full + slot * 8, (it / kStages) & 1, sm.wait))) return false;
+        if (!mbar_wait(sm.full + slot * 8, (it / kStages) & 1, sm.wait)) {
+            gave_up = true;
+            return false;
+        }
         const uint32_t tile = sm.slots + slot * kSlotBytes;
         const StageHdr h = read_hdr(tile + kHdrOffset);
         if (h.flags & kFlagEnd) return false;
         if (!ONLY && h.rp != RP) return true;
-        consume_stage<MODE, RP, H, ONLY>(p, sm, h, maps, tile, sm.empty + slot * 8, acc, warp, lane);
+        if (!consume_stage<MODE, RP, H, ONLY>(p, sm, h, maps, tile, sm.empty + slot * 8, acc, warp, lane)) {
+            gave_up = true;
+            return false;
+        }
     }
 }
 
@@ -1100,19 +1108,15 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     sm.withhold = p.test_hook == PLORA_HOOK_WITHHOLD_RELEASE && warp == 0;
-    if (MODE != kShrinkOnly && p.early_tables) {
-        // A launch that has nothing to do (every segment of the batch went to the tensor-core path, or
-        // the pool's rank class has no unit in this batch) leaves before it sets up its ring.  The
-        // tables it looks at are older than the previous kernel of the stream, hence complete.  It
-        // still joins the stream order, so that its completion implies that of everything before it.
-        // (The shrink-only kernel always has the rows of tokens without an adapter to clear.)
-        int n = *p.bk.n_bgmv_units;
-        // (the class launch that advances the epoch for its call stays: the other classes' words need it)
-        if (n != 0 && RPK && p.by_class && !(MODE == kFused && p.bump_epoch)) {
-            constexpr int kClass = RPK == 8 ? 0 : RPK == 16 ? 1 : RPK == 32 ? 2 : RPK == 64 ? 3 : 4;
-            n = p.bk.cls_start[kClass + 1] - p.bk.cls_start[kClass];
-        }
-        if (n == 0) {
+    if (MODE != kShrinkOnly && p.maybe_empty && p.early_tables) {
+        // A launch that has nothing to do (every segment of the batch went to the tensor-core path)
+        // leaves before it sets up its ring.  The host asks for the check only for batches that can
+        // have tensor-core segments: the load below delays the start of every CTA by a trip to L2,
+        // which the small launches of a decode step would feel.  The count is older than the previous
+        // kernel of the stream, hence complete.  The CTA still joins the stream order, so that the
+        // launch's completion implies that of everything before it.  (The shrink-only kernel always
+        // has the rows of tokens without an adapter to clear.)
+        if (*p.bk.n_bgmv_units == 0) {
             if (tid == 0) grid_dependency_wait();
             return;
         }
@@ -1400,22 +1404,23 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
     // of another class turns up (tasks are sorted by class, so a CTA switches a few times per launch).
     float acc[kMaxRowsPerLane][kTokChunk];
     uint32_t it = 0;
+    bool gave_up = false;   // this lane: from here to the end of the kernel there is no warp-level operation
     if (RPK) {
-        consume_class<MODE, RPK ? RPK : 8, H, true>(p, sm, it, acc, warp, lane);
+        consume_class<MODE, RPK ? RPK : 8, H, true>(p, sm, it, gave_up, acc, warp, lane);
     } else {
         for (bool more = true; more;) {
             // whose stage is next?  (the class's loop waits for it again: the phase is complete by then)
             const uint32_t slot = it % kStages;
-            if (!__all_sync(0xffffffffu, mbar_wait(sm.full + slot * 8, (it / kStages) & 1, sm.wait))) break;
+            if (!mbar_wait(sm.full + slot * 8, (it / kStages) & 1, sm.wait)) break;
             const int flags = (int)lds32(sm.slots + slot * kSlotBytes + kHdrOffset);
             const int rp = (int)lds32(sm.slots + slot * kSlotBytes + kHdrOffset + 36);
             if (flags & kFlagEnd) break;
             switch (rp) {
-                case 8: more = consume_class<MODE, 8, H, false>(p, sm, it, acc, warp, lane); break;
-                case 16: more = consume_class<MODE, 16, H, false>(p, sm, it, acc, warp, lane); break;
-                case 32: more = consume_class<MODE, 32, H, false>(p, sm, it, acc, warp, lane); break;
-                case 64: more = consume_class<MODE, 64, H, false>(p, sm, it, acc, warp, lane); break;
-                default: more = consume_class<MODE, 128, H, false>(p, sm, it, acc, warp, lane); break;
+                case 8: more = consume_class<MODE, 8, H, false>(p, sm, it, gave_up, acc, warp, lane); break;
+                case 16: more = consume_class<MODE, 16, H, false>(p, sm, it, gave_up, acc, warp, lane); break;
+                case 32: more = consume_class<MODE, 32, H, false>(p, sm, it, gave_up, acc, warp, lane); break;
+                case 64: more = consume_class<MODE, 64, H, false>(p, sm, it, gave_up, acc, warp, lane); break;
+                default: more = consume_class<MODE, 128, H, false>(p, sm, it, gave_up, acc, warp, lane); break;
             }
         }
     }
@@ -1503,6 +1508,7 @@ cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const
     p.wait_cycles = dbg.wait_cycles > 0 ? dbg.wait_cycles : kWaitCycles;
     p.test_hook = dbg.test_hook;
     p.early_tables = early_tables ? 1 : 0;
+    p.maybe_empty = dbg.maybe_empty ? 1 : 0;
     p.defer_wait = 0;
     p.bump_epoch = 1;
     cudaLaunchAttribute attr[1];

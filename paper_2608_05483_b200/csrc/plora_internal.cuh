@@ -121,10 +121,12 @@ struct ClassCache {
     uint64_t sig = 0;
     bool valid = false;
 };
-// Diagnostics of the bounded waits (plora_set_wait_limit, plora_set_test_hook).
+// Per-launch settings that come from the context: the diagnostics of the bounded waits
+// (plora_set_wait_limit, plora_set_test_hook) and what the host knows about the batch.
 struct DebugCfg {
     long long wait_cycles = 0;   // 0: the kernels' default
     int32_t test_hook = 0;       // PLORA_HOOK_*
+    bool maybe_empty = false;    // the bucket may hold tensor-core segments only (BGMV launches look before they set up)
 };
 cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const BucketDev& bk, int n_tok,
                         const void* const* x, float* const* y, void* m, int ldm, bool m16, bool fp16, int32_t* status,

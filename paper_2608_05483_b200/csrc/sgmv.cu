@@ -124,7 +124,7 @@ struct WaitCtl {
     int32_t* status;
     long long limit;
 };
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, const WaitCtl& w) {
+__device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, const WaitCtl& w) {
     const long long t0 = clock64();
     for (;;) {
         if (*w.abort_flag) return false;
@@ -142,7 +142,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const W
     return mbar_wait_slow(bar, parity, w);
 }
 // Winding down after a give-up: wait for a phase whatever the abort flag says, for at most the limit.
-__device__ __noinline__ bool mbar_drain(uint32_t bar, uint32_t parity, long long limit) {
+__device__ __forceinline__ bool mbar_drain(uint32_t bar, uint32_t parity, long long limit) {
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity))
         if (clock64() - t0 > limit) return false;

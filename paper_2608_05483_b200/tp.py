@@ -14,8 +14,10 @@ exchange is the small m.  Everything numerical runs in the library's shrink and 
 this module holds the index arithmetic and the call sequence, and takes the all-reduce as a
 callable (torch.distributed.all_reduce on an NCCL group in production, anything else in a test).
 
-Not measured on several GPUs: the test pool gives one GPU per call.  Covered by a two-rank gloo test
-of the arithmetic on CPU and by a one-GPU test that runs both ranks' shards one after the other.
+The benchmark's --tp mode runs this wave with torch.distributed.all_reduce on an NCCL group, one rank per
+GPU.  Covered by a two-rank gloo test of the arithmetic on CPU, by a one-GPU test that runs both ranks'
+shards one after the other, and by a CPU test that the wave's three steps run in order on the caller's
+stream.
 """
 from __future__ import annotations
 
@@ -79,6 +81,11 @@ class TensorParallelDelta:
         m = self._m.get(key)
         if m is None:
             m = self._m[key] = torch.empty((n_tok, ldm), dtype=torch.float32, device=x_shard.device)
-        self.ctx.shrink(x_shard, ids, layer, proj, m, stream=stream)
-        self.all_reduce(m)
-        self.ctx.expand(m, ids, layer, proj, y_shard, stream=stream)
+        # All three steps are queued on one stream, in this order.  torch.distributed orders a collective
+        # against the stream that is current when it is called, so a caller's stream is made current for the
+        # whole wave: the all-reduce then starts after the shrink kernel and the expand kernel after the sum.
+        import contextlib
+        with (torch.cuda.stream(stream) if stream is not None else contextlib.nullcontext()):
+            self.ctx.shrink(x_shard, ids, layer, proj, m, stream=stream)
+            self.all_reduce(m)
+            self.ctx.expand(m, ids, layer, proj, y_shard, stream=stream)

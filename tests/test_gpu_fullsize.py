@@ -63,3 +63,20 @@ def test_algorithmic_bytes_of_the_decode_config():
     b = algorithmic_bytes(wl.ids, wl.ranks, 4096, 4096)
     assert b["adapter"] == b["distinct"] * (4096 + 4096) * 16 * 2
     assert b["x"] == 256 * 4096 * 2 and b["y"] == 256 * 4096 * 8
+
+
+@pytest.mark.parametrize("cfg", [2, 3, 4, 5, 6])
+def test_whole_output_of_one_projection_per_shape(cfg):
+    """Every element of the [n_tok, d_out] output, for the first projection of each distinct shape, through the
+    call the benchmark's step makes (q goes with its k and v), against the oracle at full size."""
+    from bench import oracle_sample, parity_pools
+    wl = make_workload(cfg, n_layers=1)
+    dw = DeviceWorkload(wl, 0)
+    try:
+        dw.ctx.set_path(P.PATH_AUTO)
+        pools, _, err, _, _ = oracle_sample(dw, 0, check_gpu=True, pools=parity_pools(wl))
+        assert len(pools) == (3 if cfg == 3 else 1)
+        assert err <= TOL_FP32_PATH, (cfg, err)
+        assert dw.ctx.device_status() == 0
+    finally:
+        dw.close()

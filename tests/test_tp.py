@@ -160,3 +160,44 @@ def test_both_shards_through_the_kernels_on_one_gpu(world):
     assert np.max(np.abs(got - ref)) <= TOL_FP32_PATH * delta + 1e-6 * np.max(np.abs(ref))
     for tp in ranks_tp:
         tp.ctx.close()
+
+
+def test_the_wave_runs_its_three_steps_in_order_on_the_callers_stream(monkeypatch):
+    """The all-reduce must be called between the two kernels while the caller's stream is the current one
+    (torch.distributed orders a collective against the current stream)."""
+    import contextlib
+
+    log = []
+
+    class FakeCtx:
+        def pool_max_rank(self, layer, proj):
+            return 8
+
+        def shrink(self, x, ids, layer, proj, m, stream=None):
+            log.append(("shrink", stream, current[0]))
+
+        def expand(self, m, ids, layer, proj, y, stream=None):
+            log.append(("expand", stream, current[0]))
+
+    current = [None]
+
+    @contextlib.contextmanager
+    def fake_stream_ctx(s):
+        prev, current[0] = current[0], s
+        try:
+            yield
+        finally:
+            current[0] = prev
+
+    monkeypatch.setattr(torch.cuda, "stream", fake_stream_ctx)
+    tp = TensorParallelDelta(FakeCtx(), 0, 2, all_reduce=lambda m: log.append(("all_reduce", None, current[0])))
+    x = torch.zeros((4, 16))
+    ids = torch.zeros(4, dtype=torch.int32)
+    y = torch.zeros((4, 16))
+    mine = object()
+    tp.lora_delta(x, ids, 0, 0, y, stream=mine)
+    assert [e[0] for e in log] == ["shrink", "all_reduce", "expand"]
+    assert all(e[2] is mine for e in log) and log[0][1] is mine and log[2][1] is mine
+    log.clear()
+    tp.lora_delta(x, ids, 0, 0, y)            # no stream given: nothing is made current
+    assert [e[0] for e in log] == ["shrink", "all_reduce", "expand"] and all(e[2] is None for e in log)
