@@ -65,11 +65,13 @@ enum {
 
 /* Which kernels plora_lora_delta uses. */
 enum {
-    PLORA_PATH_AUTO = 0,    /* fused BGMV for short segments; in batches of 512+ tokens SGMV takes the long
-                               ones, provided they make at least 128 tiles of 64 rows together */
+    PLORA_PATH_AUTO = 0,    /* fused BGMV for short segments; in batches of 512+ tokens the tensor-core
+                               segmented GEMM takes the long ones: a CTA per tile of 64 rows when they make
+                               at least 128 tiles together, a cluster of eight CTAs per tile when fewer */
     PLORA_PATH_UNFUSED = 1, /* BGMV shrink kernel then BGMV expand kernel, m in HBM workspace */
     PLORA_PATH_FUSED = 2,   /* fused BGMV for every segment */
-    PLORA_PATH_SGMV = 3     /* tensor-core segmented GEMM for every segment */
+    PLORA_PATH_SGMV = 3,    /* tensor-core segmented GEMM for every segment, a CTA per tile */
+    PLORA_PATH_SGMV_SPLIT = 4 /* tensor-core segmented GEMM for every segment, a cluster of eight CTAs per tile */
 };
 
 /*

@@ -25,7 +25,7 @@ ERR_CUDA = -5
 ERR_TIMEOUT = -6
 ERR_UNSUPPORTED = -7
 
-PATH_AUTO, PATH_UNFUSED, PATH_FUSED, PATH_SGMV = 0, 1, 2, 3
+PATH_AUTO, PATH_UNFUSED, PATH_FUSED, PATH_SGMV, PATH_SGMV_SPLIT = 0, 1, 2, 3, 4
 
 EXPORTS = (
     "plora_create", "plora_destroy", "plora_pool_slab_bytes", "plora_register_pool", "plora_pool_max_rank",

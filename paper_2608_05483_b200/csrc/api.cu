@@ -142,30 +142,49 @@ size_t layout_pool(const plora_pool_desc* d, std::vector<AdapterEntry>* table, i
 
 int32_t effective_sgmv_min(const plora_ctx* ctx, int32_t n_tok) {
     switch (ctx->path) {
-        case PLORA_PATH_SGMV: return 1;
-        case PLORA_PATH_AUTO:
-            // kSgmvMinTiles tiles hold at least kSgmvMinTiles * sgmv_min_rows tokens: a smaller batch
-            // cannot have a tensor-core segment, and is spared the launch that would find none
-            return n_tok >= kSgmvMinBatch && (long long)n_tok >= (long long)kSgmvMinTiles * ctx->sgmv_min_rows
-                       ? ctx->sgmv_min_rows
-                       : INT_MAX;
+        case PLORA_PATH_SGMV:
+        case PLORA_PATH_SGMV_SPLIT: return 1;
+        case PLORA_PATH_AUTO: return n_tok >= kSgmvMinBatch ? ctx->sgmv_min_rows : INT_MAX;
         default: return INT_MAX;
     }
+}
+
+// Which tensor-core launches a call makes.  The wide shape needs kSgmvMinTiles tiles, which hold at least
+// kSgmvMinTiles * sgmv_min_rows tokens: a smaller batch cannot reach it and is spared the launch that would find
+// no tile.  The host does not know how many tiles a batch has; of the two launches of a large batch one finds none.
+bool wide_launch(const plora_ctx* ctx, int32_t n_tok) {
+    if (ctx->path == PLORA_PATH_SGMV) return true;
+    return ctx->path == PLORA_PATH_AUTO && ctx->bucket_sgmv_min != INT_MAX &&
+           (long long)n_tok >= (long long)kSgmvMinTiles * ctx->bucket_sgmv_min;
+}
+// under AUTO the bucket kernel sends kSgmvMinTiles tiles or more to the wide shape
+int split_max_tiles(const plora_ctx* ctx) { return ctx->path == PLORA_PATH_AUTO ? kSgmvMinTiles - 1 : INT_MAX; }
+// AUTO: the split shape serves the batches that are too small for the wide one.  (Launching both for a large batch
+// and letting the bucket kernel's tile count decide cost the prefill step 5 %: a launch of up to 127 clusters that
+// all find nothing still takes 6 us.  A large batch whose long segments make fewer than kSgmvMinTiles tiles keeps
+// them on BGMV.)
+bool split_launch(const plora_ctx* ctx, int32_t n_tok) {
+    return ctx->path == PLORA_PATH_SGMV_SPLIT ||
+           (ctx->path == PLORA_PATH_AUTO && ctx->bucket_sgmv_min != INT_MAX && !wide_launch(ctx, n_tok));
 }
 
 plora_status do_bucket(plora_ctx* ctx, const int32_t* ids, int32_t n_tok, int32_t n_adapters, cudaStream_t st,
                        bool is_explicit) {
     const int32_t thr = effective_sgmv_min(ctx, n_tok);
     int nl = 0;
-    cudaError_t e = launch_bucket(ids, n_tok, n_adapters, thr, ctx->path == PLORA_PATH_AUTO ? kSgmvMinTiles : 0, ctx->bk,
-                                  ctx->status_dev, st, &nl);
+    const int min_tiles = ctx->path == PLORA_PATH_AUTO ? kSgmvMinTiles : ctx->path == PLORA_PATH_SGMV_SPLIT ? INT_MAX : 0;
+    const bool split_ok = ctx->path == PLORA_PATH_SGMV_SPLIT ||
+                          (ctx->path == PLORA_PATH_AUTO && thr != INT_MAX && (long long)n_tok < (long long)kSgmvMinTiles * thr);
+    cudaError_t e = launch_bucket(ids, n_tok, n_adapters, thr, min_tiles, split_ok, ctx->bk, ctx->status_dev, st, &nl);
     ctx->launches += nl;
     if (e != cudaSuccess) { ctx->bucket_valid = false; return PLORA_ERR_CUDA; }
     ctx->cur_ids = ids;
     ctx->cur_ntok = n_tok;
     ctx->cur_nadapters = n_adapters;
     ctx->bucket_sgmv_min = thr;
-    ctx->dbg.maybe_empty = thr != INT_MAX;   // segments may have gone to the tensor-core path, perhaps all of them
+    // every segment may have gone to the tensor-core path (a prefill batch): the BGMV launches then look before they
+    // set up; a smaller batch always keeps short segments, and is spared the look
+    ctx->dbg.maybe_empty = thr != INT_MAX && (long long)n_tok >= (long long)kSgmvMinTiles * thr;
     ctx->bucket_valid = true;
     ctx->bucket_explicit = is_explicit;
     ctx->bucket_gen = ctx->call_gen;
@@ -264,6 +283,7 @@ PLORA_API plora_status plora_create(plora_ctx** out, int device, int32_t max_tok
     ctx->bk.n_active = scal + 1;
     ctx->bk.n_bgmv_units = scal + 2;
     ctx->bk.n_sgmv_tiles = scal + 3;
+    ctx->bk.sgmv_split = scal + 4;
     ctx->status_dev = scal + 8;
     ctx->bk.bgmv_units = (WorkUnit*)(blk + o_bg);
     ctx->bk.sgmv_tiles = (WorkUnit*)(blk + o_sg);
@@ -435,7 +455,7 @@ PLORA_API plora_status plora_bucket_view(plora_ctx* ctx, const int32_t** perm, c
 }
 
 PLORA_API plora_status plora_set_path(plora_ctx* ctx, int32_t path, int32_t sgmv_min_rows) {
-    if (!ctx || path < PLORA_PATH_AUTO || path > PLORA_PATH_SGMV || sgmv_min_rows < 0) return PLORA_ERR_INVALID_ARG;
+    if (!ctx || path < PLORA_PATH_AUTO || path > PLORA_PATH_SGMV_SPLIT || sgmv_min_rows < 0) return PLORA_ERR_INVALID_ARG;
     ctx->path = path;
     ctx->sgmv_min_rows = sgmv_min_rows > 0 ? sgmv_min_rows : kDefaultSgmvMinRows;
     return PLORA_OK;
@@ -488,12 +508,13 @@ plora_status delta_one(plora_ctx* ctx, const void* x, const int32_t* ids, int32_
                             ctx->status_dev, ctx->sm_count, ctx->launches_since_bucket++ > 0, &ctx->cls_cache, pool->rank_sig, st, &nl, false, ctx->fp16, ctx->dbg);
     } else {
         // a batch shorter than the threshold cannot hold a segment for the tensor-core path
-        const bool may_bgmv = ctx->path != PLORA_PATH_SGMV;
-        const bool may_sgmv = ctx->bucket_sgmv_min != INT_MAX;
+        const bool may_bgmv = ctx->path != PLORA_PATH_SGMV && ctx->path != PLORA_PATH_SGMV_SPLIT;
         if (may_bgmv)
             e = launch_bgmv_one(kFused, pool->dev, ctx->bk, n_tok, x, y, nullptr, 0, ctx->status_dev, ctx->sm_count, ctx->launches_since_bucket++ > 0, &ctx->cls_cache, pool->rank_sig, st, &nl, false, ctx->fp16, ctx->dbg);
-        if (e == cudaSuccess && may_sgmv)
-            e = launch_sgmv(pool->dev, ctx->bk, n_tok, ctx->bucket_sgmv_min, x, y, ctx->fp16, ctx->status_dev, ctx->sm_count, may_bgmv, ctx->dbg, st, &nl);
+        if (e == cudaSuccess && wide_launch(ctx, n_tok))
+            e = launch_sgmv(pool->dev, ctx->bk, n_tok, ctx->bucket_sgmv_min, x, y, ctx->fp16, ctx->status_dev, ctx->sm_count, may_bgmv, false, 0, ctx->dbg, st, &nl);
+        if (e == cudaSuccess && split_launch(ctx, n_tok))
+            e = launch_sgmv(pool->dev, ctx->bk, n_tok, ctx->bucket_sgmv_min, x, y, ctx->fp16, ctx->status_dev, ctx->sm_count, may_bgmv || wide_launch(ctx, n_tok), true, split_max_tiles(ctx), ctx->dbg, st, &nl);
     }
     ctx->launches += nl;
     return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
@@ -527,7 +548,7 @@ PLORA_API plora_status plora_lora_delta_group(plora_ctx* ctx, int32_t n, const v
                recs[g]->dev.n_adapters == recs[0]->dev.n_adapters && recs[g]->dev.max_rp == recs[0]->dev.max_rp &&
                recs[g]->dev.rp_mask == recs[0]->dev.rp_mask &&
                (recs[g]->rank_sig == recs[0]->rank_sig || (recs[0]->dev.rp_mask & (recs[0]->dev.rp_mask - 1)) == 0);
-    if (!same || ctx->path == PLORA_PATH_UNFUSED || ctx->path == PLORA_PATH_SGMV) {
+    if (!same || ctx->path == PLORA_PATH_UNFUSED || ctx->path == PLORA_PATH_SGMV || ctx->path == PLORA_PATH_SGMV_SPLIT) {
         // pools of different shape, or a path without a grouped kernel: one projection after the other
         for (int g = 0; g < n; ++g) {
             plora_status rc = delta_one(ctx, x[g], ids, n_tok, layers[g], projs[g], y[g], stream);
@@ -545,9 +566,10 @@ PLORA_API plora_status plora_lora_delta_group(plora_ctx* ctx, int32_t n, const v
     int nl = 0;
     cudaError_t e = launch_bgmv(kFused, pools, n, ctx->bk, n_tok, x, y, nullptr, 0, false, ctx->fp16, ctx->status_dev, ctx->sm_count,
                                 ctx->launches_since_bucket++ > 0, &ctx->cls_cache, recs[0]->rank_sig, ctx->dbg, st, &nl);
-    if (e == cudaSuccess && ctx->bucket_sgmv_min != INT_MAX)
-        for (int g = 0; g < n && e == cudaSuccess; ++g)
-            e = launch_sgmv(pools[g], ctx->bk, n_tok, ctx->bucket_sgmv_min, x[g], y[g], ctx->fp16, ctx->status_dev, ctx->sm_count, true, ctx->dbg, st, &nl);
+    for (int g = 0; g < n && e == cudaSuccess && wide_launch(ctx, n_tok); ++g)
+        e = launch_sgmv(pools[g], ctx->bk, n_tok, ctx->bucket_sgmv_min, x[g], y[g], ctx->fp16, ctx->status_dev, ctx->sm_count, true, false, 0, ctx->dbg, st, &nl);
+    for (int g = 0; g < n && e == cudaSuccess && split_launch(ctx, n_tok); ++g)
+        e = launch_sgmv(pools[g], ctx->bk, n_tok, ctx->bucket_sgmv_min, x[g], y[g], ctx->fp16, ctx->status_dev, ctx->sm_count, true, true, split_max_tiles(ctx), ctx->dbg, st, &nl);
     ctx->launches += nl;
     return e == cudaSuccess ? PLORA_OK : PLORA_ERR_CUDA;
 }

@@ -77,7 +77,7 @@ __device__ void write_units(WorkUnit* out, int n_units, const int* ustart, const
 
 __global__ void __launch_bounds__(kThreads, 1)
 bucket_kernel(const int32_t* __restrict__ ids, int T, int N, int nch, int sgmv_min_rows, int sgmv_min_tiles,
-              BucketDev bk, int32_t* status) {
+              int split_ok, BucketDev bk, int32_t* status) {
     extern __shared__ int smem[];
     const int nb = N + 1;                 // bins: ids 0..N-1, then "no adapter"
     int* cnt = smem;                      // [nch][nb]   per-chunk counts, later per-chunk cursors
@@ -124,10 +124,13 @@ bucket_kernel(const int32_t* __restrict__ ids, int T, int N, int nch, int sgmv_m
     block_exclusive_scan(start, nb, wsum);
     if (tid == 0) start[nb] = T;
     const int n_seg = block_exclusive_scan(segidx, nb, wsum);
-    // Long segments go to the tensor-core path only if together they make enough tiles to occupy
-    // the GPU; a handful of tiles would each be one long serial job, so they stay with BGMV.
+    // Long segments go to the tensor-core path.  If together they make enough tiles to occupy the
+    // GPU, a CTA takes whole tiles (wide shape); a handful of tiles would each be one long serial
+    // job, so they go to the split shape (a cluster of CTAs per tile) where the caller has it, and
+    // stay with BGMV otherwise.
     const int n_sg_cand = block_exclusive_scan(usg, nb, wsum);
-    const bool use_sg = n_sg_cand >= sgmv_min_tiles;
+    const bool wide = n_sg_cand >= sgmv_min_tiles;
+    const bool use_sg = wide || (split_ok && n_sg_cand > 0);
     const int n_sg = use_sg ? n_sg_cand : 0;
     for (int b = tid; b < nb; b += kThreads) {
         const int run = total[b];
@@ -176,6 +179,7 @@ bucket_kernel(const int32_t* __restrict__ ids, int T, int N, int nch, int sgmv_m
         *bk.n_active = n_active;
         *bk.n_bgmv_units = n_bg;
         *bk.n_sgmv_tiles = n_sg;
+        *bk.sgmv_split = (use_sg && !wide) ? 1 : 0;
     }
     __syncthreads();   // perm is complete (written by this block) before the units quote it
     write_units(bk.bgmv_units, n_bg, ubg, start, total, segidx, N, kTokChunk, bk.perm);
@@ -199,12 +203,12 @@ int bucket_max_adapters() {
 }
 
 cudaError_t launch_bucket(const int32_t* ids, int n_tok, int n_adapters, int sgmv_min_rows, int sgmv_min_tiles,
-                          BucketDev bk, int32_t* status, cudaStream_t stream, int* n_launches) {
+                          bool split_ok, BucketDev bk, int32_t* status, cudaStream_t stream, int* n_launches) {
     int nch = kWarps;
     while (nch > 1 && bucket_smem_bytes(n_adapters, nch) > kBucketSmemLimit) nch >>= 1;
     const size_t smem = bucket_smem_bytes(n_adapters, nch);
     if (smem > kBucketSmemLimit) return cudaErrorInvalidValue;
-    bucket_kernel<<<1, kThreads, smem, stream>>>(ids, n_tok, n_adapters, nch, sgmv_min_rows, sgmv_min_tiles, bk, status);
+    bucket_kernel<<<1, kThreads, smem, stream>>>(ids, n_tok, n_adapters, nch, sgmv_min_rows, sgmv_min_tiles, split_ok ? 1 : 0, bk, status);
     ++*n_launches;
     return cudaGetLastError();
 }

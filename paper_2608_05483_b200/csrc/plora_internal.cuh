@@ -86,6 +86,7 @@ struct BucketDev {
     int32_t* n_bgmv_units;
     WorkUnit* sgmv_tiles;
     int32_t* n_sgmv_tiles;
+    int32_t* sgmv_split;    // 1: the tiles are few and go to the split launch shape (a cluster per tile), 0: to the wide one
     // cross-CTA hand-over of the fused BGMV kernel: every partial m value travels as one
     // 64-bit word {value, launch epoch}, so a reader can tell on its own whether it has arrived
     unsigned long long* m_part;
@@ -100,8 +101,10 @@ struct BucketDev {
 constexpr int kRankClasses = 5;   // padded ranks 8, 16, 32, 64, 128
 
 // Launchers (each returns the cudaError_t of its launch).
+// sgmv_min_tiles: from this many tensor-core tiles on they go to the wide launch shape; fewer go to the split
+// shape if split_ok, else their segments stay with BGMV
 cudaError_t launch_bucket(const int32_t* ids, int n_tok, int n_adapters, int sgmv_min_rows, int sgmv_min_tiles,
-                          BucketDev bk, int32_t* status, cudaStream_t stream, int* n_launches);
+                          bool split_ok, BucketDev bk, int32_t* status, cudaStream_t stream, int* n_launches);
 cudaError_t launch_repack(const AdapterEntry* table_dev, const void* const* A_dev, const void* const* B_dev,
                           int n_adapters, int d_in, int d_out, uint8_t* slab, cudaStream_t stream, int* n_launches);
 
@@ -135,8 +138,8 @@ cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const
 // after_bgmv_of_same_call: the launch follows fused BGMV launches of the same call (other tokens of the
 // same batch) and may overlap them
 cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, int sgmv_min_rows, const void* x, float* y,
-                        bool fp16, int32_t* status, int sm_count, bool after_bgmv_of_same_call, const DebugCfg& dbg,
-                        cudaStream_t stream, int* n_launches);
+                        bool fp16, int32_t* status, int sm_count, bool after_bgmv_of_same_call, bool split,
+                        int split_max_tiles, const DebugCfg& dbg, cudaStream_t stream, int* n_launches);
 // per-device function attributes (dynamic shared memory); called by plora_create
 cudaError_t bucket_configure();
 cudaError_t bgmv_configure();

@@ -27,6 +27,16 @@
 // bound by HBM traffic on the activations (x read once, y updated once), not by the tensor
 // pipe.  Every wait is bounded: when one runs out the kernel records PLORA_ERR_TIMEOUT, every
 // role leaves its loop, and the tensor memory is freed before the CTA exits.
+//
+// Two launch shapes share the code.  Wide: persistent CTAs, a CTA runs whole tiles (a batch with
+// enough tiles to occupy the GPU, prefill).  Split: a batch with only a handful of long segments
+// (the paper's per-adapter batches go up to 256 requests, Section V-A, also inside an otherwise
+// decode-shaped step) gives too few tiles for that, and a tile is a long serial job.  There a
+// thread-block cluster of kClusterSize CTAs takes one tile: CTA c shrinks over its eighth of d_in,
+// the partial m of the cluster meet through distributed shared memory (each CTA sums eight of the
+// 64 rows in a fixed order, scales, splits into hi + lo and stores the finished rows into every
+// CTA's operand buffers), and CTA c expands its eighth of d_out.  Every CTA fetches its own
+// operands; nothing is multicast.
 #include <cuda.h>
 #include <cuda_fp16.h>
 
@@ -62,6 +72,8 @@ constexpr int kStagingBytes = kEpiWarps * kRowsPerWarp * kStagePitch;
 constexpr int kSmemBudget = 227 * 1024;                    // of an SM
 constexpr int kSmemPerCta = kSmemBudget / 2 - 1024;        // two CTAs per SM, so that one tile's shrink overlaps another's expand
 constexpr long long kWaitCycles = 4000000000ll;            // default limit of a wait: about two seconds of SM clock
+constexpr int kClusterSize = 8;                            // split shape: CTAs per tile
+constexpr int kRedRows = kRows / kClusterSize;             // rows of the tile a CTA of the cluster sums
 
 // Shared memory, sized for R = max(16, largest padded rank of the pool):
 //   ring of n_stages x (x block 8 KiB + weight sub-tile R x 128 B)       1024-byte aligned
@@ -71,13 +83,16 @@ __host__ __device__ inline int w_stage_bytes(int R) { return R * 128; }
 __host__ __device__ inline int stage_bytes(int R) { return kXStageBytes + w_stage_bytes(R); }
 __host__ __device__ inline int m_bytes(int R) { return (R / 8) * kRows * 16; }
 constexpr int kTailBytes = kStagingBytes + kRows * 4 + 256;
-__host__ __device__ inline int stages_for(int R) {
-    int n = (kSmemPerCta - 1024 - kTailBytes - 2 * m_bytes(R)) / stage_bytes(R);
-    if (n < 3) n = (kSmemBudget - 1024 - kTailBytes - 2 * m_bytes(R)) / stage_bytes(R);   // rank 128: one CTA per SM
+// split shape: where the cluster's partial sums of this CTA's kRedRows rows arrive, [source CTA][row][R] floats
+__host__ __device__ inline int red_bytes(int R, bool split) { return split ? kClusterSize * kRedRows * R * 4 : 0; }
+__host__ __device__ inline int stages_for(int R, bool split) {
+    const int fixed = 1024 + kTailBytes + 2 * m_bytes(R) + red_bytes(R, split);
+    int n = (kSmemPerCta - fixed) / stage_bytes(R);
+    if (n < 3) n = (kSmemBudget - fixed) / stage_bytes(R);   // rank 128: one CTA per SM
     return n > kMaxStages ? kMaxStages : n;
 }
-__host__ __device__ inline int smem_bytes(int R) {
-    return 1024 + stages_for(R) * stage_bytes(R) + 2 * m_bytes(R) + kTailBytes;
+__host__ __device__ inline int smem_bytes(int R, bool split) {
+    return 1024 + stages_for(R, split) * stage_bytes(R) + 2 * m_bytes(R) + red_bytes(R, split) + kTailBytes;
 }
 
 struct Params {
@@ -220,6 +235,72 @@ __device__ __forceinline__ uint32_t f32_to_bf16_bits(float f) {
     return (u + 0x7fffu + ((u >> 16) & 1u)) >> 16;
 }
 
+// ---- thread-block cluster pieces of the split shape ---------------------------------------------------
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// The address, in the cluster's shared window, of `addr` (an address in this CTA's shared memory) in CTA `rank`.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void st_cluster_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared::cluster.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+// One arrival on a barrier of another CTA of the cluster; everything this thread has observed or written before
+// (its own stores, and those of the threads it has met at a CTA barrier) is visible to whoever acquires the phase.
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void fence_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
+// All threads of all CTAs of the cluster (the hardware's own barrier; used at the two ends of the kernel only, where
+// every thread is certain to arrive: after the barriers are set up, and before any CTA gives up its shared memory).
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+// What a CTA does of which tiles: the wide shape walks whole tiles, the split shape takes one tile and an
+// eighth of each of its two loops.
+struct Span {
+    int t0, t_step;      // tiles t0, t0 + t_step, ... below the tile count
+    int kc0, kc1;        // shrink stages (64 columns of d_in each)
+    int nc0, nc1;        // expand blocks (64 columns of d_out each)
+};
+template <bool SPLIT>
+__device__ __forceinline__ Span make_span(int nK, int nN) {
+    Span sp;
+    if (SPLIT) {
+        const int c = (int)cluster_rank();
+        sp.t0 = blockIdx.x / kClusterSize;
+        sp.t_step = 1 << 30;
+        sp.kc0 = c * nK / kClusterSize;
+        sp.kc1 = (c + 1) * nK / kClusterSize;
+        sp.nc0 = c * nN / kClusterSize;
+        sp.nc1 = (c + 1) * nN / kClusterSize;
+    } else {
+        sp.t0 = blockIdx.x;
+        sp.t_step = gridDim.x;
+        sp.kc0 = 0; sp.kc1 = nK;
+        sp.nc0 = 0; sp.nc1 = nN;
+    }
+    return sp;
+}
+
 struct Smem {
     uint32_t ring;        // stage 0 (1024-byte aligned); stage = x block, then the weight sub-tile
     uint32_t m_hi, m_lo;  // K-major operand of the expand, chunk kc (8 columns) of row r at kc * 2048 + r * 16
@@ -230,15 +311,19 @@ struct Smem {
     uint32_t m_ready;     // the epilogue has stored m hi / lo (and is done with the shrink accumulator)
     uint32_t d2_full, d2_empty;   // [kD2Bufs] each
     uint32_t wind_down;   // after a give-up: the MMAs issued so far have completed
+    uint32_t red;         // split shape: partial sums from the cluster (see red_bytes)
+    uint32_t part_in;     // split shape: every CTA of the cluster has delivered its partial rows (kClusterSize arrivals)
+    uint32_t m_in;        // split shape: every CTA of the cluster has delivered its finished rows of m
     WaitCtl wait;         // abort flag of the CTA, status word, limit of a wait
     uint32_t* tmem_slot;
     uint32_t* armed;      // [kMaxStages]: 1 + the running number of the stage a slot was last armed for (0: never)
 };
 
-__device__ __forceinline__ Smem carve(uint8_t* raw, const Params& p) {
+__device__ __forceinline__ Smem carve(uint8_t* raw, const Params& p, bool split) {
     uint8_t* base = raw + ((1024u - (smem_u32(raw) & 1023u)) & 1023u);
     uint8_t* m = base + p.n_stages * stage_bytes(p.R);
-    uint8_t* staging = m + 2 * m_bytes(p.R);
+    uint8_t* red = m + 2 * m_bytes(p.R);
+    uint8_t* staging = red + red_bytes(p.R, split);
     uint8_t* tok = staging + kStagingBytes;
     uint8_t* bars = tok + kRows * 4;
     Smem s;
@@ -254,7 +339,10 @@ __device__ __forceinline__ Smem carve(uint8_t* raw, const Params& p) {
     s.d2_full = s.m_ready + 8;
     s.d2_empty = s.d2_full + kD2Bufs * 8;
     s.wind_down = s.d2_empty + kD2Bufs * 8;
-    uint8_t* words = bars + (2 * kMaxStages + 3 + 2 * kD2Bufs) * 8;
+    s.part_in = s.wind_down + 8;
+    s.m_in = s.part_in + 8;
+    s.red = smem_u32(red);
+    uint8_t* words = bars + (2 * kMaxStages + 5 + 2 * kD2Bufs) * 8;
     s.wait.abort_flag = reinterpret_cast<volatile int*>(words);
     s.wait.status = p.status;
     s.wait.limit = p.wait_cycles;
@@ -267,12 +355,14 @@ __device__ __forceinline__ Smem carve(uint8_t* raw, const Params& p) {
 // Lane g owns rows 4g .. 4g + 3 of every tile: one gather instruction per lane and stage.  Rows
 // beyond the tile's count repeat its last token (their results are never written); groups that
 // lie entirely beyond it are not copied at all.
+template <bool SPLIT>
 __device__ __forceinline__ void producer_warp(const Params& p, const Smem& sm, const CUtensorMap* tm_x,
                                               const CUtensorMap* tm_box, int n_tiles, int warp, int lane) {
     const int nK = (p.pool.d_in + kKC - 1) / kKC, nN = (p.pool.d_out + kKC - 1) / kKC;
+    const Span sp = make_span<SPLIT>(nK, nN);
     const int stage = stage_bytes(p.R);
     uint32_t it = 0;
-    for (int t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+    for (int t = sp.t0; t < n_tiles; t += sp.t_step) {
         const WorkUnit wu = p.bk.sgmv_tiles[t];
         const AdapterEntry e = p.pool.table[wu.adapter];
         const int cnt = wu.cnt;
@@ -290,11 +380,13 @@ __device__ __forceinline__ void producer_warp(const Params& p, const Smem& sm, c
         const uint32_t xbytes = (uint32_t)((cnt + 3) / 4) * 512u, wbytes = (uint32_t)e.rp * 128u;
         const uint8_t* a_src = p.pool.slab + e.offA;
         const uint8_t* b_src = p.pool.slab + e.offB;
-        for (int c = 0; c < nK + nN; ++c, ++it) {
+        const int n_shrink = sp.kc1 - sp.kc0, n_all = n_shrink + sp.nc1 - sp.nc0;
+        for (int j = 0; j < n_all; ++j, ++it) {
             if ((int)(it % kProducerWarps) != warp) continue;   // another copy warp's stage
             const uint32_t slot = it % p.n_stages;
             const uint32_t dst = sm.ring + slot * stage, bar = sm.full + slot * 8;
-            const bool shrink = c < nK;
+            const bool shrink = j < n_shrink;
+            const int c = shrink ? sp.kc0 + j : nK + sp.nc0 + (j - n_shrink);   // stage number in the tile's whole sequence
             int ok = 1;
             if (lane == 0) {
                 ok = mbar_wait(sm.empty + slot * 8, ((it / p.n_stages) & 1) ^ 1, sm.wait);
@@ -317,25 +409,27 @@ __device__ __forceinline__ void producer_warp(const Params& p, const Smem& sm, c
 }
 
 // ---- MMA warp, one lane --------------------------------------------------------------------
+template <bool SPLIT>
 __device__ __forceinline__ void mma_thread(const Params& p, const Smem& sm, uint32_t tmem, int n_tiles) {
     const int nK = (p.pool.d_in + kKC - 1) / kKC, nN = (p.pool.d_out + kKC - 1) / kKC;
+    const Span sp = make_span<SPLIT>(nK, nN);
     const int stage = stage_bytes(p.R);
     uint32_t it = 0, d2 = 0, tile_idx = 0;
     const bool withhold = p.test_hook == PLORA_HOOK_WITHHOLD_RELEASE;   // test hook: shrink stages are never handed back
-    for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++tile_idx) {
+    for (int t = sp.t0; t < n_tiles; t += sp.t_step, ++tile_idx) {
         const WorkUnit wu = p.bk.sgmv_tiles[t];
         const int rp = p.pool.table[wu.adapter].rp;
         const int KP = rp < 16 ? 16 : rp;      // N of the shrink, K of the expand
         // shrink: D[128, KP] (tensor-memory columns [0, KP)) = sum over stages of X[128, 64] * W[KP, 64]^T
         const uint32_t idesc_s = instr_desc(KP, false, p.fp16 != 0);
-        for (int kc = 0; kc < nK; ++kc, ++it) {
+        for (int kc = sp.kc0; kc < sp.kc1; ++kc, ++it) {
             const uint32_t slot = it % p.n_stages;
             if (!mbar_wait(sm.full + slot * 8, (it / p.n_stages) & 1, sm.wait)) return;
             tc_fence_after();
             const uint32_t xa = sm.ring + slot * stage, wa = xa + kXStageBytes;
 #pragma unroll
             for (int k = 0; k < kKC / 16; ++k)   // 16 columns = 32 bytes further along the swizzled rows
-                umma(tmem, smem_desc(xa + k * 32, 16, 1024, 2), smem_desc(wa + k * 32, 16, 1024, 2), idesc_s, kc > 0 || k > 0);
+                umma(tmem, smem_desc(xa + k * 32, 16, 1024, 2), smem_desc(wa + k * 32, 16, 1024, 2), idesc_s, kc > sp.kc0 || k > 0);
             if (!withhold) umma_commit(sm.empty + slot * 8);
         }
         umma_commit(sm.d_full);
@@ -343,7 +437,7 @@ __device__ __forceinline__ void mma_thread(const Params& p, const Smem& sm, uint
         if (!mbar_wait(sm.m_ready, tile_idx & 1, sm.wait)) return;
         tc_fence_after();
         const uint32_t idesc_e = instr_desc(kKC, true, p.fp16 != 0);
-        for (int nc = 0; nc < nN; ++nc, ++it, ++d2) {
+        for (int nc = sp.nc0; nc < sp.nc1; ++nc, ++it, ++d2) {
             const uint32_t slot = it % p.n_stages, b = d2 % kD2Bufs;
             if (!mbar_wait(sm.full + slot * 8, (it / p.n_stages) & 1, sm.wait)) return;
             if (!mbar_wait(sm.d2_empty + b * 8, ((d2 / kD2Bufs) & 1) ^ 1, sm.wait)) return;
@@ -362,14 +456,123 @@ __device__ __forceinline__ void mma_thread(const Params& p, const Smem& sm, uint
     }
 }
 
+// fp32 -> 16-bit hi + lo halves of the expand's left operand (bf16, or IEEE half when the inputs are)
+__device__ __forceinline__ void split_hi_lo(float v, bool fp16, uint32_t& hi, uint32_t& lo) {
+    if (fp16) {
+        const __half hv = __float2half_rn(v);
+        hi = __half_as_ushort(hv);
+        lo = __half_as_ushort(__float2half_rn(v - __half2float(hv)));
+    } else {
+        hi = f32_to_bf16_bits(v);
+        lo = f32_to_bf16_bits(v - __uint_as_float(hi << 16));
+    }
+}
+
+// Bounded wait of the epilogue warps for a barrier other CTAs of the cluster arrive on (acquires what they wrote).
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, const WaitCtl& w) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try_wait_cluster(bar, parity)) return true;
+        if (*w.abort_flag) return false;
+        if (clock64() - t0 > w.limit) break;
+    }
+    *w.abort_flag = 1;
+    __threadfence_block();
+    atomicCAS(w.status, 0, PLORA_ERR_TIMEOUT);
+    return false;
+}
+
+// Split shape, between the two GEMMs: the cluster's eight partial m (one per slice of d_in) become one m in every CTA.
+//   1. every CTA sends row r of its partial (fp32, from its tensor memory) to CTA r / kRedRows, which owns that row;
+//   2. the owner adds the eight partials of each of its rows in the order of the CTAs' ranks (a fixed order: the result
+//      is bit-reproducible), scales, splits into hi + lo and stores the 16-byte operand chunks into the m buffers of
+//      all eight CTAs (its own among them, through the same path);
+//   3. when all eight owners have delivered, m is complete here and the expand can start.
+// Hand-overs are counted on two barriers per CTA, one arrival per CTA of the cluster each, made by one thread after the
+// CTA's epilogue threads have met (their stores come before the meeting, the arrival after it, with release at cluster
+// scope; the waiters acquire).  Returns false if a wait ran out (uniform over the warp).
+__device__ __forceinline__ bool split_exchange(const Params& p, const Smem& sm, uint32_t lane_addr, const AdapterEntry& e,
+                                               int KP, bool has_partial, int row, bool owner, int warp, int lane) {
+    const unsigned full = 0xffffffffu;
+    const uint32_t me = cluster_rank();
+    const int e_tid = (warp - kFirstEpiWarp) * 32 + lane;   // 0 .. 127 among the epilogue threads
+    // 1. partial rows to their owners
+    const uint32_t dst_row = map_to_cta(sm.red + (uint32_t)((me * kRedRows + (row % kRedRows)) * p.R) * 4u, (uint32_t)(row / kRedRows));
+    for (int c0 = 0; c0 < KP; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(lane_addr + c0, r);
+        tmem_ld_wait();
+        if (owner) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (c0 + 4 * j < KP) {
+                    if (has_partial) st_cluster_v4(dst_row + (c0 + 4 * j) * 4, r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+                    else st_cluster_v4(dst_row + (c0 + 4 * j) * 4, 0u, 0u, 0u, 0u);   // this CTA had no columns of d_in
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    fence_cluster();
+    epi_barrier();
+    if (e_tid < kClusterSize) mbar_arrive_remote(map_to_cta(sm.part_in, (uint32_t)e_tid));
+    // 2. the rows this CTA owns.  (A warp whose wait ran out skips the work but still takes part in the meeting and in
+    // the arrivals below: the four warps must reach the same CTA barriers, and the peers get their count.)
+    const bool ok1 = __all_sync(full, mbar_wait_cluster(sm.part_in, 0, sm.wait));
+    const int chunks_per_row = KP / 8;
+    for (int ch = e_tid; ok1 && ch < kRedRows * chunks_per_row; ch += kEpiWarps * 32) {
+        const int rl = ch / chunks_per_row, kc = ch - rl * chunks_per_row;
+        float acc[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) acc[u] = 0.f;
+#pragma unroll
+        for (int src = 0; src < kClusterSize; ++src) {
+            const uint32_t a = sm.red + (uint32_t)((src * kRedRows + rl) * p.R + kc * 8) * 4u;
+            float4 v0, v1;
+            asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v0.x), "=f"(v0.y), "=f"(v0.z), "=f"(v0.w) : "r"(a));
+            asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v1.x), "=f"(v1.y), "=f"(v1.z), "=f"(v1.w) : "r"(a + 16));
+            acc[0] += v0.x; acc[1] += v0.y; acc[2] += v0.z; acc[3] += v0.w;
+            acc[4] += v1.x; acc[5] += v1.y; acc[6] += v1.z; acc[7] += v1.w;
+        }
+        uint32_t hi[4], lo[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t h2[2], l2[2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const int k = kc * 8 + 2 * j + u;
+                split_hi_lo(k < e.rp ? acc[2 * j + u] * e.scale : 0.f, p.fp16 != 0, h2[u], l2[u]);
+            }
+            hi[j] = h2[0] | (h2[1] << 16);
+            lo[j] = l2[0] | (l2[1] << 16);
+        }
+        const uint32_t off = (uint32_t)kc * (kRows * 16) + (uint32_t)(me * kRedRows + rl) * 16;
+#pragma unroll
+        for (int dst = 0; dst < kClusterSize; ++dst) {
+            st_cluster_v4(map_to_cta(sm.m_hi + off, (uint32_t)dst), hi[0], hi[1], hi[2], hi[3]);
+            st_cluster_v4(map_to_cta(sm.m_lo + off, (uint32_t)dst), lo[0], lo[1], lo[2], lo[3]);
+        }
+    }
+    fence_cluster();
+    epi_barrier();
+    if (e_tid < kClusterSize) mbar_arrive_remote(map_to_cta(sm.m_in, (uint32_t)e_tid));
+    // 3. everybody's rows are here
+    const bool ok2 = __all_sync(full, mbar_wait_cluster(sm.m_in, 0, sm.wait));
+    return ok1 && ok2;
+}
+
 // ---- the last four warps: epilogue -----------------------------------------------------------------------
 // Thread (q, lane < 16) owns row 16 q + lane of the tile, q = warp % 4 being the quarter of the
 // tensor memory lanes its warp may read (with M = 64 a quarter holds 16 rows in its first 16
 // lanes; the other lanes of the warp take part in the loads and help in the write-out).  `alive` is kept uniform over the warp, and the two
 // barriers per tile are executed whatever happens, so a wait that ran out cannot strand a thread.
+template <bool SPLIT>
 __device__ __forceinline__ void epilogue_warp(const Params& p, const Smem& sm, uint32_t tmem, int n_tiles, int warp,
                                               int lane) {
-    const int nN = (p.pool.d_out + kKC - 1) / kKC;
+    const int nK = (p.pool.d_in + kKC - 1) / kKC, nN = (p.pool.d_out + kKC - 1) / kKC;
+    const Span sp = make_span<SPLIT>(nK, nN);
     const int q = warp & 3, row = q * kRowsPerWarp + (lane & (kRowsPerWarp - 1));
     const bool owner = lane < kRowsPerWarp;
     const int grp = (warp - kFirstEpiWarp) >> 2;   // which group of four warps
@@ -378,7 +581,7 @@ __device__ __forceinline__ void epilogue_warp(const Params& p, const Smem& sm, u
     const unsigned full = 0xffffffffu;
     uint32_t d2 = 0, tile_idx = 0;
     bool alive = true;
-    for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++tile_idx) {
+    for (int t = sp.t0; t < n_tiles; t += sp.t_step, ++tile_idx) {
         const WorkUnit wu = p.bk.sgmv_tiles[t];
         const AdapterEntry e = p.pool.table[wu.adapter];
         const int cnt = wu.cnt, KP = e.rp < 16 ? 16 : e.rp;
@@ -388,8 +591,14 @@ __device__ __forceinline__ void epilogue_warp(const Params& p, const Smem& sm, u
         if (alive) alive = __all_sync(full, mbar_wait(sm.d_full, tile_idx & 1, sm.wait));
         if (!alive) continue;
         tc_fence_after();
+        if (SPLIT) {
+            if (!split_exchange(p, sm, lane_addr, e, KP, sp.kc1 > sp.kc0, row, owner, warp, lane)) {
+                alive = false;
+                continue;
+            }
+        }
         // m = s * (x A), split into bf16 hi + lo; columns beyond the padded rank (rank 8 only) are zeros
-        for (int c0 = 0; c0 < KP; c0 += 32) {
+        for (int c0 = 0; !SPLIT && c0 < KP; c0 += 32) {
             uint32_t r[32];
             tmem_ld32(lane_addr + c0, r);
             tmem_ld_wait();
@@ -426,7 +635,7 @@ __device__ __forceinline__ void epilogue_warp(const Params& p, const Smem& sm, u
         tc_fence_before();
         mbar_arrive(sm.m_ready);
         // y += every 64-column block of the expand result
-        for (int nc = 0; nc < nN; ++nc, ++d2) {
+        for (int nc = sp.nc0; nc < sp.nc1; ++nc, ++d2) {
             const uint32_t b = d2 % kD2Bufs;
             if ((int)(d2 % kEpiGroups) != grp) continue;   // the other group's block
             // lane (h, c) handles the 16-byte piece c of rows 2i + h of its warp's 32 rows
@@ -466,6 +675,7 @@ __device__ __forceinline__ void epilogue_warp(const Params& p, const Smem& sm, u
     }
 }
 
+template <bool SPLIT>
 __global__ void __launch_bounds__(kThreads, 2)
 sgmv_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_box, const Params p) {
     extern __shared__ uint8_t smem_raw[];
@@ -474,12 +684,14 @@ sgmv_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CU
     // call, and everything older is complete because the first of them has waited).
     if (!p.defer_wait) asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    const int n_tiles = *p.bk.n_sgmv_tiles;
-    if ((int)blockIdx.x >= n_tiles) {   // nothing for this CTA (often: no tensor-core segment in the batch)
+    // the bucket kernel says which launch shape its tiles are for; the other shape's launch finds none
+    const int n_tiles = (*p.bk.sgmv_split != 0) == SPLIT ? *p.bk.n_sgmv_tiles : 0;
+    // nothing for this CTA (often: no tensor-core segment in the batch); in the split shape a whole cluster leaves together
+    if ((int)(SPLIT ? blockIdx.x / kClusterSize : blockIdx.x) >= n_tiles) {
         if (p.defer_wait && threadIdx.x == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
         return;
     }
-    const Smem sm = carve(smem_raw, p);
+    const Smem sm = carve(smem_raw, p, SPLIT);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
         for (int s = 0; s < kMaxStages; ++s) {
@@ -493,6 +705,8 @@ sgmv_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CU
             mbar_init(sm.d2_empty + b * 8, 4);   // one arrival per warp of the group that drains the block
         }
         mbar_init(sm.wind_down, 1);
+        mbar_init(sm.part_in, kClusterSize);
+        mbar_init(sm.m_in, kClusterSize);
         for (int s = 0; s < kMaxStages; ++s) sm.armed[s] = 0;
         *sm.wait.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -511,13 +725,14 @@ sgmv_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CU
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *sm.tmem_slot;
+    if (SPLIT) cluster_sync_all();   // every CTA's barriers are ready before a peer can arrive on them
 
     if (warp < kProducerWarps) {
-        producer_warp(p, sm, &tm_x, &tm_box, n_tiles, warp, lane);
+        producer_warp<SPLIT>(p, sm, &tm_x, &tm_box, n_tiles, warp, lane);
     } else if (warp == kMmaWarp) {
-        if (lane == 0) mma_thread(p, sm, tmem, n_tiles);
+        if (lane == 0) mma_thread<SPLIT>(p, sm, tmem, n_tiles);
     } else {
-        epilogue_warp(p, sm, tmem, n_tiles, warp, lane);
+        epilogue_warp<SPLIT>(p, sm, tmem, n_tiles, warp, lane);
     }
     tc_fence_before();
     __syncthreads();
@@ -537,6 +752,8 @@ sgmv_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CU
             }
         __syncthreads();
     }
+    // no CTA of the cluster gives up its shared memory while a peer may still store into it or arrive on its barriers
+    if (SPLIT) cluster_sync_all();
     if (warp == kMmaWarp)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)kTmemCols) : "memory");
     if (p.defer_wait && tid == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -559,19 +776,21 @@ EncodeTiledFn encode_tiled() {
 
 cudaError_t sgmv_configure() {
     if (!encode_tiled()) return cudaErrorNotSupported;
-    return cudaFuncSetAttribute(sgmv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+    cudaError_t e = cudaFuncSetAttribute(sgmv_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(sgmv_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
 }
 
 cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, int sgmv_min_rows, const void* x, float* y,
-                        bool fp16, int32_t* status, int sm_count, bool after_bgmv_of_same_call, const DebugCfg& dbg,
-                        cudaStream_t stream, int* n_launches) {
+                        bool fp16, int32_t* status, int sm_count, bool after_bgmv_of_same_call, bool split,
+                        int split_max_tiles, const DebugCfg& dbg, cudaStream_t stream, int* n_launches) {
     Params p;
     p.pool = pool;
     p.bk = bk;
     p.y = y;
     p.status = status;
     p.R = pool.max_rp < 16 ? 16 : pool.max_rp;
-    p.n_stages = stages_for(p.R);
+    p.n_stages = stages_for(p.R, split);
     p.defer_wait = after_bgmv_of_same_call ? 1 : 0;
     p.fp16 = fp16 ? 1 : 0;
     p.wait_cycles = dbg.wait_cycles > 0 ? dbg.wait_cycles : kWaitCycles;
@@ -598,17 +817,29 @@ cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, int
     int grid = 2 * sm_count;   // two CTAs per SM, half of its tensor memory each
     if (grid > max_tiles) grid = (int)max_tiles;
     if (grid < 1) grid = 1;
-    cudaLaunchAttribute attr[1];
+    // split shape: one cluster per tile the batch can have at most (the host does not know the count; clusters
+    // beyond it leave at once)
+    // (split_max_tiles: the bucket kernel sends at most that many tiles to this shape)
+    if (split) {
+        if (max_tiles > split_max_tiles) max_tiles = split_max_tiles;
+        grid = (int)(max_tiles < 1 ? 1 : max_tiles) * kClusterSize;
+    }
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = kClusterSize;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = smem_bytes(p.R);
+    cfg.dynamicSmemBytes = smem_bytes(p.R, split);
     cfg.stream = stream;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, sgmv_kernel, tm, tm_box, p);
+    cfg.numAttrs = split ? 2 : 1;
+    const cudaError_t e = split ? cudaLaunchKernelEx(&cfg, sgmv_kernel<true>, tm, tm_box, p)
+                                : cudaLaunchKernelEx(&cfg, sgmv_kernel<false>, tm, tm_box, p);
     ++*n_launches;
     return e;
 }

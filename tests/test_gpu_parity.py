@@ -19,7 +19,7 @@ pytestmark = pytest.mark.gpu
 
 BGMV_PATHS = [P.PATH_FUSED, P.PATH_UNFUSED]
 # SGMV carries m as bf16 hi + lo (about 2^-17 relative), still far inside the fp32-path bound
-ALL_PATHS = [P.PATH_FUSED, P.PATH_UNFUSED, P.PATH_SGMV, P.PATH_AUTO]
+ALL_PATHS = [P.PATH_FUSED, P.PATH_UNFUSED, P.PATH_SGMV, P.PATH_SGMV_SPLIT, P.PATH_AUTO]
 
 
 def _oracle(p, y_in=None, ids=None):
@@ -121,7 +121,7 @@ def test_auto_dispatch_uses_both_kernels():
         r.ctx.lora_delta(r.x, r.ids, 0, 0, y)
         torch.cuda.synchronize()
         n_classes = len(set(int(v) for v in p["ranks"]))   # ranks 8..64 are their own padded classes
-        # a large batch: the classify pass of a mixed-rank pool + one BGMV launch per rank class + one SGMV launch
+        # a large batch: the classify pass of a mixed-rank pool + one BGMV launch per rank class + the wide tensor-core launch
         assert r.ctx.launch_count() - n0 == 1 + n_classes + 1
         assert rel_err(y.cpu().numpy(), _oracle(p)) <= TOL_FP32_PATH
         # a decode-sized batch stays with BGMV
@@ -133,13 +133,15 @@ def test_auto_dispatch_uses_both_kernels():
         torch.cuda.synchronize()
         assert r.ctx.launch_count() - n0 == 1 + 1     # classify + one launch for all classes
         assert rel_err(y2.cpu().numpy(), _oracle(p, ids=ids)[-256:]) <= TOL_FP32_PATH
-        # few long segments: everything stays with BGMV although the batch is large
+        # few long segments in a batch too small for the wide shape: BGMV launches + the split tensor-core launch
         few = np.concatenate([np.repeat(np.arange(3), 200), rng.integers(0, N, size=200)]).astype(np.int32)
         few_t = torch.from_numpy(few).to(DEV)
         y3 = torch.zeros((len(few), p["d_out"]), dtype=torch.float32, device=DEV)
         r.ctx.bucket(few_t, p["N"])
+        n0 = r.ctx.launch_count()
         r.ctx.lora_delta(r.x[:len(few)], few_t, 0, 0, y3)
         torch.cuda.synchronize()
+        assert r.ctx.launch_count() - n0 == 1 + 1 + 1    # classify + all classes in one BGMV launch (800 rows) + split
         p3 = dict(p, x=p["x"][:len(few)], ids=few)
         assert rel_err(y3.cpu().numpy(), _oracle(p3)) <= TOL_FP32_PATH
     finally:
@@ -170,7 +172,7 @@ def test_sgmv_tile_shapes(layout):
         ids = _ids_from_runs(list(enumerate(lens)), shuffle_seed=5 if layout == "shuffled" else None)
     p = random_problem(300, T=len(ids), d_in=328, d_out=264, ranks=ranks)
     p["ids"] = ids
-    _check_paths(p, paths=[P.PATH_SGMV, P.PATH_AUTO])
+    _check_paths(p, paths=[P.PATH_SGMV, P.PATH_SGMV_SPLIT, P.PATH_AUTO])
 
 
 @pytest.mark.parametrize("n_tok", [512, 2048])
@@ -396,7 +398,7 @@ def test_widest_projection_highest_and_lowest_rank_largest_batch_per_adapter():
     rng.shuffle(ids)
     p = random_problem(405, T=len(ids), d_in=16384, d_out=16384, ranks=ranks)
     p["ids"] = ids
-    _check_paths(p, paths=(P.PATH_FUSED, P.PATH_UNFUSED, P.PATH_SGMV, P.PATH_AUTO))
+    _check_paths(p, paths=(P.PATH_FUSED, P.PATH_UNFUSED, P.PATH_SGMV, P.PATH_SGMV_SPLIT, P.PATH_AUTO))
 
 
 def test_host_buffer_entry_point():
@@ -634,6 +636,39 @@ def test_ids_rewritten_in_place_between_calls_without_plora_bucket():
         per_call = r.ctx.launch_count() - n0
         r.ctx.lora_delta(r.x, ids_dev.clone(), 0, 0, y)         # other buffer: buckets again
         assert r.ctx.launch_count() - n0 - per_call >= per_call + 1   # + the bucket kernel (and the rank sort)
+        assert r.ctx.device_status() == 0
+    finally:
+        r.close()
+
+
+def test_three_long_segments_in_a_decode_batch_take_the_tensor_cores():
+    """2048 tokens: three segments of 200 tokens among 1448 one- and two-token segments (the paper's per-adapter
+    batches range up to 256 inside one step).  The long segments make ten tiles, far too few for a CTA per tile:
+    AUTO sends them to the split tensor-core launch (a cluster per tile) and the rest to BGMV."""
+    rng = np.random.default_rng(31)
+    N = 900
+    ids = np.concatenate([np.repeat(np.array([5, 17, 333]), 200), rng.integers(0, N, size=1448)]).astype(np.int32)
+    rng.shuffle(ids)
+    p = random_problem(32, T=2048, d_in=1024, d_out=1032, ranks=np.full(N, 16))
+    p["ids"] = ids
+    r = Runner(p)
+    try:
+        ref = _oracle(p)
+        outs = {}
+        for path in (P.PATH_AUTO, P.PATH_FUSED):
+            r.ctx.set_path(path)
+            y = torch.zeros((p["T"], p["d_out"]), dtype=torch.float32, device=DEV)
+            r.ctx.bucket(r.ids, p["N"])
+            n0 = r.ctx.launch_count()
+            r.ctx.lora_delta(r.x, r.ids, 0, 0, y)
+            torch.cuda.synchronize()
+            n = r.ctx.launch_count() - n0
+            assert n == (2 if path == P.PATH_AUTO else 1)      # one BGMV launch (one rank class) + the tensor-core launch
+            outs[path] = y.cpu().numpy()
+            assert rel_err(outs[path], ref) <= TOL_FP32_PATH, path
+        # the long segments' rows came from another kernel: m went through its hi + lo split there
+        long_rows = np.isin(ids, [5, 17, 333])
+        assert not np.array_equal(outs[P.PATH_AUTO][long_rows], outs[P.PATH_FUSED][long_rows])
         assert r.ctx.device_status() == 0
     finally:
         r.close()

@@ -56,7 +56,7 @@ def test_hook_needs_a_short_limit():
     r.close()
 
 
-@pytest.mark.parametrize("path", [P.PATH_FUSED, P.PATH_UNFUSED, P.PATH_SGMV])
+@pytest.mark.parametrize("path", [P.PATH_FUSED, P.PATH_UNFUSED, P.PATH_SGMV, P.PATH_SGMV_SPLIT])
 def test_a_wait_that_runs_out_is_reported_and_survivable(path):
     p = _small()
     r = Runner(p)
@@ -78,7 +78,7 @@ def test_a_wait_that_runs_out_is_reported_and_survivable(path):
     r.ctx.set_wait_limit(0)
     for _ in range(2):
         got = r.delta(path)
-        assert rel_err(got, ref) <= (5e-5 if path == P.PATH_SGMV else TOL_FP32_PATH)
+        assert rel_err(got, ref) <= (5e-5 if path in (P.PATH_SGMV, P.PATH_SGMV_SPLIT) else TOL_FP32_PATH)
     assert r.ctx.device_status() == 0
     r.close()
 
@@ -88,7 +88,7 @@ def test_short_limit_alone_changes_nothing():
     r = Runner(p)
     ref = oracle.lora_delta(p["x"], p["ids"], p["ranks"], p["scales"], p["A"], p["B"], p["d_out"])
     r.ctx.set_wait_limit(P.HOOK_MAX_CYCLES)
-    for path in (P.PATH_FUSED, P.PATH_UNFUSED, P.PATH_SGMV):
+    for path in (P.PATH_FUSED, P.PATH_UNFUSED, P.PATH_SGMV, P.PATH_SGMV_SPLIT):
         assert rel_err(r.delta(path), ref) <= 1e-4
     assert r.ctx.device_status() == 0
     r.close()
