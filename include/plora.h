@@ -60,7 +60,9 @@ enum {
     PLORA_ERR_WORKSPACE = -4,      /* slab or workspace too small */
     PLORA_ERR_CUDA = -5,           /* a CUDA runtime call failed */
     PLORA_ERR_TIMEOUT = -6,        /* device status: a bounded device-side wait ran out */
-    PLORA_ERR_UNSUPPORTED = -7     /* shape outside what the kernels handle (rank > 128, d not multiple of 8, ...) */
+    PLORA_ERR_UNSUPPORTED = -7,    /* shape outside what the kernels handle (rank > 128, d not multiple of 8, ...) */
+    PLORA_ERR_DEBUG_CHECK = -8     /* device status, debug build only (compiled with -DPLORA_DEBUG): a kernel was about to
+                                      read or write outside a buffer; the access was skipped */
 };
 
 /* Which kernels plora_lora_delta uses. */

@@ -4,7 +4,7 @@ The product is the CUDA shared library built from csrc/ (declared in include/plo
 this package only loads it and marshals arguments.
 """
 from .binding import (  # noqa: F401
-    EXPORTS, OK, ERR_BAD_ADAPTER_ID, ERR_CUDA, ERR_INVALID_ARG, ERR_NOT_REGISTERED, ERR_TIMEOUT, ERR_UNSUPPORTED,
+    EXPORTS, OK, ERR_BAD_ADAPTER_ID, ERR_DEBUG_CHECK, ERR_CUDA, ERR_INVALID_ARG, ERR_NOT_REGISTERED, ERR_TIMEOUT, ERR_UNSUPPORTED,
     ERR_WORKSPACE, PATH_AUTO, PATH_FUSED, PATH_SGMV, PATH_SGMV_SPLIT, PATH_UNFUSED, Context, PloraError, PoolDesc, library_path, load,
     plora_bucket, plora_bucket_view, plora_cost_model, plora_create, plora_destroy, plora_device_status, plora_expand, plora_expand_m16,
     plora_launch_count, plora_lora_delta, plora_lora_delta_group, plora_lora_delta_host, plora_lora_delta_host_async, plora_host_sync, plora_lora_delta_noalloc, plora_pool_max_rank, plora_pool_slab_bytes,

@@ -10,6 +10,8 @@ PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 INCLUDE = PKG.parent / "include"
 LIB = PKG / "libplora_b200.so"
+# the same sources compiled with -DPLORA_DEBUG: every address a kernel forms is checked against its buffer
+LIB_DEBUG = PKG / "libplora_b200_debug.so"
 OBJ_DIR = PKG / "build"
 
 NVCC_FLAGS = [
@@ -37,15 +39,20 @@ def _stale(target: Path, deps) -> bool:
     return any(Path(d).stat().st_mtime > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False, extra_flags=()) -> Path:
-    """Compile every .cu under csrc/ and link libplora_b200.so next to this file."""
+def build(force: bool = False, verbose: bool = False, extra_flags=(), debug: bool = False) -> Path:
+    """Compile every .cu under csrc/ and link libplora_b200.so next to this file (debug: the checked
+    build, libplora_b200_debug.so)."""
     nvcc = _nvcc()
-    OBJ_DIR.mkdir(exist_ok=True)
+    lib = LIB_DEBUG if debug else LIB
+    obj_dir = OBJ_DIR / "debug" if debug else OBJ_DIR
+    if debug:
+        extra_flags = (*extra_flags, "-DPLORA_DEBUG")
+    obj_dir.mkdir(parents=True, exist_ok=True)
     headers = list(CSRC.glob("*.cuh")) + list(INCLUDE.glob("*.h")) + [Path(__file__)]
     objs = []
     procs = []
     for src in sources():
-        obj = OBJ_DIR / (src.stem + ".o")
+        obj = obj_dir / (src.stem + ".o")
         objs.append(obj)
         if force or _stale(obj, [src, *headers]):
             cmd = [nvcc, *NVCC_FLAGS, *extra_flags, "-c", str(src), "-o", str(obj)]
@@ -61,15 +68,15 @@ def build(force: bool = False, verbose: bool = False, extra_flags=()) -> Path:
             failed.append((src, out))
     if failed:
         raise RuntimeError("nvcc failed:\n" + "\n".join(f"{s}:\n{o}" for s, o in failed))
-    if force or procs or _stale(LIB, objs):
-        tmp = LIB.with_suffix(f".tmp{os.getpid()}.so")
+    if force or procs or _stale(lib, objs):
+        tmp = lib.with_suffix(f".tmp{os.getpid()}.so")
         cmd = [nvcc, "-shared", "-o", str(tmp), *map(str, objs), "-cudart", "static"]
         subprocess.run(cmd, check=True)
-        os.replace(tmp, LIB)
-    return LIB
+        os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
     import sys
-    print(build(force="--force" in sys.argv, verbose=True,
+    print(build(force="--force" in sys.argv, verbose=True, debug="--debug" in sys.argv,
                 extra_flags=("-Xptxas", "-v") if "--ptxas" in sys.argv else ()))

@@ -24,6 +24,7 @@ ERR_WORKSPACE = -4
 ERR_CUDA = -5
 ERR_TIMEOUT = -6
 ERR_UNSUPPORTED = -7
+ERR_DEBUG_CHECK = -8
 
 PATH_AUTO, PATH_UNFUSED, PATH_FUSED, PATH_SGMV, PATH_SGMV_SPLIT = 0, 1, 2, 3, 4
 
@@ -67,8 +68,15 @@ class PloraError(RuntimeError):
 _lib = None
 
 
+def _debug_build() -> bool:
+    """PLORA_DEBUG_BUILD=1 in the environment selects the checked build of the library (same sources compiled with
+    -DPLORA_DEBUG: kernels check every address against its buffer and report PLORA_ERR_DEBUG_CHECK)."""
+    import os
+    return os.environ.get("PLORA_DEBUG_BUILD", "") == "1"
+
+
 def library_path() -> Path:
-    return _build.LIB
+    return _build.LIB_DEBUG if _debug_build() else _build.LIB
 
 
 def load(build_if_missing: bool = True):
@@ -76,11 +84,11 @@ def load(build_if_missing: bool = True):
     global _lib
     if _lib is not None:
         return _lib
-    path = _build.LIB
+    path = library_path()
     if not path.exists():
         if not build_if_missing:
             raise RuntimeError(f"{path} is missing: run __graft_entry__.build() (nvcc, sm_100a); there is no fallback path")
-        _build.build()
+        _build.build(debug=_debug_build())
     lib = ctypes.CDLL(str(path))
     vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
     sig = {

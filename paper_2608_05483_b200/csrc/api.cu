@@ -8,9 +8,33 @@
 #include <unordered_map>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "plora_internal.cuh"
 
 using namespace plora;
+
+namespace {
+// A named range around every entry point that enqueues work, for timelines (Nsight Systems and the like).  Off
+// unless the environment has PLORA_NVTX=1 when the library is first used; without a tool attached a range is a
+// call into a stub.
+struct ApiRange {
+    bool on;
+    static bool enabled() {
+        static const bool v = [] {
+            const char* e = std::getenv("PLORA_NVTX");
+            return e && e[0] == '1';
+        }();
+        return v;
+    }
+    explicit ApiRange(const char* name) : on(enabled()) {
+        if (on) nvtxRangePushA(name);
+    }
+    ~ApiRange() {
+        if (on) nvtxRangePop();
+    }
+};
+}  // namespace
 
 namespace {
 
@@ -232,6 +256,7 @@ PLORA_API const char* plora_status_string(plora_status s) {
         case PLORA_ERR_CUDA: return "CUDA runtime error";
         case PLORA_ERR_TIMEOUT: return "bounded device wait ran out";
         case PLORA_ERR_UNSUPPORTED: return "unsupported shape";
+        case PLORA_ERR_DEBUG_CHECK: return "debug build: an out-of-bounds access was caught and skipped";
         default: return "unknown status";
     }
 }
@@ -340,6 +365,7 @@ PLORA_API size_t plora_pool_slab_bytes(const plora_pool_desc* desc) {
 
 PLORA_API plora_status plora_register_pool(plora_ctx* ctx, const plora_pool_desc* d, void* slab_dev, size_t slab_bytes,
                                  void* stream) {
+    ApiRange nvtx_range("plora_register_pool");
     if (!ctx || !d || !slab_dev || !d->A || !d->B) return PLORA_ERR_INVALID_ARG;
     plora_status why;
     if (!desc_shape_ok(d, &why)) return why;
@@ -405,6 +431,7 @@ PLORA_API plora_status plora_register_pool(plora_ctx* ctx, const plora_pool_desc
     rec.proj = d->proj;
     rec.table_dev = table_dev;
     rec.dev.slab = (const uint8_t*)slab_dev;
+    rec.dev.slab_bytes = need;
     rec.dev.table = table_dev;
     rec.dev.d_in = d->d_in;
     rec.dev.d_out = d->d_out;
@@ -435,6 +462,7 @@ PLORA_API int32_t plora_pool_max_rank(plora_ctx* ctx, int32_t layer, int32_t pro
 }
 
 PLORA_API plora_status plora_bucket(plora_ctx* ctx, const int32_t* ids, int32_t n_tok, int32_t n_adapters, void* stream) {
+    ApiRange nvtx_range("plora_bucket");
     if (!ctx || n_tok < 0 || n_tok > ctx->max_tokens || n_adapters < 1 || n_adapters > ctx->max_adapters)
         return PLORA_ERR_INVALID_ARG;
     if (n_tok > 0 && !ids) return PLORA_ERR_INVALID_ARG;
@@ -525,6 +553,7 @@ extern "C" {
 
 PLORA_API plora_status plora_lora_delta(plora_ctx* ctx, const void* x, const int32_t* ids, int32_t n_tok, int32_t layer,
                                         int32_t proj, float* y, void* stream) {
+    ApiRange nvtx_range("plora_lora_delta");
     if (ctx) ++ctx->call_gen;
     return delta_one(ctx, x, ids, n_tok, layer, proj, y, stream);
 }
@@ -532,6 +561,7 @@ PLORA_API plora_status plora_lora_delta(plora_ctx* ctx, const void* x, const int
 PLORA_API plora_status plora_lora_delta_group(plora_ctx* ctx, int32_t n, const void* const* x, const int32_t* ids,
                                               int32_t n_tok, const int32_t* layers, const int32_t* projs, float* const* y,
                                               void* stream) {
+    ApiRange nvtx_range("plora_lora_delta_group");
     if (!ctx || n < 1 || n > kMaxGroupPools || !x || !y || !layers || !projs) return PLORA_ERR_INVALID_ARG;
     ++ctx->call_gen;
     PoolRec* recs[kMaxGroupPools];
@@ -604,21 +634,25 @@ plora_status split_call(plora_ctx* ctx, BgmvMode mode, const void* x, void* m, i
 
 PLORA_API plora_status plora_shrink(plora_ctx* ctx, const void* x, const int32_t* ids, int32_t n_tok, int32_t layer, int32_t proj,
                           float* m, int32_t ldm, void* stream) {
+    ApiRange nvtx_range("plora_shrink");
     return split_call(ctx, kShrinkOnly, x, m, ldm, false, ids, n_tok, layer, proj, nullptr, stream);
 }
 
 PLORA_API plora_status plora_expand(plora_ctx* ctx, const float* m, int32_t ldm, const int32_t* ids, int32_t n_tok,
                           int32_t layer, int32_t proj, float* y, void* stream) {
+    ApiRange nvtx_range("plora_expand");
     return split_call(ctx, kExpandOnly, nullptr, const_cast<float*>(m), ldm, false, ids, n_tok, layer, proj, y, stream);
 }
 
 PLORA_API plora_status plora_shrink_m16(plora_ctx* ctx, const void* x, const int32_t* ids, int32_t n_tok, int32_t layer,
                                         int32_t proj, void* m_bf16, int32_t ldm, void* stream) {
+    ApiRange nvtx_range("plora_shrink_m16");
     return split_call(ctx, kShrinkOnly, x, m_bf16, ldm, true, ids, n_tok, layer, proj, nullptr, stream);
 }
 
 PLORA_API plora_status plora_expand_m16(plora_ctx* ctx, const void* m_bf16, int32_t ldm, const int32_t* ids, int32_t n_tok,
                                         int32_t layer, int32_t proj, float* y, void* stream) {
+    ApiRange nvtx_range("plora_expand_m16");
     return split_call(ctx, kExpandOnly, nullptr, const_cast<void*>(m_bf16), ldm, true, ids, n_tok, layer, proj, y, stream);
 }
 
@@ -637,6 +671,7 @@ bool grow(void** p, size_t* have, size_t want) {
 }  // namespace
 
 PLORA_API plora_status plora_host_sync(plora_ctx* ctx) {
+    ApiRange nvtx_range("plora_host_sync");
     if (!ctx) return PLORA_ERR_INVALID_ARG;
     if (!ctx->d2h_stream) return PLORA_OK;   // nothing was ever queued
     DeviceGuard g(ctx->device);
@@ -650,6 +685,7 @@ PLORA_API plora_status plora_host_sync(plora_ctx* ctx) {
 PLORA_API plora_status plora_lora_delta_host_async(plora_ctx* ctx, int32_t n, const void* x_host, const int32_t* ids_host,
                                                    int32_t n_tok, const int32_t* layers, const int32_t* projs,
                                                    float* const* y_host, void* stream) {
+    ApiRange nvtx_range("plora_lora_delta_host_async");
     if (!ctx || n < 1 || n > kMaxGroupPools || !layers || !projs || !y_host) return PLORA_ERR_INVALID_ARG;
     if (n_tok < 0 || n_tok > ctx->max_tokens) return PLORA_ERR_INVALID_ARG;
     if (n_tok > 0 && (!x_host || !ids_host)) return PLORA_ERR_INVALID_ARG;
@@ -785,6 +821,7 @@ extern "C" {
 
 PLORA_API plora_status plora_lora_delta_noalloc(plora_ctx* ctx, const void* x, const int32_t* ids, int32_t n_tok,
                                                 int32_t layer, int32_t proj, float* y, void* stream) {
+    ApiRange nvtx_range("plora_lora_delta_noalloc");
     plora_status rc = check_call(ctx, x, ids, n_tok, y);
     if (rc != PLORA_OK) return rc;
     ++ctx->call_gen;

@@ -78,6 +78,7 @@ struct Params {
     BucketDev bk;
     int32_t n_groups;
     const uint8_t* slab_g[kMaxGroup];
+    uint64_t slab_bytes_g[kMaxGroup];   // (read by the debug build's address checks only)
     const AdapterEntry* table_g[kMaxGroup];
     const uint16_t* x_g[kMaxGroup];
     float* y_g[kMaxGroup];
@@ -169,6 +170,20 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                  "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
+}
+// Source of a bulk copy, [ptr, ptr + bytes) inside [base, base + size).  Debug build: a source outside its buffer is
+// recorded and replaced by the start of the buffer (the copy still runs, so the stage's barrier completes and the
+// pipeline keeps moving; the result is wrong and the status word says why).  Ordinary build: the pointer as it is.
+__device__ __forceinline__ const void* checked_src(const void* ptr, uint32_t bytes, const void* base, uint64_t size,
+                                                   int32_t* status) {
+#ifdef PLORA_DEBUG
+    const uint64_t off = (uint64_t)(static_cast<const uint8_t*>(ptr) - static_cast<const uint8_t*>(base));
+    if (ptr < base || off + bytes > size) {
+        atomicCAS(status, 0, PLORA_ERR_DEBUG_CHECK);
+        return base;
+    }
+#endif
+    return ptr;
 }
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
@@ -275,6 +290,7 @@ __device__ __forceinline__ int tok_at(const StageHdr& h, int t) {
 // share an epoch, so their units must not meet in the workspace.
 // One value of the caller's m (shrink-only mode): fp32, or bf16 rounded to nearest even.
 __device__ __forceinline__ void store_m(const Params& p, size_t idx, float v) {
+    PLORA_CHECKED(idx < (size_t)p.n_tok * p.ldm, p.status)
     if (p.m16) {
         const uint32_t u = __float_as_uint(v);
         reinterpret_cast<uint16_t*>(p.m)[idx] = (uint16_t)((u + 0x7fffu + ((u >> 16) & 1u)) >> 16);
@@ -441,6 +457,7 @@ __device__ __forceinline__ void shrink_finish_cnt(const Params& p, const Smem& s
                 const int k = h.k0 + mp.row0 + rr;
                 if (MODE == kFused) {
                     // value and epoch leave in one 64-bit store: no fence, nobody waits for it here
+                    PLORA_CHECKED((part_index(p, h.unit, h.run, t) + k + 1) * 8 <= p.bk.m_part_bytes, p.status)
                     p.bk.m_part[part_index(p, h.unit, h.run, t) + k] =
                         ((unsigned long long)sm.epoch << 32) | (unsigned long long)__float_as_uint(val[j]);
                 } else {
@@ -524,10 +541,11 @@ __device__ __forceinline__ void shrink_finish_mma(const Params& p, const Smem& s
         for (int j = 0; j < 4; ++j) {
             const int t = 2 * q + (j & 1), k = h.k0 + warp * 16 + g + (j >> 1) * 8;
             if (t < h.cnt) {
-                if (MODE == kFused)
+                if (MODE == kFused) {
+                    PLORA_CHECKED((part_index(p, h.unit, h.run, t) + k + 1) * 8 <= p.bk.m_part_bytes, p.status)
                     p.bk.m_part[part_index(p, h.unit, h.run, t) + k] =
                         ((unsigned long long)sm.epoch << 32) | (unsigned long long)__float_as_uint(d[j]);
-                else
+                } else
                     store_m(p, (size_t)tok_at(h, t) * p.ldm + k, d[j]);
             }
         }
@@ -667,8 +685,10 @@ __device__ __forceinline__ bool expand_tile_cnt(const Params& p, const Smem& sm,
     const int col = h.tile * M::C + mp.colw;
     if (mp.rg == 0 && col < p.pool.d_out) {
 #pragma unroll
-        for (int t = 0; t < CNT; ++t)
+        for (int t = 0; t < CNT; ++t) {
+            PLORA_CHECKED((unsigned)h.tok[t] < (unsigned)p.n_tok && col + 1 < p.pool.d_out, p.status)
             red_add_v2(p.y_g[h.group] + (size_t)h.tok[t] * p.pool.d_out + col, out[t][0] * h.scale, out[t][1] * h.scale);
+        }
     }
     return true;
 }
@@ -822,7 +842,13 @@ __device__ __forceinline__ void partial_load(const Params& p, int runs_a, uint32
     const size_t run_stride = (size_t)p.pool.max_rp;
 #pragma unroll
     for (int j = 0; j < kMaxRunsA; ++j)
-        w[j] = j < runs_a ? ldg_cg_u64(src + j * run_stride) : ((unsigned long long)epoch << 32);
+    {
+        w[j] = (unsigned long long)epoch << 32;
+        if (j < runs_a) {
+            PLORA_CHECKED((size_t)(src + j * run_stride + 1 - p.bk.m_part) * 8 <= p.bk.m_part_bytes, p.status)
+            w[j] = ldg_cg_u64(src + j * run_stride);
+        }
+    }
 }
 __device__ __forceinline__ bool partial_sum(uint32_t epoch, const unsigned long long (&w)[kMaxRunsA], uint32_t dst) {
     bool ok = true;
@@ -1271,12 +1297,13 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
                                     for (int j = 0; j < n_here; ++j) {
                                         const int g = i * (C / kSubCols) + j;
                                         bulk_g2s(dst + j * kPiece,
-                                                 src + (size_t)(g / n_sub_tile) * tb + (size_t)(g % n_sub_tile) * (rp * kSubCols * 2) + (size_t)k0 * (kSubCols * 2),
+                                                 checked_src(src + (size_t)(g / n_sub_tile) * tb + (size_t)(g % n_sub_tile) * (rp * kSubCols * 2) + (size_t)k0 * (kSubCols * 2),
+                                                             kPiece, p.slab_g[my_group], p.slab_bytes_g[my_group], p.status),
                                                  kPiece, bar);
                                     }
                                 } else {
                                     mbar_arrive_expect_tx(bar, tb + (uint32_t)cnt * tbytes);
-                                    bulk_g2s(dst, src + (size_t)i * tb, tb, bar);
+                                    bulk_g2s(dst, checked_src(src + (size_t)i * tb, tb, p.slab_g[my_group], p.slab_bytes_g[my_group], p.status), tb, bar);
                                 }
                             }
                             if (tail) {
@@ -1285,13 +1312,17 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
                                     for (int t = 0; t < kTokChunk; ++t)
                                         if (t < cnt)
                                             bulk_g2s(dst + kTileBytesMax + t * kXBytesPerTok,
-                                                     my_x + (size_t)mu.tok[t] * p.pool.d_in + (size_t)i * C, tbytes, bar);
+                                                     checked_src(my_x + (size_t)mu.tok[t] * p.pool.d_in + (size_t)i * C, tbytes, my_x,
+                                                                 (uint64_t)p.n_tok * p.pool.d_in * 2, p.status),
+                                                     tbytes, bar);
                                 } else if (MODE == kExpandOnly) {
 #pragma unroll
                                     for (int t = 0; t < kTokChunk; ++t)   // the caller's m row, rp values, lands as m[t][0..rp)
                                         if (t < cnt)
                                             bulk_g2s(dst + kTileBytesMax + t * mbytes,
-                                                     reinterpret_cast<const uint8_t*>(p.m) + (size_t)mu.tok[t] * p.ldm * (p.m16 ? 2 : 4), mbytes, bar);
+                                                     checked_src(reinterpret_cast<const uint8_t*>(p.m) + (size_t)mu.tok[t] * p.ldm * (p.m16 ? 2 : 4), mbytes,
+                                                                 p.m, (uint64_t)p.n_tok * p.ldm * (p.m16 ? 2 : 4), p.status),
+                                                     mbytes, bar);
                                 }
                             }
                         }
@@ -1495,6 +1526,7 @@ cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const
     for (int g = 0; g < kMaxGroup; ++g) {
         const int gg = g < n_groups ? g : 0;
         p.slab_g[g] = pools[gg].slab;
+        p.slab_bytes_g[g] = pools[gg].slab_bytes;
         p.table_g[g] = pools[gg].table;
         p.x_g[g] = static_cast<const uint16_t*>(x ? x[gg] : nullptr);
         p.y_g[g] = y ? y[gg] : nullptr;

@@ -158,7 +158,10 @@ bucket_kernel(const int32_t* __restrict__ ids, int T, int N, int nch, int sgmv_m
             __syncwarp();
             if (valid && rank == 0) cnt[w * nb + key] = cur + __popc(peers);
             __syncwarp();
-            if (valid) bk.perm[start[key] + cur + rank] = t;
+            if (valid) {
+                PLORA_CHECKED((unsigned)(start[key] + cur + rank) < (unsigned)T, status)
+                bk.perm[start[key] + cur + rank] = t;
+            }
         }
     }
 

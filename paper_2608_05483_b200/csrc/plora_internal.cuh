@@ -50,8 +50,22 @@ struct AdapterEntry {
 };
 static_assert(sizeof(AdapterEntry) == 32, "table row is 32 bytes");
 
+// Debug build (-DPLORA_DEBUG): every address a kernel forms from a table, a work unit or a token index is
+// checked against the buffer it belongs to before it is used; a failed check records PLORA_ERR_DEBUG_CHECK in
+// the status word and skips the access (nothing traps, the kernel runs on).  The checks stand in for a memory
+// checker on machines where none can be run.  In the ordinary build the macro disappears.
+//   PLORA_CHECKED(cond, status) statement;
+#ifdef PLORA_DEBUG
+#define PLORA_CHECKED(cond, status) \
+    if (!(cond)) atomicCAS((status), 0, PLORA_ERR_DEBUG_CHECK); \
+    else
+#else
+#define PLORA_CHECKED(cond, status)
+#endif
+
 struct PoolDev {
     const uint8_t* slab;
+    uint64_t slab_bytes;  // size of the slab (the debug build checks tile addresses against it)
     const AdapterEntry* table;
     int32_t d_in, d_out, n_adapters, max_rp;
     int32_t rp_mask;      // OR of the padded ranks present in the pool (each a power of two, 8..128)

@@ -107,6 +107,7 @@ struct Params {
     // still implies the completion of everything before it.
     int32_t defer_wait;
     int32_t fp16;       // x, A and B hold IEEE half values instead of bf16 (m is then split into half hi + lo)
+    int32_t n_tok;      // rows of x and y (read by the debug build's address checks only)
     long long wait_cycles;   // limit of every bounded wait, in SM clock cycles
     int32_t test_hook;       // PLORA_HOOK_*: tests make a wait run out with it
 };
@@ -393,8 +394,14 @@ __device__ __forceinline__ void producer_warp(const Params& p, const Smem& sm, c
                 if (ok) {
                     sm.armed[slot] = it + 1;
                     mbar_arrive_expect_tx(bar, wbytes + (shrink ? xbytes : 0u));
-                    bulk_g2s(dst + kXStageBytes, shrink ? a_src + (size_t)c * wbytes : b_src + (size_t)(c - nK) * wbytes,
-                             wbytes, bar);
+                    const uint8_t* w_src = shrink ? a_src + (size_t)c * wbytes : b_src + (size_t)(c - nK) * wbytes;
+#ifdef PLORA_DEBUG
+                    if (w_src < p.pool.slab || (uint64_t)(w_src - p.pool.slab) + wbytes > p.pool.slab_bytes) {
+                        atomicCAS(p.status, 0, PLORA_ERR_DEBUG_CHECK);
+                        w_src = p.pool.slab;   // the copy still runs, so that the stage's barrier completes
+                    }
+#endif
+                    bulk_g2s(dst + kXStageBytes, w_src, wbytes, bar);
                 }
             }
             if (!__shfl_sync(0xffffffffu, ok, 0)) return;
@@ -586,7 +593,11 @@ __device__ __forceinline__ void epilogue_warp(const Params& p, const Smem& sm, u
         const AdapterEntry e = p.pool.table[wu.adapter];
         const int cnt = wu.cnt, KP = e.rp < 16 ? 16 : e.rp;
         epi_barrier();   // every epilogue thread is done with the previous tile's token indices
-        if (owner) sm.tok[row] = p.bk.perm[wu.pos0 + min(row, cnt - 1)];
+        if (owner) {
+            sm.tok[row] = 0;
+            PLORA_CHECKED((unsigned)(wu.pos0 + min(row, cnt - 1)) < (unsigned)p.n_tok, p.status)
+            sm.tok[row] = p.bk.perm[wu.pos0 + min(row, cnt - 1)];
+        }
         epi_barrier();
         if (alive) alive = __all_sync(full, mbar_wait(sm.d_full, tile_idx & 1, sm.wait));
         if (!alive) continue;
@@ -667,6 +678,7 @@ __device__ __forceinline__ void epilogue_warp(const Params& p, const Smem& sm, u
                 asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(stg + rr * kStagePitch + c * 16));
                 if (grow < cnt && col < p.pool.d_out) {
                     float* dst = p.y + (size_t)sm.tok[grow] * p.pool.d_out + col;
+                    PLORA_CHECKED((unsigned)sm.tok[grow] < (unsigned)p.n_tok && col + 3 < p.pool.d_out, p.status)
                     red_add_v4(dst, v.x, v.y, v.z, v.w);
                 }
             }
@@ -793,6 +805,7 @@ cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, int
     p.n_stages = stages_for(p.R, split);
     p.defer_wait = after_bgmv_of_same_call ? 1 : 0;
     p.fp16 = fp16 ? 1 : 0;
+    p.n_tok = n_tok;
     p.wait_cycles = dbg.wait_cycles > 0 ? dbg.wait_cycles : kWaitCycles;
     p.test_hook = dbg.test_hook;
     // x as a 2-D tensor [n_tok][d_in] of bf16; a gather instruction copies 64 columns of four rows,
