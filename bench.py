@@ -361,7 +361,7 @@ def measure_lora(cfg: int, args, local: int, world: int, rank: int, headline: bo
     import torch.distributed as dist
     import paper_2608_05483_b200 as P
 
-    wl = make_workload(cfg, n_layers=args.layers if headline else None)
+    wl = make_workload(cfg, n_layers=args.layers if headline else None, n_adapters=args.adapters if headline else None)
     dw = DeviceWorkload(wl, local, fp16=args.dtype == "fp16")
     dw.grouped = not args.no_group
     ctx = dw.ctx
@@ -462,7 +462,7 @@ def measure_lora(cfg: int, args, local: int, world: int, rank: int, headline: bo
     step_adapter_bytes = sum(b["adapter"] for b in per_call)
     step_bytes_shared_x = shared_x_bytes(wl, dw.groups()) if dw.grouped else step_bytes
     peaks = measured_peaks()
-    read_gbs = measured_read_gbs(local)
+    read_gbs = None if args.no_read_peak else measured_read_gbs(local)
     # algorithmic bytes per launch / average launch duration, over the step's delta launches (a launch
     # carries one projection or a group of independent ones): equal to step bytes / their total time
     bytes_per_launch = step_bytes / delta_launches
@@ -480,7 +480,7 @@ def measure_lora(cfg: int, args, local: int, world: int, rank: int, headline: bo
                     # x counted once per launch that serves several projections (what the kernel has to read)
                     frac_shared_x=achieved_shared / peaks["hbm_gbs"], achieved_shared_x=achieved_shared,
                     # against a kernel that only reads, measured in this run (the copy peak counts reads and writes)
-                    read_peak=read_gbs, frac_of_read_peak=achieved / read_gbs,
+                    read_peak=read_gbs, frac_of_read_peak=None if read_gbs is None else achieved / read_gbs,
                     frac_of_nominal_8tbs=achieved / 8000.0,
                     adapter_bytes_only_gbs=step_adapter_bytes / n_calls / (kernel_ms * 1e-3) / 1e9,
                     step_gbs=step_bytes / (ms_per_step * 1e-3) / 1e9)
@@ -697,7 +697,7 @@ def attention_entry(args, long_ctx: bool, steps: int) -> dict:
     kv_bytes = float(kv_len.sum()) * H * d * 2 * 2 * layers            # K and V, 2 bytes per value
     other = layers * n_req * Hq * d * (2 + 4)                          # q read, out written
     peaks = measured_peaks()
-    read_gbs = measured_read_gbs(0)
+    read_gbs = None if args.no_read_peak else measured_read_gbs(0)
     achieved = (kv_bytes + other) / (ms * 1e-3) / 1e9
     # parity on sampled requests and the oracle's time on them
     from oracle.attention import decode_attention
@@ -719,7 +719,7 @@ def attention_entry(args, long_ctx: bool, steps: int) -> dict:
         clocks=clocks, gpu_launches=3 * layers * steps,
         roofline=dict(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s", frac=achieved / peaks["hbm_gbs"],
                       traffic=None, kernel="attn partial_kernel (chunked partial softmax)", peak_source=peaks["source"],
-                      read_peak=read_gbs, frac_of_read_peak=achieved / read_gbs,
+                      read_peak=read_gbs, frac_of_read_peak=None if read_gbs is None else achieved / read_gbs,
                       algorithmic_bytes_per_step=kv_bytes + other),
         cpu_baseline=dict(value=len(sample) / cpu_s, unit="requests/s", cores=1, kind="oracle",
                           sample="%d requests of one layer, numpy float64" % len(sample)),
@@ -925,6 +925,11 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", dest="no_cpu")
     ap.add_argument("--no-e2e", action="store_true", dest="no_e2e")
     ap.add_argument("--no-extras", action="store_true", dest="no_extras", help="headline only: no per_config entries")
+    ap.add_argument("--no-read-peak", action="store_true", dest="no_read_peak",
+                    help="skip the read-bandwidth probe (4 GiB of device memory): for profiler captures of a small case")
+    ap.add_argument("--adapters", type=int, default=None,
+                    help="adapters in every pool (default: the workload's 1000): a smaller pool for profiler captures, "
+                         "the launch shape per adapter touched is unchanged")
     ap.add_argument("--tp", action="store_true",
                     help="the tensor-parallel adapter wave over --gpus ranks instead of replicas of the step")
     ap.add_argument("--tp-backend", default="nccl", choices=["nccl", "gloo"], dest="tp_backend")

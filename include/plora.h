@@ -67,7 +67,7 @@ enum {
 
 /* Which kernels plora_lora_delta uses. */
 enum {
-    PLORA_PATH_AUTO = 0,    /* fused BGMV for short segments; in batches of 512+ tokens the tensor-core
+    PLORA_PATH_AUTO = 0,    /* fused BGMV for short segments; in batches of 1024+ tokens the tensor-core
                                segmented GEMM takes the long ones: a CTA per tile of 64 rows when they make
                                at least 128 tiles together, a cluster of eight CTAs per tile when fewer */
     PLORA_PATH_UNFUSED = 1, /* BGMV shrink kernel then BGMV expand kernel, m in HBM workspace */
@@ -187,7 +187,7 @@ PLORA_API plora_status plora_bucket_view(plora_ctx *ctx, const int32_t **perm, c
  * (Section VI-B).  Each element of y receives exactly one addition, so results are
  * bit-reproducible run to run.
  * Tensor memory.  Segments that take the tensor-core path (PLORA_PATH_AUTO on batches
- * of 512+ tokens, PLORA_PATH_SGMV always) run in a kernel whose CTAs each allocate 256
+ * of 1024+ tokens, PLORA_PATH_SGMV and PLORA_PATH_SGMV_SPLIT always) run in a kernel whose CTAs each allocate 256
  * of an SM's 512 tensor-memory columns, two CTAs per SM (one per SM for pools with
  * ranks above 64).  The allocation instruction has no time limit: it blocks while
  * another kernel resident on the same SM (a base-model GEMM on a second stream, say)

@@ -59,7 +59,10 @@ struct DeviceGuard {
 };
 
 constexpr int kDefaultSgmvMinRows = 32;   // AUTO: segments at least this long take the tensor-core path ...
-constexpr int kSgmvMinBatch = 512;        // ... in batches at least this large (a decode batch stays one launch)
+// ... in batches at least this large (a decode batch stays one launch).  The host cannot know whether a batch has such
+// a segment, and a tensor-core launch that finds none still takes its place in the stream's chain of launches (2 to
+// 4 us each): measured on 512 uniformly tagged tokens (the 13B decode workload) it cost 2.5 % of the step.
+constexpr int kSgmvMinBatch = 1024;
 // ... and only if they make at least this many 64-row tiles together: a tile is one CTA's serial chain
 // over the whole width (with 8 tiles allowed, the mixed batch of config 5 took 0.52 ms instead of 0.34)
 constexpr int kSgmvMinTiles = 128;
