@@ -96,19 +96,27 @@ __device__ __forceinline__ long long wait_limit(const int32_t* status) {
     return v > 0 ? v : kWaitCycles;
 }
 // Bounded wait on an mbarrier phase; false when the CTA has given up (here or elsewhere).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
-    if (mbar_try_wait(bar, parity)) return true;
+// (The slow path is a real call here: inlined, its timing variables raised the register pressure of the grouped-query
+// variants, which sit at their register limit, and doubled their spills; the call costs those kernels nothing measurable.
+// The BGMV kernel is the opposite case: there a called slow path cost 4 %, see bgmv.cu.)
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
     const long long t0 = clock64();
+    long long limit = 0;
     for (;;) {
         for (int i = 0; i < 64; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > wait_limit(status)) break;
+        if (limit == 0) limit = wait_limit(status);
+        if (clock64() - t0 > limit) break;
     }
     *abort_flag = 1;
     __threadfence_block();
     atomicCAS(status, 0, PLORA_ERR_TIMEOUT);
     return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag, status);
 }
 // The copy thread's last look at a stage before it leaves: waits whatever the abort flag says, for at
 // most the limit (a CTA must not retire with a copy still on its way into its shared memory).
@@ -240,6 +248,7 @@ partial_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         }
         mbar_init(meet, kConsumerWarps);   // where the consumer warps meet at the end of an item (a bounded wait, like all others)
         *abort_flag = 0;
+        abort_flag[1] = p.w.status[kHookWord] == PLORA_HOOK_WITHHOLD_RELEASE;   // test hook: warp 0 never hands a stage back
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -314,7 +323,9 @@ partial_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     uint32_t meetings = 0;
     bool alive = true;
     // test hook: warp 0 never hands a stage back, so the copy thread's wait for a free stage runs out
-    const bool withhold = warp == 0 && p.w.status[kHookWord] == PLORA_HOOK_WITHHOLD_RELEASE;
+    // (the hook's flag sits in shared memory next to the abort flag and is looked up at every release: a value kept in
+    // a register for the whole kernel pushed the grouped-query variants, which are at their register limit, into spills)
+    volatile int* hook_flag = abort_flag + 1;
     // A lane whose wait for a stage fails leaves the loop and, with it, the kernel, without another
     // warp-level operation (shuffles and warp barriers are defined over the lanes that have not exited);
     // at the meetings, which are rare, the warp votes so that its lanes go on or stop together.
@@ -513,10 +524,10 @@ partial_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the stage goes back to the copy engine
             }
             __syncwarp();
-            if (lane == 0 && !withhold) mbar_arrive(empty + slot * 8);
+            if (lane == 0 && !(warp == 0 && *hook_flag)) mbar_arrive(empty + slot * 8);
         } else {
             __syncwarp();
-            if (lane == 0 && !withhold) mbar_arrive(empty + slot * 8);
+            if (lane == 0 && !(warp == 0 && *hook_flag)) mbar_arrive(empty + slot * 8);
             if (h.flags & kFlagLast) {
                 // anchor merge of the eight warps' shares of this item
                 float* mine = merge + warp * kMergeStride;
