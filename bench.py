@@ -47,16 +47,18 @@ FALLBACK_HBM_GBS = 6650.0   # used only when MEASURED_PEAKS.json is absent
 # library at the commit named in NCU_TRAFFIC_BUILD; the roofline entry scales the figure to the average
 # launch (a launch may carry a group of projections).  A capture says nothing about a later build of the
 # kernels: the line prints the build next to the figure, and null for a workload that was not captured.
-NCU_TRAFFIC_BUILD = "a048f9c"
+NCU_TRAFFIC_BUILD = "a5cdd72"
 NCU_TRAFFIC_BYTES = {
-    "decode7b": 40.17e6,   # q/k/v launch 116.44 + 3.84 MB, o launch 40.31 + 0.09 MB, over four projections
-    # captured on the four 5120 -> 5120 projections (567.3 MB each against 565.0 MB of algorithmic bytes);
-    # the step's 5120 <-> 13824 projections are scaled by their algorithmic bytes
-    "decode13b": ("of_algorithmic", 567.3 / 565.0),
-    "prefill": 622.7e6,    # the tensor-core kernel, one projection
-    "mixed": 518.8e6,      # the four rank-class launches of one projection
-    "skew7b": 91.5e6,      # q/k/v launch 272.8 MB, o launch 93.3 MB, over four projections
+    "decode7b": 40.2e6,    # q/k/v launch 120.46 MB, o launch 40.32 MB, over four projections
+    # captured with 150 adapters per pool (2103.4 MB of traffic for 2116.3 MB of algorithmic bytes over one layer's
+    # four launches); the full workload's algorithmic bytes are scaled by this ratio
+    "decode13b": ("of_algorithmic", 2103.4 / 2116.3),
+    "prefill": 622.2e6,    # the wide tensor-core kernel, one projection
+    "mixed": 525.7e6,      # the four rank-class launches and the split tensor-core launch of one projection
+    "skew7b": 93.2e6,      # q/k/v launch 276.93 MB, o launch 95.85 MB, over four projections
 }
+# decode attention, per call (one layer's cache) of the partial kernel, at the default shapes with one query head per KV head
+NCU_ATTN_TRAFFIC_BYTES = {False: 2604.8e6, True: 3241.3e6}   # short requests / long requests
 
 
 # ----------------------------------------------------------------------------------
@@ -718,7 +720,9 @@ def attention_entry(args, long_ctx: bool, steps: int) -> dict:
                     l2="inputs larger than L2: a step streams %.2f GB of KV cache" % (kv_bytes / 1e9)),
         clocks=clocks, gpu_launches=3 * layers * steps,
         roofline=dict(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s", frac=achieved / peaks["hbm_gbs"],
-                      traffic=None, kernel="attn partial_kernel (chunked partial softmax)", peak_source=peaks["source"],
+                      traffic=NCU_ATTN_TRAFFIC_BYTES[long_ctx] * layers if G == 1 and not args.attn_requests else None,
+                      traffic_from_build=NCU_TRAFFIC_BUILD if G == 1 and not args.attn_requests else None,
+                      kernel="attn partial_kernel (chunked partial softmax)", peak_source=peaks["source"],
                       read_peak=read_gbs, frac_of_read_peak=None if read_gbs is None else achieved / read_gbs,
                       algorithmic_bytes_per_step=kv_bytes + other),
         cpu_baseline=dict(value=len(sample) / cpu_s, unit="requests/s", cores=1, kind="oracle",
