@@ -64,3 +64,19 @@ def test_reregistration_replaces_the_pool():
     r.slab = r.ctx.register_pool(0, 0, 64, 64, p["ranks"], p["scales"], p["A"], zB)
     assert np.all(r.delta(P.PATH_FUSED) == 0) and np.any(first != 0)
     r.close()
+
+
+def test_read_bandwidth_probe():
+    # the probe folds what it reads into per-block checksums: their XOR is the XOR of all words of the buffer
+    n = (8 << 20) + 4096 + 16                      # not a multiple of the kernel's stride: the tail loop runs too
+    buf = torch.randint(-2**31, 2**31 - 1, (n // 4,), dtype=torch.int32, device=DEV)
+    sink = torch.zeros(1 << 14, dtype=torch.int32, device=DEV)
+    assert P.plora_stream_read(buf.data_ptr(), n, sink.data_ptr(), sink.numel() * 4) == P.OK
+    torch.cuda.synchronize()
+    want = np.bitwise_xor.reduce(buf.cpu().numpy().view(np.uint32))
+    got = np.bitwise_xor.reduce(sink.cpu().numpy().view(np.uint32))
+    assert got == want
+    assert P.plora_stream_read(buf.data_ptr(), n, sink.data_ptr(), 16) == P.ERR_WORKSPACE        # sink too small
+    assert P.plora_stream_read(buf.data_ptr() + 4, n - 16, sink.data_ptr(), 1 << 16) == P.ERR_INVALID_ARG
+    assert P.plora_stream_read(buf.data_ptr(), n - 8, sink.data_ptr(), 1 << 16) == P.ERR_INVALID_ARG
+    assert P.plora_stream_read(0, n, sink.data_ptr(), 1 << 16) == P.ERR_INVALID_ARG

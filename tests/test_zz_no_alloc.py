@@ -48,6 +48,15 @@ def test_two_calls_in_a_row_match_the_ordinary_entry_point():
             assert np.max(np.abs(got - want)) <= TOL_FP32_PATH * scale + 1e-6 * np.max(np.abs(want))
         assert r.ctx.launch_count() > before
         assert r.ctx.device_status() == 0
+        # after the first call on the device (which looked the array's address up), a call allocates nothing:
+        # the device's free memory is the same before and after, with everything the call needs made beforehand
+        ids = torch.from_numpy(np.ascontiguousarray(ids_a, np.int32)).to(DEV)
+        y = torch.from_numpy(p["y_in"]).to(DEV)
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
+        rc = P.plora_lora_delta_noalloc(r.ctx.handle, r.x.data_ptr(), ids.data_ptr(), p["T"], 0, 0, y.data_ptr())
+        torch.cuda.synchronize()
+        assert rc == P.OK and torch.cuda.mem_get_info()[0] == free_before
     finally:
         r.close()
 
