@@ -1515,7 +1515,7 @@ cudaError_t bgmv_configure() {
 cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const BucketDev& bk, int n_tok,
                         const void* const* x, float* const* y, void* m, int ldm, bool m16, bool fp16, int32_t* status,
                         int sm_count, bool early_tables, ClassCache* cls_cache, uint64_t rank_sig, const DebugCfg& dbg,
-                        cudaStream_t stream, int* n_launches) {
+                        cudaStream_t stream, int* n_launches, BetweenLaunch between, void* between_arg) {
     if (n_groups < 1 || n_groups > kMaxGroup || (mode != kFused && n_groups != 1)) return cudaErrorInvalidValue;
     const PoolDev& pool = pools[0];
     Params p;
@@ -1563,6 +1563,12 @@ cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const
             cls_cache->sig = rank_sig;
             cls_cache->valid = true;
         }
+    }
+    if (between) {
+        const cudaError_t e = between(between_arg, n_launches);
+        if (e != cudaSuccess) return e;
+        p.early_tables = 1;                          // what follows comes after a kernel that is not the bucket kernel,
+        p.defer_wait = mode == kFused ? 1 : 0;       // and that kernel has joined the stream's order for the whole call
     }
     // one launch per padded-rank class present in the pool
     if (p.by_class && mode == kFused && (long long)n_tok * n_groups <= kMixedLaunchMaxRows) {

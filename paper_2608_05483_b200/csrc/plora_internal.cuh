@@ -145,10 +145,15 @@ struct DebugCfg {
     int32_t test_hook = 0;       // PLORA_HOOK_*
     bool maybe_empty = false;    // the bucket may hold tensor-core segments only (BGMV launches look before they set up)
 };
+// between: a launch the caller wants between the classify pass (if one is needed) and the BGMV launches, nullptr for
+// none: the split tensor-core launch of the same call, which works on other tokens.  It joins the stream's order (the
+// BGMV launches behind it then need not), and its CTAs, one per SM for a few tens of microseconds, overlap the BGMV
+// launches instead of trailing them.  It gets its argument and the launch counter and returns its launch's error.
+typedef cudaError_t (*BetweenLaunch)(void* arg, int* n_launches);
 cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const BucketDev& bk, int n_tok,
                         const void* const* x, float* const* y, void* m, int ldm, bool m16, bool fp16, int32_t* status,
                         int sm_count, bool early_tables, ClassCache* cls_cache, uint64_t rank_sig, const DebugCfg& dbg,
-                        cudaStream_t stream, int* n_launches);
+                        cudaStream_t stream, int* n_launches, BetweenLaunch between = nullptr, void* between_arg = nullptr);
 // after_bgmv_of_same_call: the launch follows fused BGMV launches of the same call (other tokens of the
 // same batch) and may overlap them
 cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, int sgmv_min_rows, const void* x, float* y,

@@ -672,3 +672,40 @@ def test_three_long_segments_in_a_decode_batch_take_the_tensor_cores():
         assert r.ctx.device_status() == 0
     finally:
         r.close()
+
+
+def test_grouped_call_with_long_segments_in_a_mid_sized_batch():
+    """q, k, v of a layer in one call on a 1536-token batch with a few long segments: the three split tensor-core
+    launches go ahead of the one BGMV launch of the group; results as from three separate calls, and as the oracle's."""
+    rng = np.random.default_rng(41)
+    N = 400
+    ids = np.concatenate([np.repeat(np.array([3, 77]), 150), rng.integers(-1, N, size=1236)]).astype(np.int32)
+    rng.shuffle(ids)
+    p = random_problem(42, T=len(ids), d_in=512, d_out=520, ranks=np.full(N, 32))
+    p["ids"] = ids
+    ctx = P.Context(p["T"], N)
+    try:
+        xd = bits_to_dev(p["x"])
+        idt = torch.from_numpy(ids).to(DEV)
+        Bs = []
+        for proj in range(3):
+            B = [f32_to_bf16_bits(np.random.default_rng(100 + proj).standard_normal(b.shape, dtype=np.float32) / np.float32(np.sqrt(32))) for b in p["B"]]
+            Bs.append(B)
+            ctx.register_pool(0, proj, p["d_in"], p["d_out"], p["ranks"], p["scales"], p["A"], B)
+        ctx.set_path(P.PATH_AUTO)
+        ys = [torch.zeros((p["T"], p["d_out"]), dtype=torch.float32, device=DEV) for _ in range(3)]
+        ctx.bucket(idt, N)
+        n0 = ctx.launch_count()
+        ctx.lora_delta_group([xd] * 3, idt, [0] * 3, [0, 1, 2], ys)
+        torch.cuda.synchronize()
+        assert ctx.launch_count() - n0 == 3 + 1            # three split launches, one BGMV launch for the group
+        for proj in range(3):
+            want = oracle.lora_delta(p["x"], ids, p["ranks"], p["scales"], p["A"], Bs[proj], p["d_out"])
+            assert rel_err(ys[proj].cpu().numpy(), want) <= TOL_FP32_PATH, proj
+            alone = torch.zeros_like(ys[proj])
+            ctx.lora_delta(xd, idt, 0, proj, alone)
+            torch.cuda.synchronize()
+            assert rel_err(alone.cpu().numpy(), want) <= TOL_FP32_PATH
+        assert ctx.device_status() == 0
+    finally:
+        ctx.close()
