@@ -709,3 +709,46 @@ def test_grouped_call_with_long_segments_in_a_mid_sized_batch():
         assert ctx.device_status() == 0
     finally:
         ctx.close()
+
+
+@pytest.mark.parametrize("rank", [8, 32])
+def test_grouped_call_on_a_prefill_batch(rank):
+    """q, k, v of a layer on a batch whose long segments all go to the wide tensor-core shape: one BGMV launch for the
+    group's short segments and one tensor-core launch per projection (their own A, B and scales); results as the
+    oracle's, and as from separate calls."""
+    rng = np.random.default_rng(51)
+    N, n_seg = 200, 130
+    ids = np.concatenate([np.repeat(rng.permutation(N)[:n_seg], 64), rng.integers(-1, N, size=180)]).astype(np.int32)
+    p = random_problem(52 + rank, T=len(ids), d_in=328, d_out=264, ranks=np.full(N, rank))
+    p["ids"] = ids
+    ctx = P.Context(p["T"], N)
+    try:
+        xd = bits_to_dev(p["x"])
+        idt = torch.from_numpy(ids).to(DEV)
+        pools = []
+        for proj in range(3):
+            r2 = np.random.default_rng(200 + proj)
+            A = [f32_to_bf16_bits(r2.standard_normal(a.shape, dtype=np.float32) / np.float32(np.sqrt(p["d_in"]))) for a in p["A"]]
+            B = [f32_to_bf16_bits(r2.standard_normal(b.shape, dtype=np.float32) / np.float32(np.sqrt(rank))) for b in p["B"]]
+            sc = r2.choice(np.array([0.5, 1.0, 2.0], np.float32), size=N).astype(np.float32)
+            pools.append((A, B, sc))
+            ctx.register_pool(0, proj, p["d_in"], p["d_out"], p["ranks"], sc, A, B)
+        ctx.set_path(P.PATH_AUTO)
+        ys = [torch.from_numpy(p["y_in"]).to(DEV) for _ in range(3)]
+        ctx.bucket(idt, N)
+        n0 = ctx.launch_count()
+        ctx.lora_delta_group([xd] * 3, idt, [0] * 3, [0, 1, 2], ys)
+        torch.cuda.synchronize()
+        assert ctx.launch_count() - n0 == 1 + 3            # one BGMV launch for the group, one tensor-core launch per projection
+        for proj, (A, B, sc) in enumerate(pools):
+            want = oracle.lora_delta(p["x"], ids, p["ranks"], sc, A, B, p["d_out"], p["y_in"])
+            scale = np.max(np.abs(want - p["y_in"]))
+            got = ys[proj].cpu().numpy()
+            assert np.max(np.abs(got - want)) <= TOL_FP32_PATH * scale + 1e-6 * np.max(np.abs(want)), proj
+            alone = torch.from_numpy(p["y_in"]).to(DEV)
+            ctx.lora_delta(xd, idt, 0, proj, alone)
+            torch.cuda.synchronize()
+            assert np.max(np.abs(alone.cpu().numpy() - want)) <= TOL_FP32_PATH * scale + 1e-6 * np.max(np.abs(want))
+        assert ctx.device_status() == 0
+    finally:
+        ctx.close()
