@@ -367,7 +367,8 @@ def measure_lora(cfg: int, args, local: int, world: int, rank: int, headline: bo
     dw = DeviceWorkload(wl, local, fp16=args.dtype == "fp16")
     dw.grouped = not args.no_group
     ctx = dw.ctx
-    ctx.set_path({"auto": P.PATH_AUTO, "fused": P.PATH_FUSED, "unfused": P.PATH_UNFUSED, "sgmv": P.PATH_SGMV}[args.path])
+    ctx.set_path({"auto": P.PATH_AUTO, "fused": P.PATH_FUSED, "unfused": P.PATH_UNFUSED, "sgmv": P.PATH_SGMV,
+                  "sgmv_split": P.PATH_SGMV_SPLIT}[args.path])
     n_calls = len(wl.pools)
     steps = args.steps if headline else max(10, min(args.steps, 50))
     warmup = max(3, args.warmup)
@@ -922,7 +923,7 @@ def main():
     ap.add_argument("--cpu-pools", type=int, default=64, dest="cpu_pools")
     ap.add_argument("--cpu-seconds", type=float, default=20.0, dest="cpu_seconds",
                     help="target CPU time of the oracle sample (cpu_baseline leg)")
-    ap.add_argument("--path", default="auto", choices=["auto", "fused", "unfused", "sgmv"])
+    ap.add_argument("--path", default="auto", choices=["auto", "fused", "unfused", "sgmv", "sgmv_split"])
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp16"], help="16-bit type of x, A and B (fp16 = the paper's own)")
     ap.add_argument("--no-group", action="store_true", dest="no_group",
                     help="one call per projection instead of grouping q/k/v and up/gate")
