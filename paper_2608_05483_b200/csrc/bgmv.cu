@@ -897,8 +897,11 @@ __device__ __forceinline__ bool gather_m(const Params& p, int rp, int runs_a, ui
 // the large ones far behind (measured 2x slower than one launch per class), so the classes are cut to
 // tasks of about the same size, chosen so that a CTA gets about kTasksPerCta tasks per phase: between
 // kTaskBytesMin and kTaskBytesMax of adapter bytes.  A unit of padded rank 128 then makes up to 16
-// shrink tasks (4 column runs x 4 row slices) and 16 expand tasks, one of rank 8 one and one.
-constexpr int kTaskBytesMin = 16 * 1024, kTaskBytesMax = 32 * 1024, kTasksPerCta = 4;
+// shrink tasks (4 column runs x 4 row slices) and 16 expand tasks, one of rank 8 at least one and one.
+// (Between 32 and 256 KiB: with tasks of 16 to 32 KiB, one or two stages each, the hand-over of a partial m per task
+// and the gather before every expand task weighed more than the finer balance gained; the paper's skewed decode mix
+// on 8 layers took 0.906 ms per step with those, 0.857 ms with these, and no more with a ceiling of 512 KiB or 1 MiB.)
+constexpr int kTaskBytesMin = 32 * 1024, kTaskBytesMax = 256 * 1024, kTasksPerCta = 4;
 // The one launch pays off for small batches, where the per-class launches are mostly fixed cost
 // (256 tokens, ranks 8..128, q/k/v grouped: 1.10 -> 1.00 ms for 8 layers); with many units per
 // class the per-class launches, each with loops compiled for its rank, are faster (2048 tokens,
@@ -1011,7 +1014,7 @@ __device__ __forceinline__ Plan<RPK ? 1 : kRankClasses> make_plan(const Params& 
             tot_a += (long long)pl.n[i] * p.pool.d_in * rp * 2;
             tot_b += (long long)pl.n[i] * p.pool.d_out * rp * 2;
         }
-        // task size: about three tasks per CTA and phase, between two tiles and eight
+        // task size: about kTasksPerCta tasks per CTA and phase, within the bounds above
         const int tgt_a = clamp_int((int)(tot_a / (kTasksPerCta * (long long)gridDim.x)), kTaskBytesMin, kTaskBytesMax);
         const int tgt_b = clamp_int((int)(tot_b / (kTasksPerCta * (long long)gridDim.x)), kTaskBytesMin, kTaskBytesMax);
 #pragma unroll
