@@ -15,7 +15,11 @@ entry point (pinned host memory, copies inside the timed region); `roofline`
 compares the dominant kernel's algorithmic bytes per launch with the measured
 HBM copy bandwidth and with a read-only streaming bandwidth measured in the same
 run; `cpu_baseline` is the float64 oracle timed on this machine's host cores on a
-bounded sample.  Without --config the headline (config 2) is followed, in the
+bounded sample.  The step's x, ids and y are resident before the step starts, and the
+benchmark says so to the library (plora_set_inputs_resident; --resident 0 withholds
+the hint): the fused kernels then read x while the previous launch drains.
+`roofline.frac_without_inputs_hint` is the same set of launches without the hint.
+Without --config the headline (config 2) is followed, in the
 same process, by the other benchmark workloads (configs 3 to 6 and decode
 attention), each with its own roofline, full-size parity figure, oracle time and
 clocks, under the key `per_config`.  --impl reference times the oracle alone.
@@ -150,7 +154,7 @@ class ClockSampler:
 class DeviceWorkload:
     """Pools registered in a library context plus per-call activations, all resident in HBM."""
 
-    def __init__(self, wl, device_index: int, max_tokens=None, fp16: bool = False):
+    def __init__(self, wl, device_index: int, max_tokens=None, fp16: bool = False, resident: bool = True):
         import torch
         import paper_2608_05483_b200 as P
         self.P, self.torch, self.wl = P, torch, wl
@@ -160,6 +164,8 @@ class DeviceWorkload:
         self.ctx = P.Context(max_tokens or wl.n_tok, wl.n_adapters, device=device_index)
         if fp16:
             self.ctx.set_input_type(True)
+        # every x of the step sits in HBM before the step starts: the kernels may read it while the previous one drains
+        self.ctx.set_inputs_resident(resident)
         self.ids = torch.from_numpy(wl.ids).to(self.dev)
         g = torch.Generator(device=self.dev)
         g.manual_seed(wl.seed)
@@ -364,7 +370,7 @@ def measure_lora(cfg: int, args, local: int, world: int, rank: int, headline: bo
     import paper_2608_05483_b200 as P
 
     wl = make_workload(cfg, n_layers=args.layers if headline else None, n_adapters=args.adapters if headline else None)
-    dw = DeviceWorkload(wl, local, fp16=args.dtype == "fp16")
+    dw = DeviceWorkload(wl, local, fp16=args.dtype == "fp16", resident=bool(args.resident))
     dw.grouped = not args.no_group
     ctx = dw.ctx
     ctx.set_path({"auto": P.PATH_AUTO, "fused": P.PATH_FUSED, "unfused": P.PATH_UNFUSED, "sgmv": P.PATH_SGMV,
@@ -460,6 +466,24 @@ def measure_lora(cfg: int, args, local: int, world: int, rank: int, headline: bo
     deltas_ms = e0.elapsed_time(e1) / reps                 # all delta launches of one step
     kernel_ms = deltas_ms / n_calls                        # per (layer, proj) delta, however they are grouped
 
+    # the same launches without the inputs-resident hint (every kernel touches x only after the one before it has
+    # completed): what a caller gets who cannot make that statement about its x
+    deltas_ms_no_hint = None
+    if args.resident and not args.no_extras:
+        ctx.set_inputs_resident(False)
+        g2, _ = capture(dw.deltas)
+        for _ in range(3):
+            g2.replay() if g2 is not None else dw.deltas()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(reps):
+            g2.replay() if g2 is not None else dw.deltas()
+        e1.record()
+        torch.cuda.synchronize()
+        deltas_ms_no_hint = e0.elapsed_time(e1) / reps
+        ctx.set_inputs_resident(True)
+        del g2
+
     per_call = [algorithmic_bytes(wl.ids, wl.ranks, p.d_in, p.d_out) for p in wl.pools]
     step_bytes = sum(b["total"] for b in per_call)
     step_adapter_bytes = sum(b["adapter"] for b in per_call)
@@ -485,6 +509,8 @@ def measure_lora(cfg: int, args, local: int, world: int, rank: int, headline: bo
                     # against a kernel that only reads, measured in this run (the copy peak counts reads and writes)
                     read_peak=read_gbs, frac_of_read_peak=None if read_gbs is None else achieved / read_gbs,
                     frac_of_nominal_8tbs=achieved / 8000.0,
+                    frac_without_inputs_hint=None if deltas_ms_no_hint is None
+                    else step_bytes / (deltas_ms_no_hint * 1e-3) / 1e9 / peaks["hbm_gbs"],
                     adapter_bytes_only_gbs=step_adapter_bytes / n_calls / (kernel_ms * 1e-3) / 1e9,
                     step_gbs=step_bytes / (ms_per_step * 1e-3) / 1e9)
     return dict(wl=wl, dw=dw, ms_per_step=ms_per_step, steps=steps, warmup=warmup, clocks=clocks, launches=int(launches),
@@ -529,6 +555,7 @@ def config_entry(m: dict, args, cfg: int) -> dict:
                 layers=len({p.layer for p in wl.pools}), calls_per_step=m["n_calls"],
                 ranks=sorted({int(r) for r in wl.ranks}), ids=wl.meta.get("ids"), accumulate="fp32", y="fp32",
                 distinct_adapters=m["distinct"], path=args.path, cuda_graph=bool(args.graph), grouped_calls=not args.no_group,
+                inputs_resident_hint=bool(args.resident),
                 l2="inputs larger than L2: a step streams %.2f GB through %d distinct slabs" % (m["step_bytes"] / 1e9, m["n_calls"]))
 
 
@@ -925,6 +952,8 @@ def main():
                     help="target CPU time of the oracle sample (cpu_baseline leg)")
     ap.add_argument("--path", default="auto", choices=["auto", "fused", "unfused", "sgmv", "sgmv_split"])
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp16"], help="16-bit type of x, A and B (fp16 = the paper's own)")
+    ap.add_argument("--resident", type=int, default=1, choices=[0, 1],
+                    help="1: tell the library that the step's inputs are resident before the step starts (plora_set_inputs_resident)")
     ap.add_argument("--no-group", action="store_true", dest="no_group",
                     help="one call per projection instead of grouping q/k/v and up/gate")
     ap.add_argument("--no-cpu", action="store_true", dest="no_cpu")

@@ -327,6 +327,20 @@ PLORA_API plora_status plora_set_path(plora_ctx *ctx, int32_t path, int32_t sgmv
 PLORA_API plora_status plora_set_input_type(plora_ctx *ctx, int32_t type);
 
 /*
+ * Hint about the inputs of the following calls (no counterpart in the paper; default 0).  The fused decode
+ * kernels are launched so that they may start while the previous kernel of the stream is still running
+ * (programmatic dependent launch).  By default they read x only after that kernel has completed, because
+ * it may be the kernel that produces x.  With resident = 1 the caller states that the x of every
+ * following call was complete in memory before the previous kernel of the stream began: true when deltas
+ * are issued back to back on inputs produced earlier (q/k/v of a layer, a benchmark on resident inputs),
+ * false when the kernel right before a call writes its x and signals its dependents early.  The kernels
+ * then stream and multiply x while the previous kernel drains; they still write nothing (workspace, y)
+ * and read no y before it has completed, and the results are bit-identical to those with resident = 0.
+ * Wrong use is a data race on x, nothing else.  The tensor-core path and the unfused halves ignore the hint.
+ */
+PLORA_API plora_status plora_set_inputs_resident(plora_ctx *ctx, int32_t resident);
+
+/*
  * Diagnostics of the bounded device-side waits (no counterpart in the paper).  Every wait inside the
  * kernels (on a shared-memory barrier, or on partial sums from another CTA) gives up after a number of
  * SM clock cycles, records PLORA_ERR_TIMEOUT in the status word, and the kernel winds down: no role

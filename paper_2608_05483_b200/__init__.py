@@ -10,5 +10,5 @@ from .binding import (  # noqa: F401
     plora_launch_count, plora_lora_delta, plora_lora_delta_group, plora_lora_delta_host, plora_lora_delta_host_async, plora_host_sync, plora_lora_delta_noalloc, plora_pool_max_rank, plora_pool_slab_bytes,
     plora_register_pool, plora_set_path, plora_shrink, plora_shrink_m16, status_string,
     attn_decode, plora_attn_decode, plora_attn_set_debug, plora_attn_status, plora_attn_workspace_bytes,
-    plora_set_test_hook, plora_set_wait_limit, plora_stream_read, HOOK_NONE, HOOK_WITHHOLD_RELEASE, HOOK_MAX_CYCLES,
+    plora_set_test_hook, plora_set_wait_limit, plora_set_inputs_resident, plora_stream_read, HOOK_NONE, HOOK_WITHHOLD_RELEASE, HOOK_MAX_CYCLES,
 )

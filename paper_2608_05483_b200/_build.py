@@ -32,6 +32,16 @@ def sources():
     return sorted(CSRC.glob("*.cu"))
 
 
+def _included_sources(src: Path):
+    """Sources a .cu file includes (a translation unit that compiles another one's templates)."""
+    out = []
+    for line in src.read_text().splitlines():
+        line = line.strip()
+        if line.startswith('#include "') and line.endswith('.cu"'):
+            out.append(CSRC / line[len('#include "'):-1])
+    return out
+
+
 def _stale(target: Path, deps) -> bool:
     if not target.exists():
         return True
@@ -54,7 +64,7 @@ def build(force: bool = False, verbose: bool = False, extra_flags=(), debug: boo
     for src in sources():
         obj = obj_dir / (src.stem + ".o")
         objs.append(obj)
-        if force or _stale(obj, [src, *headers]):
+        if force or _stale(obj, [src, *_included_sources(src), *headers]):
             cmd = [nvcc, *NVCC_FLAGS, *extra_flags, "-c", str(src), "-o", str(obj)]
             if verbose:
                 print(" ".join(cmd))

@@ -34,7 +34,7 @@ EXPORTS = (
     "plora_shrink_m16", "plora_expand_m16", "plora_set_input_type",
     "plora_lora_delta_host", "plora_lora_delta_host_async", "plora_host_sync", "plora_lora_delta_noalloc", "plora_set_path", "plora_device_status", "plora_launch_count", "plora_status_string",
     "plora_cost_model", "plora_attn_workspace_bytes", "plora_attn_decode", "plora_attn_status", "plora_attn_set_debug",
-    "plora_set_wait_limit", "plora_set_test_hook", "plora_stream_read",
+    "plora_set_wait_limit", "plora_set_test_hook", "plora_set_inputs_resident", "plora_stream_read",
 )
 
 HOOK_NONE, HOOK_WITHHOLD_RELEASE, HOOK_MAX_CYCLES = 0, 1, 1 << 24
@@ -120,6 +120,7 @@ def load(build_if_missing: bool = True):
         "plora_attn_set_debug": (i32, [vp, i64, i32, vp]),
         "plora_set_wait_limit": (i32, [vp, i64]),
         "plora_set_test_hook": (i32, [vp, i32]),
+        "plora_set_inputs_resident": (i32, [vp, i32]),
         "plora_stream_read": (i32, [vp, ctypes.c_size_t, vp, ctypes.c_size_t, vp]),
         "plora_cost_model": (i32, [ctypes.POINTER(CostHw), i32, vp, vp, ctypes.c_double, ctypes.c_double, ctypes.c_double,
                                    ctypes.POINTER(CostTerms)]),
@@ -187,6 +188,10 @@ def plora_set_wait_limit(ctx, cycles: int):
 
 def plora_set_test_hook(ctx, hook: int):
     return load().plora_set_test_hook(ctx, int(hook))
+
+
+def plora_set_inputs_resident(ctx, resident: bool):
+    return load().plora_set_inputs_resident(ctx, 1 if resident else 0)
 
 
 def plora_stream_read(buf_ptr, nbytes: int, sink_ptr, sink_bytes: int, stream=0):
@@ -477,6 +482,9 @@ class Context:
 
     def set_test_hook(self, hook: int):
         _check(plora_set_test_hook(self._h, hook), "plora_set_test_hook")
+
+    def set_inputs_resident(self, resident: bool):
+        _check(plora_set_inputs_resident(self._h, resident), "plora_set_inputs_resident")
 
     def set_input_type(self, fp16: bool):
         _check(load().plora_set_input_type(self._h, 1 if fp16 else 0), "plora_set_input_type")

@@ -330,7 +330,7 @@ PLORA_API plora_status plora_create(plora_ctx** out, int device, int32_t max_tok
             return PLORA_ERR_CUDA;
         }
     }
-    if (bucket_configure() != cudaSuccess || bgmv_configure() != cudaSuccess || sgmv_configure() != cudaSuccess ||
+    if (bucket_configure() != cudaSuccess || bgmv_configure() != cudaSuccess || sgmv_configure() != cudaSuccess || bgmv_configure_lazy() != cudaSuccess ||
         cudaDeviceSynchronize() != cudaSuccess) {
         cudaFree(blk);
         delete ctx;
@@ -504,6 +504,12 @@ PLORA_API plora_status plora_set_test_hook(plora_ctx* ctx, int32_t hook) {
     if (hook != PLORA_HOOK_NONE && (ctx->dbg.wait_cycles < 1 || ctx->dbg.wait_cycles > PLORA_HOOK_MAX_CYCLES))
         return PLORA_ERR_INVALID_ARG;
     ctx->dbg.test_hook = hook;
+    return PLORA_OK;
+}
+
+PLORA_API plora_status plora_set_inputs_resident(plora_ctx* ctx, int32_t resident) {
+    if (!ctx || (resident != 0 && resident != 1)) return PLORA_ERR_INVALID_ARG;
+    ctx->dbg.inputs_resident = resident != 0;
     return PLORA_OK;
 }
 

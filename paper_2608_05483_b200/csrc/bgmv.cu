@@ -96,9 +96,14 @@ struct Params {
     // still implies the completion of everything before it) and leaves the epoch to the last of them.
     int32_t defer_wait;
     int32_t bump_epoch;
+
     int32_t* status;
     long long wait_cycles;    // limit of every bounded wait, in SM clock cycles
     int32_t test_hook;        // PLORA_HOOK_*: tests make a wait run out with it
+    // The caller states that x was complete before the previous kernel of the stream began
+    // (plora_set_inputs_resident): the launch uses the kernels that stream and multiply x before they join
+    // the stream order, and join when they first have something to write (host side only).
+    int32_t inputs_resident;
 };
 
 // ---- PTX wrappers -----------------------------------------------------------------
@@ -242,10 +247,22 @@ struct Smem {
     uint32_t m_empty;    // m_empty[kMRing]: every consumer warp is done with the entry
     uint32_t epoch;      // this launch's epoch (fused mode)
     bool withhold;       // test hook: this warp never hands a stage back
+    bool joined;         // lazy launches: this thread has joined the stream order and knows the epoch
 };
 // A consumer warp is done with a stage.
 __device__ __forceinline__ void release_stage(const Smem& sm, uint32_t empty_bar, int lane) {
     if (lane == 0 && !sm.withhold) mbar_arrive(empty_bar);
+}
+
+// A consumer thread that put off joining the stream order does so now: from here on it may write
+// (partial words, y), and it knows the launch's epoch.
+__device__ __forceinline__ void join_stream(const Params& p, Smem& sm) {
+    if (!sm.joined) {
+        grid_dependency_wait();
+        grid_launch_dependents();
+        sm.epoch = *p.bk.epoch;
+        sm.joined = true;
+    }
 }
 
 // What a stage holds (written by the producer into the stage, read by every consumer warp).
@@ -756,7 +773,7 @@ struct LaneMaps {
 
 // One stage, consumer side.
 // (false: this lane gave up inside the stage)
-template <int MODE, int RP, bool H, bool TC>
+template <int MODE, int RP, bool H, bool TC, bool LAZY>
 __device__ __forceinline__ bool consume_stage(const Params& p, const Smem& sm, const StageHdr& h,
                                               const LaneMaps<RP, SliceCfg<MODE, RP>::kSliceRp>& maps, uint32_t tile, uint32_t empty_bar,
                                               float (&acc)[kMaxRowsPerLane][kTokChunk], int warp, int lane) {
@@ -780,6 +797,7 @@ __device__ __forceinline__ bool consume_stage(const Params& p, const Smem& sm, c
                 __syncwarp();
                 release_stage(sm, empty_bar, lane);
                 if (h.flags & kFlagLast) {
+                    if (LAZY) join_stream(p, const_cast<Smem&>(sm));   // (the kernel's own, non-const, object)
                     if (tc) shrink_finish_mma<MODE, RPS < 16 ? 16 : RPS>(p, sm, h, acc[0], warp, lane);
                     else shrink_finish<MODE, RPS>(p, sm, h, maps.s2, acc, warp, lane);
                 }
@@ -787,15 +805,23 @@ __device__ __forceinline__ bool consume_stage(const Params& p, const Smem& sm, c
                 shrink_tile_mma<RP < 16 ? 16 : RP, H>(p, h, tile, acc[0], warp, lane);
                 __syncwarp();
                 release_stage(sm, empty_bar, lane);
-                if (h.flags & kFlagLast) shrink_finish_mma<MODE, RP < 16 ? 16 : RP>(p, sm, h, acc[0], warp, lane);
+                if (h.flags & kFlagLast) {
+                    if (LAZY) join_stream(p, const_cast<Smem&>(sm));   // (the kernel's own, non-const, object)
+                    shrink_finish_mma<MODE, RP < 16 ? 16 : RP>(p, sm, h, acc[0], warp, lane);
+                }
             } else {
                 shrink_tile<RP, H>(p, h, maps.s, tile, acc);
                 __syncwarp();
                 release_stage(sm, empty_bar, lane);
-                if (h.flags & kFlagLast) shrink_finish<MODE, RP>(p, sm, h, maps.s, acc, warp, lane);
+                if (h.flags & kFlagLast) {
+                    if (LAZY) join_stream(p, const_cast<Smem&>(sm));   // (the kernel's own, non-const, object)
+                    shrink_finish<MODE, RP>(p, sm, h, maps.s, acc, warp, lane);
+                }
             }
         }
     } else {
+        // (a lazy launch needs no join here: the m this tile waits for is published by the gather warp, which
+        // joined the stream order before it read the first partial word, and the expand does not use the epoch)
         if (MODE != kShrinkOnly) return expand_tile<MODE, RP, H>(p, sm, h, maps.e, tile, empty_bar, lane);
     }
     return true;
@@ -804,7 +830,7 @@ __device__ __forceinline__ bool consume_stage(const Params& p, const Smem& sm, c
 // Consumes stages from stage `it` on for as long as they belong to padded rank RP (a one-class
 // launch: to the end).  Returns true when stage `it` is another class's (it has not been touched),
 // false when nothing follows or this lane gave up (gave_up: it must leave the kernel now).
-template <int MODE, int RP, bool H, bool ONLY>
+template <int MODE, int RP, bool H, bool ONLY, bool LAZY>
 __device__ __forceinline__ bool consume_class(const Params& p, const Smem& sm, uint32_t& it, bool& gave_up,
                                               float (&acc)[kMaxRowsPerLane][kTokChunk], int warp, int lane) {
     LaneMaps<RP, SliceCfg<MODE, RP>::kSliceRp> maps;   // per-lane constants of both phases
@@ -819,7 +845,7 @@ __device__ __forceinline__ bool consume_class(const Params& p, const Smem& sm, u
         const StageHdr h = read_hdr(tile + kHdrOffset);
         if (h.flags & kFlagEnd) return false;
         if (!ONLY && h.rp != RP) return true;
-        if (!consume_stage<MODE, RP, H, ONLY>(p, sm, h, maps, tile, sm.empty + slot * 8, acc, warp, lane)) {
+        if (!consume_stage<MODE, RP, H, ONLY, LAZY>(p, sm, h, maps, tile, sm.empty + slot * 8, acc, warp, lane)) {
             gave_up = true;
             return false;
         }
@@ -1049,6 +1075,7 @@ __device__ __forceinline__ Plan<RPK ? 1 : kRankClasses> make_plan(const Params& 
     return pl;
 }
 
+#ifndef PLORA_BGMV_LAZY_UNIT
 // Classify pass (pools of mixed ranks): sorts the bucket's units by the padded rank of the unit's
 // adapter, keeping their order inside a class, so that every class gets a dense list.  The ranks
 // are those of the call's first pool; the pools of a group, and every later call that reuses the
@@ -1117,11 +1144,14 @@ __global__ void __launch_bounds__(kClassifyThreads) classify_kernel(const Params
     }
 }
 
+#endif   // PLORA_BGMV_LAZY_UNIT
+
 // One instantiation per padded rank RPK.  The kernel handles the units whose adapter has that
 // padded rank and skips the others: a pool of mixed ranks is served by one launch per rank
 // class present in it, each with loops specialised (and registers allocated) for its rank.
-template <int MODE, int RPK, bool H>
+template <int MODE, int RPK, bool H, bool LAZY>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params p) {
+    static_assert(!LAZY || MODE == kFused, "only the fused kernel puts off its join");
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     Smem sm;
     sm.slots = smem_u32(smem_raw);
@@ -1173,13 +1203,22 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
     // issues the slab tiles of the ring's first turn while the previous kernel drains (config 2:
     // 1.134 -> 1.118 ms per step).  (Pulling tiles towards L2 with prefetches at that point, instead
     // of copying them into the ring, was tried earlier and was slower.)
+    if (LAZY) sm.joined = true;
     if (warp != kProducerWarp) {
-        if (!p.defer_wait) grid_dependency_wait();
-        // Signalled only after this CTA has seen the previous kernel complete (or, for a class launch
-        // that defers its wait, after the first class launch of the call has): when the next kernel of
-        // the stream starts, everything older than this call is therefore complete.
-        grid_launch_dependents();
-        sm.epoch = MODE == kFused ? *p.bk.epoch : 0u;
+        if (LAZY && !p.defer_wait && warp < kConsumerWarps) {
+            // The consumers of a launch whose x is known to be complete start on their first shrink task
+            // at once and join at its hand-over (join_stream); the gather warp below joins now, so the
+            // CTA still signals only after it has seen the previous kernel complete.
+            sm.joined = false;
+            sm.epoch = 0u;
+        } else {
+            if (!p.defer_wait) grid_dependency_wait();
+            // Signalled only after this CTA has seen the previous kernel complete (or, for a class launch
+            // that defers its wait, after the first class launch of the call has): when the next kernel of
+            // the stream starts, everything older than this call is therefore complete.
+            grid_launch_dependents();
+            sm.epoch = MODE == kFused ? *p.bk.epoch : 0u;
+        }
     }
 
     if (MODE == kShrinkOnly && warp != kProducerWarp) {
@@ -1204,6 +1243,8 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
         // the serial part of the producer is a few dozen instructions per stage.  In fused mode
         // the whole warp first gathers an expand task's m into the m ring.
         bool waited = p.defer_wait != 0;
+        // (x complete before the previous kernel began, tables older than it: nothing this warp reads can change)
+        if (LAZY && p.early_tables) waited = true;
         if (!waited && !p.early_tables) {
             grid_dependency_wait();
             waited = true;
@@ -1440,7 +1481,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
     uint32_t it = 0;
     bool gave_up = false;   // this lane: from here to the end of the kernel there is no warp-level operation
     if (RPK) {
-        consume_class<MODE, RPK ? RPK : 8, H, true>(p, sm, it, gave_up, acc, warp, lane);
+        consume_class<MODE, RPK ? RPK : 8, H, true, LAZY>(p, sm, it, gave_up, acc, warp, lane);
     } else {
         for (bool more = true; more;) {
             // whose stage is next?  (the class's loop waits for it again: the phase is complete by then)
@@ -1450,14 +1491,15 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
             const int rp = (int)lds32(sm.slots + slot * kSlotBytes + kHdrOffset + 36);
             if (flags & kFlagEnd) break;
             switch (rp) {
-                case 8: more = consume_class<MODE, 8, H, false>(p, sm, it, gave_up, acc, warp, lane); break;
-                case 16: more = consume_class<MODE, 16, H, false>(p, sm, it, gave_up, acc, warp, lane); break;
-                case 32: more = consume_class<MODE, 32, H, false>(p, sm, it, gave_up, acc, warp, lane); break;
-                case 64: more = consume_class<MODE, 64, H, false>(p, sm, it, gave_up, acc, warp, lane); break;
-                default: more = consume_class<MODE, 128, H, false>(p, sm, it, gave_up, acc, warp, lane); break;
+                case 8: more = consume_class<MODE, 8, H, false, LAZY>(p, sm, it, gave_up, acc, warp, lane); break;
+                case 16: more = consume_class<MODE, 16, H, false, LAZY>(p, sm, it, gave_up, acc, warp, lane); break;
+                case 32: more = consume_class<MODE, 32, H, false, LAZY>(p, sm, it, gave_up, acc, warp, lane); break;
+                case 64: more = consume_class<MODE, 64, H, false, LAZY>(p, sm, it, gave_up, acc, warp, lane); break;
+                default: more = consume_class<MODE, 128, H, false, LAZY>(p, sm, it, gave_up, acc, warp, lane); break;
             }
         }
     }
+    if (LAZY) join_stream(p, sm);   // (a CTA without a shrink task has not joined yet)
     if (tid == 0 && p.defer_wait) grid_dependency_wait();
     if (MODE == kFused && tid == 0 && p.bump_epoch) {
         // the last CTA to finish opens the next epoch: words written by this call can never
@@ -1471,29 +1513,51 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
 
 using KernelFn = void (*)(const Params);
 
-template <int MODE, bool H>
+template <int MODE, bool H, bool LAZY>
 KernelFn pick_rank(int rp) {
     switch (rp) {
-        case 0: return MODE == kFused ? bgmv_kernel<kFused, 0, H> : nullptr;   // all classes of a mixed pool, fused only
-        case 8: return bgmv_kernel<MODE, 8, H>;
-        case 16: return bgmv_kernel<MODE, 16, H>;
-        case 32: return bgmv_kernel<MODE, 32, H>;
-        case 64: return bgmv_kernel<MODE, 64, H>;
-        default: return bgmv_kernel<MODE, 128, H>;
+        case 0: return MODE == kFused ? bgmv_kernel<kFused, 0, H, LAZY> : nullptr;   // all classes of a mixed pool, fused only
+        case 8: return bgmv_kernel<MODE, 8, H, LAZY>;
+        case 16: return bgmv_kernel<MODE, 16, H, LAZY>;
+        case 32: return bgmv_kernel<MODE, 32, H, LAZY>;
+        case 64: return bgmv_kernel<MODE, 64, H, LAZY>;
+        default: return bgmv_kernel<MODE, 128, H, LAZY>;
     }
 }
+
+#ifdef PLORA_BGMV_LAZY_UNIT
+}  // namespace
+
+// The fused kernels whose consumers put off joining the stream order (plora_set_inputs_resident) are compiled in a
+// translation unit of their own, bgmv_lazy.cu, which includes this file with PLORA_BGMV_LAZY_UNIT defined and gets
+// the kernel template and this function, nothing else: the other kernels of the library keep the code they had
+// before these existed, byte for byte and in the same order (several of them run side by side in a mixed-rank
+// call, and their speed there proved sensitive to what else the module holds).
+const void* bgmv_lazy_kernel(int rp, bool fp16) {
+    return fp16 ? reinterpret_cast<const void*>(pick_rank<kFused, true, true>(rp))
+                : reinterpret_cast<const void*>(pick_rank<kFused, false, true>(rp));
+}
+#else
 
 template <bool H>
 KernelFn pick_mode(BgmvMode mode, int rp) {
     switch (mode) {
-        case kFused: return pick_rank<kFused, H>(rp);
-        case kShrinkOnly: return pick_rank<kShrinkOnly, H>(rp);
-        default: return pick_rank<kExpandOnly, H>(rp);
+        case kFused: return pick_rank<kFused, H, false>(rp);
+        case kShrinkOnly: return pick_rank<kShrinkOnly, H, false>(rp);
+        default: return pick_rank<kExpandOnly, H, false>(rp);
     }
 }
 
-KernelFn pick_kernel(BgmvMode mode, int rp, bool fp16) {
-    return fp16 ? pick_mode<true>(mode, rp) : pick_mode<false>(mode, rp);
+// lazy: the fused kernel whose consumers put off joining the stream order (plora_set_inputs_resident)
+const void* pick_kernel(BgmvMode mode, int rp, bool fp16, bool lazy) {
+    if (lazy && mode == kFused) return bgmv_lazy_kernel(rp, fp16);
+    return reinterpret_cast<const void*>(fp16 ? pick_mode<true>(mode, rp) : pick_mode<false>(mode, rp));
+}
+
+// One launch of a BGMV kernel with the given configuration.
+cudaError_t launch_kernel(const cudaLaunchConfig_t& cfg, const void* fn, const Params& p) {
+    void* args[1] = {const_cast<Params*>(&p)};
+    return cudaLaunchKernelExC(&cfg, fn, args);
 }
 
 int clamp_runs(int tiles) { return tiles < 1 ? 1 : (tiles > kMaxRuns ? kMaxRuns : tiles); }
@@ -1507,10 +1571,21 @@ cudaError_t bgmv_configure() {
         for (int rp : rps) {
             if (rp == 0 && m != kFused) continue;
             for (int h = 0; h < 2; ++h) {
-                cudaError_t e = cudaFuncSetAttribute(pick_kernel((BgmvMode)m, rp, h != 0),
+                cudaError_t e = cudaFuncSetAttribute(pick_kernel((BgmvMode)m, rp, h != 0, false),
                                                      cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
                 if (e != cudaSuccess) return e;
             }
+        }
+    return cudaSuccess;
+}
+
+// The kernels of bgmv_lazy.cu, configured (and thereby loaded) after every other module of the library.
+cudaError_t bgmv_configure_lazy() {
+    const int rps[6] = {0, 8, 16, 32, 64, 128};
+    for (int rp : rps)
+        for (int h = 0; h < 2; ++h) {
+            cudaError_t e = cudaFuncSetAttribute(bgmv_lazy_kernel(rp, h != 0), cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+            if (e != cudaSuccess) return e;
         }
     return cudaSuccess;
 }
@@ -1544,6 +1619,7 @@ cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const
     p.test_hook = dbg.test_hook;
     p.early_tables = early_tables ? 1 : 0;
     p.maybe_empty = dbg.maybe_empty ? 1 : 0;
+    p.inputs_resident = dbg.inputs_resident && mode == kFused ? 1 : 0;
     p.defer_wait = 0;
     p.bump_epoch = 1;
     cudaLaunchAttribute attr[1];
@@ -1589,7 +1665,7 @@ cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const
         cfg.stream = stream;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        const cudaError_t e = cudaLaunchKernelEx(&cfg, pick_kernel(mode, 0, fp16), p);
+        const cudaError_t e = launch_kernel(cfg, pick_kernel(mode, 0, fp16, p.inputs_resident != 0 && !p.defer_wait), p);
         ++*n_launches;
         return e;
     }
@@ -1632,7 +1708,7 @@ cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const
         cfg.stream = stream;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        const cudaError_t e = cudaLaunchKernelEx(&cfg, pick_kernel(mode, rp, fp16), p);
+        const cudaError_t e = launch_kernel(cfg, pick_kernel(mode, rp, fp16, p.inputs_resident != 0 && !p.defer_wait), p);
         ++*n_launches;
         if (e != cudaSuccess) return e;
         p.early_tables = 1;   // the next class's launch follows a kernel that is not the bucket kernel
@@ -1640,5 +1716,7 @@ cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const
     }
     return cudaSuccess;
 }
+
+#endif   // PLORA_BGMV_LAZY_UNIT
 
 }  // namespace plora

@@ -144,6 +144,7 @@ struct DebugCfg {
     long long wait_cycles = 0;   // 0: the kernels' default
     int32_t test_hook = 0;       // PLORA_HOOK_*
     bool maybe_empty = false;    // the bucket may hold tensor-core segments only (BGMV launches look before they set up)
+    bool inputs_resident = false;   // plora_set_inputs_resident: x of a call was complete before the previous kernel of the stream began
 };
 // between: a launch the caller wants between the classify pass (if one is needed) and the BGMV launches, nullptr for
 // none: the split tensor-core launch of the same call, which works on other tokens.  It joins the stream's order (the
@@ -154,6 +155,8 @@ cudaError_t launch_bgmv(BgmvMode mode, const PoolDev* pools, int n_groups, const
                         const void* const* x, float* const* y, void* m, int ldm, bool m16, bool fp16, int32_t* status,
                         int sm_count, bool early_tables, ClassCache* cls_cache, uint64_t rank_sig, const DebugCfg& dbg,
                         cudaStream_t stream, int* n_launches, BetweenLaunch between = nullptr, void* between_arg = nullptr);
+// The fused BGMV kernel of padded rank rp (0: all classes) whose consumers put off joining the stream order.
+const void* bgmv_lazy_kernel(int rp, bool fp16);
 // after_bgmv_of_same_call: the launch follows fused BGMV launches of the same call (other tokens of the
 // same batch) and may overlap them
 cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, int sgmv_min_rows, const void* x, float* y,
@@ -163,6 +166,7 @@ cudaError_t launch_sgmv(const PoolDev& pool, const BucketDev& bk, int n_tok, int
 cudaError_t bucket_configure();
 cudaError_t bgmv_configure();
 cudaError_t sgmv_configure();
+cudaError_t bgmv_configure_lazy();   // after the others: see bgmv_lazy_kernel
 int bucket_max_adapters();      // largest pool the single-CTA bucketing kernel handles
 
 }  // namespace plora

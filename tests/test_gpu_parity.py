@@ -752,3 +752,90 @@ def test_grouped_call_on_a_prefill_batch(rank):
         assert ctx.device_status() == 0
     finally:
         ctx.close()
+
+
+@pytest.mark.parametrize("ranks, T, dims", [
+    ([16] * 40, 96, (1024, 768)),                      # one rank class: the one-rank kernel
+    ([8, 16, 32, 64, 128, 24] * 6, 120, (776, 520)),   # a small batch on a pool of mixed ranks: one launch for all classes
+    ([8, 16, 32, 64] * 10, 1400, (256, 320)),          # a large batch on mixed ranks: one launch per class, overlapping
+])
+def test_inputs_resident_hint_changes_nothing_in_the_result(ranks, T, dims):
+    # With the hint the fused kernels read x and start multiplying before the previous kernel of the stream has
+    # ended; they write only after it has.  A chain of back-to-back deltas into one y (each depends on the one
+    # before through y) must give the same bits with and without the hint, eagerly and from a CUDA graph.
+    p = random_problem(900 + T, T=T, d_in=dims[0], d_out=dims[1], ranks=ranks, with_minus_one=True)
+    r = Runner(p)
+    try:
+        r.ctx.set_path(P.PATH_FUSED)
+        y_in = torch.from_numpy(p["y_in"]).to(DEV)
+        y = y_in.clone()
+
+        def step():
+            r.ctx.bucket(r.ids, p["N"])
+            for _ in range(4):
+                r.ctx.lora_delta(r.x, r.ids, 0, 0, y)
+
+        results = {}
+        for hint in (False, True, False):
+            r.ctx.set_inputs_resident(hint)
+            y.copy_(y_in)
+            step()
+            torch.cuda.synchronize()
+            results.setdefault(hint, []).append(y.cpu().numpy().copy())
+        ref = _oracle(p)
+        want = p["y_in"].astype(np.float64) + 4 * ref
+        assert np.max(np.abs(results[True][0] - want)) <= TOL_FP32_PATH * np.max(np.abs(ref)) + 4e-6 * np.max(np.abs(want))
+        assert results[True][0].tobytes() == results[False][0].tobytes() == results[False][1].tobytes()
+        r.ctx.set_inputs_resident(True)
+        s = torch.cuda.Stream()
+        s.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(s):
+            step()
+        torch.cuda.current_stream().wait_stream(s)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            step()
+        for _ in range(10):
+            y.copy_(y_in)
+            g.replay()
+            torch.cuda.synchronize()
+            assert y.cpu().numpy().tobytes() == results[True][0].tobytes()
+        assert r.ctx.device_status() == 0
+    finally:
+        r.close()
+
+
+def test_inputs_resident_hint_with_grouped_projections():
+    # q, k and v of a layer in one launch, then o, several layers back to back, hint on: equal to the oracle
+    # and to the run without the hint
+    rng = np.random.default_rng(77)
+    N, T, d = 48, 64, 512
+    ranks = rng.choice([8, 16, 64], size=N)
+    probs = [random_problem(950 + i, T=T, d_in=d, d_out=d, ranks=ranks) for i in range(8)]
+    ids = probs[0]["ids"]
+    ctx = P.Context(T, N)
+    try:
+        for i, p in enumerate(probs):
+            ctx.register_pool(i // 4, i % 4, d, d, p["ranks"], p["scales"], p["A"], p["B"])
+        x = bits_to_dev(probs[0]["x"])
+        ids_t = torch.from_numpy(ids).to(DEV)
+        outs = {}
+        for hint in (False, True):
+            ctx.set_inputs_resident(hint)
+            ys = [torch.zeros((T, d), dtype=torch.float32, device=DEV) for _ in probs]
+            ctx.bucket(ids_t, N)
+            for layer in range(2):
+                ctx.lora_delta_group([x, x, x], ids_t, [layer] * 3, [0, 1, 2], ys[4 * layer:4 * layer + 3])
+                ctx.lora_delta(x, ids_t, layer, 3, ys[4 * layer + 3])
+            torch.cuda.synchronize()
+            outs[hint] = [y.cpu().numpy() for y in ys]
+        for i, p in enumerate(probs):
+            q = dict(p)
+            q["ids"], q["x"] = ids, probs[0]["x"]
+            ref = oracle.lora_delta(q["x"], q["ids"], q["ranks"], q["scales"], q["A"], q["B"], d, np.zeros((T, d), np.float32))
+            assert rel_err(outs[True][i], ref) <= TOL_FP32_PATH
+            assert outs[True][i].tobytes() == outs[False][i].tobytes()
+        assert ctx.device_status() == 0
+    finally:
+        ctx.close()

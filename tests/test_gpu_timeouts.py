@@ -83,6 +83,32 @@ def test_a_wait_that_runs_out_is_reported_and_survivable(path):
     r.close()
 
 
+def test_a_wait_that_runs_out_in_a_launch_that_joins_late():
+    # the same with the inputs-resident hint: the consumers of the fused kernel have not joined the stream order
+    # when the copy warp gives up; two calls in a row, so that the second starts under the first one's wind-down
+    p = _small()
+    r = Runner(p)
+    ref = oracle.lora_delta(p["x"], p["ids"], p["ranks"], p["scales"], p["A"], p["B"], p["d_out"])
+    r.ctx.set_path(P.PATH_FUSED)
+    r.ctx.set_inputs_resident(True)
+    r.ctx.set_wait_limit(LIMIT)
+    r.ctx.set_test_hook(P.HOOK_WITHHOLD_RELEASE)
+    buf = _guarded_y(p["T"], p["d_out"])
+    r.ctx.bucket(r.ids, p["N"])
+    r.ctx.lora_delta(r.x, r.ids, 0, 0, buf[1:p["T"] + 1])
+    r.ctx.lora_delta(r.x, r.ids, 0, 0, buf[1:p["T"] + 1])
+    torch.cuda.synchronize()
+    assert r.ctx.device_status() == P.ERR_TIMEOUT
+    out = buf.cpu().numpy()
+    assert np.all(out[0] == 777.0) and np.all(out[-1] == 777.0), "rows around y were written"
+    r.ctx.set_test_hook(P.HOOK_NONE)
+    r.ctx.set_wait_limit(0)
+    for _ in range(2):
+        assert rel_err(r.delta(P.PATH_FUSED), ref) <= TOL_FP32_PATH
+    assert r.ctx.device_status() == 0
+    r.close()
+
+
 def test_short_limit_alone_changes_nothing():
     p = random_problem(12, T=150, d_in=776, d_out=520, ranks=[8, 24, 64, 5, 16], with_minus_one=True)
     r = Runner(p)
