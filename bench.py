@@ -48,19 +48,21 @@ from workloads import gen_pool_device, make_workload  # noqa: E402
 FALLBACK_HBM_GBS = 6650.0   # used only when MEASURED_PEAKS.json is absent
 
 # DRAM bytes (read + write) per (layer, proj) delta of the dominant kernel, from ncu captures of this
-# library at the commit named in NCU_TRAFFIC_BUILD; the roofline entry scales the figure to the average
-# launch (a launch may carry a group of projections).  A capture says nothing about a later build of the
-# kernels: the line prints the build next to the figure, and null for a workload that was not captured.
-NCU_TRAFFIC_BUILD = "a5cdd72"
+# library; the roofline entry scales the figure to the average launch (a launch may carry a group of
+# projections).  A capture says nothing about a later build of the kernels: the line prints the commit the
+# kernels of the capture were built from next to the figure, and null for a workload that was not captured.
+NCU_TRAFFIC_BUILD = "a5cdd72"          # the tensor-core kernels, the one-rank kernels of the mixed workload, attention
+NCU_TRAFFIC_BUILD_LAZY = "c047e8b"     # the fused kernels that join the stream order late (the decode workloads)
 NCU_TRAFFIC_BYTES = {
-    "decode7b": 40.2e6,    # q/k/v launch 120.46 MB, o launch 40.32 MB, over four projections
-    # captured with 150 adapters per pool (2103.4 MB of traffic for 2116.3 MB of algorithmic bytes over one layer's
+    "decode7b": 40.4e6,    # q/k/v launch 122.19 / 120.63 MB, o launch 40.30 / 40.35 MB, over four projections
+    # captured with 150 adapters per pool (2106.4 MB of traffic for 2116.3 MB of algorithmic bytes over one layer's
     # four launches); the full workload's algorithmic bytes are scaled by this ratio
-    "decode13b": ("of_algorithmic", 2103.4 / 2116.3),
+    "decode13b": ("of_algorithmic", 2106.4 / 2116.3),
     "prefill": 622.2e6,    # the wide tensor-core kernel, one projection
     "mixed": 525.7e6,      # the four rank-class launches and the split tensor-core launch of one projection
-    "skew7b": 93.2e6,      # q/k/v launch 276.93 MB, o launch 95.85 MB, over four projections
+    "skew7b": 93.0e6,      # q/k/v launch 276.22 MB, o launch 95.58 MB, over four projections
 }
+NCU_TRAFFIC_LAZY = ("decode7b", "decode13b", "skew7b")
 # decode attention, per call (one layer's cache) of the partial kernel, at the default shapes with one query head per KV head
 NCU_ATTN_TRAFFIC_BYTES = {False: 2604.8e6, True: 3241.3e6}   # short requests / long requests
 
@@ -500,7 +502,7 @@ def measure_lora(cfg: int, args, local: int, world: int, rank: int, headline: bo
     roofline = dict(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s", frac=achieved / peaks["hbm_gbs"],
                     traffic=None if traffic is None else (traffic[1] * bytes_per_launch if isinstance(traffic, tuple)
                                                            else traffic * n_calls / delta_launches),
-                    traffic_from_build=None if traffic is None else NCU_TRAFFIC_BUILD,
+                    traffic_from_build=None if traffic is None else (NCU_TRAFFIC_BUILD_LAZY if wl.name in NCU_TRAFFIC_LAZY else NCU_TRAFFIC_BUILD),
                     kernel="sgmv_kernel (tensor-core segmented GEMM)" if wl.name == "prefill" else "bgmv_kernel (fused shrink+expand)",
                     peak_source=peaks["source"], avg_launch_us=launch_us, launches_per_step=delta_launches,
                     per_projection_us=kernel_ms * 1e3, algorithmic_bytes_per_launch=bytes_per_launch,
