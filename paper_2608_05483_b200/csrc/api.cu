@@ -216,7 +216,7 @@ plora_status do_bucket(plora_ctx* ctx, const int32_t* ids, int32_t n_tok, int32_
     ctx->bucket_explicit = is_explicit;
     ctx->bucket_gen = ctx->call_gen;
     ctx->launches_since_bucket = 0;
-    ctx->cls_cache.valid = false;
+    ctx->cls_cache.reset();
     return PLORA_OK;
 }
 

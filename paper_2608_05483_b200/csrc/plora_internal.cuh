@@ -109,8 +109,8 @@ struct BucketDev {
     uint32_t* exit_count;   // CTAs of the running launch that have finished
     // pools of mixed ranks: the (projection, unit) pairs of a call sorted by padded-rank class, so
     // that the launch of a class walks only its own units (written by the classify pass)
-    int32_t* cls_list;      // kMaxGroupPools * max_tokens entries: projection * n_units + unit
-    int32_t* cls_start;     // kRankClasses + 1 offsets into cls_list
+    int32_t* cls_list;      // room for kMaxGroupPools * max_tokens entries; a sort fills n_units of them (unit numbers), the second sort starts n_tok entries in
+    int32_t* cls_start;     // kRankClasses + 1 offsets into cls_list (the second sort's: 8 words further on)
 };
 constexpr int kRankClasses = 5;   // padded ranks 8, 16, 32, 64, 128
 
@@ -134,9 +134,12 @@ constexpr int kMaxGroupPools = 4;
 // calls of a step share one sort.  The owner resets it whenever the bucket is rebuilt.  The pools of a
 // group must have the same ranks if they hold more than one rank class.  rank_sig: a hash of the
 // padded ranks of the call's pools (host side only).
+// Two sorts are kept side by side: [0] the class lists in bucket order (one launch per class), [1] ordered by token
+// count inside a class as well (one launch for all classes); a step whose calls use both kinds sorts twice, not per call.
 struct ClassCache {
-    uint64_t sig = 0;
-    bool valid = false;
+    uint64_t sig[2] = {0, 0};
+    bool valid[2] = {false, false};
+    void reset() { valid[0] = valid[1] = false; }
 };
 // Per-launch settings that come from the context: the diagnostics of the bounded waits
 // (plora_set_wait_limit, plora_set_test_hook) and what the host knows about the batch.
