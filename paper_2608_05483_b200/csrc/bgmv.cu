@@ -246,9 +246,9 @@ struct Smem {
     uint32_t m_ring;     // shared address of the m ring (fused mode): kMRing entries of kMRingBytes
     uint32_t m_full;     // m_full[kMRing]: the gather warp has written the entry
     uint32_t m_empty;    // m_empty[kMRing]: every consumer warp is done with the entry
-    uint32_t epoch;      // this launch's epoch (fused mode)
+    mutable uint32_t epoch;   // this launch's epoch (fused mode); mutable: a thread that joins late learns it then
     bool withhold;       // test hook: this warp never hands a stage back
-    bool joined;         // lazy launches: this thread has joined the stream order and knows the epoch
+    mutable bool joined;      // lazy launches: this thread has joined the stream order and knows the epoch
 };
 // A consumer warp is done with a stage.
 __device__ __forceinline__ void release_stage(const Smem& sm, uint32_t empty_bar, int lane) {
@@ -257,7 +257,7 @@ __device__ __forceinline__ void release_stage(const Smem& sm, uint32_t empty_bar
 
 // A consumer thread that put off joining the stream order does so now: from here on it may write
 // (partial words, y), and it knows the launch's epoch.
-__device__ __forceinline__ void join_stream(const Params& p, Smem& sm) {
+__device__ __forceinline__ void join_stream(const Params& p, const Smem& sm) {
     if (!sm.joined) {
         grid_dependency_wait();
         grid_launch_dependents();
@@ -798,7 +798,7 @@ __device__ __forceinline__ bool consume_stage(const Params& p, const Smem& sm, c
                 __syncwarp();
                 release_stage(sm, empty_bar, lane);
                 if (h.flags & kFlagLast) {
-                    if (LAZY) join_stream(p, const_cast<Smem&>(sm));   // (the kernel's own, non-const, object)
+                    if (LAZY) join_stream(p, sm);
                     if (tc) shrink_finish_mma<MODE, RPS < 16 ? 16 : RPS>(p, sm, h, acc[0], warp, lane);
                     else shrink_finish<MODE, RPS>(p, sm, h, maps.s2, acc, warp, lane);
                 }
@@ -807,7 +807,7 @@ __device__ __forceinline__ bool consume_stage(const Params& p, const Smem& sm, c
                 __syncwarp();
                 release_stage(sm, empty_bar, lane);
                 if (h.flags & kFlagLast) {
-                    if (LAZY) join_stream(p, const_cast<Smem&>(sm));   // (the kernel's own, non-const, object)
+                    if (LAZY) join_stream(p, sm);
                     shrink_finish_mma<MODE, RP < 16 ? 16 : RP>(p, sm, h, acc[0], warp, lane);
                 }
             } else {
@@ -815,7 +815,7 @@ __device__ __forceinline__ bool consume_stage(const Params& p, const Smem& sm, c
                 __syncwarp();
                 release_stage(sm, empty_bar, lane);
                 if (h.flags & kFlagLast) {
-                    if (LAZY) join_stream(p, const_cast<Smem&>(sm));   // (the kernel's own, non-const, object)
+                    if (LAZY) join_stream(p, sm);
                     shrink_finish<MODE, RP>(p, sm, h, maps.s, acc, warp, lane);
                 }
             }
