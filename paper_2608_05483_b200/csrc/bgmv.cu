@@ -927,8 +927,11 @@ __device__ __forceinline__ bool gather_m(const Params& p, int rp, int runs_a, ui
 // shrink tasks (4 column runs x 4 row slices) and 16 expand tasks, one of rank 8 at least one and one.
 // (Between 32 and 256 KiB: with tasks of 16 to 32 KiB, one or two stages each, the hand-over of a partial m per task
 // and the gather before every expand task weighed more than the finer balance gained; the paper's skewed decode mix
-// on 8 layers took 0.906 ms per step with those, 0.857 ms with these, and no more with a ceiling of 512 KiB or 1 MiB.)
-constexpr int kTaskBytesMin = 32 * 1024, kTaskBytesMax = 256 * 1024, kTasksPerCta = 4;
+// on 8 layers took 0.906 ms per step with those, 0.857 ms with these, and no more with a ceiling of 512 KiB or 1 MiB.
+// Two tasks per CTA and phase: since consecutive launches overlap (a launch's CTAs start on their inputs under the
+// previous launch's tail), an uneven end costs less than the hand-overs of finer tasks; the same mix with four, three,
+// two, one task per CTA: 0.820, 0.817, 0.795, 0.869 ms, and two with a ceiling of 512 KiB loses 7 % on uniform ids.)
+constexpr int kTaskBytesMin = 32 * 1024, kTaskBytesMax = 256 * 1024, kTasksPerCta = 2;
 // The one launch pays off for small batches, where the per-class launches are mostly fixed cost
 // (256 tokens, ranks 8..128, q/k/v grouped: 1.10 -> 1.00 ms for 8 layers); with many units per
 // class the per-class launches, each with loops compiled for its rank, are faster (2048 tokens,
