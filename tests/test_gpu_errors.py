@@ -7,6 +7,10 @@ import paper_2608_05483_b200 as P
 from gpu_util import DEV, Runner
 from helpers import random_problem
 
+
+def load_raw():
+    return P.load()
+
 pytestmark = pytest.mark.gpu
 
 
@@ -30,6 +34,9 @@ def test_error_statuses():
     m = torch.zeros((8, 4), dtype=torch.float32, device=DEV)
     assert P.plora_shrink(h, x, ids, 8, 0, 0, m.data_ptr(), 4) == P.ERR_INVALID_ARG        # ldm below the padded rank
     assert P.plora_set_path(h, 17, 0) == P.ERR_INVALID_ARG
+    assert load_raw().plora_set_inputs_resident(None, 1) == P.ERR_INVALID_ARG
+    assert load_raw().plora_set_inputs_resident(h, 2) == P.ERR_INVALID_ARG
+    assert P.plora_set_inputs_resident(h, True) == P.OK and P.plora_set_inputs_resident(h, False) == P.OK
     assert r.ctx.launch_count() == n0
     assert P.plora_lora_delta(h, x, ids, 0, 0, 0, y.data_ptr()) == P.OK                   # empty batch is fine
     r.close()
