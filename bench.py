@@ -53,6 +53,7 @@ FALLBACK_HBM_GBS = 6650.0   # used only when MEASURED_PEAKS.json is absent
 # kernels of the capture were built from next to the figure, and null for a workload that was not captured.
 NCU_TRAFFIC_BUILD = "a5cdd72"          # the tensor-core kernels, the one-rank kernels of the mixed workload, attention
 NCU_TRAFFIC_BUILD_LAZY = "c047e8b"     # the fused kernels that join the stream order late (the decode workloads)
+NCU_TRAFFIC_BUILD_SKEW = "468045f"     # the all-classes kernel with two tasks per CTA and phase
 NCU_TRAFFIC_BYTES = {
     "decode7b": 40.4e6,    # q/k/v launch 122.19 / 120.63 MB, o launch 40.30 / 40.35 MB, over four projections
     # captured with 150 adapters per pool (2106.4 MB of traffic for 2116.3 MB of algorithmic bytes over one layer's
@@ -60,7 +61,7 @@ NCU_TRAFFIC_BYTES = {
     "decode13b": ("of_algorithmic", 2106.4 / 2116.3),
     "prefill": 622.2e6,    # the wide tensor-core kernel, one projection
     "mixed": 525.7e6,      # the four rank-class launches and the split tensor-core launch of one projection
-    "skew7b": 93.0e6,      # q/k/v launch 276.22 MB, o launch 95.58 MB, over four projections
+    "skew7b": 93.3e6,      # q/k/v launch 277.26 MB, o launch 95.93 MB, over four projections
 }
 NCU_TRAFFIC_LAZY = ("decode7b", "decode13b", "skew7b")
 # decode attention, per call (one layer's cache) of the partial kernel, at the default shapes with one query head per KV head
@@ -502,7 +503,7 @@ def measure_lora(cfg: int, args, local: int, world: int, rank: int, headline: bo
     roofline = dict(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s", frac=achieved / peaks["hbm_gbs"],
                     traffic=None if traffic is None else (traffic[1] * bytes_per_launch if isinstance(traffic, tuple)
                                                            else traffic * n_calls / delta_launches),
-                    traffic_from_build=None if traffic is None else (NCU_TRAFFIC_BUILD_LAZY if wl.name in NCU_TRAFFIC_LAZY else NCU_TRAFFIC_BUILD),
+                    traffic_from_build=None if traffic is None else (NCU_TRAFFIC_BUILD_SKEW if wl.name == "skew7b" else NCU_TRAFFIC_BUILD_LAZY if wl.name in NCU_TRAFFIC_LAZY else NCU_TRAFFIC_BUILD),
                     kernel="sgmv_kernel (tensor-core segmented GEMM)" if wl.name == "prefill" else "bgmv_kernel (fused shrink+expand)",
                     peak_source=peaks["source"], avg_launch_us=launch_us, launches_per_step=delta_launches,
                     per_projection_us=kernel_ms * 1e3, algorithmic_bytes_per_launch=bytes_per_launch,
