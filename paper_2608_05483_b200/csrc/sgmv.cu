@@ -36,7 +36,7 @@
 // the partial m of the cluster meet through distributed shared memory (each CTA sums eight of the
 // 64 rows in a fixed order, scales, splits into hi + lo and stores the finished rows into every
 // CTA's operand buffers), and CTA c expands its eighth of d_out.  Every CTA fetches its own
-// operands; nothing is multicast.
+// operands: no copy is shared between the CTAs of a cluster.
 #include <cuda.h>
 #include <cuda_fp16.h>
 
