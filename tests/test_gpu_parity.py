@@ -839,3 +839,48 @@ def test_inputs_resident_hint_with_grouped_projections():
         assert ctx.device_status() == 0
     finally:
         ctx.close()
+
+
+def test_a_step_that_uses_both_kinds_of_mixed_rank_launch():
+    # 400 tokens on a pool of mixed ranks: q, k and v grouped make 1200 rows (one launch per rank class, class lists
+    # in bucket order), o alone 400 rows (one launch for all classes, lists ordered by token count).  Both sorts are
+    # kept side by side: the first step sorts twice, later steps on the same bucket not at all; results are
+    # bit-identical from step to step and equal to the oracle.
+    rng = np.random.default_rng(911)
+    N, T, d = 40, 400, 264
+    ranks = rng.choice([8, 16, 32, 64, 128], size=N)
+    probs = [random_problem(912 + j, T=T, d_in=d, d_out=d, ranks=ranks) for j in range(4)]
+    ids_np = probs[0]["ids"].copy()
+    ids_np[:160] = np.repeat(np.arange(40, dtype=np.int32), 4)        # units of four tokens next to single ones
+    for pr in probs:
+        pr["ids"], pr["x"] = ids_np, probs[0]["x"]
+    ctx = P.Context(T, N)
+    try:
+        for j, pr in enumerate(probs):
+            ctx.register_pool(0, j, d, d, pr["ranks"], pr["scales"], pr["A"], pr["B"])
+        ctx.set_path(P.PATH_FUSED)
+        ids = torch.from_numpy(ids_np).to(DEV)
+        x = bits_to_dev(probs[0]["x"])
+        ctx.bucket(ids, N)
+        n_classes = len(set(int(r) for r in ranks))
+        first = None
+        for step in range(3):
+            ys = [torch.from_numpy(probs[j]["y_in"]).to(DEV) for j in range(4)]
+            n0 = ctx.launch_count()
+            ctx.lora_delta_group([x, x, x], ids, [0, 0, 0], [0, 1, 2], ys[:3])
+            ctx.lora_delta(x, ids, 0, 3, ys[3])
+            torch.cuda.synchronize()
+            sorts = 2 if step == 0 else 0
+            assert ctx.launch_count() - n0 == sorts + n_classes + 1, step
+            got = [y.cpu().numpy() for y in ys]
+            if first is None:
+                first = got
+            for j in range(4):
+                assert got[j].tobytes() == first[j].tobytes(), (step, j)
+        for j in range(4):
+            ref = _oracle(probs[j], y_in=probs[j]["y_in"])
+            delta = np.max(np.abs(ref - probs[j]["y_in"]))
+            assert np.max(np.abs(first[j] - ref)) <= TOL_FP32_PATH * delta + 1e-6 * np.max(np.abs(ref)), j
+        assert ctx.device_status() == 0
+    finally:
+        ctx.close()
