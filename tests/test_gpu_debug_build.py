@@ -15,7 +15,7 @@ pytestmark = pytest.mark.gpu
 ROOT = Path(__file__).resolve().parent.parent
 CASES = ("tiny_config or odd_ranks or ragged_dims or token_counts or sgmv_tile_shapes or random_shapes or "
          "mixed_rank_calls or grouped_projections or three_long_segments or empty_and_all_minus_one or "
-         "shrink_and_expand_entry_points or two_byte_m or out_of_range_id or inputs_resident_hint")
+         "shrink_and_expand_entry_points or two_byte_m or out_of_range_id or inputs_resident_hint or both_kinds")
 
 
 def test_parity_cases_pass_under_the_checked_build():

@@ -14,7 +14,7 @@ pytestmark = pytest.mark.gpu
 ROOT = Path(__file__).resolve().parent.parent
 CASES = ("tiny_config or reduced_benchmark_configs or odd_ranks or ragged_dims or token_counts or random_shapes or "
          "mixed_rank_calls or cuda_graph_replay or grouped_projections or half_precision or auto_dispatch or "
-         "three_long_segments or empty_and_all_minus_one or out_of_range_id")
+         "three_long_segments or empty_and_all_minus_one or out_of_range_id or both_kinds")
 
 
 def test_parity_cases_pass_with_the_hint_on():
