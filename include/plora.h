@@ -337,6 +337,8 @@ PLORA_API plora_status plora_set_input_type(plora_ctx *ctx, int32_t type);
  * then stream and multiply x while the previous kernel drains; they still write nothing (workspace, y)
  * and read no y before it has completed, and the results are bit-identical to those with resident = 0.
  * Wrong use is a data race on x, nothing else.  The tensor-core path and the unfused halves ignore the hint.
+ * Host-side setting of the context, no device work; PLORA_ERR_INVALID_ARG for a null context or a value
+ * other than 0 or 1.
  */
 PLORA_API plora_status plora_set_inputs_resident(plora_ctx *ctx, int32_t resident);
 
