@@ -1053,8 +1053,11 @@ __device__ __forceinline__ Plan<RPK ? 1 : kRankClasses> make_plan(const Params& 
             const int half_a = p.pool.d_in * rp * 2, half_b = p.pool.d_out * rp * 2;   // bytes of a unit's A and B
             int s_runs = clamp_int((half_a + tgt_a / 2) / tgt_a, 1, min(kMaxRunsA, tiles_for(p.pool.d_in, rp)));
             int slices = 1;
-            if (rp > kSliceRows && half_a / s_runs > 2 * tgt_a) {
-                // the column runs alone leave the tasks too large: cut along the rank too
+            if (rp > kSliceRows && half_a / s_runs > 4 * tgt_a) {
+                // the column runs alone leave the tasks far too large (a handful of units in a small batch): cut
+                // along the rank too.  (Only then: slice stages cost four copies each and run the rank-32 loops;
+                // with the threshold at twice the target the skewed decode mix took 0.795 ms per step, at four
+                // times, eight times or without slices 0.779.)
                 slices = rp / kSliceRows;
                 s_runs = clamp_int((half_a / slices + tgt_a / 2) / tgt_a, 1, min(kMaxRunsA, tiles_for(p.pool.d_in, kSliceRows)));
             }
