@@ -931,7 +931,9 @@ __device__ __forceinline__ bool gather_m(const Params& p, int rp, int runs_a, ui
 // Two tasks per CTA and phase: since consecutive launches overlap (a launch's CTAs start on their inputs under the
 // previous launch's tail), an uneven end costs less than the hand-overs of finer tasks; the same mix with four, three,
 // two, one task per CTA: 0.820, 0.817, 0.795, 0.869 ms, and two with a ceiling of 512 KiB loses 7 % on uniform ids.)
-constexpr int kTaskBytesMin = 32 * 1024, kTaskBytesMax = 256 * 1024, kTasksPerCta = 2;
+// The expand phase does with one task per CTA (an expand task has no hand-over at its end, but a gather at its start):
+// 0.779 -> 0.768 ms on the same mix, better on six of seven other small mixed-rank batches.
+constexpr int kTaskBytesMin = 32 * 1024, kTaskBytesMax = 256 * 1024, kTasksPerCta = 2, kExpandTasksPerCta = 1;
 // The one launch pays off for small batches, where the per-class launches are mostly fixed cost
 // (256 tokens, ranks 8..128, q/k/v grouped: 1.10 -> 1.00 ms for 8 layers); with many units per
 // class the per-class launches, each with loops compiled for its rank, are faster (2048 tokens,
@@ -1044,9 +1046,9 @@ __device__ __forceinline__ Plan<RPK ? 1 : kRankClasses> make_plan(const Params& 
             tot_a += (long long)pl.n[i] * p.pool.d_in * rp * 2;
             tot_b += (long long)pl.n[i] * p.pool.d_out * rp * 2;
         }
-        // task size: about kTasksPerCta tasks per CTA and phase, within the bounds above
+        // task size: about kTasksPerCta shrink tasks and kExpandTasksPerCta expand tasks per CTA, within the bounds above
         const int tgt_a = clamp_int((int)(tot_a / (kTasksPerCta * (long long)gridDim.x)), kTaskBytesMin, kTaskBytesMax);
-        const int tgt_b = clamp_int((int)(tot_b / (kTasksPerCta * (long long)gridDim.x)), kTaskBytesMin, kTaskBytesMax);
+        const int tgt_b = clamp_int((int)(tot_b / (kExpandTasksPerCta * (long long)gridDim.x)), kTaskBytesMin, kTaskBytesMax);
 #pragma unroll
         for (int i = 0; i < NC; ++i) {
             const int rp = pl.rp[i];
