@@ -53,7 +53,7 @@ FALLBACK_HBM_GBS = 6650.0   # used only when MEASURED_PEAKS.json is absent
 # kernels of the capture were built from next to the figure, and null for a workload that was not captured.
 NCU_TRAFFIC_BUILD = "a5cdd72"          # the tensor-core kernels, the one-rank kernels of the mixed workload, attention
 NCU_TRAFFIC_BUILD_LAZY = "c047e8b"     # the fused kernels that join the stream order late (the decode workloads)
-NCU_TRAFFIC_BUILD_SKEW = "468045f"     # the all-classes kernel with two tasks per CTA and phase
+NCU_TRAFFIC_BUILD_SKEW = "ce7d1ff"     # the all-classes kernel with its final task plan
 NCU_TRAFFIC_BYTES = {
     "decode7b": 40.4e6,    # q/k/v launch 122.19 / 120.63 MB, o launch 40.30 / 40.35 MB, over four projections
     # captured with 150 adapters per pool (2106.4 MB of traffic for 2116.3 MB of algorithmic bytes over one layer's
@@ -61,7 +61,7 @@ NCU_TRAFFIC_BYTES = {
     "decode13b": ("of_algorithmic", 2106.4 / 2116.3),
     "prefill": 622.2e6,    # the wide tensor-core kernel, one projection
     "mixed": 525.7e6,      # the four rank-class launches and the split tensor-core launch of one projection
-    "skew7b": 93.3e6,      # q/k/v launch 277.26 MB, o launch 95.93 MB, over four projections
+    "skew7b": 93.5e6,      # q/k/v launch 277.62 MB, o launch 96.26 MB, over four projections
 }
 NCU_TRAFFIC_LAZY = ("decode7b", "decode13b", "skew7b")
 # decode attention, per call (one layer's cache) of the partial kernel, at the default shapes with one query head per KV head
