@@ -922,7 +922,7 @@ __device__ __forceinline__ bool gather_m(const Params& p, int rp, int runs_a, ui
 //
 // Mixed launch: tasks of very different sizes under a static round-robin leave the CTAs that drew
 // the large ones far behind (measured 2x slower than one launch per class), so the classes are cut to
-// tasks of about the same size, chosen so that a CTA gets about kTasksPerCta tasks per phase: between
+// tasks of about the same size, chosen so that a CTA gets a few tasks per phase (TaskPlanCfg): between
 // kTaskBytesMin and kTaskBytesMax of adapter bytes.  A unit of padded rank 128 then makes up to 16
 // shrink tasks (4 column runs x 4 row slices) and 16 expand tasks, one of rank 8 at least one and one.
 // (Between 32 and 256 KiB: with tasks of 16 to 32 KiB, one or two stages each, the hand-over of a partial m per task
@@ -933,7 +933,16 @@ __device__ __forceinline__ bool gather_m(const Params& p, int rp, int runs_a, ui
 // two, one task per CTA: 0.820, 0.817, 0.795, 0.869 ms, and two with a ceiling of 512 KiB loses 7 % on uniform ids.)
 // The expand phase does with one task per CTA (an expand task has no hand-over at its end, but a gather at its start):
 // 0.779 -> 0.768 ms on the same mix, better on six of seven other small mixed-rank batches.
-constexpr int kTaskBytesMin = 32 * 1024, kTaskBytesMax = 256 * 1024, kTasksPerCta = 2, kExpandTasksPerCta = 1;
+// These coarse tasks are for the kernels that join the stream order late, whose launches overlap; a launch that waits
+// at its start for the one before it keeps four tasks per CTA and phase and slices from twice the target size on
+// (without the hint the same mix takes 0.854 ms per step with those, about 0.905 ms with the coarse plan).
+constexpr int kTaskBytesMin = 32 * 1024, kTaskBytesMax = 256 * 1024;
+template <bool LAZY>
+struct TaskPlanCfg {
+    static constexpr int kShrinkTasksPerCta = LAZY ? 2 : 4;
+    static constexpr int kExpandTasksPerCta = LAZY ? 1 : 4;
+    static constexpr int kSliceFactor = LAZY ? 4 : 2;   // row slices when a column run exceeds this many targets
+};
 // The one launch pays off for small batches, where the per-class launches are mostly fixed cost
 // (256 tokens, ranks 8..128, q/k/v grouped: 1.10 -> 1.00 ms for 8 layers); with many units per
 // class the per-class launches, each with loops compiled for its rank, are faster (2048 tokens,
@@ -1012,7 +1021,7 @@ __device__ __forceinline__ int expand_runs(const Params& p, int n_vunits) {
     return runs;
 }
 
-template <int MODE, int RPK>
+template <int MODE, int RPK, bool LAZY>
 __device__ __forceinline__ Plan<RPK ? 1 : kRankClasses> make_plan(const Params& p, int n_units) {
     constexpr int NC = RPK ? 1 : kRankClasses;
     Plan<NC> pl;
@@ -1046,16 +1055,17 @@ __device__ __forceinline__ Plan<RPK ? 1 : kRankClasses> make_plan(const Params& 
             tot_a += (long long)pl.n[i] * p.pool.d_in * rp * 2;
             tot_b += (long long)pl.n[i] * p.pool.d_out * rp * 2;
         }
-        // task size: about kTasksPerCta shrink tasks and kExpandTasksPerCta expand tasks per CTA, within the bounds above
-        const int tgt_a = clamp_int((int)(tot_a / (kTasksPerCta * (long long)gridDim.x)), kTaskBytesMin, kTaskBytesMax);
-        const int tgt_b = clamp_int((int)(tot_b / (kExpandTasksPerCta * (long long)gridDim.x)), kTaskBytesMin, kTaskBytesMax);
+        // task size: a few shrink and expand tasks per CTA (TaskPlanCfg), within the bounds above
+        using Cfg = TaskPlanCfg<LAZY>;
+        const int tgt_a = clamp_int((int)(tot_a / (Cfg::kShrinkTasksPerCta * (long long)gridDim.x)), kTaskBytesMin, kTaskBytesMax);
+        const int tgt_b = clamp_int((int)(tot_b / (Cfg::kExpandTasksPerCta * (long long)gridDim.x)), kTaskBytesMin, kTaskBytesMax);
 #pragma unroll
         for (int i = 0; i < NC; ++i) {
             const int rp = pl.rp[i];
             const int half_a = p.pool.d_in * rp * 2, half_b = p.pool.d_out * rp * 2;   // bytes of a unit's A and B
             int s_runs = clamp_int((half_a + tgt_a / 2) / tgt_a, 1, min(kMaxRunsA, tiles_for(p.pool.d_in, rp)));
             int slices = 1;
-            if (rp > kSliceRows && half_a / s_runs > 4 * tgt_a) {
+            if (rp > kSliceRows && half_a / s_runs > Cfg::kSliceFactor * tgt_a) {
                 // the column runs alone leave the tasks far too large (a handful of units in a small batch): cut
                 // along the rank too.  (Only then: slice stages cost four copies each and run the rank-32 loops;
                 // with the threshold at twice the target the skewed decode mix took 0.795 ms per step, at four
@@ -1262,7 +1272,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
             waited = true;
         }
         const int n_units = *p.bk.n_bgmv_units;
-        const auto plan = make_plan<MODE, RPK>(p, n_units);   // the tasks of this launch
+        const auto plan = make_plan<MODE, RPK, LAZY>(p, n_units);   // the tasks of this launch
         const int n_tasks = plan.n_tasks;
         const int stride = gridDim.x;
         const unsigned full = 0xffffffffu;
@@ -1420,7 +1430,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) bgmv_kernel(const Params
         // epoch), sums them in run order into the next m-ring entry and publishes the entry.
         if (MODE != kFused) return;
         const int n_units = *p.bk.n_bgmv_units;
-        const auto plan = make_plan<MODE, RPK>(p, n_units);
+        const auto plan = make_plan<MODE, RPK, LAZY>(p, n_units);
         const int n_shrink = plan.n_shrink, n_tasks = plan.n_tasks;
         const int stride = gridDim.x;
         const unsigned full = 0xffffffffu;
